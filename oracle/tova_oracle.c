@@ -1,0 +1,205 @@
+/*
+ * TEST INFRASTRUCTURE - CPU checker for the TOVA decode step.
+ *
+ * A plain, slow, deliberately unoptimised statement of what one decoding step
+ * of one transformer layer computes when the layer is run as a bounded
+ * multi-state RNN with the TOVA compression policy.  It exists only so that
+ * tests, the smoke check and the CPU-baseline leg of the benchmark have
+ * something to compare the GPU library with.  It shares no code with the GPU
+ * library and must never be called from it.
+ *
+ * What it follows, step by step and in the paper's order:
+ *   - Eq. 6 (Section 3.2): the new (k_t, v_t) is appended to the multi-state
+ *     (K_{t-1}, V_{t-1}) first;
+ *   - Eq. 4 / Eq. 7: the layer output is Softmax(q_t K_t^T) V_t over ALL rows
+ *     of the appended state, including the row that is about to be dropped;
+ *   - Section 3.3: g(t) = min(t, k): nothing is dropped while the state has
+ *     at most k rows;
+ *   - Section 4, Eq. 9 and Algorithm 1: once the appended state has k+1 rows,
+ *     the last query's attention weights are averaged over the heads of the
+ *     layer, the row with the lowest average is deleted from K and V.
+ *
+ * Readings where the paper is silent (stated once more in the design notes):
+ *   - a scale factor multiplies the logits (the paper omits 1/sqrt(d));
+ *   - under grouped-query attention all H query heads are averaged and the one
+ *     victim is removed from every KV head;
+ *   - ties of the arg-min go to the lowest row index, the new token being the
+ *     last row;
+ *   - the state is kept in place: the new token takes the victim's row, so
+ *     row order is not position order; positions travel with the rows.
+ *
+ * Precision: every operation is carried out in REAL (float for the parity
+ * checker, double for the reference the float build is itself checked with).
+ * Sums run in ascending index order; the soft-max divides (no reciprocal).
+ *
+ * Parity pins (tests marked "not gpu"): textbook soft-max attention in double
+ * on tiny states, library causal attention when k >= stream length, the
+ * size invariant len_t = min(t, k), a hand-worked 3-row example in exact
+ * rational arithmetic, an order-preserving restatement of Algorithm 1, and
+ * permutation / shift invariances.
+ */
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifndef REAL
+#define REAL float
+#endif
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static REAL real_exp(REAL x) { return sizeof(REAL) == 4 ? (REAL)expf((float)x) : (REAL)exp((double)x); }
+
+/*
+ * One token for one sequence.
+ *   len      in/out  live rows n (0 <= n <= cap)
+ *   pos      in/out  [cap]          original position of each row, -1 if unused
+ *   K, V     in/out  [Hkv][cap][D]
+ *   q        in      [H][D]
+ *   k_new,v_new in   [Hkv][D]
+ *   forced   in      -1, or the candidate index (0..cap) to drop instead of
+ *                    the arg-min when a drop is due
+ *   out      out     [H][D]
+ *   evicted_pos out  position dropped; -1 when nothing was dropped
+ *   victim   out     candidate index dropped (cap = the new token), -1 if none
+ *   argmin   out     the arg-min itself (differs from victim only when forced), -1 if none
+ *   gap      out     mean[dropped] - min(mean) (0 unless forced differs)
+ *   mean_out out     [cap+1] head-averaged weights, or NULL
+ *   work     scratch [H+1][cap+1] REAL (weights per head, then their mean)
+ */
+static void step_one(int H, int Hkv, int D, int cap, REAL scale,
+                     int *len, int *pos, REAL *K, REAL *V,
+                     const REAL *q, const REAL *k_new, const REAL *v_new,
+                     int pos_t, int forced,
+                     REAL *out, int *evicted_pos, int *victim, int *argmin, REAL *gap,
+                     REAL *mean_out, REAL *work)
+{
+    const int n = *len;          /* rows before the append */
+    const int m = n + 1;         /* rows after the append (Eq. 6) */
+    const int G = H / Hkv;
+    const int ld = cap + 1;
+
+    /* Attention weights of the new query over the appended state (Eq. 4). */
+    for (int h = 0; h < H; ++h) {
+        const int kv = h / G;
+        REAL *p = work + (size_t)h * ld;
+        for (int j = 0; j < m; ++j) {
+            const REAL *krow = (j < n) ? K + ((size_t)kv * cap + j) * D : k_new + (size_t)kv * D;
+            REAL s = 0;
+            for (int d = 0; d < D; ++d) s += q[(size_t)h * D + d] * krow[d];
+            p[j] = scale * s;
+        }
+        REAL mx = p[0];
+        for (int j = 1; j < m; ++j) if (p[j] > mx) mx = p[j];
+        REAL l = 0;
+        for (int j = 0; j < m; ++j) { p[j] = real_exp(p[j] - mx); l += p[j]; }
+        for (int j = 0; j < m; ++j) p[j] = p[j] / l;
+        /* Layer output before any row is dropped (Eq. 7). */
+        for (int d = 0; d < D; ++d) {
+            REAL o = 0;
+            for (int j = 0; j < m; ++j) {
+                const REAL *vrow = (j < n) ? V + ((size_t)kv * cap + j) * D : v_new + (size_t)kv * D;
+                o += p[j] * vrow[d];
+            }
+            out[(size_t)h * D + d] = o;
+        }
+    }
+
+    *gap = 0;
+    if (m <= cap) {              /* Algorithm 1: num_kv <= cache_max_size -> keep all */
+        for (int kv = 0; kv < Hkv; ++kv) {
+            memcpy(K + ((size_t)kv * cap + n) * D, k_new + (size_t)kv * D, sizeof(REAL) * D);
+            memcpy(V + ((size_t)kv * cap + n) * D, v_new + (size_t)kv * D, sizeof(REAL) * D);
+        }
+        pos[n] = pos_t;
+        *len = m;
+        *evicted_pos = -1;
+        *victim = -1;
+        *argmin = -1;
+        if (mean_out) for (int j = 0; j < ld; ++j) mean_out[j] = 0;
+        return;
+    }
+
+    /* Average the last query's weights over the heads, take the arg-min
+     * (Algorithm 1), lowest index on ties. */
+    REAL *mean = work + (size_t)H * ld;
+    int jmin = 0;
+    for (int j = 0; j < m; ++j) {
+        REAL a = 0;
+        for (int h = 0; h < H; ++h) a += work[(size_t)h * ld + j];
+        mean[j] = a / (REAL)H;
+        if (mean[j] < mean[jmin]) jmin = j;
+    }
+    if (mean_out) for (int j = 0; j < m; ++j) mean_out[j] = mean[j];
+    int drop = jmin;
+    *argmin = jmin;
+    if (forced >= 0 && forced < m) {
+        drop = forced;
+        *gap = mean[drop] - mean[jmin];
+    }
+
+    /* Delete row `drop` from K and V (Eq. 9): in place, the new token takes
+     * the freed row; dropping the new token itself changes nothing. */
+    *victim = drop;
+    if (drop < cap) {
+        *evicted_pos = pos[drop];
+        for (int kv = 0; kv < Hkv; ++kv) {
+            memcpy(K + ((size_t)kv * cap + drop) * D, k_new + (size_t)kv * D, sizeof(REAL) * D);
+            memcpy(V + ((size_t)kv * cap + drop) * D, v_new + (size_t)kv * D, sizeof(REAL) * D);
+        }
+        pos[drop] = pos_t;
+    } else {
+        *evicted_pos = pos_t;
+    }
+}
+
+/*
+ * One token for each of B independent sequences (Algorithm 1 assumes batch 1:
+ * sequences never interact).  Layouts: len [B], pos [B][cap],
+ * K,V [B][Hkv][cap][D], q/out [B][H][D], k_new/v_new [B][Hkv][D],
+ * forced/evicted_pos/victim/argmin/gap [B] (forced may be NULL),
+ * mean_out [B][cap+1] or NULL.  Sequences are spread over `nthreads` threads;
+ * nothing else is parallel.  Returns 0, or -1 on a bad argument.
+ */
+int tova_oracle_step(int B, int H, int Hkv, int D, int cap, REAL scale,
+                     int *len, int *pos, REAL *K, REAL *V,
+                     const REAL *q, const REAL *k_new, const REAL *v_new,
+                     int pos_t, const int *forced,
+                     REAL *out, int *evicted_pos, int *victim, int *argmin, REAL *gap,
+                     REAL *mean_out, int nthreads)
+{
+    if (B < 1 || H < 1 || Hkv < 1 || D < 1 || cap < 1 || H % Hkv != 0) return -1;
+    const size_t ld = (size_t)cap + 1;
+    if (nthreads < 1) nthreads = 1;
+    int bad = 0;
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(nthreads) schedule(static)
+#endif
+    for (int b = 0; b < B; ++b) {
+        REAL *work = (REAL *)malloc(sizeof(REAL) * (size_t)(H + 1) * ld);
+        if (!work) { bad = 1; continue; }
+        if (len[b] < 0 || len[b] > cap) { bad = 1; free(work); continue; }
+        step_one(H, Hkv, D, cap, scale,
+                 len + b, pos + (size_t)b * cap,
+                 K + (size_t)b * Hkv * cap * D, V + (size_t)b * Hkv * cap * D,
+                 q + (size_t)b * H * D, k_new + (size_t)b * Hkv * D, v_new + (size_t)b * Hkv * D,
+                 pos_t, forced ? forced[b] : -1,
+                 out + (size_t)b * H * D, evicted_pos + b, victim + b, argmin + b, gap + b,
+                 mean_out ? mean_out + (size_t)b * ld : NULL, work);
+        free(work);
+    }
+    return bad ? -1 : 0;
+}
+
+int tova_oracle_real_bytes(void) { return (int)sizeof(REAL); }
+
+int tova_oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

@@ -1,0 +1,107 @@
+"""TEST INFRASTRUCTURE - ctypes front end of the CPU checker in tova_oracle.c.
+
+Only tests, the smoke check and the CPU-baseline leg of the benchmark may use
+this module.  It compiles tova_oracle.c with gcc twice (REAL=float, the parity
+checker; REAL=double, the reference the float build is itself checked with)
+and keeps one bounded multi-state per layer in numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "tova_oracle.c")
+_LIBS = {}
+
+
+def build(force: bool = False) -> None:
+    """Compile both precisions of the checker next to its source."""
+    for tag, real in (("f32", "float"), ("f64", "double")):
+        so = os.path.join(_HERE, f"libtova_oracle_{tag}.so")
+        if not force and os.path.exists(so) and os.path.getmtime(so) >= os.path.getmtime(_SRC):
+            continue
+        tmp = so + f".tmp{os.getpid()}"
+        cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", f"-DREAL={real}",
+               "-o", tmp, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, so)
+
+
+def _lib(precision: str):
+    if precision not in _LIBS:
+        build()
+        tag = {"f32": "f32", "f64": "f64"}[precision]
+        lib = ctypes.CDLL(os.path.join(_HERE, f"libtova_oracle_{tag}.so"))
+        lib.tova_oracle_step.restype = ctypes.c_int
+        lib.tova_oracle_real_bytes.restype = ctypes.c_int
+        lib.tova_oracle_max_threads.restype = ctypes.c_int
+        _LIBS[precision] = lib
+    return _LIBS[precision]
+
+
+def host_threads() -> int:
+    """Threads the checker may use: the cores this process is allowed on."""
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:  # pragma: no cover
+        return max(1, os.cpu_count() or 1)
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+class OracleCache:
+    """Bounded multi-state (K, V) of one layer for B independent sequences."""
+
+    def __init__(self, batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
+                 capacity: int, sm_scale: float = 0.0, precision: str = "f32",
+                 threads: Optional[int] = None):
+        if n_q_heads % n_kv_heads:
+            raise ValueError("n_q_heads must be a multiple of n_kv_heads")
+        self.B, self.H, self.Hkv, self.D, self.cap = batch, n_q_heads, n_kv_heads, head_dim, capacity
+        self.scale = float(sm_scale) if sm_scale else 1.0 / float(np.sqrt(head_dim))
+        self.precision = precision
+        self.real = np.float32 if precision == "f32" else np.float64
+        self.creal = ctypes.c_float if precision == "f32" else ctypes.c_double
+        self.lib = _lib(precision)
+        assert self.lib.tova_oracle_real_bytes() == np.dtype(self.real).itemsize
+        self.threads = threads or host_threads()
+        self.len = np.zeros(batch, np.int32)
+        self.pos = np.full((batch, capacity), -1, np.int32)
+        self.K = np.zeros((batch, n_kv_heads, capacity, head_dim), self.real)
+        self.V = np.zeros_like(self.K)
+
+    def step(self, q, k_new, v_new, pos_t: int, forced=None, want_mean: bool = False):
+        """Feed one token to every sequence.
+
+        Returns (out [B,H,D], evicted_pos [B], victim [B], argmin [B], gap [B],
+        mean [B,cap+1] or None).
+        `forced` [B] int: candidate index to drop instead of the arg-min
+        (-1 = no override)."""
+        B, H, Hkv, D, cap = self.B, self.H, self.Hkv, self.D, self.cap
+        q = np.ascontiguousarray(q, self.real).reshape(B, H, D)
+        k_new = np.ascontiguousarray(k_new, self.real).reshape(B, Hkv, D)
+        v_new = np.ascontiguousarray(v_new, self.real).reshape(B, Hkv, D)
+        out = np.empty((B, H, D), self.real)
+        ev = np.empty(B, np.int32)
+        victim = np.empty(B, np.int32)
+        argmin = np.empty(B, np.int32)
+        gap = np.zeros(B, self.real)
+        mean = np.zeros((B, cap + 1), self.real) if want_mean else None
+        f = None if forced is None else np.ascontiguousarray(forced, np.int32)
+        rc = self.lib.tova_oracle_step(
+            ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D),
+            ctypes.c_int(cap), self.creal(self.scale),
+            _ptr(self.len), _ptr(self.pos), _ptr(self.K), _ptr(self.V),
+            _ptr(q), _ptr(k_new), _ptr(v_new), ctypes.c_int(int(pos_t)), _ptr(f),
+            _ptr(out), _ptr(ev), _ptr(victim), _ptr(argmin), _ptr(gap), _ptr(mean),
+            ctypes.c_int(self.threads))
+        if rc != 0:
+            raise RuntimeError("tova_oracle_step rejected its arguments")
+        return out, ev, victim, argmin, gap, mean
