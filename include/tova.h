@@ -1,0 +1,143 @@
+/*
+ * tova.h - C ABI of the bounded multi-state (KV cache) decode step with TOVA
+ * eviction, for NVIDIA B200 (sm_100a).
+ *
+ * A transformer layer is run as a bounded multi-state RNN (Section 3.3 of
+ * "Transformers are Multi-State RNNs"): the state of a layer is the pair
+ * (K, V) with at most `capacity` rows per sequence.  One decoding step appends
+ * the new token's (k, v) to the state (Eq. 6), attends with the new query over
+ * all rows (Eq. 4, Eq. 7) and, once the appended state holds capacity+1 rows,
+ * drops the row whose attention weight, averaged over the query heads of the
+ * layer, is lowest (Section 4, Eq. 9, Algorithm 1).
+ *
+ * General conventions
+ *  - One tova_cache holds the state of ONE layer for `batch` independent
+ *    sequences that advance in lock step (one token each per call).
+ *  - Unless a parameter says "host", every tensor pointer is a DEVICE pointer,
+ *    16-byte aligned, contiguous in the stated layout, owned by the caller.
+ *    The library allocates no device memory: the caller provides one block of
+ *    tova_cache_bytes() bytes at init, which must outlive the handle.
+ *  - q, k, v have the cache's dtype (fp32 or bf16); outputs are fp32.
+ *  - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL =
+ *    the default stream) and return without synchronising.  All calls on one
+ *    cache must be issued on one stream or otherwise ordered by the caller.
+ *  - Return value: TOVA_OK or a negative tova_status.  Argument errors are
+ *    detected on the host before anything is launched.  There is no CPU
+ *    fallback: without a usable CUDA device the calls fail with TOVA_ERR_CUDA.
+ *  - Keys are cached as given (callers pass post-RoPE q and k); positions are
+ *    metadata that travel with the rows, so eviction never re-rotates a key.
+ */
+#ifndef TOVA_H_
+#define TOVA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tova_cache tova_cache; /* opaque host handle */
+
+enum { TOVA_DTYPE_FP32 = 0, TOVA_DTYPE_BF16 = 1 };
+
+/* Pass as `pos` / `first_pos`: the token's position is the previous token's
+ * position in this cache plus one (0 for the first token), taken from a
+ * counter on the device; a recorded sequence of steps (a CUDA graph) can then
+ * be replayed and still give every token a fresh position. */
+#define TOVA_POS_AUTO (-1)
+
+typedef enum {
+  TOVA_OK = 0,
+  TOVA_ERR_NULL = -1,        /* a required pointer is NULL                        */
+  TOVA_ERR_BAD_SHAPE = -2,   /* batch/heads/capacity/n_tokens out of range        */
+  TOVA_ERR_UNSUPPORTED = -3, /* head_dim not in {64,128}, unknown dtype           */
+  TOVA_ERR_ALIGN = -4,       /* a device pointer is not 16-byte aligned           */
+  TOVA_ERR_WORKSPACE = -5,   /* dev_bytes < tova_cache_bytes()                    */
+  TOVA_ERR_FULL = -6,        /* evict == 0 and the state already holds capacity   */
+  TOVA_ERR_CUDA = -7,        /* a CUDA runtime call or launch failed              */
+  TOVA_ERR_DEVICE = -8       /* a kernel reported a failed internal check         */
+} tova_status;
+
+typedef struct {
+  int32_t batch;      /* B >= 1 sequences                                          */
+  int32_t n_q_heads;  /* H >= 1 query heads                                        */
+  int32_t n_kv_heads; /* Hkv >= 1, H % Hkv == 0 (H == Hkv: MHA, else GQA)          */
+  int32_t head_dim;   /* D in {64, 128}                                            */
+  int32_t capacity;   /* k >= 1 rows per sequence (the multi-state size)           */
+  int32_t dtype;      /* TOVA_DTYPE_FP32 or TOVA_DTYPE_BF16 for q, k, v, K, V      */
+  float sm_scale;     /* logit scale; 0 selects 1/sqrt(head_dim)                   */
+  int32_t evict;      /* 1: TOVA policy; 0: unbounded arm (a full state is an error) */
+} tova_config;
+
+/* Device bytes a cache of this shape needs (K, V, positions, lengths, the
+ * logit / partial-result scratch, counters, status, host-call staging).
+ * Returns 0 when the configuration is invalid. */
+size_t tova_cache_bytes(const tova_config* cfg);
+
+/* Create a cache in caller-provided device memory `dev_mem` (256-byte aligned,
+ * dev_bytes >= tova_cache_bytes(cfg)) and enqueue its initialisation (empty
+ * state: length 0, positions -1).  The multi-state H_0 is empty (Section 3.1).
+ * `*out` receives a host handle to be released with tova_cache_destroy. */
+int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, size_t dev_bytes,
+                    void* cuda_stream);
+
+/* One decoding step of the layer for every sequence (Eq. 6, Eq. 4, Eq. 7,
+ * then Algorithm 1 / Eq. 9):
+ *   q [B,H,D], k and v [B,Hkv,D]   the new token's projections (cache dtype)
+ *   pos                            its original position (metadata), or TOVA_POS_AUTO
+ *   out [B,H,D] fp32               attention output over all n+1 rows, the
+ *                                  row dropped at this step included
+ *   evicted_pos [B] int32 or NULL  position of the dropped token; -1 when the
+ *                                  state was not full; `pos` when the new
+ *                                  token itself was dropped
+ * The new token takes the dropped row's slot in place (slot order is not
+ * position order).  Ties of the arg-min go to the lowest slot, the new token
+ * counting as slot `capacity`. */
+int tova_decode_step(tova_cache* c, const void* q, const void* k, const void* v, int32_t pos,
+                     float* out, int32_t* evicted_pos, void* cuda_stream);
+
+/* The same per-token policy run over n_tokens consecutive prompt tokens at
+ * positions first_pos, first_pos+1, ...: identical results to n_tokens calls
+ * of tova_decode_step.
+ *   q [T,B,H,D], k and v [T,B,Hkv,D]; out [T,B,H,D] fp32 or NULL;
+ *   evicted_pos [T,B] or NULL. */
+int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int32_t n_tokens,
+                 int32_t first_pos, float* out, int32_t* evicted_pos, void* cuda_stream);
+
+/* tova_decode_step with HOST buffers: q, k, v are copied to the device, the
+ * step runs, out (and evicted_pos if not NULL) are copied back, all on
+ * `cuda_stream`; returns after the stream has been synchronised.  Pinned host
+ * memory makes the copies asynchronous, pageable memory works too. */
+int tova_decode_step_host(tova_cache* c, const void* q_host, const void* k_host,
+                          const void* v_host, int32_t pos, float* out_host,
+                          int32_t* evicted_pos_host, void* cuda_stream);
+
+/* Copy the state out (device to DEVICE buffers of the caller; any may be NULL):
+ *   len [B] int32, positions [B,capacity] int32 in slot order (-1 = unused),
+ *   k_out, v_out [B,Hkv,capacity,D] in the cache dtype,
+ *   status [1] int32: 0, or a nonzero code left by a failed device-side check. */
+int tova_cache_read(const tova_cache* c, int32_t* len, int32_t* positions, void* k_out,
+                    void* v_out, int32_t* status, void* cuda_stream);
+
+/* Tuning: rows of the state one thread block of the streaming kernel covers
+ * (32, 64, 128 or 256; 0 restores the automatic choice made at init).  Results
+ * do not depend on it beyond floating-point summation order. */
+int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows);
+
+/* Rows each sequence holds now, min(tokens fed, capacity) = g(t) of Section
+ * 3.3, tracked on the host (sequences advance in lock step). */
+int32_t tova_cache_len(const tova_cache* c);
+
+/* Kernel launches issued for this cache so far (for benchmarks). */
+int64_t tova_cache_launches(const tova_cache* c);
+
+/* Release the host handle (device memory stays with the caller). */
+int tova_cache_destroy(tova_cache* c);
+
+const char* tova_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TOVA_H_ */

@@ -1,0 +1,11 @@
+"""B200-native TOVA decode step: bounded multi-state attention with eviction.
+
+The product is the CUDA library behind include/tova.h; this package holds its
+sources (csrc/), the in-tree build, a ctypes binding with the same names, and
+the seeded synthetic workloads.
+"""
+from .binding import (TOVA_DTYPE_BF16, TOVA_DTYPE_FP32, TovaCache, TovaError, lib, strerror,
+                      to_device, tova_cache_bytes, tova_config)
+
+__all__ = ["TOVA_DTYPE_BF16", "TOVA_DTYPE_FP32", "TovaCache", "TovaError", "lib", "strerror",
+           "to_device", "tova_cache_bytes", "tova_config"]

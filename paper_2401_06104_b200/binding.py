@@ -1,0 +1,177 @@
+"""Thin ctypes binding of the C ABI in include/tova.h.
+
+Argument marshalling only: every step of the decode path runs in the CUDA
+library.  torch is used for device memory and streams.  Loading fails loudly
+if the library has not been built; nothing here computes on the CPU.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+TOVA_DTYPE_FP32 = 0
+TOVA_DTYPE_BF16 = 1
+
+
+class TovaError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: status {code} ({strerror(code)})")
+        self.code = code
+
+
+class tova_config(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
+                ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("capacity", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("sm_scale", ctypes.c_float), ("evict", ctypes.c_int32)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded CUDA library (built on first use if nvcc is present)."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB_PATH
+        if not os.path.exists(path):
+            path = _build.build()
+        L = ctypes.CDLL(path)
+        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+        L.tova_cache_bytes.restype = ctypes.c_size_t
+        L.tova_cache_bytes.argtypes = [ctypes.POINTER(tova_config)]
+        L.tova_cache_init.restype = ctypes.c_int
+        L.tova_cache_init.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(tova_config), vp,
+                                      ctypes.c_size_t, vp]
+        L.tova_decode_step.restype = ctypes.c_int
+        L.tova_decode_step.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp]
+        L.tova_prefill.restype = ctypes.c_int
+        L.tova_prefill.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp]
+        L.tova_decode_step_host.restype = ctypes.c_int
+        L.tova_decode_step_host.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp]
+        L.tova_cache_read.restype = ctypes.c_int
+        L.tova_cache_read.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+        L.tova_cache_set_chunk_rows.restype = ctypes.c_int
+        L.tova_cache_set_chunk_rows.argtypes = [vp, i32]
+        L.tova_cache_len.restype = i32
+        L.tova_cache_len.argtypes = [vp]
+        L.tova_cache_launches.restype = i64
+        L.tova_cache_launches.argtypes = [vp]
+        L.tova_cache_destroy.restype = ctypes.c_int
+        L.tova_cache_destroy.argtypes = [vp]
+        L.tova_strerror.restype = ctypes.c_char_p
+        L.tova_strerror.argtypes = [ctypes.c_int]
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().tova_strerror(int(code)).decode()
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        raise TovaError(rc, what)
+
+
+def _p(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream: Optional[torch.cuda.Stream]):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def tova_cache_bytes(cfg: tova_config) -> int:
+    return int(lib().tova_cache_bytes(ctypes.byref(cfg)))
+
+
+class TovaCache:
+    """State of one layer for `batch` sequences; the names follow the C ABI."""
+
+    def __init__(self, batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int, capacity: int,
+                 dtype: int = TOVA_DTYPE_BF16, sm_scale: float = 0.0, evict: bool = True,
+                 device: str = "cuda:0", stream: Optional[torch.cuda.Stream] = None):
+        self.cfg = tova_config(batch, n_q_heads, n_kv_heads, head_dim, capacity, dtype,
+                               float(sm_scale), 1 if evict else 0)
+        nbytes = tova_cache_bytes(self.cfg)
+        if nbytes == 0:
+            raise TovaError(-2, "tova_cache_bytes rejected the configuration")
+        self.device = torch.device(device)
+        self.tdtype = torch.bfloat16 if dtype == TOVA_DTYPE_BF16 else torch.float32
+        self.nbytes = nbytes
+        with torch.cuda.device(self.device):
+            self.mem = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+            off = (-self.mem.data_ptr()) % 256
+            self._base = self.mem.data_ptr() + off
+            h = ctypes.c_void_p()
+            _check(lib().tova_cache_init(ctypes.byref(h), ctypes.byref(self.cfg),
+                                         ctypes.c_void_p(self._base), nbytes, _stream(stream)),
+                   "tova_cache_init")
+        self._h = h
+
+    # -- C ABI calls ---------------------------------------------------------
+    def tova_decode_step(self, q, k, v, pos: int, out, evicted_pos=None, stream=None) -> None:
+        _check(lib().tova_decode_step(self._h, _p(q), _p(k), _p(v), int(pos), _p(out),
+                                      _p(evicted_pos), _stream(stream)), "tova_decode_step")
+
+    def tova_prefill(self, q, k, v, n_tokens: int, first_pos: int, out=None, evicted_pos=None,
+                     stream=None) -> None:
+        _check(lib().tova_prefill(self._h, _p(q), _p(k), _p(v), int(n_tokens), int(first_pos),
+                                  _p(out), _p(evicted_pos), _stream(stream)), "tova_prefill")
+
+    def tova_decode_step_host(self, q, k, v, pos: int, out, evicted_pos=None, stream=None) -> None:
+        """q, k, v, out, evicted_pos are HOST tensors (pinned for async copies)."""
+        _check(lib().tova_decode_step_host(self._h, _p(q), _p(k), _p(v), int(pos), _p(out),
+                                           _p(evicted_pos), _stream(stream)), "tova_decode_step_host")
+
+    def tova_cache_read(self, want_kv: bool = False, stream=None):
+        """Returns dict(len [B], positions [B,cap], status int, K, V or None) on the host."""
+        c = self.cfg
+        ln = torch.empty(c.batch, dtype=torch.int32, device=self.device)
+        ps = torch.empty(c.batch, c.capacity, dtype=torch.int32, device=self.device)
+        stt = torch.empty(1, dtype=torch.int32, device=self.device)
+        K = V = None
+        if want_kv:
+            K = torch.empty(c.batch, c.n_kv_heads, c.capacity, c.head_dim, dtype=self.tdtype,
+                            device=self.device)
+            V = torch.empty_like(K)
+        _check(lib().tova_cache_read(self._h, _p(ln), _p(ps), _p(K), _p(V), _p(stt), _stream(stream)),
+               "tova_cache_read")
+        torch.cuda.synchronize(self.device)
+        return {"len": ln.cpu(), "positions": ps.cpu(), "status": int(stt.item()),
+                "K": None if K is None else K.float().cpu(), "V": None if V is None else V.float().cpu()}
+
+    def tova_cache_set_chunk_rows(self, rows: int) -> None:
+        _check(lib().tova_cache_set_chunk_rows(self._h, int(rows)), "tova_cache_set_chunk_rows")
+
+    def tova_cache_len(self) -> int:
+        return int(lib().tova_cache_len(self._h))
+
+    def tova_cache_launches(self) -> int:
+        return int(lib().tova_cache_launches(self._h))
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h:
+            lib().tova_cache_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def to_device(x, dtype: int, device="cuda:0") -> torch.Tensor:
+    """Upload a float32 numpy array (bf16-representable for bf16) in the cache dtype."""
+    t = torch.from_numpy(x)
+    if dtype == TOVA_DTYPE_BF16:
+        t = t.to(torch.bfloat16)
+    return t.to(device)

@@ -1,0 +1,393 @@
+// Host side of the C ABI declared in include/tova.h: argument checks, the
+// layout of the caller-provided device block, launch configuration.  Every
+// step of the decode path runs in the kernels of tova_kernels.cuh; there is no
+// CPU fallback.
+#include "../../include/tova.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "tova_kernels.cuh"
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct Layout {
+  size_t K, V, pos, len, logits, part_ml, part_acc, blockmin, counter, status, cur_pos;
+  size_t st_q, st_k, st_v, st_out, st_ev;  // staging for host-buffer calls
+  size_t total;
+  int ld, pc, nx_max;
+};
+
+bool config_ok(const tova_config* c, int* why) {
+  if (!c) { *why = TOVA_ERR_NULL; return false; }
+  if (c->batch < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->capacity < 1 ||
+      c->n_q_heads % c->n_kv_heads != 0 || c->batch > 65535 || c->n_kv_heads > 65535 ||
+      c->n_q_heads > 4096 || c->capacity > (1 << 24)) {
+    *why = TOVA_ERR_BAD_SHAPE;
+    return false;
+  }
+  if ((c->head_dim != 64 && c->head_dim != 128) ||
+      (c->dtype != TOVA_DTYPE_FP32 && c->dtype != TOVA_DTYPE_BF16)) {
+    *why = TOVA_ERR_UNSUPPORTED;
+    return false;
+  }
+  if (!(c->sm_scale >= 0.f) || !std::isfinite(c->sm_scale)) { *why = TOVA_ERR_BAD_SHAPE; return false; }
+  return true;
+}
+
+Layout make_layout(const tova_config& c) {
+  Layout L{};
+  const size_t B = c.batch, H = c.n_q_heads, Hkv = c.n_kv_heads, D = c.head_dim, cap = c.capacity;
+  const size_t E = c.dtype == TOVA_DTYPE_BF16 ? 2 : 4;
+  L.ld = (int)((cap + 1 + 3) / 4 * 4);
+  // scratch is sized for the smallest chunk (one warp = 32 rows per split CTA)
+  L.pc = (int)((cap + tova::ROWS_PER_WARP - 1) / tova::ROWS_PER_WARP) + 1;
+  L.nx_max = (int)((cap + 1 + tova::COMBINE_ROWS - 1) / tova::COMBINE_ROWS);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L.K = take(B * Hkv * cap * D * E);
+  L.V = take(B * Hkv * cap * D * E);
+  L.pos = take(B * cap * 4);
+  L.len = take(B * 4);
+  L.logits = take(B * H * L.ld * 4);
+  L.part_ml = take(B * H * L.pc * 8);
+  L.part_acc = take(B * H * (size_t)(L.pc - 1) * D * 4);
+  L.blockmin = take(B * L.nx_max * 8);
+  L.counter = take(B * 4);
+  L.status = take(4);
+  L.cur_pos = take(4);
+  L.st_q = take(B * H * D * E);
+  L.st_k = take(B * Hkv * D * E);
+  L.st_v = take(B * Hkv * D * E);
+  L.st_out = take(B * H * D * 4);
+  L.st_ev = take(B * 4);
+  L.total = off;
+  return L;
+}
+
+}  // namespace
+
+struct tova_cache {
+  tova_config cfg;
+  Layout lay;
+  unsigned char* base;
+  int32_t len;          // rows per sequence (host mirror; sequences move in lock step)
+  int64_t launches;
+  int chunk_warps;      // warps (x32 rows) per split CTA
+  int sm_count;
+  int device;
+  float scale2;
+  size_t elem, row_bytes;
+};
+
+namespace {
+
+using tova::StepParams;
+
+template <typename T, int D, int NW, int GB>
+cudaError_t launch_split(int dev, const StepParams& p, dim3 grid, cudaStream_t st) {
+  const size_t rb = (size_t)D * sizeof(T);
+  const size_t smem = 2 * (size_t)NW * tova::ROWS_PER_WARP * rb +
+                      sizeof(float) * ((size_t)NW * GB * 32 + (size_t)NW * GB * 2 + (size_t)NW * GB * D);
+  auto kern = tova::tova_split_kernel<T, D, NW, GB>;
+  static bool attr_set[64] = {};  // per instantiation and device: the attribute is per function
+  if (!attr_set[dev & 63]) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set[dev & 63] = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(NW * 32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
+template <typename T, int D, int GB>
+cudaError_t launch_split_nw(int dev, int nw, const StepParams& p, dim3 grid, cudaStream_t st) {
+  switch (nw) {
+    case 1: return launch_split<T, D, 1, GB>(dev, p, grid, st);
+    case 2: return launch_split<T, D, 2, GB>(dev, p, grid, st);
+    case 4: return launch_split<T, D, 4, GB>(dev, p, grid, st);
+    default: return launch_split<T, D, 8, GB>(dev, p, grid, st);
+  }
+}
+
+template <typename T, int D>
+cudaError_t launch_split_g(int dev, int G, int nw, const StepParams& p, dim3 grid, cudaStream_t st) {
+  // heads of a query group handled per pass over the shared-memory tile
+  constexpr bool wide = (D * sizeof(T) == 512);  // fp32, D = 128: 32 partial sums per head
+  if (G == 1 || wide) return launch_split_nw<T, D, 1>(dev, nw, p, grid, st);
+  if (G == 2) return launch_split_nw<T, D, 2>(dev, nw, p, grid, st);
+  return launch_split_nw<T, D, 4>(dev, nw, p, grid, st);
+}
+
+template <typename T, int D>
+cudaError_t launch_combine(const StepParams& p, cudaStream_t st) {
+  const size_t smem = sizeof(float) * (2 * (size_t)p.H + (size_t)p.pc);
+  auto kern = tova::tova_combine_kernel<T, D>;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(p.nx, p.B);
+  cfg.blockDim = dim3(tova::COMBINE_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
+template <typename T, int D>
+cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st) {
+  dim3 grid(p.n_chunks > 0 ? p.n_chunks : 1, p.Hkv, p.B);
+  cudaError_t e = launch_split_g<T, D>(c->device, p.G, c->chunk_warps, p, grid, st);
+  if (e != cudaSuccess) return e;
+  e = launch_combine<T, D>(p, st);
+  if (e != cudaSuccess) return e;
+  c->launches += 2;
+  return cudaSuccess;
+}
+
+// Rows per split CTA: the largest of 256/128/64/32 that still gives every SM
+// about four CTAs when the state is full.
+int pick_chunk_warps(const tova_config& cfg, int sm_count) {
+  const long long pairs = (long long)cfg.batch * cfg.n_kv_heads;
+  const long long want = 4LL * sm_count;
+  for (int nw = 8; nw >= 2; nw >>= 1) {
+    const long long chunks = (cfg.capacity + 32LL * nw - 1) / (32LL * nw);
+    if (pairs * chunks >= want) return nw;
+  }
+  return 1;
+}
+
+int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_t pos, float* out,
+              int32_t* evicted_pos, cudaStream_t st) {
+  const tova_config& cfg = c->cfg;
+  const int n = c->len;
+  if (n >= cfg.capacity && !cfg.evict) return TOVA_ERR_FULL;
+  StepParams p{};
+  unsigned char* base = c->base;
+  p.K = base + c->lay.K;
+  p.V = base + c->lay.V;
+  p.pos = reinterpret_cast<int32_t*>(base + c->lay.pos);
+  p.len = reinterpret_cast<int32_t*>(base + c->lay.len);
+  p.logits = reinterpret_cast<float*>(base + c->lay.logits);
+  p.part_ml = reinterpret_cast<float2*>(base + c->lay.part_ml);
+  p.part_acc = reinterpret_cast<float*>(base + c->lay.part_acc);
+  p.blockmin = reinterpret_cast<float2*>(base + c->lay.blockmin);
+  p.counter = reinterpret_cast<unsigned*>(base + c->lay.counter);
+  p.status = reinterpret_cast<int32_t*>(base + c->lay.status);
+  p.cur_pos = reinterpret_cast<int32_t*>(base + c->lay.cur_pos);
+  p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.evicted = evicted_pos; p.pos_t = pos;
+  p.B = cfg.batch; p.H = cfg.n_q_heads; p.Hkv = cfg.n_kv_heads; p.G = cfg.n_q_heads / cfg.n_kv_heads;
+  p.cap = cfg.capacity; p.ld = c->lay.ld; p.pc = c->lay.pc;
+  p.n = n;
+  p.chunk_rows = c->chunk_warps * tova::ROWS_PER_WARP;
+  p.n_chunks = (n + p.chunk_rows - 1) / p.chunk_rows;
+  p.do_evict = (n == cfg.capacity) ? 1 : 0;
+  p.nx = p.do_evict ? (n + 1 + tova::COMBINE_ROWS - 1) / tova::COMBINE_ROWS : 1;
+  if (!p.do_evict) {
+    // no scoring: spread the output merge over a few CTAs per sequence
+    int nx = (c->sm_count + cfg.batch - 1) / cfg.batch;
+    if (nx > cfg.n_q_heads) nx = cfg.n_q_heads;
+    if (nx > c->lay.nx_max) nx = c->lay.nx_max;
+    p.nx = nx < 1 ? 1 : nx;
+  }
+  p.scale2 = c->scale2;
+  cudaError_t e;
+  if (cfg.dtype == TOVA_DTYPE_BF16) {
+    e = cfg.head_dim == 128 ? launch_step<__nv_bfloat16, 128>(c, p, st) : launch_step<__nv_bfloat16, 64>(c, p, st);
+  } else {
+    e = cfg.head_dim == 128 ? launch_step<float, 128>(c, p, st) : launch_step<float, 64>(c, p, st);
+  }
+  if (e != cudaSuccess) return TOVA_ERR_CUDA;
+  if (c->len < cfg.capacity) c->len += 1;
+  return TOVA_OK;
+}
+
+int check_step_args(const tova_cache* c, const void* q, const void* k, const void* v, const void* out) {
+  if (!c || !q || !k || !v || !out) return TOVA_ERR_NULL;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return TOVA_ERR_ALIGN;
+  return TOVA_OK;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------
+// C ABI
+// ---------------------------------------------------------------------------
+extern "C" {
+
+size_t tova_cache_bytes(const tova_config* cfg) {
+  int why;
+  if (!config_ok(cfg, &why)) return 0;
+  return make_layout(*cfg).total;
+}
+
+int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, size_t dev_bytes,
+                    void* cuda_stream) {
+  if (!out) return TOVA_ERR_NULL;
+  *out = nullptr;
+  int why;
+  if (!config_ok(cfg, &why)) return why;
+  if (!dev_mem) return TOVA_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(dev_mem) % ALIGN != 0) return TOVA_ERR_ALIGN;
+  const Layout lay = make_layout(*cfg);
+  if (dev_bytes < lay.total) return TOVA_ERR_WORKSPACE;
+
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TOVA_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return TOVA_ERR_CUDA;
+
+  tova_cache* c = new (std::nothrow) tova_cache();
+  if (!c) return TOVA_ERR_CUDA;
+  c->cfg = *cfg;
+  if (c->cfg.sm_scale == 0.f) c->cfg.sm_scale = 1.f / std::sqrt((float)cfg->head_dim);
+  c->lay = lay;
+  c->base = static_cast<unsigned char*>(dev_mem);
+  c->len = 0;
+  c->launches = 0;
+  c->sm_count = sms;
+  c->device = dev;
+  c->chunk_warps = pick_chunk_warps(*cfg, sms);
+  c->scale2 = c->cfg.sm_scale * 1.4426950408889634f;
+  c->elem = cfg->dtype == TOVA_DTYPE_BF16 ? 2 : 4;
+  c->row_bytes = c->elem * cfg->head_dim;
+
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t n = (size_t)cfg->batch * cfg->capacity;
+  const int threads = 256;
+  const unsigned blocks = (unsigned)((n + threads - 1) / threads);
+  tova::tova_init_kernel<<<blocks, threads, 0, st>>>(
+      reinterpret_cast<int32_t*>(c->base + lay.pos), reinterpret_cast<int32_t*>(c->base + lay.len),
+      reinterpret_cast<unsigned*>(c->base + lay.counter), reinterpret_cast<int32_t*>(c->base + lay.status),
+      reinterpret_cast<int32_t*>(c->base + lay.cur_pos), cfg->batch, cfg->capacity);
+  if (cudaGetLastError() != cudaSuccess) { delete c; return TOVA_ERR_CUDA; }
+  c->launches += 1;
+  *out = c;
+  return TOVA_OK;
+}
+
+int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows) {
+  if (!c) return TOVA_ERR_NULL;
+  if (rows == 0) { c->chunk_warps = pick_chunk_warps(c->cfg, c->sm_count); return TOVA_OK; }
+  if (rows != 32 && rows != 64 && rows != 128 && rows != 256) return TOVA_ERR_BAD_SHAPE;
+  c->chunk_warps = rows / 32;
+  return TOVA_OK;
+}
+
+int tova_decode_step(tova_cache* c, const void* q, const void* k, const void* v, int32_t pos, float* out,
+                     int32_t* evicted_pos, void* cuda_stream) {
+  int rc = check_step_args(c, q, k, v, out);
+  if (rc != TOVA_OK) return rc;
+  return step_impl(c, q, k, v, pos, out, evicted_pos, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int32_t n_tokens,
+                 int32_t first_pos, float* out, int32_t* evicted_pos, void* cuda_stream) {
+  if (!c) return TOVA_ERR_NULL;
+  if (n_tokens < 0) return TOVA_ERR_BAD_SHAPE;
+  if (n_tokens == 0) return TOVA_OK;
+  float* scratch_out = reinterpret_cast<float*>(c->base + c->lay.st_out);
+  int rc = check_step_args(c, q, k, v, out ? (const void*)out : (const void*)scratch_out);
+  if (rc != TOVA_OK) return rc;
+  if (!c->cfg.evict && (int64_t)c->len + n_tokens > c->cfg.capacity) return TOVA_ERR_FULL;
+  const size_t B = c->cfg.batch, H = c->cfg.n_q_heads, Hkv = c->cfg.n_kv_heads, D = c->cfg.head_dim;
+  const size_t q_stride = B * H * D * c->elem, kv_stride = B * Hkv * D * c->elem;
+  for (int32_t t = 0; t < n_tokens; ++t) {
+    rc = step_impl(c, static_cast<const unsigned char*>(q) + t * q_stride,
+                   static_cast<const unsigned char*>(k) + t * kv_stride,
+                   static_cast<const unsigned char*>(v) + t * kv_stride,
+                   first_pos < 0 ? first_pos : first_pos + t,
+                   out ? out + (size_t)t * B * H * D : scratch_out,
+                   evicted_pos ? evicted_pos + (size_t)t * B : nullptr, static_cast<cudaStream_t>(cuda_stream));
+    if (rc != TOVA_OK) return rc;
+  }
+  return TOVA_OK;
+}
+
+int tova_decode_step_host(tova_cache* c, const void* q_host, const void* k_host, const void* v_host,
+                          int32_t pos, float* out_host, int32_t* evicted_pos_host, void* cuda_stream) {
+  if (!c || !q_host || !k_host || !v_host || !out_host) return TOVA_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t B = c->cfg.batch, H = c->cfg.n_q_heads, Hkv = c->cfg.n_kv_heads, D = c->cfg.head_dim;
+  const size_t qb = B * H * D * c->elem, kb = B * Hkv * D * c->elem, ob = B * H * D * sizeof(float);
+  unsigned char* base = c->base;
+  if (cudaMemcpyAsync(base + c->lay.st_q, q_host, qb, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(base + c->lay.st_k, k_host, kb, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(base + c->lay.st_v, v_host, kb, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return TOVA_ERR_CUDA;
+  int rc = step_impl(c, base + c->lay.st_q, base + c->lay.st_k, base + c->lay.st_v, pos,
+                     reinterpret_cast<float*>(base + c->lay.st_out),
+                     reinterpret_cast<int32_t*>(base + c->lay.st_ev), st);
+  if (rc != TOVA_OK) return rc;
+  if (cudaMemcpyAsync(out_host, base + c->lay.st_out, ob, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return TOVA_ERR_CUDA;
+  if (evicted_pos_host &&
+      cudaMemcpyAsync(evicted_pos_host, base + c->lay.st_ev, B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return TOVA_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TOVA_ERR_CUDA;
+  return TOVA_OK;
+}
+
+int tova_cache_read(const tova_cache* c, int32_t* len, int32_t* positions, void* k_out, void* v_out,
+                    int32_t* status, void* cuda_stream) {
+  if (!c) return TOVA_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t B = c->cfg.batch, Hkv = c->cfg.n_kv_heads, cap = c->cfg.capacity;
+  const size_t kvb = B * Hkv * cap * c->row_bytes;
+  const unsigned char* base = c->base;
+  bool ok = true;
+  if (len) ok &= cudaMemcpyAsync(len, base + c->lay.len, B * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (positions)
+    ok &= cudaMemcpyAsync(positions, base + c->lay.pos, B * cap * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (k_out) ok &= cudaMemcpyAsync(k_out, base + c->lay.K, kvb, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (v_out) ok &= cudaMemcpyAsync(v_out, base + c->lay.V, kvb, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (status) ok &= cudaMemcpyAsync(status, base + c->lay.status, 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  return ok ? TOVA_OK : TOVA_ERR_CUDA;
+}
+
+int32_t tova_cache_len(const tova_cache* c) { return c ? c->len : -1; }
+int64_t tova_cache_launches(const tova_cache* c) { return c ? c->launches : -1; }
+
+int tova_cache_destroy(tova_cache* c) {
+  if (!c) return TOVA_ERR_NULL;
+  delete c;
+  return TOVA_OK;
+}
+
+const char* tova_strerror(int status) {
+  switch (status) {
+    case TOVA_OK: return "ok";
+    case TOVA_ERR_NULL: return "a required pointer is NULL";
+    case TOVA_ERR_BAD_SHAPE: return "shape or size out of range";
+    case TOVA_ERR_UNSUPPORTED: return "unsupported head_dim or dtype";
+    case TOVA_ERR_ALIGN: return "pointer not aligned as required";
+    case TOVA_ERR_WORKSPACE: return "device block smaller than tova_cache_bytes()";
+    case TOVA_ERR_FULL: return "state is full and eviction is off";
+    case TOVA_ERR_CUDA: return "CUDA runtime call or kernel launch failed";
+    case TOVA_ERR_DEVICE: return "a device-side check failed";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

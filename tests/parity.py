@@ -1,0 +1,151 @@
+"""Lock-step comparison of the CUDA library with the CPU checker.
+
+Both sides consume the same seeded tokens.  The GPU runs blocks of tokens
+through the C ABI (tova_prefill or tova_decode_step); the checker replays every
+token.  Rule for the victim: the checker is told which candidate the GPU
+dropped and reports how far that candidate's head-averaged weight lies above
+the minimum; a gap below 1e-6 is accepted (either choice is right when the two
+lowest averages are that close) and the checker follows the GPU's choice,
+otherwise the test fails at that token.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+import paper_2401_06104_b200 as tova
+from paper_2401_06104_b200 import workloads as W
+from oracle.tova_oracle import OracleCache
+
+GAP_TOL = 1e-6
+
+
+def out_tol(w: W.Workload) -> float:
+    """Max-abs tolerance on attention outputs: 2e-3 for bf16 inputs with fp32
+    accumulation, 1e-5 for fp32 inputs."""
+    return 2e-3 if w.dtype == W.DTYPE_BF16 else 1e-5
+
+
+@dataclass
+class ParityReport:
+    steps: int = 0
+    evictions: int = 0
+    resyncs: int = 0            # checker's own arg-min differed (gap < 1e-6)
+    self_evictions: int = 0
+    max_err: float = 0.0
+    max_gap: float = 0.0
+    evicted_log: List[np.ndarray] = field(default_factory=list)
+
+
+def make_cache(w: W.Workload, sm_scale: float = 0.0, evict: bool = True, chunk_rows: int = 0):
+    c = tova.TovaCache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, dtype=w.dtype,
+                       sm_scale=sm_scale, evict=evict)
+    if chunk_rows:
+        c.tova_cache_set_chunk_rows(chunk_rows)
+    return c
+
+
+def gpu_block(cache, w: W.Workload, q, k, v, first_pos: int, use_prefill: bool = True):
+    """Run a block of tokens on the GPU; returns (out [T,B,H,D], evicted [T,B]) on the host."""
+    T = q.shape[0]
+    dq, dk, dv = (tova.to_device(a, w.dtype) for a in (q, k, v))
+    out = torch.empty(T, w.batch, w.n_q_heads, w.head_dim, dtype=torch.float32, device="cuda:0")
+    ev = torch.full((T, w.batch), -12345, dtype=torch.int32, device="cuda:0")
+    if use_prefill:
+        cache.tova_prefill(dq, dk, dv, T, first_pos, out, ev)
+    else:
+        for t in range(T):
+            cache.tova_decode_step(dq[t], dk[t], dv[t], first_pos + t, out[t], ev[t])
+    torch.cuda.synchronize()
+    return out.cpu().numpy(), ev.cpu().numpy()
+
+
+def run_lockstep(w: W.Workload, n_tokens: int, *, seqs: Optional[Sequence[int]] = None,
+                 block: int = 64, use_prefill: bool = True, chunk_rows: int = 0,
+                 sm_scale: float = 0.0, layer: int = 0, cache=None, oracle=None,
+                 first_pos: int = 0, check_state_every: int = 4, direct_fill: bool = False) -> ParityReport:
+    """Feed n_tokens tokens to both sides and compare at every token.
+
+    direct_fill: while the state is filling nothing is dropped (Section 3.3), so
+    the checker's state after the first `capacity` tokens is those tokens in
+    order; it is then written from the generated tokens instead of replayed, and
+    only the slot table is compared for that phase (the checker's cost per
+    token grows with the state; this keeps capacity-4096 cases affordable)."""
+    seqs = list(range(w.batch)) if seqs is None else list(seqs)
+    own = cache is None
+    cache = cache or make_cache(w, sm_scale=sm_scale, chunk_rows=chunk_rows)
+    orc = oracle or OracleCache(len(seqs), w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity,
+                                sm_scale=sm_scale, precision="f32")
+    tol = out_tol(w)
+    rep = ParityReport()
+    done = 0
+    blocks = 0
+    while done < n_tokens:
+        T = min(block, n_tokens - done)
+        p0 = first_pos + done
+        q, k, v = W.tokens(w, p0, T, layer)
+        g_out, g_ev = gpu_block(cache, w, q, k, v, p0, use_prefill)
+        for t in range(T):
+            pos_t = p0 + t
+            if direct_fill and orc.len[0] < w.capacity:
+                n = int(orc.len[0])
+                assert np.all(g_ev[t] == -1)
+                orc.K[:, :, n] = k[t][seqs]
+                orc.V[:, :, n] = v[t][seqs]
+                orc.pos[:, n] = pos_t
+                orc.len[:] = n + 1
+                continue
+            forced = np.full(len(seqs), -1, np.int32)
+            full = orc.len[0] == w.capacity
+            if full:
+                for i, b in enumerate(seqs):
+                    e = int(g_ev[t, b])
+                    if e == pos_t:
+                        forced[i] = w.capacity
+                    else:
+                        hit = np.nonzero(orc.pos[i] == e)[0]
+                        assert hit.size == 1, f"token {pos_t} seq {b}: GPU dropped position {e}, not in the checker's state"
+                        forced[i] = int(hit[0])
+            o_out, o_ev, victim, argmin, gap, _ = orc.step(q[t][seqs], k[t][seqs], v[t][seqs], pos_t, forced=forced)
+            assert np.all(gap < GAP_TOL), f"token {pos_t}: GPU victim lies {gap.max():.3e} above the minimum"
+            assert np.array_equal(o_ev, g_ev[t, seqs]), f"token {pos_t}: evicted {g_ev[t, seqs]} vs {o_ev}"
+            err = float(np.abs(g_out[t][seqs] - o_out).max())
+            assert err <= tol, f"token {pos_t}: output error {err:.3e} > {tol}"
+            rep.max_err = max(rep.max_err, err)
+            rep.max_gap = max(rep.max_gap, float(gap.max()))
+            if full:
+                rep.evictions += len(seqs)
+                rep.resyncs += int(np.sum(victim != argmin))
+                rep.self_evictions += int(np.sum(victim == w.capacity))
+        rep.evicted_log.append(g_ev)
+        done += T
+        rep.steps = done
+        blocks += 1
+        if blocks % check_state_every == 0 or done == n_tokens:
+            st = cache.tova_cache_read()
+            assert st["status"] == 0, f"device status {st['status']}"
+            assert np.array_equal(st["len"].numpy()[seqs], orc.len), "state sizes differ"
+            assert np.array_equal(st["positions"].numpy()[seqs], orc.pos), f"slot table differs after {done} tokens"
+    rep.cache = cache
+    rep.oracle = orc
+    return rep
+
+
+def replay_slot_table(evicted: np.ndarray, capacity: int, first_pos: int = 0) -> np.ndarray:
+    """Integer replay of a position log [T,B]: which positions must be held
+    after T tokens, as sets per sequence (slot order is not recoverable from
+    the log alone)."""
+    T, B = evicted.shape
+    held = [set() for _ in range(B)]
+    for t in range(T):
+        for b in range(B):
+            held[b].add(first_pos + t)
+            e = int(evicted[t, b])
+            if e >= 0:
+                assert e in held[b], (t, b, e)
+                held[b].remove(e)
+            assert len(held[b]) <= capacity
+    return held

@@ -1,0 +1,171 @@
+"""GPU parity: the CUDA library, called through the C ABI, against the CPU
+checker on the same seeded inputs.  Retained positions are compared slot by
+slot (bit-exact), outputs within 2e-3 (bf16 inputs) / 1e-5 (fp32 inputs)."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2401_06104_b200 as tova
+from paper_2401_06104_b200 import workloads as W
+from oracle.tova_oracle import OracleCache
+from parity import gpu_block, make_cache, out_tol, replay_slot_table, run_lockstep
+from test_oracle_pins import parse_golden
+
+pytestmark = pytest.mark.gpu
+
+LLAMA = W.WORKLOADS["llama2_7b_layer"]
+MISTRAL = W.WORKLOADS["mistral_7b_gqa"]
+YI = W.WORKLOADS["yi_6b_long"]
+
+
+def test_hand_worked_example_on_gpu():
+    """The 3-row example (exact tie, self-eviction, slot order != position order)."""
+    toks, steps = parse_golden()
+    D = 64
+    c = tova.TovaCache(1, 2, 2, D, 3, dtype=tova.TOVA_DTYPE_FP32, sm_scale=1.0)
+    out = torch.empty(1, 2, D, device="cuda:0")
+    ev = torch.empty(1, dtype=torch.int32, device="cuda:0")
+    for (t, e, rows_after, o0, o1) in steps:
+        q = np.zeros((1, 2, D), np.float32); q[..., 0] = 1.0
+        k = np.zeros((1, 2, D), np.float32); v = np.zeros((1, 2, D), np.float32)
+        a0, v0, a1, v1 = toks[t]
+        k[0, 0, 0], k[0, 1, 0] = np.log(a0), np.log(a1)
+        v[0, 0, 0], v[0, 1, 0] = v0, v1
+        c.tova_decode_step(*(tova.to_device(a, 0) for a in (q, k, v)), t, out, ev)
+        st = c.tova_cache_read()
+        assert int(ev.item()) == e, t
+        assert st["positions"][0].tolist() == rows_after, t
+        o = out.cpu().numpy()
+        assert abs(o[0, 0, 0] - float(o0)) < 1e-4 and abs(o[0, 1, 0] - float(o1)) < 1e-4
+        assert np.all(o[0, :, 1:] == 0)
+        assert st["status"] == 0 and c.tova_cache_len() == min(t + 1, 3)
+
+
+@pytest.mark.parametrize("name", ["tiny", "tiny_unit"])
+def test_tiny_reference_config_full_stream(name):
+    """1 layer, batch 1, 4 MHA heads, D 64, fp32, capacity 64, 32 + 512 tokens."""
+    w = W.WORKLOADS[name]
+    rep = run_lockstep(w, w.prompt + w.decode, block=32)
+    assert rep.evictions == w.prompt + w.decode - w.capacity
+    print(f"{name}: resyncs {rep.resyncs}/{rep.evictions} self {rep.self_evictions} "
+          f"max_err {rep.max_err:.2e} max_gap {rep.max_gap:.2e}")
+
+
+@pytest.mark.parametrize("chunk_rows", [0, 32, 64, 128, 256])
+def test_llama_shape_reduced_every_chunk_size(chunk_rows):
+    """bf16 MHA, capacity 203: several tiles plus a ragged tail at every chunk size."""
+    w = LLAMA.scaled(batch=2, n_q_heads=6, n_kv_heads=6, capacity=203)
+    rep = run_lockstep(w, 460, chunk_rows=chunk_rows, block=50)
+    assert rep.evictions == 2 * (460 - 203)
+
+
+@pytest.mark.parametrize("H,Hkv,D,dtype,cap,B", [
+    (8, 2, 128, W.DTYPE_BF16, 200, 3),      # G = 4 (Mistral-like)
+    (16, 2, 128, W.DTYPE_BF16, 130, 2),     # G = 8 (Yi-like)
+    (6, 2, 128, W.DTYPE_BF16, 77, 2),       # G = 3: group not a multiple of the head block
+    (32, 2, 64, W.DTYPE_BF16, 65, 1),       # G = 16, D = 64
+    (4, 2, 64, W.DTYPE_BF16, 64, 2),        # G = 2, D = 64
+    (4, 4, 128, W.DTYPE_FP32, 97, 2),       # fp32, D = 128
+    (8, 2, 64, W.DTYPE_FP32, 40, 2),        # fp32 GQA, D = 64
+    (2, 1, 128, W.DTYPE_BF16, 1, 2),        # capacity 1: every step evicts
+    (4, 4, 128, W.DTYPE_BF16, 33, 1),       # one row past a tile
+])
+def test_head_layouts_and_dtypes(H, Hkv, D, dtype, cap, B):
+    w = MISTRAL.scaled(batch=B, n_q_heads=H, n_kv_heads=Hkv, head_dim=D, dtype=dtype, capacity=cap)
+    rep = run_lockstep(w, cap + 150, block=40)
+    assert rep.evictions == B * 150
+
+
+def test_yi_shape_reduced_with_periodic_heavy_keys():
+    w = YI.scaled(batch=2, capacity=256, heavy_period=64)
+    rep = run_lockstep(w, 256 + 300, block=64)
+    assert rep.evictions == 2 * 300
+
+
+def test_prefill_equals_decode_steps_bitwise():
+    w = LLAMA.scaled(batch=2, n_q_heads=8, n_kv_heads=8, capacity=100)
+    T = 260
+    q, k, v = W.tokens(w, 0, T)
+    a, b = make_cache(w), make_cache(w)
+    oa, ea = gpu_block(a, w, q, k, v, 0, use_prefill=True)
+    ob, eb = gpu_block(b, w, q, k, v, 0, use_prefill=False)
+    assert np.array_equal(oa, ob) and np.array_equal(ea, eb)
+    sa, sb = a.tova_cache_read(want_kv=True), b.tova_cache_read(want_kv=True)
+    for key in ("len", "positions", "K", "V"):
+        assert torch.equal(sa[key], sb[key]), key
+    assert a.tova_cache_launches() == b.tova_cache_launches() == 1 + 2 * T
+
+
+def test_cached_rows_are_the_inserted_tokens():
+    """tova_cache_read returns, per slot, exactly the k/v of the position it reports."""
+    w = MISTRAL.scaled(batch=2, n_q_heads=8, n_kv_heads=2, capacity=48)
+    T = 150
+    q, k, v = W.tokens(w, 0, T)
+    c = make_cache(w)
+    gpu_block(c, w, q, k, v, 0)
+    st = c.tova_cache_read(want_kv=True)
+    pos = st["positions"].numpy()
+    for b in range(w.batch):
+        assert len(set(pos[b].tolist())) == w.capacity
+        for s in range(w.capacity):
+            assert np.array_equal(st["K"][b, :, s].numpy(), k[pos[b, s], b])
+            assert np.array_equal(st["V"][b, :, s].numpy(), v[pos[b, s], b])
+
+
+def test_sequences_are_independent_on_gpu():
+    w = LLAMA.scaled(batch=3, n_q_heads=4, n_kv_heads=4, capacity=70)
+    T = 200
+    q, k, v = W.tokens(w, 0, T)
+    full = make_cache(w)
+    of, ef = gpu_block(full, w, q, k, v, 0)
+    for b in range(w.batch):
+        w1 = w.scaled(batch=1)
+        one = make_cache(w1)
+        o1, e1 = gpu_block(one, w1, q[:, b:b + 1], k[:, b:b + 1], v[:, b:b + 1], 0)
+        assert np.array_equal(o1[:, 0], of[:, b]) and np.array_equal(e1[:, 0], ef[:, b])
+
+
+def test_unbounded_arm_matches_checker_and_reports_full():
+    w = LLAMA.scaled(batch=2, n_q_heads=4, n_kv_heads=4, capacity=150)
+    cache = make_cache(w, evict=False)
+    rep = run_lockstep(w, 150, cache=cache, block=50)
+    assert rep.evictions == 0 and cache.tova_cache_len() == 150
+    q, k, v = W.tokens(w, 150, 1)
+    out = torch.empty(2, 4, 128, device="cuda:0")
+    with pytest.raises(tova.TovaError) as e:
+        cache.tova_decode_step(*(tova.to_device(a[0], w.dtype) for a in (q, k, v)), 150, out)
+    assert e.value.code == -6
+
+
+def test_host_buffer_entry_point_matches_device_path():
+    w = LLAMA.scaled(batch=2, n_q_heads=4, n_kv_heads=4, capacity=40)
+    T = 90
+    q, k, v = W.tokens(w, 0, T)
+    dev = make_cache(w)
+    o_dev, e_dev = gpu_block(dev, w, q, k, v, 0)
+    host = make_cache(w)
+    hq, hk, hv = (torch.from_numpy(a).to(torch.bfloat16).pin_memory() for a in (q, k, v))
+    out = torch.empty(w.batch, w.n_q_heads, w.head_dim, dtype=torch.float32).pin_memory()
+    ev = torch.empty(w.batch, dtype=torch.int32).pin_memory()
+    for t in range(T):
+        host.tova_decode_step_host(hq[t], hk[t], hv[t], t, out, ev)
+        assert np.array_equal(out.numpy(), o_dev[t]) and np.array_equal(ev.numpy(), e_dev[t])
+
+
+def test_step_argument_errors():
+    w = LLAMA.scaled(batch=1, n_q_heads=2, n_kv_heads=2, capacity=8)
+    c = make_cache(w)
+    q = torch.zeros(1, 2, 128, dtype=torch.bfloat16, device="cuda:0")
+    out = torch.zeros(1, 2, 128, device="cuda:0")
+    with pytest.raises(tova.TovaError) as e:
+        c.tova_decode_step(q, q, None, 0, out)
+    assert e.value.code == -1
+    mis = torch.zeros(2 * 128 + 8, dtype=torch.bfloat16, device="cuda:0")[4:4 + 256].view(1, 2, 128)
+    with pytest.raises(tova.TovaError) as e:
+        c.tova_decode_step(mis, q, q, 0, out)
+    assert e.value.code == -4
+    with pytest.raises(tova.TovaError):
+        c.tova_cache_set_chunk_rows(48)
+    assert c.tova_cache_len() == 0
