@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the TOVA decode path on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--capacity C]
+  python bench.py --impl reference ...        # the CPU checker, timed on the host cores
+
+A "step" is one decode step of one layer for the whole batch: split-K
+attention over the full bounded state, combine, TOVA eviction and in-place
+insert.  Steps rotate over enough independent layer caches that the working
+set exceeds the L2 cache, the way the layers of a model follow each other.
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "tova_decode_tokens_per_s_per_layer"
+UNIT = "tokens/s"
+RING = 128                      # distinct pre-generated tokens per workload
+WORKING_SET = 1 << 30           # rotate layer caches until this many bytes are touched per round
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16384)
+    ap.add_argument("--warmup", type=int, default=2048)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2_7b_layer")
+    ap.add_argument("--capacity", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--layers", type=int, default=0, help="independent layer caches to rotate over (0 = auto)")
+    ap.add_argument("--chunk-rows", type=int, default=0)
+    ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of CUDA graphs")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    return ap.parse_args()
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def pick_workload(args):
+    from paper_2401_06104_b200 import workloads as W
+    w = W.WORKLOADS[args.workload]
+    if args.capacity:
+        w = w.scaled(capacity=args.capacity)
+    if args.batch:
+        w = w.scaled(batch=args.batch)
+    return w
+
+
+# ----------------------------------------------------------------------------
+# clocks: sampled with NVML (read-only) while the timed region runs
+# ----------------------------------------------------------------------------
+class ClockSampler:
+    BAD = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown"}
+    NOTE = {0x4: "sw_power_cap"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            if vis:
+                index = int(vis.split(",")[index]) if vis.split(",")[index].isdigit() else index
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                for bit, name in {**self.BAD, **self.NOTE}.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------
+# the CPU checker as a timed baseline (never tuned for this)
+# ----------------------------------------------------------------------------
+def time_oracle(w, ring, seconds: float, max_seqs: int = 0):
+    """Steady-state decode steps of the CPU checker on a full state.  The state
+    is written directly from ring tokens (while filling nothing is dropped), then
+    steps are timed.  Returns (tokens/s, threads, description)."""
+    from oracle.tova_oracle import OracleCache, host_threads
+    threads = host_threads()
+    S = min(w.batch, max_seqs or max(threads, 1))
+    q, k, v = ring
+    orc = OracleCache(S, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, precision="f32", threads=threads)
+    R = q.shape[0]
+    for n in range(w.capacity):
+        orc.K[:, :, n] = k[n % R][:S]
+        orc.V[:, :, n] = v[n % R][:S]
+        orc.pos[:, n] = n
+    orc.len[:] = w.capacity
+    pos = w.capacity
+    t0 = time.perf_counter()
+    orc.step(q[0][:S], k[0][:S], v[0][:S], pos); pos += 1
+    one = max(time.perf_counter() - t0, 1e-6)
+    n_steps = int(min(max(seconds / one, 4), 4096))
+    t0 = time.perf_counter()
+    for i in range(n_steps):
+        r = (i + 1) % R
+        orc.step(q[r][:S], k[r][:S], v[r][:S], pos); pos += 1
+    dt = time.perf_counter() - t0
+    used = min(threads, S)
+    return S * n_steps / dt, used, f"{n_steps} steady-state steps of {S} of {w.batch} sequences on a full state (k={w.capacity})"
+
+
+def workload_config(w, extra):
+    cfg = {"workload": w.name, "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
+           "head_dim": w.head_dim, "capacity": w.capacity,
+           "storage": "bf16" if w.elem_bytes == 2 else "fp32"}
+    cfg.update(extra)
+    return cfg
+
+
+def run_reference(args):
+    """--impl reference: the CPU checker alone, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from paper_2401_06104_b200 import workloads as W
+    w = pick_workload(args)
+    ring = W.tokens(w, 0, RING)
+    # every "step" is a bounded sample; the whole run stays within minutes
+    budget = min(60.0, max(4.0, 0.004 * (args.steps + args.warmup)))
+    val, cores, sample = time_oracle(w, ring, budget)
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.batch / val,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": workload_config(w, {"sample": sample}),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ----------------------------------------------------------------------------
+# the CUDA path
+# ----------------------------------------------------------------------------
+def kernel_digest() -> str:
+    """Hash of the kernel sources: DRAM counters in profiles/ apply to one digest only."""
+    import hashlib
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_2401_06104_b200", "csrc")
+    for f in sorted(os.listdir(d)):
+        with open(os.path.join(d, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(w, layers_bytes_per_step):
+    """DRAM bytes per split-kernel launch from the committed ncu summary, or None
+    when there is none for this workload or the kernels changed since."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        with open(path) as fh:
+            rec = json.load(fh)
+        if rec.get("kernel_digest") != kernel_digest():
+            return None
+        e = rec["workloads"].get(f"{w.name}:k{w.capacity}:b{w.batch}")
+        return None if e is None else float(e["dram_bytes_per_launch"])
+    except Exception:
+        return None
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2401_06104_b200 as tova
+    from paper_2401_06104_b200 import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the decode path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    w = pick_workload(args)
+    B, H, Hkv, D, cap = w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity
+    step_bytes = w.step_bytes()
+    L = args.layers or max(1, -(-WORKING_SET // step_bytes))
+    ring = W.tokens(w, 0, RING)                                   # seeded, host
+    dq, dk, dv = (tova.to_device(a, w.dtype, dev) for a in ring)
+
+    caches = []
+    for l in range(L):
+        c = tova.TovaCache(B, H, Hkv, D, cap, dtype=w.dtype, device=dev)
+        if args.chunk_rows:
+            c.tova_cache_set_chunk_rows(args.chunk_rows)
+        caches.append(c)
+    outs = torch.empty(L, B, H, D, dtype=torch.float32, device=dev)
+    evs = torch.empty(L, B, dtype=torch.int32, device=dev)
+
+    # steady state: fill every layer past its capacity (positions from the device counter)
+    for l, c in enumerate(caches):
+        fed, r = 0, (17 * l) % RING
+        while fed < cap + 64:
+            T = min(RING - r, cap + 64 - fed)
+            c.tova_prefill(dq[r:], dk[r:], dv[r:], T, -1, None, None)
+            fed += T
+            r = (r + T) % RING
+    torch.cuda.synchronize()
+    for c in caches:
+        assert c.tova_cache_len() == cap
+
+    counter = [0]
+
+    def step(i):
+        l = i % L
+        r = (i // L + 29 * l) % RING
+        caches[l].tova_decode_step(dq[r], dk[r], dv[r], -1, outs[l], evs[l])
+
+    def run_direct(n):
+        for _ in range(n):
+            step(counter[0])
+            counter[0] += 1
+
+    run_direct(min(64, max(args.warmup, 3)))                      # sets function attributes before capture
+    torch.cuda.synchronize()
+
+    graph, G = None, 0
+    launch_mode = "stream"
+    if not args.no_graph and args.steps >= 2 * L:
+        G = min(args.steps, 512)
+        G = max(L, G // L * L)
+        try:
+            graph = torch.cuda.CUDAGraph()
+            base = counter[0]
+            with torch.cuda.graph(graph):
+                for j in range(G):
+                    step(base + j)
+            launch_mode = "cuda_graph"
+        except Exception as e:  # pragma: no cover
+            print(f"bench.py: graph capture failed ({e}); launching from the host", file=sys.stderr)
+            graph, G = None, 0
+            torch.cuda.synchronize()
+
+    def run(n):
+        if graph is not None:
+            for _ in range(n // G):
+                graph.replay()
+            n = n % G
+        run_direct(n)
+
+    launches_before = sum(c.tova_cache_launches() for c in caches)
+    run(max(args.warmup, 3))
+    sampler = ClockSampler(local)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    run(args.steps)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if world > 1:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    for c in caches:
+        assert c.tova_cache_read()["status"] == 0, "a kernel reported a failed check"
+
+    ms_per_step = ms / args.steps
+    value = world * B * args.steps / (ms * 1e-3)
+    gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+    peak, peak_kind = load_peaks()
+
+    # end to end: host buffers in, host buffers out, through tova_decode_step_host
+    e2e = None
+    if not args.no_e2e:
+        hq, hk, hv = (torch.from_numpy(a).to(dq.dtype).pin_memory() for a in ring)
+        hout = torch.empty(B, H, D, dtype=torch.float32).pin_memory()
+        hev = torch.empty(B, dtype=torch.int32).pin_memory()
+        n_e = min(args.steps, 2048)
+        for i in range(8):
+            caches[i % L].tova_decode_step_host(hq[i % RING], hk[i % RING], hv[i % RING], -1, hout, hev)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for i in range(n_e):
+            r = (i // L + 29 * (i % L)) % RING
+            caches[i % L].tova_decode_step_host(hq[r], hk[r], hv[r], -1, hout, hev)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([dt], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        e2e = {"value": world * B * n_e / dt, "unit": UNIT, "steps": n_e,
+               "h2d_bytes_per_step": int(hq[0].nbytes + hk[0].nbytes + hv[0].nbytes),
+               "d2h_bytes_per_step": int(hout.nbytes + hev.nbytes)}
+
+    if rank != 0:
+        return 0
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        val, cores, sample = time_oracle(w, ring, args.cpu_seconds)
+        cpu = {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(w, {
+            "layers_rotated": L, "working_set_bytes": L * step_bytes, "l2": "inputs larger than L2",
+            "launch": launch_mode, "graph_steps": G, "bytes_per_step": step_bytes,
+            "parallelism": "replicas only" if world > 1 else "single GPU"}),
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                     "traffic": recorded_traffic(w, step_bytes), "peak_kind": peak_kind,
+                     "frac_of_nominal_8TBs": gbs / 8000.0,
+                     "note": "algorithmic bytes (K/V read + one slot written) / whole-step time (split + combine kernels)"},
+        "cpu_baseline": cpu,
+        "e2e": e2e,
+        "gpu_launches": 2 * args.steps,
+        "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
