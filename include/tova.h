@@ -56,7 +56,8 @@ typedef enum {
   TOVA_ERR_WORKSPACE = -5,   /* dev_bytes < tova_cache_bytes()                    */
   TOVA_ERR_FULL = -6,        /* evict == 0 and the state already holds capacity   */
   TOVA_ERR_CUDA = -7,        /* a CUDA runtime call or launch failed              */
-  TOVA_ERR_DEVICE = -8       /* a kernel reported a failed internal check         */
+  TOVA_ERR_DEVICE = -8,      /* a kernel reported a failed internal check         */
+  TOVA_ERR_STATIC_LIMIT = -9 /* tova_decode_step_static: shape exceeds the built-in scratch */
 } tova_status;
 
 typedef struct {
@@ -136,6 +137,48 @@ int64_t tova_cache_launches(const tova_cache* c);
 int tova_cache_destroy(tova_cache* c);
 
 const char* tova_strerror(int status);
+
+/* One decode step WITHOUT any workspace from the caller and without a cache
+ * handle (the paper has no counterpart: this is a packaging variant of
+ * tova_decode_step, same kernels, same results).
+ *
+ * Who needs it: code that runs where device memory cannot be requested - a
+ * plugin or callback inside another framework's execution engine that owns
+ * the allocator, code between the begin and end of someone else's stream
+ * capture, a process whose memory budget was fixed at start-up.  Such callers
+ * usually do hold the K/V tensors themselves but have nowhere to put the
+ * scratch the two kernels exchange (logits, per-chunk soft-max partials,
+ * per-block minima, tickets).  For this call that scratch is an array
+ * compiled into the library: TOVA_STATIC_SCRATCH_BYTES (8 MiB) of device
+ * memory that every GPU context loading the library holds until it exits.
+ *
+ *   cfg                          shape, dtype, scale, policy (as for tova_cache_init)
+ *   K, V [B,Hkv,capacity,D]      the caller's state, updated in place
+ *   positions [B,capacity] int32 slot table, updated in place (caller sets
+ *                                unused slots to -1 before the first token)
+ *   n_live                       rows each sequence holds before this token,
+ *                                min(tokens fed so far, capacity): the caller
+ *                                tracks it
+ *   q, k, v, pos, out, evicted_pos   as for tova_decode_step (pos >= 0)
+ *
+ * Scratch need: about 4*B*H*(capacity+5) bytes of logits plus
+ * B*H*(D*4+8)*ceil(capacity/chunk) bytes of partials (chunk = 32..256 rows,
+ * chosen from the shape); the LLaMA-2-7B layer at batch 8, capacity 512 takes
+ * under 1 MiB.  A shape that needs more than the array holds is refused with
+ * TOVA_ERR_STATIC_LIMIT before anything is launched.
+ *
+ * The call allocates nothing, on the device or through any library.  Its first
+ * use on a device looks up the array's device address (cudaGetSymbolAddress)
+ * and the SM count; make that first call outside any stream capture.  All calls
+ * on a device share the one array, which keeps whatever the previous call left:
+ * the call clears its tickets and status itself (a memset on `cuda_stream`),
+ * but two calls whose kernels overlap on the GPU - different streams, or
+ * different host threads without ordering - race on it.  Issue them on one
+ * stream or order them with events. */
+#define TOVA_STATIC_SCRATCH_BYTES (8u << 20)
+int tova_decode_step_static(const tova_config* cfg, void* K, void* V, int32_t* positions,
+                            int32_t n_live, const void* q, const void* k, const void* v, int32_t pos,
+                            float* out, int32_t* evicted_pos, void* cuda_stream);
 
 #ifdef __cplusplus
 }

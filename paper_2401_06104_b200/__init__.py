@@ -5,7 +5,7 @@ sources (csrc/), the in-tree build, a ctypes binding with the same names, and
 the seeded synthetic workloads.
 """
 from .binding import (TOVA_DTYPE_BF16, TOVA_DTYPE_FP32, TovaCache, TovaError, lib, strerror,
-                      to_device, tova_cache_bytes, tova_config)
+                      to_device, tova_cache_bytes, tova_config, tova_decode_step_static)
 
 __all__ = ["TOVA_DTYPE_BF16", "TOVA_DTYPE_FP32", "TovaCache", "TovaError", "lib", "strerror",
-           "to_device", "tova_cache_bytes", "tova_config"]
+           "to_device", "tova_cache_bytes", "tova_config", "tova_decode_step_static"]

@@ -386,8 +386,127 @@ const char* tova_strerror(int status) {
     case TOVA_ERR_FULL: return "state is full and eviction is off";
     case TOVA_ERR_CUDA: return "CUDA runtime call or kernel launch failed";
     case TOVA_ERR_DEVICE: return "a device-side check failed";
+    case TOVA_ERR_STATIC_LIMIT:
+      return "this shape needs more scratch than the library's built-in 8 MiB array holds";
     default: return "unknown status";
   }
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// A decode step for callers that cannot allocate device memory.
+// ---------------------------------------------------------------------------
+// The scratch the two kernels exchange (logits, chunk partials, per-block
+// minima, tickets, status words) normally lives in the block the caller
+// allocates for tova_cache_init.  Here it lives in an array that is part of the
+// loaded module, so the call needs no workspace from anybody.  Every device
+// context that loads the library carries these bytes until it exits.
+namespace {
+
+constexpr size_t STATIC_SCRATCH_BYTES = (size_t)TOVA_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+struct StaticDevice {
+  bool ready;
+  unsigned char* scratch;  // device address of g_static_scratch on this device
+  int sm_count;
+};
+StaticDevice g_static_dev[64] = {};
+
+struct StaticLayout {
+  size_t logits, part_ml, part_acc, blockmin, control, total;
+  int ld, pc, nx_max;
+};
+
+StaticLayout make_static_layout(const tova_config& c, int chunk_rows) {
+  StaticLayout L{};
+  const size_t B = c.batch, H = c.n_q_heads, D = c.head_dim, cap = c.capacity;
+  L.ld = (int)((cap + 1 + 3) / 4 * 4);
+  L.pc = (int)((cap + chunk_rows - 1) / chunk_rows) + 1;
+  L.nx_max = (int)((cap + 1 + tova::COMBINE_ROWS - 1) / tova::COMBINE_ROWS);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L.control = take(B * 4 /*tickets*/ + B * 4 /*len*/ + 8 /*status, cur_pos*/);
+  L.logits = take(B * H * L.ld * 4);
+  L.part_ml = take(B * H * L.pc * 8);
+  L.part_acc = take(B * H * (size_t)(L.pc - 1) * D * 4);
+  L.blockmin = take(B * L.nx_max * 8);
+  L.total = off;
+  return L;
+}
+
+}  // namespace
+
+extern "C" int tova_decode_step_static(const tova_config* cfg, void* K, void* V, int32_t* positions,
+                                       int32_t n_live, const void* q, const void* k, const void* v,
+                                       int32_t pos, float* out, int32_t* evicted_pos, void* cuda_stream) {
+  int why;
+  if (!config_ok(cfg, &why)) return why;
+  if (!K || !V || !positions || !q || !k || !v || !out) return TOVA_ERR_NULL;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+    return TOVA_ERR_ALIGN;
+  if (n_live < 0 || n_live > cfg->capacity || pos < 0) return TOVA_ERR_BAD_SHAPE;
+  if (n_live == cfg->capacity && !cfg->evict) return TOVA_ERR_FULL;
+
+  // One-time set-up per device, with that device current: the array's name is
+  // only a host-side handle, kernels need the address the runtime reports.
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return TOVA_ERR_CUDA;
+  StaticDevice& sd = g_static_dev[dev];
+  if (!sd.ready) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return TOVA_ERR_CUDA;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return TOVA_ERR_CUDA;
+    sd.scratch = static_cast<unsigned char*>(ptr);
+    sd.sm_count = sms;
+    sd.ready = true;
+  }
+
+  const int chunk_warps = pick_chunk_warps(*cfg, sd.sm_count);
+  const int chunk_rows = chunk_warps * tova::ROWS_PER_WARP;
+  const StaticLayout lay = make_static_layout(*cfg, chunk_rows);
+  if (lay.total > STATIC_SCRATCH_BYTES) return TOVA_ERR_STATIC_LIMIT;
+
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* base = sd.scratch;
+  const size_t B = cfg->batch;
+  // tickets and status must start at zero; the array keeps the previous call's contents
+  if (cudaMemsetAsync(base + lay.control, 0, B * 8 + 8, st) != cudaSuccess) return TOVA_ERR_CUDA;
+
+  StepParams p{};
+  p.K = K;
+  p.V = V;
+  p.pos = positions;
+  p.counter = reinterpret_cast<unsigned*>(base + lay.control);
+  p.len = reinterpret_cast<int32_t*>(base + lay.control + B * 4);
+  p.status = reinterpret_cast<int32_t*>(base + lay.control + B * 8);
+  p.cur_pos = p.status + 1;
+  p.logits = reinterpret_cast<float*>(base + lay.logits);
+  p.part_ml = reinterpret_cast<float2*>(base + lay.part_ml);
+  p.part_acc = reinterpret_cast<float*>(base + lay.part_acc);
+  p.blockmin = reinterpret_cast<float2*>(base + lay.blockmin);
+  p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.evicted = evicted_pos; p.pos_t = pos;
+  p.B = cfg->batch; p.H = cfg->n_q_heads; p.Hkv = cfg->n_kv_heads; p.G = cfg->n_q_heads / cfg->n_kv_heads;
+  p.cap = cfg->capacity; p.ld = lay.ld; p.pc = lay.pc;
+  p.n = n_live;
+  p.chunk_rows = chunk_rows;
+  p.n_chunks = (n_live + chunk_rows - 1) / chunk_rows;
+  p.do_evict = (n_live == cfg->capacity) ? 1 : 0;
+  p.nx = p.do_evict ? (n_live + 1 + tova::COMBINE_ROWS - 1) / tova::COMBINE_ROWS : 1;
+  const float scale = cfg->sm_scale == 0.f ? 1.f / std::sqrt((float)cfg->head_dim) : cfg->sm_scale;
+  p.scale2 = scale * 1.4426950408889634f;
+
+  tova_cache shim{};  // launch_step only reads these three fields and counts launches
+  shim.device = dev;
+  shim.chunk_warps = chunk_warps;
+  cudaError_t e;
+  if (cfg->dtype == TOVA_DTYPE_BF16) {
+    e = cfg->head_dim == 128 ? launch_step<__nv_bfloat16, 128>(&shim, p, st)
+                             : launch_step<__nv_bfloat16, 64>(&shim, p, st);
+  } else {
+    e = cfg->head_dim == 128 ? launch_step<float, 128>(&shim, p, st) : launch_step<float, 64>(&shim, p, st);
+  }
+  return e == cudaSuccess ? TOVA_OK : TOVA_ERR_CUDA;
+}
