@@ -121,9 +121,9 @@ int tova_decode_step_host(tova_cache* c, const void* q_host, const void* k_host,
 int tova_cache_read(const tova_cache* c, int32_t* len, int32_t* positions, void* k_out,
                     void* v_out, int32_t* status, void* cuda_stream);
 
-/* Tuning: rows of the state one thread block of the streaming kernel covers
- * (32, 64, 128 or 256; 0 restores the automatic choice made at init).  Results
- * do not depend on it beyond floating-point summation order. */
+/* Tuning: rows of the state one warp of the streaming kernel covers (a multiple
+ * of 32 up to 8192; 0 restores the automatic choice made at init).  Results do
+ * not depend on it beyond floating-point summation order. */
 int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows);
 
 /* Rows each sequence holds now, min(tokens fed, capacity) = g(t) of Section

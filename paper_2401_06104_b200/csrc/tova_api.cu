@@ -42,14 +42,22 @@ bool config_ok(const tova_config* c, int* why) {
   return true;
 }
 
+// Upper bound of combine CTAs per sequence: enough to score 128 candidates each,
+// and enough to spread a small batch over the whole GPU.
+constexpr int NX_SPREAD = 512;
+int nx_limit(int capacity) {
+  const int by_rows = (capacity + 1 + tova::COMBINE_THREADS - 1) / tova::COMBINE_THREADS;
+  return by_rows > NX_SPREAD ? by_rows : NX_SPREAD;
+}
+
 Layout make_layout(const tova_config& c) {
   Layout L{};
   const size_t B = c.batch, H = c.n_q_heads, Hkv = c.n_kv_heads, D = c.head_dim, cap = c.capacity;
   const size_t E = c.dtype == TOVA_DTYPE_BF16 ? 2 : 4;
   L.ld = (int)((cap + 1 + 3) / 4 * 4);
-  // scratch is sized for the smallest chunk (one warp = 32 rows per split CTA)
-  L.pc = (int)((cap + tova::ROWS_PER_WARP - 1) / tova::ROWS_PER_WARP) + 1;
-  L.nx_max = (int)((cap + 1 + tova::COMBINE_ROWS - 1) / tova::COMBINE_ROWS);
+  // scratch is sized for the smallest chunk (32 rows per split warp)
+  L.pc = (int)((cap + tova::TILE_ROWS - 1) / tova::TILE_ROWS) + 1;
+  L.nx_max = nx_limit(c.capacity);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   L.K = take(B * Hkv * cap * D * E);
@@ -59,7 +67,7 @@ Layout make_layout(const tova_config& c) {
   L.logits = take(B * H * L.ld * 4);
   L.part_ml = take(B * H * L.pc * 8);
   L.part_acc = take(B * H * (size_t)(L.pc - 1) * D * 4);
-  L.blockmin = take(B * L.nx_max * 8);
+  L.blockmin = take(B * L.nx_max * 16);
   L.counter = take(B * 4);
   L.status = take(4);
   L.cur_pos = take(4);
@@ -80,7 +88,7 @@ struct tova_cache {
   unsigned char* base;
   int32_t len;          // rows per sequence (host mirror; sequences move in lock step)
   int64_t launches;
-  int chunk_warps;      // warps (x32 rows) per split CTA
+  int chunk_rows;       // rows of the state per split warp
   int sm_count;
   int device;
   float scale2;
@@ -91,21 +99,31 @@ namespace {
 
 using tova::StepParams;
 
-template <typename T, int D, int NW, int GB>
+// Heads one split warp carries (GU) and heads per pass over a tile (GB).
+inline int unit_heads(int G) { return G <= 1 ? 1 : G == 2 ? 2 : G <= 4 ? 4 : tova::MAX_UNIT_HEADS; }
+
+inline size_t split_smem_bytes(const tova_config& cfg) {
+  const size_t rb = (size_t)cfg.head_dim * (cfg.dtype == TOVA_DTYPE_BF16 ? 2 : 4);
+  const int gu = unit_heads(cfg.n_q_heads / cfg.n_kv_heads);
+  return (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + sizeof(float) * gu * 32;
+}
+
+template <typename T, int D, int GU, int GB>
 cudaError_t launch_split(int dev, const StepParams& p, dim3 grid, cudaStream_t st) {
   const size_t rb = (size_t)D * sizeof(T);
-  const size_t smem = 2 * (size_t)NW * tova::ROWS_PER_WARP * rb +
-                      sizeof(float) * ((size_t)NW * GB * 32 + (size_t)NW * GB * 2 + (size_t)NW * GB * D);
-  auto kern = tova::tova_split_kernel<T, D, NW, GB>;
+  const size_t smem = (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + sizeof(float) * GU * 32;
+  auto kern = tova::tova_split_kernel<T, D, GU, GB>;
   static bool attr_set[64] = {};  // per instantiation and device: the attribute is per function
   if (!attr_set[dev & 63]) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     if (e != cudaSuccess) return e;
     attr_set[dev & 63] = true;
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = grid;
-  cfg.blockDim = dim3(NW * 32);
+  cfg.blockDim = dim3(32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute at[1];
@@ -116,37 +134,25 @@ cudaError_t launch_split(int dev, const StepParams& p, dim3 grid, cudaStream_t s
   return cudaLaunchKernelEx(&cfg, kern, p);
 }
 
-template <typename T, int D, int GB>
-cudaError_t launch_split_nw(int dev, int nw, const StepParams& p, dim3 grid, cudaStream_t st) {
-  switch (nw) {
-    case 1: return launch_split<T, D, 1, GB>(dev, p, grid, st);
-    case 2: return launch_split<T, D, 2, GB>(dev, p, grid, st);
-    case 4: return launch_split<T, D, 4, GB>(dev, p, grid, st);
-    default: return launch_split<T, D, 8, GB>(dev, p, grid, st);
-  }
-}
-
 template <typename T, int D>
-cudaError_t launch_split_g(int dev, int G, int nw, const StepParams& p, dim3 grid, cudaStream_t st) {
-  // heads of a query group handled per pass over the shared-memory tile
-  constexpr bool wide = (D * sizeof(T) == 512);  // fp32, D = 128: 32 partial sums per head
-  if (G == 1 || wide) return launch_split_nw<T, D, 1>(dev, nw, p, grid, st);
-  if (G == 2) return launch_split_nw<T, D, 2>(dev, nw, p, grid, st);
-  return launch_split_nw<T, D, 4>(dev, nw, p, grid, st);
+cudaError_t launch_split_g(int dev, int G, const StepParams& p, dim3 grid, cudaStream_t st) {
+  constexpr bool wide = (D * sizeof(T) == 512);  // fp32, D = 128: 32 partial sums per head and lane
+  switch (unit_heads(G)) {
+    case 1: return launch_split<T, D, 1, 1>(dev, p, grid, st);
+    case 2: return launch_split<T, D, 2, wide ? 1 : 2>(dev, p, grid, st);
+    case 4: return launch_split<T, D, 4, wide ? 1 : 4>(dev, p, grid, st);
+    default: return launch_split<T, D, 8, wide ? 1 : 2>(dev, p, grid, st);
+  }
 }
 
 template <typename T, int D>
 cudaError_t launch_combine(const StepParams& p, cudaStream_t st) {
-  const size_t smem = sizeof(float) * (2 * (size_t)p.H + (size_t)p.pc);
+  const size_t smem = sizeof(float) * (2 * (size_t)p.H + tova::COMBINE_THREADS);
   auto kern = tova::tova_combine_kernel<T, D>;
-  if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-  }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(p.nx, p.B);
   cfg.blockDim = dim3(tova::COMBINE_THREADS);
-  cfg.dynamicSmemBytes = smem;
+  cfg.dynamicSmemBytes = smem;  // H <= 4096: at most 33 KiB, below the default limit
   cfg.stream = st;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -158,8 +164,8 @@ cudaError_t launch_combine(const StepParams& p, cudaStream_t st) {
 
 template <typename T, int D>
 cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st) {
-  dim3 grid(p.n_chunks > 0 ? p.n_chunks : 1, p.Hkv, p.B);
-  cudaError_t e = launch_split_g<T, D>(c->device, p.G, c->chunk_warps, p, grid, st);
+  dim3 grid(p.n_chunks > 0 ? p.n_chunks : 1, p.Hkv * p.hgroups, p.B);
+  cudaError_t e = launch_split_g<T, D>(c->device, p.G, p, grid, st);
   if (e != cudaSuccess) return e;
   e = launch_combine<T, D>(p, st);
   if (e != cudaSuccess) return e;
@@ -167,16 +173,54 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st) {
   return cudaSuccess;
 }
 
-// Rows per split CTA: the largest of 256/128/64/32 that still gives every SM
-// about four CTAs when the state is full.
-int pick_chunk_warps(const tova_config& cfg, int sm_count) {
-  const long long pairs = (long long)cfg.batch * cfg.n_kv_heads;
-  const long long want = 4LL * sm_count;
-  for (int nw = 8; nw >= 2; nw >>= 1) {
-    const long long chunks = (cfg.capacity + 32LL * nw - 1) / (32LL * nw);
-    if (pairs * chunks >= want) return nw;
+// Rows of the state per split warp.  Every SM holds `per_sm` split warps at a
+// time (shared memory bound); warps beyond one full set wait for a free slot,
+// so the choice trades rounds against per-warp fixed cost (launch, first copy,
+// partial write: about 24 rows' worth).
+int pick_chunk_rows(const tova_config& cfg, int sm_count) {
+  const size_t smem = split_smem_bytes(cfg) + 1024 /* per-CTA reserve */ + 64;
+  long long per_sm = (long long)(227 * 1024) / (long long)smem;
+  if (per_sm > 32) per_sm = 32;
+  if (per_sm < 1) per_sm = 1;
+  const long long slots = per_sm * sm_count;
+  const int G = cfg.n_q_heads / cfg.n_kv_heads;
+  const long long hgroups = (G + unit_heads(G) - 1) / unit_heads(G);
+  const long long pairs = (long long)cfg.batch * cfg.n_kv_heads * hgroups;
+  long long best_cost = -1;
+  int best = 32;
+  for (int cr = 32; cr <= 8192; cr *= 2) {
+    const long long chunks = (cfg.capacity + (long long)cr - 1) / cr;
+    const long long units = pairs * chunks;
+    const long long rounds = (units + slots - 1) / slots;
+    const long long rows = cr < cfg.capacity ? cr : cfg.capacity;
+    const long long cost = rounds * (rows + 24);
+    if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best = cr; }
+    if (cr >= cfg.capacity) break;
   }
-  return 1;
+  return best;
+}
+
+// Launch geometry of one step for n live rows.
+void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows, int sm_count, int nx_max) {
+  p.B = cfg.batch; p.H = cfg.n_q_heads; p.Hkv = cfg.n_kv_heads; p.G = cfg.n_q_heads / cfg.n_kv_heads;
+  p.cap = cfg.capacity;
+  p.n = n;
+  p.chunk_rows = chunk_rows;
+  p.n_chunks = (n + chunk_rows - 1) / chunk_rows;
+  p.hgroups = (p.G + unit_heads(p.G) - 1) / unit_heads(p.G);
+  p.do_evict = (n == cfg.capacity) ? 1 : 0;
+  // combine CTAs per sequence: about two per SM over the batch, at least enough
+  // to give every CTA no more than 128 candidates
+  int nx = (2 * sm_count + cfg.batch - 1) / cfg.batch;
+  const int need = p.do_evict ? (n + 1 + tova::COMBINE_THREADS - 1) / tova::COMBINE_THREADS : 1;
+  if (nx < need) nx = need;
+  if (nx > nx_max) nx = nx_max;
+  const int items = cfg.n_q_heads * cfg.head_dim;
+  if (!p.do_evict && nx > items / 32) nx = items / 32 > 0 ? items / 32 : 1;
+  if (p.do_evict && nx > n + 1) nx = n + 1;
+  if (nx < 1) nx = 1;
+  p.nx = nx;
+  p.cand_per_cta = (n + 1 + nx - 1) / nx;
 }
 
 int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_t pos, float* out,
@@ -193,25 +237,13 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
   p.logits = reinterpret_cast<float*>(base + c->lay.logits);
   p.part_ml = reinterpret_cast<float2*>(base + c->lay.part_ml);
   p.part_acc = reinterpret_cast<float*>(base + c->lay.part_acc);
-  p.blockmin = reinterpret_cast<float2*>(base + c->lay.blockmin);
+  p.blockmin = reinterpret_cast<float4*>(base + c->lay.blockmin);
   p.counter = reinterpret_cast<unsigned*>(base + c->lay.counter);
   p.status = reinterpret_cast<int32_t*>(base + c->lay.status);
   p.cur_pos = reinterpret_cast<int32_t*>(base + c->lay.cur_pos);
   p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.evicted = evicted_pos; p.pos_t = pos;
-  p.B = cfg.batch; p.H = cfg.n_q_heads; p.Hkv = cfg.n_kv_heads; p.G = cfg.n_q_heads / cfg.n_kv_heads;
-  p.cap = cfg.capacity; p.ld = c->lay.ld; p.pc = c->lay.pc;
-  p.n = n;
-  p.chunk_rows = c->chunk_warps * tova::ROWS_PER_WARP;
-  p.n_chunks = (n + p.chunk_rows - 1) / p.chunk_rows;
-  p.do_evict = (n == cfg.capacity) ? 1 : 0;
-  p.nx = p.do_evict ? (n + 1 + tova::COMBINE_ROWS - 1) / tova::COMBINE_ROWS : 1;
-  if (!p.do_evict) {
-    // no scoring: spread the output merge over a few CTAs per sequence
-    int nx = (c->sm_count + cfg.batch - 1) / cfg.batch;
-    if (nx > cfg.n_q_heads) nx = cfg.n_q_heads;
-    if (nx > c->lay.nx_max) nx = c->lay.nx_max;
-    p.nx = nx < 1 ? 1 : nx;
-  }
+  p.ld = c->lay.ld; p.pc = c->lay.pc;
+  fill_geometry(p, cfg, n, c->chunk_rows, c->sm_count, c->lay.nx_max);
   p.scale2 = c->scale2;
   cudaError_t e;
   if (cfg.dtype == TOVA_DTYPE_BF16) {
@@ -268,7 +300,7 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   c->launches = 0;
   c->sm_count = sms;
   c->device = dev;
-  c->chunk_warps = pick_chunk_warps(*cfg, sms);
+  c->chunk_rows = pick_chunk_rows(*cfg, sms);
   c->scale2 = c->cfg.sm_scale * 1.4426950408889634f;
   c->elem = cfg->dtype == TOVA_DTYPE_BF16 ? 2 : 4;
   c->row_bytes = c->elem * cfg->head_dim;
@@ -289,9 +321,9 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
 
 int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows) {
   if (!c) return TOVA_ERR_NULL;
-  if (rows == 0) { c->chunk_warps = pick_chunk_warps(c->cfg, c->sm_count); return TOVA_OK; }
-  if (rows != 32 && rows != 64 && rows != 128 && rows != 256) return TOVA_ERR_BAD_SHAPE;
-  c->chunk_warps = rows / 32;
+  if (rows == 0) { c->chunk_rows = pick_chunk_rows(c->cfg, c->sm_count); return TOVA_OK; }
+  if (rows < 32 || rows > 8192 || rows % tova::TILE_ROWS != 0) return TOVA_ERR_BAD_SHAPE;
+  c->chunk_rows = rows;
   return TOVA_OK;
 }
 
@@ -424,14 +456,15 @@ StaticLayout make_static_layout(const tova_config& c, int chunk_rows) {
   const size_t B = c.batch, H = c.n_q_heads, D = c.head_dim, cap = c.capacity;
   L.ld = (int)((cap + 1 + 3) / 4 * 4);
   L.pc = (int)((cap + chunk_rows - 1) / chunk_rows) + 1;
-  L.nx_max = (int)((cap + 1 + tova::COMBINE_ROWS - 1) / tova::COMBINE_ROWS);
+  L.nx_max = 64 > (int)((cap + 1 + tova::COMBINE_THREADS - 1) / tova::COMBINE_THREADS)
+                 ? 64 : (int)((cap + 1 + tova::COMBINE_THREADS - 1) / tova::COMBINE_THREADS);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   L.control = take(B * 4 /*tickets*/ + B * 4 /*len*/ + 8 /*status, cur_pos*/);
   L.logits = take(B * H * L.ld * 4);
   L.part_ml = take(B * H * L.pc * 8);
   L.part_acc = take(B * H * (size_t)(L.pc - 1) * D * 4);
-  L.blockmin = take(B * L.nx_max * 8);
+  L.blockmin = take(B * L.nx_max * 16);
   L.total = off;
   return L;
 }
@@ -464,8 +497,7 @@ extern "C" int tova_decode_step_static(const tova_config* cfg, void* K, void* V,
     sd.ready = true;
   }
 
-  const int chunk_warps = pick_chunk_warps(*cfg, sd.sm_count);
-  const int chunk_rows = chunk_warps * tova::ROWS_PER_WARP;
+  const int chunk_rows = pick_chunk_rows(*cfg, sd.sm_count);
   const StaticLayout lay = make_static_layout(*cfg, chunk_rows);
   if (lay.total > STATIC_SCRATCH_BYTES) return TOVA_ERR_STATIC_LIMIT;
 
@@ -486,21 +518,15 @@ extern "C" int tova_decode_step_static(const tova_config* cfg, void* K, void* V,
   p.logits = reinterpret_cast<float*>(base + lay.logits);
   p.part_ml = reinterpret_cast<float2*>(base + lay.part_ml);
   p.part_acc = reinterpret_cast<float*>(base + lay.part_acc);
-  p.blockmin = reinterpret_cast<float2*>(base + lay.blockmin);
+  p.blockmin = reinterpret_cast<float4*>(base + lay.blockmin);
   p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.evicted = evicted_pos; p.pos_t = pos;
-  p.B = cfg->batch; p.H = cfg->n_q_heads; p.Hkv = cfg->n_kv_heads; p.G = cfg->n_q_heads / cfg->n_kv_heads;
-  p.cap = cfg->capacity; p.ld = lay.ld; p.pc = lay.pc;
-  p.n = n_live;
-  p.chunk_rows = chunk_rows;
-  p.n_chunks = (n_live + chunk_rows - 1) / chunk_rows;
-  p.do_evict = (n_live == cfg->capacity) ? 1 : 0;
-  p.nx = p.do_evict ? (n_live + 1 + tova::COMBINE_ROWS - 1) / tova::COMBINE_ROWS : 1;
+  p.ld = lay.ld; p.pc = lay.pc;
+  fill_geometry(p, *cfg, n_live, chunk_rows, sd.sm_count, lay.nx_max);
   const float scale = cfg->sm_scale == 0.f ? 1.f / std::sqrt((float)cfg->head_dim) : cfg->sm_scale;
   p.scale2 = scale * 1.4426950408889634f;
 
-  tova_cache shim{};  // launch_step only reads these three fields and counts launches
+  tova_cache shim{};  // launch_step only reads the device and counts launches
   shim.device = dev;
-  shim.chunk_warps = chunk_warps;
   cudaError_t e;
   if (cfg->dtype == TOVA_DTYPE_BF16) {
     e = cfg->head_dim == 128 ? launch_step<__nv_bfloat16, 128>(&shim, p, st)

@@ -57,6 +57,19 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
   return false;
 }
 
+// All lanes of a warp wait for the same barrier phase; the verdict is made
+// uniform so that the warp never splits on it.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity) {
+  return __all_sync(0xffffffffu, mbar_wait_bounded(bar, parity)) != 0;
+}
+
+// Orders this thread's earlier generic-proxy accesses to shared memory before
+// later asynchronous-proxy (bulk copy) writes to it: needed before a buffer
+// that was just read is handed back to the copy engine.
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
 // Global -> shared bulk copy (TMA engine, 1-D form).  dst, src and bytes must
 // be multiples of 16.  Completion is signalled on `bar` as transaction bytes.
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {

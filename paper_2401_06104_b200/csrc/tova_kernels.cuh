@@ -1,11 +1,12 @@
 // The two device stages of one TOVA decode step (sm_100a).
 //
-//   split kernel    : streams the cached K/V rows of one (sequence, KV head,
-//                     chunk of rows) through shared memory with bulk
-//                     asynchronous copies, computes the logits of the query
-//                     heads that share the KV head (Eq. 4), a soft-max partial
-//                     (max, sum, weighted V sum) per head and chunk (Eq. 7),
-//                     and keeps every logit in an fp32 scratch.
+//   split kernel    : one warp streams the cached K/V rows of one (sequence, KV
+//                     head, chunk of rows) through a private shared-memory ring
+//                     fed by bulk asynchronous copies, computes the logits of
+//                     the query heads that share the KV head (Eq. 4), keeps an
+//                     online soft-max (max, sum, weighted V sum) per head and
+//                     writes it as the chunk's partial (Eq. 7); every logit is
+//                     kept in an fp32 scratch.
 //   combine kernel  : merges the partials into the attention output, forms the
 //                     head-averaged weights from the kept logits, takes the
 //                     arg-min and overwrites the victim's row with the new
@@ -19,10 +20,10 @@
 
 namespace tova {
 
-constexpr int ROWS_PER_WARP = 32;   // cache rows one warp owns in the split kernel
-constexpr int MAX_SPLIT_WARPS = 8;  // warps per CTA in the split kernel: 1, 2, 4 or 8
+constexpr int TILE_ROWS = 32;       // cache rows per pipeline stage of the split kernel
+constexpr int SPLIT_BUFFERS = 3;    // tile buffers of a split warp's ring (K and V tiles alternate)
+constexpr int MAX_UNIT_HEADS = 8;   // query heads one split warp carries
 constexpr int COMBINE_THREADS = 128;
-constexpr int COMBINE_ROWS = 128;   // candidate rows scored per combine CTA
 
 struct StepParams {
   // state
@@ -34,7 +35,7 @@ struct StepParams {
   float* logits;      // [B,H,ld]   base-2 logits of candidates 0..n (n = the new token)
   float2* part_ml;    // [B,H,pc]   (max2, sum) per chunk; entry n_chunks = the new token
   float* part_acc;    // [B,H,pc-1,D] un-normalised weighted V sums per chunk
-  float2* blockmin;   // [B,nx_max] (lowest mean weight, its candidate index as int bits)
+  float4* blockmin;   // [B,nx_max] (lowest mean weight, its candidate index, its position, -)
   unsigned* counter;  // [B] tickets of the combine CTAs
   int32_t* status;    // [1]
   int32_t* cur_pos;   // [1] position of the token being processed (set by the split kernel)
@@ -49,8 +50,10 @@ struct StepParams {
   int32_t B, H, Hkv, G, cap, ld, pc;
   int32_t n;          // live rows before this step (same for every sequence)
   int32_t n_chunks;   // ceil(n / chunk_rows)
-  int32_t chunk_rows; // rows per split CTA = 32 * warps
+  int32_t chunk_rows; // rows per split warp, a multiple of TILE_ROWS
+  int32_t hgroups;    // ceil(G / heads per split warp)
   int32_t nx;         // combine CTAs per sequence
+  int32_t cand_per_cta;  // candidates scored per combine CTA (<= COMBINE_THREADS)
   int32_t do_evict;   // n == cap and the policy is on
   float scale2;       // sm_scale * log2(e)
 };
@@ -58,69 +61,86 @@ struct StepParams {
 // ---------------------------------------------------------------------------
 // split kernel
 // ---------------------------------------------------------------------------
-// grid = (max(n_chunks,1), Hkv, B), block = NW warps.  Warp w of chunk c owns
-// rows [c*32*NW + 32*w, +32).  Every lane reads 16 bytes of a row; LPR lanes
-// cover a row, so a warp reads RPW = 32/LPR rows per pass and needs LPR passes.
-template <typename T, int D, int NW, int GB>
-__global__ void __launch_bounds__(NW * 32) tova_split_kernel(const StepParams p) {
+// grid = (max(n_chunks,1), Hkv*hgroups, B), block = one warp.  The warp owns
+// rows [c*chunk_rows, +chunk_rows) of one KV head and up to GU query heads of
+// its group.  The operand tiles K_0 V_0 K_1 V_1 ... (32 rows each) travel through
+// a ring of SPLIT_BUFFERS buffers: lane 0 issues the copy of operand tile u+NB
+// into a buffer as soon as the warp has consumed tile u from it, so nothing but
+// this warp ever waits on these barriers.
+// Every lane reads 16 bytes of a row; LPR lanes cover a row, so the warp reads
+// RPW = 32/LPR rows per pass and a tile takes LPR passes.
+template <typename T, int D, int GU, int GB>
+__global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
   constexpr int EPL = Vec16<T>::N;          // elements per lane
   constexpr int RB = D * (int)sizeof(T);    // bytes per row
   constexpr int LPR = RB / 16;              // lanes per row
   constexpr int RPW = 32 / LPR;             // rows per pass
-  constexpr int NP = LPR;                   // passes per warp tile (RPW * NP = 32)
+  constexpr int NP = LPR;                   // passes per tile (RPW * NP = 32)
+  constexpr int TILE_BYTES = TILE_ROWS * RB;
+  constexpr int NB = SPLIT_BUFFERS;
   static_assert(LPR >= 8 && LPR <= 32, "row must be 128..512 bytes");
+  static_assert(GU % GB == 0, "head block must divide the unit");
 
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  unsigned char* k_tile = smem_raw;                                   // [NW][32][RB]
-  unsigned char* v_tile = smem_raw + (size_t)NW * ROWS_PER_WARP * RB; // [NW][32][RB]
-  float* w_p = reinterpret_cast<float*>(v_tile + (size_t)NW * ROWS_PER_WARP * RB);  // [NW][GB][32]
-  float* w_ml = w_p + NW * GB * 32;                                   // [NW][GB][2]
-  float* w_acc = w_ml + NW * GB * 2;                                  // [NW][GB][D]
-  __shared__ __align__(8) uint64_t bars[MAX_SPLIT_WARPS][2];
+  unsigned char* ring = smem_raw;                                    // [NB][TILE_BYTES]
+  float* w_p = reinterpret_cast<float*>(smem_raw + NB * TILE_BYTES); // [GU][32] weights of a tile
+  __shared__ __align__(8) uint64_t bars[NB];
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int lane = threadIdx.x;
   const int lig = lane % LPR;   // lane in row group
   const int sub = lane / LPR;   // which of the RPW rows of a pass
-  const int c = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
-  const int row0 = c * p.chunk_rows + warp * ROWS_PER_WARP;            // first row of this warp
-  const int nvalid = min(max(p.n - row0, 0), ROWS_PER_WARP);           // live rows of this warp
-  const int my_row = lig * RPW + sub;                                  // row this lane ends up owning
+  const int c = blockIdx.x, b = blockIdx.z;
+  const int kvh = blockIdx.y / p.hgroups, hg = blockIdx.y % p.hgroups;
+  const int g_begin = hg * GU;
+  const int g_cnt = min(GU, p.G - g_begin);                 // real heads of this unit
+  const int row_begin = c * p.chunk_rows;
+  const int rows = min(max(p.n - row_begin, 0), p.chunk_rows);
+  const int ntiles = (rows + TILE_ROWS - 1) / TILE_ROWS;
+  const int my_row = lig * RPW + sub;                       // tile row this lane ends up owning
 
-  if (lane == 0 && nvalid > 0) {
-    mbar_init(&bars[warp][0], 1);
-    mbar_init(&bars[warp][1], 1);
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < NB; ++s) mbar_init(&bars[s], 1);
     mbar_fence_init();
   }
   __syncwarp();
 
-  // Everything above touches no global memory; below we read what the previous
-  // kernels in the stream wrote.
+  // Nothing above touches global memory; below we read what earlier kernels in
+  // the stream wrote.
   pdl_wait();
   pdl_launch_dependents();
 
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0)
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0)
     *p.cur_pos = (p.pos_t < 0) ? *p.cur_pos + 1 : p.pos_t;
 
-  const size_t kv_row0 = ((size_t)b * p.Hkv + kvh) * p.cap + row0;
-  unsigned char* my_k = k_tile + (size_t)warp * ROWS_PER_WARP * RB;
-  unsigned char* my_v = v_tile + (size_t)warp * ROWS_PER_WARP * RB;
-  if (lane == 0 && nvalid > 0) {
-    const uint32_t bytes = (uint32_t)nvalid * RB;
-    mbar_expect_tx(&bars[warp][0], bytes);
-    bulk_g2s(my_k, static_cast<const unsigned char*>(p.K) + kv_row0 * RB, bytes, &bars[warp][0]);
-    mbar_expect_tx(&bars[warp][1], bytes);
-    bulk_g2s(my_v, static_cast<const unsigned char*>(p.V) + kv_row0 * RB, bytes, &bars[warp][1]);
+  const unsigned char* k_src =
+      static_cast<const unsigned char*>(p.K) + (((size_t)b * p.Hkv + kvh) * p.cap + row_begin) * RB;
+  const unsigned char* v_src =
+      static_cast<const unsigned char*>(p.V) + (((size_t)b * p.Hkv + kvh) * p.cap + row_begin) * RB;
+
+  const int n_ops = 2 * ntiles;        // operand tiles: u = 2t is K_t, u = 2t+1 is V_t
+  auto issue = [&](int u) {            // lane 0 only
+    const int t = u >> 1;
+    const uint32_t bytes = (uint32_t)min(TILE_ROWS, rows - t * TILE_ROWS) * RB;
+    uint64_t* bar = &bars[u % NB];
+    mbar_expect_tx(bar, bytes);
+    bulk_g2s(ring + (size_t)(u % NB) * TILE_BYTES, ((u & 1) ? v_src : k_src) + (size_t)t * TILE_BYTES, bytes,
+             bar);
+  };
+  if (lane == 0) {
+    for (int u = 0; u < min(NB, n_ops); ++u) issue(u);
   }
 
-  const T* qbase = static_cast<const T*>(p.q) + ((size_t)b * p.H + (size_t)kvh * p.G) * D;
+  const T* qbase = static_cast<const T*>(p.q) + ((size_t)b * p.H + (size_t)kvh * p.G + g_begin) * D;
+  const size_t bh0 = (size_t)b * p.H + (size_t)kvh * p.G + g_begin;
 
-  // The new token (candidate n): its logit per head, done once per (b, kvh)
-  // by warp 0 of chunk 0 while the copies are in flight.
-  if (c == 0 && warp == 0) {
+  // The new token (candidate n): its logit per head, by the warp of chunk 0
+  // while its first copies are in flight.
+  if (c == 0) {
     const T* kn = static_cast<const T*>(p.k_new) + ((size_t)b * p.Hkv + kvh) * D;
     float kf[EPL];
     Vec16<T>::unpack(*reinterpret_cast<const uint4*>(kn + lig * EPL), kf);
-    for (int g = 0; g < p.G; ++g) {
+    for (int g = 0; g < g_cnt; ++g) {
       float qf[EPL];
       Vec16<T>::unpack(*reinterpret_cast<const uint4*>(qbase + (size_t)g * D + lig * EPL), qf);
       float s = 0.f;
@@ -130,186 +150,163 @@ __global__ void __launch_bounds__(NW * 32) tova_split_kernel(const StepParams p)
       for (int o = LPR / 2; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
       s *= p.scale2;
       if (lane == 0) {
-        const size_t bh = (size_t)b * p.H + (size_t)kvh * p.G + g;
-        p.logits[bh * p.ld + p.n] = s;
-        p.part_ml[bh * p.pc + p.n_chunks] = make_float2(s, 1.f);
+        p.logits[(bh0 + g) * p.ld + p.n] = s;
+        p.part_ml[(bh0 + g) * p.pc + p.n_chunks] = make_float2(s, 1.f);
       }
     }
   }
-  if (c >= p.n_chunks) return;  // empty state: only the new token exists
+  if (ntiles == 0) return;  // empty state: only the new token exists
 
-  bool k_ready = false, v_ready = false, failed = false;
-
-  for (int g0 = 0; g0 < p.G; g0 += GB) {
-    // ---- logits of GB heads for this warp's 32 rows -----------------------
-    float qf[GB][EPL];
+  // q of the unit's heads, kept packed (16 bytes per head and lane)
+  uint4 qpk[GU];
 #pragma unroll
-    for (int gb = 0; gb < GB; ++gb) {
-      const int g = min(g0 + gb, p.G - 1);
-      Vec16<T>::unpack(*reinterpret_cast<const uint4*>(qbase + (size_t)g * D + lig * EPL), qf[gb]);
-    }
-    float s[GB];
-    float m[GB], l[GB];
-    if (nvalid > 0) {
-      if (!k_ready) {
-        k_ready = true;
-        if (!mbar_wait_bounded(&bars[warp][0], 0)) failed = true;
-      }
+  for (int g = 0; g < GU; ++g)
+    qpk[g] = *reinterpret_cast<const uint4*>(qbase + (size_t)min(g, g_cnt - 1) * D + lig * EPL);
+
+  float m[GU], l[GU], acc[GU][EPL];
+#pragma unroll
+  for (int g = 0; g < GU; ++g) {
+    m[g] = -INFINITY;
+    l[g] = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[g][e] = 0.f;
+  }
+
+  bool failed = false;
+  int t = 0;
+  for (; t < ntiles; ++t) {
+    const int uk = 2 * t, uv = 2 * t + 1;
+    const int nvalid = min(TILE_ROWS, rows - t * TILE_ROWS);
+    const unsigned char* kt = ring + (size_t)(uk % NB) * TILE_BYTES;
+    const unsigned char* vt = ring + (size_t)(uv % NB) * TILE_BYTES;
+
+    // ---- logits of the tile's 32 rows, GB heads at a time --------------------
+    if (!warp_wait(&bars[uk % NB], (uint32_t)(uk / NB) & 1u)) { failed = true; break; }
+    float s[GU];
+#pragma unroll
+    for (int g0 = 0; g0 < GU; g0 += GB) {
+      float qf[GB][EPL];
+#pragma unroll
+      for (int gb = 0; gb < GB; ++gb) Vec16<T>::unpack(qpk[g0 + gb], qf[gb]);
       float part[GB][NP];
-      if (!failed) {
 #pragma unroll
-        for (int i = 0; i < NP; ++i) {
-          const int r = i * RPW + sub;
-          float kf[EPL];
-          Vec16<T>::unpack(*reinterpret_cast<const uint4*>(my_k + (size_t)r * RB + lig * 16), kf);
+      for (int i = 0; i < NP; ++i) {
+        const int r = i * RPW + sub;
+        float kf[EPL];
+        Vec16<T>::unpack(*reinterpret_cast<const uint4*>(kt + (size_t)r * RB + lig * 16), kf);
 #pragma unroll
-          for (int gb = 0; gb < GB; ++gb) {
-            float a = 0.f;
+        for (int gb = 0; gb < GB; ++gb) {
+          float a = 0.f;
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) a = fmaf(qf[gb][e], kf[e], a);
-            part[gb][i] = a;
-          }
+          for (int e = 0; e < EPL; ++e) a = fmaf(qf[gb][e], kf[e], a);
+          part[gb][i] = a;
         }
-      } else {
-#pragma unroll
-        for (int gb = 0; gb < GB; ++gb)
-#pragma unroll
-          for (int i = 0; i < NP; ++i) part[gb][i] = 0.f;
       }
 #pragma unroll
       for (int gb = 0; gb < GB; ++gb) {
-        float v = transpose_reduce<NP>(part[gb], lig) * p.scale2;
+        const float v = transpose_reduce<NP>(part[gb], lig) * p.scale2;
         // rows past the live range hold stale shared memory: mask them out
-        s[gb] = (my_row < nvalid) ? v : -INFINITY;
+        s[g0 + gb] = (my_row < nvalid) ? v : -INFINITY;
       }
-    } else {
-#pragma unroll
-      for (int gb = 0; gb < GB; ++gb) s[gb] = -INFINITY;
+    }
+    // the K buffer is free: refill it with the tile after next
+    __syncwarp();
+    if (lane == 0 && uk + NB < n_ops) {
+      fence_proxy_async_smem();
+      issue(uk + NB);
     }
 
-    // ---- soft-max partial of the warp, weights to shared memory -----------
+    // ---- online soft-max update, weights of the tile to shared memory --------
 #pragma unroll
-    for (int gb = 0; gb < GB; ++gb) {
-      if (g0 + gb < p.G && my_row < nvalid) {
-        const size_t bh = (size_t)b * p.H + (size_t)kvh * p.G + g0 + gb;
-        p.logits[bh * p.ld + row0 + my_row] = s[gb];
-      }
-      m[gb] = warp_max(s[gb]);
-      const float e = exp2_diff(s[gb], m[gb]);
-      l[gb] = warp_sum(e);
-      w_p[(warp * GB + gb) * 32 + my_row] = e;
+    for (int g = 0; g < GU; ++g) {
+      if (g < g_cnt && my_row < nvalid)
+        p.logits[(bh0 + g) * p.ld + row_begin + t * TILE_ROWS + my_row] = s[g];
+      const float m_new = fmaxf(m[g], warp_max(s[g]));
+      const float corr = exp2_diff(m[g], m_new);
+      const float e = exp2_diff(s[g], m_new);
+      l[g] = fmaf(l[g], corr, warp_sum(e));
+      m[g] = m_new;
+#pragma unroll
+      for (int k = 0; k < EPL; ++k) acc[g][k] *= corr;
+      w_p[g * 32 + my_row] = e;
     }
     __syncwarp();
 
-    // ---- weighted V sum ----------------------------------------------------
-    float acc[GB][EPL];
+    // ---- weighted V sum --------------------------------------------------------
+    if (!warp_wait(&bars[uv % NB], (uint32_t)(uv / NB) & 1u)) { failed = true; break; }
 #pragma unroll
-    for (int gb = 0; gb < GB; ++gb)
+    for (int i = 0; i < NP; ++i) {
+      const int r = i * RPW + sub;
+      if (r < nvalid) {
+        float vf[EPL];
+        Vec16<T>::unpack(*reinterpret_cast<const uint4*>(vt + (size_t)r * RB + lig * 16), vf);
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) acc[gb][e] = 0.f;
-    if (nvalid > 0) {
-      if (!v_ready) {
-        v_ready = true;
-        if (!failed && !mbar_wait_bounded(&bars[warp][1], 0)) failed = true;
-      }
-      if (!failed) {
+        for (int g = 0; g < GU; ++g) {
+          const float w = w_p[g * 32 + r];
 #pragma unroll
-        for (int i = 0; i < NP; ++i) {
-          const int r = i * RPW + sub;
-          if (r < nvalid) {
-            float vf[EPL];
-            Vec16<T>::unpack(*reinterpret_cast<const uint4*>(my_v + (size_t)r * RB + lig * 16), vf);
-#pragma unroll
-            for (int gb = 0; gb < GB; ++gb) {
-              const float w = w_p[(warp * GB + gb) * 32 + r];
-#pragma unroll
-              for (int e = 0; e < EPL; ++e) acc[gb][e] = fmaf(w, vf[e], acc[gb][e]);
-            }
-          }
+          for (int e = 0; e < EPL; ++e) acc[g][e] = fmaf(w, vf[e], acc[g][e]);
         }
       }
     }
-    // fold the RPW row groups of the warp together
-#pragma unroll
-    for (int gb = 0; gb < GB; ++gb)
-#pragma unroll
-      for (int e = 0; e < EPL; ++e)
-#pragma unroll
-        for (int o = LPR; o < 32; o <<= 1) acc[gb][e] += __shfl_xor_sync(0xffffffffu, acc[gb][e], o);
-
-    // ---- merge the warps of the CTA, write the chunk partial --------------
-    if (NW == 1) {
-#pragma unroll
-      for (int gb = 0; gb < GB; ++gb) {
-        if (g0 + gb < p.G && sub == 0) {
-          const size_t bh = (size_t)b * p.H + (size_t)kvh * p.G + g0 + gb;
-          float* dst = p.part_acc + (bh * (p.pc - 1) + c) * D + lig * EPL;
-#pragma unroll
-          for (int e = 0; e < EPL; e += 4)
-            *reinterpret_cast<float4*>(dst + e) =
-                make_float4(acc[gb][e], acc[gb][e + 1], acc[gb][e + 2], acc[gb][e + 3]);
-          if (lane == 0) p.part_ml[bh * p.pc + c] = make_float2(m[gb], l[gb]);
-        }
-      }
-    } else {
-      if (sub == 0) {
-#pragma unroll
-        for (int gb = 0; gb < GB; ++gb) {
-          float* dst = w_acc + (size_t)(warp * GB + gb) * D + lig * EPL;
-#pragma unroll
-          for (int e = 0; e < EPL; ++e) dst[e] = acc[gb][e];
-          if (lane == 0) {
-            w_ml[(warp * GB + gb) * 2 + 0] = m[gb];
-            w_ml[(warp * GB + gb) * 2 + 1] = l[gb];
-          }
-        }
-      }
-      __syncthreads();
-      for (int idx = threadIdx.x; idx < GB * D; idx += NW * 32) {
-        const int gb = idx / D, d = idx % D;
-        if (g0 + gb < p.G) {
-          float M = -INFINITY;
-#pragma unroll
-          for (int w = 0; w < NW; ++w) M = fmaxf(M, w_ml[(w * GB + gb) * 2]);
-          float a = 0.f, L = 0.f;
-#pragma unroll
-          for (int w = 0; w < NW; ++w) {
-            const float f = exp2_diff(w_ml[(w * GB + gb) * 2], M);
-            a = fmaf(w_acc[(size_t)(w * GB + gb) * D + d], f, a);
-            L = fmaf(w_ml[(w * GB + gb) * 2 + 1], f, L);
-          }
-          const size_t bh = (size_t)b * p.H + (size_t)kvh * p.G + g0 + gb;
-          p.part_acc[(bh * (p.pc - 1) + c) * D + d] = a;
-          if (d == 0) p.part_ml[bh * p.pc + c] = make_float2(M, L);
-        }
-      }
-      __syncthreads();
+    __syncwarp();
+    if (lane == 0 && uv + NB < n_ops) {
+      fence_proxy_async_smem();
+      issue(uv + NB);
     }
   }
-  if (failed && lane == 0) atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
+
+  if (failed) {
+    // Give copies still in flight a last bounded chance to land before the
+    // shared memory is released, and report.
+    for (int u = 2 * t; u < min(2 * t + NB, n_ops); ++u) warp_wait(&bars[u % NB], (uint32_t)(u / NB) & 1u);
+    if (lane == 0) atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
+    return;
+  }
+
+  // ---- fold the RPW row groups of the warp, write the chunk partial -----------
+#pragma unroll
+  for (int g = 0; g < GU; ++g) {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e)
+#pragma unroll
+      for (int o = LPR; o < 32; o <<= 1) acc[g][e] += __shfl_xor_sync(0xffffffffu, acc[g][e], o);
+    if (g < g_cnt && sub == 0) {
+      float* dst = p.part_acc + ((bh0 + g) * (size_t)(p.pc - 1) + c) * D + lig * EPL;
+#pragma unroll
+      for (int e = 0; e < EPL; e += 4)
+        *reinterpret_cast<float4*>(dst + e) = make_float4(acc[g][e], acc[g][e + 1], acc[g][e + 2], acc[g][e + 3]);
+      if (lane == 0) p.part_ml[(bh0 + g) * p.pc + c] = make_float2(m[g], l[g]);
+    }
+  }
 }
 
 
 // ---------------------------------------------------------------------------
 // combine-and-evict kernel
 // ---------------------------------------------------------------------------
-// grid = (nx, B), block = COMBINE_THREADS.  Every CTA of a sequence first
-// rebuilds each head's global (max2, 1/sum) from the chunk partials; CTA x then
-//   - writes the attention output of heads x, x+nx, ... (Eq. 7),
-//   - scores candidates [x*COMBINE_ROWS, +COMBINE_ROWS): the mean over heads of
-//     the soft-max weights (Algorithm 1), and leaves its lowest (value, index).
-// The last CTA of the sequence to finish (atomic ticket, no waiting) picks the
-// overall arg-min - lowest index on ties - and replaces that row by the new
-// token in K, V and the position table (Eq. 9, in place).
-// smem: float hM[H], hInvL[H], wts[pc].
+// grid = (nx, B), block = COMBINE_THREADS.  Built for few dependent memory
+// round trips, since the whole step lasts microseconds:
+//   1. every CTA rebuilds each head's global (max2, 1/sum) from the chunk
+//      partials (one round trip);
+//   2. CTA x writes its 1/nx share of the H*D attention outputs (Eq. 7), every
+//      thread merging the chunk partials of one (head, dim);
+//   3. CTA x scores candidates [x*cand_per_cta, +cand_per_cta): the mean over
+//      heads of the soft-max weights (Algorithm 1).  Threads split the heads of
+//      a candidate HS ways and the partial sums are added in a fixed order;
+//      the CTA leaves its lowest (value, index, position);
+//   4. the last CTA of the sequence to finish (atomic ticket, nobody waits)
+//      takes the overall arg-min - lowest index on ties - and replaces that row
+//      by the new token in K, V and the position table (Eq. 9, in place).
+// smem: float hM[H], hInvL[H], sc[COMBINE_THREADS].
 template <typename T, int D>
 __global__ void __launch_bounds__(COMBINE_THREADS) tova_combine_kernel(const StepParams p) {
   extern __shared__ __align__(16) float csm[];
-  float* hM = csm;              // [H]
-  float* hInvL = csm + p.H;     // [H]
-  float* wts = csm + 2 * p.H;   // [pc]
+  float* hM = csm;                 // [H]
+  float* hInvL = csm + p.H;        // [H]
+  float* sc = csm + 2 * p.H;       // [COMBINE_THREADS] partial head sums
   __shared__ float red_v[COMBINE_THREADS / 32];
   __shared__ int red_i[COMBINE_THREADS / 32];
+  __shared__ int red_p[COMBINE_THREADS / 32];
   __shared__ int s_last;
 
   const int x = blockIdx.x, b = blockIdx.y;
@@ -320,18 +317,23 @@ __global__ void __launch_bounds__(COMBINE_THREADS) tova_combine_kernel(const Ste
   pdl_launch_dependents();
   const int pos_t = *p.cur_pos;
 
-  // ---- global max and sum of every head ------------------------------------
+  // ---- 1. global max and sum of every head ------------------------------------
   for (int h = warp; h < p.H; h += COMBINE_THREADS / 32) {
     const float2* ml = p.part_ml + ((size_t)b * p.H + h) * p.pc;
-    float M = -INFINITY;
-    for (int i = lane; i < np; i += 32) M = fmaxf(M, ml[i].x);
-    M = warp_max(M);
-    float L = 0.f;
-    for (int i = lane; i < np; i += 32) {
-      const float2 e = ml[i];
-      L = fmaf(e.y, exp2_diff(e.x, M), L);
+    float M = -INFINITY, L = 0.f;
+    if (np <= 32) {
+      const float2 e = (lane < np) ? ml[lane] : make_float2(-INFINITY, 0.f);
+      M = warp_max(e.x);
+      L = warp_sum(e.y * exp2_diff(e.x, M));
+    } else {
+      for (int i = lane; i < np; i += 32) M = fmaxf(M, ml[i].x);
+      M = warp_max(M);
+      for (int i = lane; i < np; i += 32) {
+        const float2 e = ml[i];
+        L = fmaf(e.y, exp2_diff(e.x, M), L);
+      }
+      L = warp_sum(L);
     }
-    L = warp_sum(L);
     if (lane == 0) {
       hM[h] = M;
       hInvL[h] = 1.f / L;
@@ -339,21 +341,24 @@ __global__ void __launch_bounds__(COMBINE_THREADS) tova_combine_kernel(const Ste
   }
   __syncthreads();
 
-  // ---- attention output of this CTA's heads --------------------------------
-  for (int h = x; h < p.H; h += p.nx) {
-    const size_t bh = (size_t)b * p.H + h;
-    const float2* ml = p.part_ml + bh * p.pc;
-    for (int i = tid; i < np; i += COMBINE_THREADS) wts[i] = exp2_diff(ml[i].x, hM[h]) * hInvL[h];
-    __syncthreads();
-    const float* acc = p.part_acc + bh * (size_t)(p.pc - 1) * D;
-    const T* vn = static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + h / p.G) * D;
-    for (int d = tid; d < D; d += COMBINE_THREADS) {
+  // ---- 2. this CTA's share of the attention output -----------------------------
+  {
+    const int items = p.H * D;
+    const int per = (items + p.nx - 1) / p.nx;
+    const int end = min(items, (x + 1) * per);
+    for (int it = x * per + tid; it < end; it += COMBINE_THREADS) {
+      const int h = it / D, d = it % D;
+      const size_t bh = (size_t)b * p.H + h;
+      const float2* ml = p.part_ml + bh * p.pc;
+      const float* acc = p.part_acc + bh * (size_t)(p.pc - 1) * D + d;
+      const float M = hM[h], iL = hInvL[h];
       float o = 0.f;
-      for (int i = 0; i < p.n_chunks; ++i) o = fmaf(acc[(size_t)i * D + d], wts[i], o);
-      o = fmaf((float)vn[d], wts[p.n_chunks], o);
-      p.out[bh * D + d] = o;
+#pragma unroll 4
+      for (int i = 0; i < p.n_chunks; ++i) o = fmaf(acc[(size_t)i * D], exp2_diff(ml[i].x, M), o);
+      const T* vn = static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + h / p.G) * D;
+      o = fmaf((float)vn[d], exp2_diff(ml[p.n_chunks].x, M), o);
+      p.out[bh * D + d] = o * iL;
     }
-    __syncthreads();
   }
 
   constexpr int RB16 = D * (int)sizeof(T) / 16;  // 16-byte words per row
@@ -378,29 +383,46 @@ __global__ void __launch_bounds__(COMBINE_THREADS) tova_combine_kernel(const Ste
     return;
   }
 
-  // ---- head-averaged weight of this CTA's candidates ------------------------
-  const int j = x * COMBINE_ROWS + tid;
-  float val = INFINITY;
-  if (j <= p.n) {
+  // ---- 3. head-averaged weight of this CTA's candidates ------------------------
+  // wp = cand_per_cta rounded up to a power of two; thread = (candidate jl, head slice hs)
+  int wp = 1;
+  while (wp < p.cand_per_cta) wp <<= 1;
+  const int hs_n = COMBINE_THREADS / wp;
+  const int jl = tid % wp, hs = tid / wp;
+  const int j = x * p.cand_per_cta + jl;
+  const bool live = (jl < p.cand_per_cta) && (j <= p.n);
+  float a = 0.f;
+  if (live) {
     const float* lg = p.logits + (size_t)b * p.H * p.ld + j;
-    float a = 0.f;
-    for (int h = 0; h < p.H; ++h) a += exp2f(lg[(size_t)h * p.ld] - hM[h]) * hInvL[h];
-    val = a * (1.f / (float)p.H);
+#pragma unroll 4
+    for (int h = hs; h < p.H; h += hs_n) a = fmaf(exp2f(lg[(size_t)h * p.ld] - hM[h]), hInvL[h], a);
   }
-  int idx = j;
+  sc[tid] = a;
+  int cpos = pos_t;  // position held by the candidate (the new token holds pos_t)
+  if (hs == 0 && live && j < p.cap) cpos = p.pos[(size_t)b * p.cap + j];
+  __syncthreads();
+  float val = INFINITY;
+  int idx = 0x7fffffff;
+  if (hs == 0 && live) {
+    float tot = 0.f;
+    for (int k = 0; k < hs_n; ++k) tot += sc[k * wp + jl];
+    val = tot * (1.f / (float)p.H);
+    idx = j;
+  }
   // lowest (value, index) of the block
 #pragma unroll
   for (int o = 16; o >= 1; o >>= 1) {
     const float ov = __shfl_xor_sync(0xffffffffu, val, o);
     const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-    if (ov < val || (ov == val && oi < idx)) { val = ov; idx = oi; }
+    const int op = __shfl_xor_sync(0xffffffffu, cpos, o);
+    if (ov < val || (ov == val && oi < idx)) { val = ov; idx = oi; cpos = op; }
   }
-  if (lane == 0) { red_v[warp] = val; red_i[warp] = idx; }
+  if (lane == 0) { red_v[warp] = val; red_i[warp] = idx; red_p[warp] = cpos; }
   __syncthreads();
   if (tid == 0) {
     for (int w = 1; w < COMBINE_THREADS / 32; ++w)
-      if (red_v[w] < val || (red_v[w] == val && red_i[w] < idx)) { val = red_v[w]; idx = red_i[w]; }
-    p.blockmin[(size_t)b * p.nx + x] = make_float2(val, __int_as_float(idx));
+      if (red_v[w] < val || (red_v[w] == val && red_i[w] < idx)) { val = red_v[w]; idx = red_i[w]; cpos = red_p[w]; }
+    p.blockmin[(size_t)b * p.nx + x] = make_float4(val, __int_as_float(idx), __int_as_float(cpos), 0.f);
     __threadfence();
     const unsigned t = atomicAdd(p.counter + b, 1u);
     s_last = (t == (unsigned)p.nx - 1u);
@@ -409,19 +431,29 @@ __global__ void __launch_bounds__(COMBINE_THREADS) tova_combine_kernel(const Ste
   if (!s_last) return;
   __threadfence();
 
-  // ---- last CTA of the sequence: arg-min over blocks, evict, insert --------
-  if (tid == 0) {
-    const volatile float2* bm = p.blockmin + (size_t)b * p.nx;
+  // ---- 4. last CTA of the sequence: arg-min over blocks, evict, insert ---------
+  if (warp == 0) {
     float bv = INFINITY;
-    int bi = p.n;  // a valid default; every block reports a finite value in practice
-    for (int i = 0; i < p.nx; ++i) {
-      const float v = bm[i].x;
-      const int ci = __float_as_int(bm[i].y);
-      if (v < bv || (v == bv && ci < bi)) { bv = v; bi = ci; }
+    int bi = 0x7fffffff, bp = pos_t;
+    for (int i = lane; i < p.nx; i += 32) {
+      const float4 e = __ldcg(p.blockmin + (size_t)b * p.nx + i);
+      const int ci = __float_as_int(e.y);
+      if (e.x < bv || (e.x == bv && ci < bi)) { bv = e.x; bi = ci; bp = __float_as_int(e.z); }
     }
-    if (bi < 0 || bi > p.cap) { atomicExch(p.status, DEV_ERR_BAD_VICTIM); bi = p.cap; }
-    red_i[0] = bi;
-    p.counter[b] = 0;  // ready for the next step
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      const int op = __shfl_xor_sync(0xffffffffu, bp, o);
+      if (ov < bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; bp = op; }
+    }
+    if (lane == 0) {
+      if (bi < 0 || bi > p.cap) { atomicExch(p.status, DEV_ERR_BAD_VICTIM); bi = p.cap; bp = pos_t; }
+      red_i[0] = bi;
+      p.counter[b] = 0;  // ready for the next step
+      if (bi < p.cap) p.pos[(size_t)b * p.cap + bi] = pos_t;
+      if (p.evicted) p.evicted[b] = bp;  // the new token's own position if it dropped itself
+    }
   }
   __syncthreads();
   const int victim = red_i[0];
@@ -433,14 +465,6 @@ __global__ void __launch_bounds__(COMBINE_THREADS) tova_combine_kernel(const Ste
       static_cast<uint4*>(p.K)[dst] = static_cast<const uint4*>(p.k_new)[src];
       static_cast<uint4*>(p.V)[dst] = static_cast<const uint4*>(p.v_new)[src];
     }
-  }
-  if (tid == 0) {
-    int ev = pos_t;  // the new token dropped itself
-    if (victim < p.cap) {
-      ev = p.pos[(size_t)b * p.cap + victim];
-      p.pos[(size_t)b * p.cap + victim] = pos_t;
-    }
-    if (p.evicted) p.evicted[b] = ev;
   }
 }
 

@@ -53,7 +53,7 @@ def test_tiny_reference_config_full_stream(name):
           f"max_err {rep.max_err:.2e} max_gap {rep.max_gap:.2e}")
 
 
-@pytest.mark.parametrize("chunk_rows", [0, 32, 64, 128, 256])
+@pytest.mark.parametrize("chunk_rows", [0, 32, 64, 96, 128, 256, 1024])
 def test_llama_shape_reduced_every_chunk_size(chunk_rows):
     """bf16 MHA, capacity 203: several tiles plus a ragged tail at every chunk size."""
     w = LLAMA.scaled(batch=2, n_q_heads=6, n_kv_heads=6, capacity=203)
