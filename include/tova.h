@@ -148,7 +148,7 @@ const char* tova_strerror(int status);
  * capture, a process whose memory budget was fixed at start-up.  Such callers
  * usually do hold the K/V tensors themselves but have nowhere to put the
  * scratch the two kernels exchange (logits, per-chunk soft-max partials,
- * per-block minima, tickets).  For this call that scratch is an array
+ * block minima, status words).  For this call that scratch is an array
  * compiled into the library: TOVA_STATIC_SCRATCH_BYTES (8 MiB) of device
  * memory that every GPU context loading the library holds until it exits.
  *
@@ -171,7 +171,7 @@ const char* tova_strerror(int status);
  * use on a device looks up the array's device address (cudaGetSymbolAddress)
  * and the SM count; make that first call outside any stream capture.  All calls
  * on a device share the one array, which keeps whatever the previous call left:
- * the call clears its tickets and status itself (a memset on `cuda_stream`),
+ * the call clears its status words itself (a memset on `cuda_stream`),
  * but two calls whose kernels overlap on the GPU - different streams, or
  * different host threads without ordering - race on it.  Issue them on one
  * stream or order them with events. */

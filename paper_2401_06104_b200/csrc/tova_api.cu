@@ -19,10 +19,10 @@ inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 struct Layout {
-  size_t K, V, pos, len, logits, part_ml, part_acc, blockmin, counter, status, cur_pos;
+  size_t K, V, pos, len, logits, part_ml, part_acc, status, cur_pos;
   size_t st_q, st_k, st_v, st_out, st_ev;  // staging for host-buffer calls
   size_t total;
-  int ld, pc, nx_max;
+  int ld, pc;
 };
 
 bool config_ok(const tova_config* c, int* why) {
@@ -42,22 +42,13 @@ bool config_ok(const tova_config* c, int* why) {
   return true;
 }
 
-// Upper bound of combine CTAs per sequence: enough to score 128 candidates each,
-// and enough to spread a small batch over the whole GPU.
-constexpr int NX_SPREAD = 512;
-int nx_limit(int capacity) {
-  const int by_rows = (capacity + 1 + tova::COMBINE_THREADS - 1) / tova::COMBINE_THREADS;
-  return by_rows > NX_SPREAD ? by_rows : NX_SPREAD;
-}
-
 Layout make_layout(const tova_config& c) {
   Layout L{};
   const size_t B = c.batch, H = c.n_q_heads, Hkv = c.n_kv_heads, D = c.head_dim, cap = c.capacity;
   const size_t E = c.dtype == TOVA_DTYPE_BF16 ? 2 : 4;
   L.ld = (int)((cap + 1 + 3) / 4 * 4);
   // scratch is sized for the smallest chunk (32 rows per split warp)
-  L.pc = (int)((cap + tova::TILE_ROWS - 1) / tova::TILE_ROWS) + 1;
-  L.nx_max = nx_limit(c.capacity);
+  L.pc = (int)((cap + tova::MIN_CHUNK_ROWS - 1) / tova::MIN_CHUNK_ROWS) + 1;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   L.K = take(B * Hkv * cap * D * E);
@@ -67,8 +58,6 @@ Layout make_layout(const tova_config& c) {
   L.logits = take(B * H * L.ld * 4);
   L.part_ml = take(B * H * L.pc * 8);
   L.part_acc = take(B * H * (size_t)(L.pc - 1) * D * 4);
-  L.blockmin = take(B * L.nx_max * 16);
-  L.counter = take(B * 4);
   L.status = take(4);
   L.cur_pos = take(4);
   L.st_q = take(B * H * D * E);
@@ -105,13 +94,13 @@ inline int unit_heads(int G) { return G <= 1 ? 1 : G == 2 ? 2 : G <= 4 ? 4 : tov
 inline size_t split_smem_bytes(const tova_config& cfg) {
   const size_t rb = (size_t)cfg.head_dim * (cfg.dtype == TOVA_DTYPE_BF16 ? 2 : 4);
   const int gu = unit_heads(cfg.n_q_heads / cfg.n_kv_heads);
-  return (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + sizeof(float) * gu * 32;
+  return (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + sizeof(float) * gu * tova::TILE_ROWS;
 }
 
 template <typename T, int D, int GU, int GB>
 cudaError_t launch_split(int dev, const StepParams& p, dim3 grid, cudaStream_t st) {
   const size_t rb = (size_t)D * sizeof(T);
-  const size_t smem = (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + sizeof(float) * GU * 32;
+  const size_t smem = (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + sizeof(float) * GU * tova::TILE_ROWS;
   auto kern = tova::tova_split_kernel<T, D, GU, GB>;
   static bool attr_set[64] = {};  // per instantiation and device: the attribute is per function
   if (!attr_set[dev & 63]) {
@@ -145,21 +134,54 @@ cudaError_t launch_split_g(int dev, int G, const StepParams& p, dim3 grid, cudaS
   }
 }
 
-template <typename T, int D>
-cudaError_t launch_combine(const StepParams& p, cudaStream_t st) {
-  const size_t smem = sizeof(float) * (2 * (size_t)p.H + tova::COMBINE_THREADS);
-  auto kern = tova::tova_combine_kernel<T, D>;
+// Dynamic shared memory of the combine kernel: all (max, sum) partials of a
+// sequence, per-head max and 1/sum, one float per thread, and the new token's
+// rows when they are small enough to be staged.
+inline size_t combine_smem_bytes(int H, int n_partials, int threads, size_t row_bytes) {
+  size_t b = sizeof(float) * (2 * (size_t)H * n_partials + 2 * (size_t)H + threads) + 16;
+  if (2 * row_bytes <= (size_t)tova::COMBINE_ROW_STAGE_BYTES) b += 2 * row_bytes;
+  return b;
+}
+constexpr size_t COMBINE_SMEM_LIMIT = 160 * 1024;
+// upper bound used when choosing chunk sizes (largest CTA, rows staged)
+inline size_t combine_smem_bound(int H, int n_partials) {
+  return combine_smem_bytes(H, n_partials, tova::COMBINE_THREADS_LARGE, 0) + tova::COMBINE_ROW_STAGE_BYTES;
+}
+
+template <typename T, int D, int CT>
+cudaError_t launch_combine_ct(int dev, const StepParams& p, cudaStream_t st) {
+  const size_t row_bytes = (size_t)p.Hkv * D * sizeof(T);
+  const size_t smem = combine_smem_bytes(p.H, p.n_chunks + 1, CT, row_bytes);
+  auto kern = tova::tova_combine_kernel<T, D, CT>;
+  static bool attr_set[64] = {};
+  if (!attr_set[dev & 63]) {
+    cudaError_t e =
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)COMBINE_SMEM_LIMIT);
+    if (e != cudaSuccess) return e;
+    attr_set[dev & 63] = true;
+  }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(p.nx, p.B);
-  cfg.blockDim = dim3(tova::COMBINE_THREADS);
-  cfg.dynamicSmemBytes = smem;  // H <= 4096: at most 33 KiB, below the default limit
+  cfg.blockDim = dim3(CT);
+  cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
+  at[1].id = cudaLaunchAttributeClusterDimension;  // the CTAs of one sequence form a cluster
+  at[1].val.clusterDim.x = p.nx;
+  at[1].val.clusterDim.y = 1;
+  at[1].val.clusterDim.z = 1;
   cfg.attrs = at;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
+template <typename T, int D>
+cudaError_t launch_combine(int dev, const StepParams& p, cudaStream_t st) {
+  return p.combine_threads == tova::COMBINE_THREADS_LARGE
+             ? launch_combine_ct<T, D, tova::COMBINE_THREADS_LARGE>(dev, p, st)
+             : launch_combine_ct<T, D, tova::COMBINE_THREADS_SMALL>(dev, p, st);
 }
 
 template <typename T, int D>
@@ -167,7 +189,7 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st) {
   dim3 grid(p.n_chunks > 0 ? p.n_chunks : 1, p.Hkv * p.hgroups, p.B);
   cudaError_t e = launch_split_g<T, D>(c->device, p.G, p, grid, st);
   if (e != cudaSuccess) return e;
-  e = launch_combine<T, D>(p, st);
+  e = launch_combine<T, D>(c->device, p, st);
   if (e != cudaSuccess) return e;
   c->launches += 2;
   return cudaSuccess;
@@ -187,13 +209,14 @@ int pick_chunk_rows(const tova_config& cfg, int sm_count) {
   const long long hgroups = (G + unit_heads(G) - 1) / unit_heads(G);
   const long long pairs = (long long)cfg.batch * cfg.n_kv_heads * hgroups;
   long long best_cost = -1;
-  int best = 32;
-  for (int cr = 32; cr <= 8192; cr *= 2) {
+  int best = -1;  // no chunk size keeps the combine kernel's shared memory within its limit
+  for (int cr = tova::MIN_CHUNK_ROWS; cr <= 8192; cr *= 2) {
     const long long chunks = (cfg.capacity + (long long)cr - 1) / cr;
     const long long units = pairs * chunks;
     const long long rounds = (units + slots - 1) / slots;
     const long long rows = cr < cfg.capacity ? cr : cfg.capacity;
     const long long cost = rounds * (rows + 24);
+    if (combine_smem_bound(cfg.n_q_heads, (int)chunks + 1) > COMBINE_SMEM_LIMIT) continue;
     if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best = cr; }
     if (cr >= cfg.capacity) break;
   }
@@ -201,7 +224,7 @@ int pick_chunk_rows(const tova_config& cfg, int sm_count) {
 }
 
 // Launch geometry of one step for n live rows.
-void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows, int sm_count, int nx_max) {
+void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows) {
   p.B = cfg.batch; p.H = cfg.n_q_heads; p.Hkv = cfg.n_kv_heads; p.G = cfg.n_q_heads / cfg.n_kv_heads;
   p.cap = cfg.capacity;
   p.n = n;
@@ -209,16 +232,22 @@ void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows,
   p.n_chunks = (n + chunk_rows - 1) / chunk_rows;
   p.hgroups = (p.G + unit_heads(p.G) - 1) / unit_heads(p.G);
   p.do_evict = (n == cfg.capacity) ? 1 : 0;
-  // combine CTAs per sequence: about two per SM over the batch, at least enough
-  // to give every CTA no more than 128 candidates
-  int nx = (2 * sm_count + cfg.batch - 1) / cfg.batch;
-  const int need = p.do_evict ? (n + 1 + tova::COMBINE_THREADS - 1) / tova::COMBINE_THREADS : 1;
-  if (nx < need) nx = need;
-  if (nx > nx_max) nx = nx_max;
-  const int items = cfg.n_q_heads * cfg.head_dim;
-  if (!p.do_evict && nx > items / 32) nx = items / 32 > 0 ? items / 32 : 1;
-  if (p.do_evict && nx > n + 1) nx = n + 1;
+  // Combine CTAs per sequence (one cluster).  A small batch gets 512-thread CTAs
+  // (more loads in flight per sequence, one CTA per SM is enough); a large one
+  // gets 256-thread CTAs, four to an SM.  Per thread: about one output element
+  // and at most LG logits per pass.
+  const int sm_guess = 148;
+  const bool big = (long long)cfg.batch * tova::COMBINE_CLUSTER_MAX <= sm_guess;
+  const int ct = big ? tova::COMBINE_THREADS_LARGE : tova::COMBINE_THREADS_SMALL;
+  const int lg = big ? 16 : 8;
+  const long long items = (long long)cfg.n_q_heads * cfg.head_dim;
+  int nx = (int)((items + ct - 1) / ct);
+  const long long score_loads = (long long)(n + 1) * cfg.n_q_heads;
+  const int by_scores = (int)((score_loads + (long long)lg * ct - 1) / ((long long)lg * ct));
+  if (p.do_evict && nx < by_scores) nx = by_scores;
+  if (nx > tova::COMBINE_CLUSTER_MAX) nx = tova::COMBINE_CLUSTER_MAX;
   if (nx < 1) nx = 1;
+  p.combine_threads = ct;
   p.nx = nx;
   p.cand_per_cta = (n + 1 + nx - 1) / nx;
 }
@@ -237,13 +266,11 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
   p.logits = reinterpret_cast<float*>(base + c->lay.logits);
   p.part_ml = reinterpret_cast<float2*>(base + c->lay.part_ml);
   p.part_acc = reinterpret_cast<float*>(base + c->lay.part_acc);
-  p.blockmin = reinterpret_cast<float4*>(base + c->lay.blockmin);
-  p.counter = reinterpret_cast<unsigned*>(base + c->lay.counter);
   p.status = reinterpret_cast<int32_t*>(base + c->lay.status);
   p.cur_pos = reinterpret_cast<int32_t*>(base + c->lay.cur_pos);
   p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.evicted = evicted_pos; p.pos_t = pos;
   p.ld = c->lay.ld; p.pc = c->lay.pc;
-  fill_geometry(p, cfg, n, c->chunk_rows, c->sm_count, c->lay.nx_max);
+  fill_geometry(p, cfg, n, c->chunk_rows);
   p.scale2 = c->scale2;
   cudaError_t e;
   if (cfg.dtype == TOVA_DTYPE_BF16) {
@@ -301,6 +328,7 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   c->sm_count = sms;
   c->device = dev;
   c->chunk_rows = pick_chunk_rows(*cfg, sms);
+  if (c->chunk_rows < 0) { delete c; return TOVA_ERR_UNSUPPORTED; }
   c->scale2 = c->cfg.sm_scale * 1.4426950408889634f;
   c->elem = cfg->dtype == TOVA_DTYPE_BF16 ? 2 : 4;
   c->row_bytes = c->elem * cfg->head_dim;
@@ -311,7 +339,7 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   const unsigned blocks = (unsigned)((n + threads - 1) / threads);
   tova::tova_init_kernel<<<blocks, threads, 0, st>>>(
       reinterpret_cast<int32_t*>(c->base + lay.pos), reinterpret_cast<int32_t*>(c->base + lay.len),
-      reinterpret_cast<unsigned*>(c->base + lay.counter), reinterpret_cast<int32_t*>(c->base + lay.status),
+      reinterpret_cast<int32_t*>(c->base + lay.status),
       reinterpret_cast<int32_t*>(c->base + lay.cur_pos), cfg->batch, cfg->capacity);
   if (cudaGetLastError() != cudaSuccess) { delete c; return TOVA_ERR_CUDA; }
   c->launches += 1;
@@ -321,8 +349,10 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
 
 int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows) {
   if (!c) return TOVA_ERR_NULL;
-  if (rows == 0) { c->chunk_rows = pick_chunk_rows(c->cfg, c->sm_count); return TOVA_OK; }
-  if (rows < 32 || rows > 8192 || rows % tova::TILE_ROWS != 0) return TOVA_ERR_BAD_SHAPE;
+  if (rows == 0) { c->chunk_rows = pick_chunk_rows(c->cfg, c->sm_count); return TOVA_OK; }  // fits: init checked
+  if (rows < tova::MIN_CHUNK_ROWS || rows > 8192 || rows % tova::MIN_CHUNK_ROWS != 0) return TOVA_ERR_BAD_SHAPE;
+  const int chunks = (c->cfg.capacity + rows - 1) / rows;
+  if (combine_smem_bound(c->cfg.n_q_heads, chunks + 1) > COMBINE_SMEM_LIMIT) return TOVA_ERR_BAD_SHAPE;
   c->chunk_rows = rows;
   return TOVA_OK;
 }
@@ -447,8 +477,8 @@ struct StaticDevice {
 StaticDevice g_static_dev[64] = {};
 
 struct StaticLayout {
-  size_t logits, part_ml, part_acc, blockmin, control, total;
-  int ld, pc, nx_max;
+  size_t logits, part_ml, part_acc, control, total;
+  int ld, pc;
 };
 
 StaticLayout make_static_layout(const tova_config& c, int chunk_rows) {
@@ -456,15 +486,12 @@ StaticLayout make_static_layout(const tova_config& c, int chunk_rows) {
   const size_t B = c.batch, H = c.n_q_heads, D = c.head_dim, cap = c.capacity;
   L.ld = (int)((cap + 1 + 3) / 4 * 4);
   L.pc = (int)((cap + chunk_rows - 1) / chunk_rows) + 1;
-  L.nx_max = 64 > (int)((cap + 1 + tova::COMBINE_THREADS - 1) / tova::COMBINE_THREADS)
-                 ? 64 : (int)((cap + 1 + tova::COMBINE_THREADS - 1) / tova::COMBINE_THREADS);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
-  L.control = take(B * 4 /*tickets*/ + B * 4 /*len*/ + 8 /*status, cur_pos*/);
+  L.control = take(B * 4 /*len*/ + 8 /*status, cur_pos*/);
   L.logits = take(B * H * L.ld * 4);
   L.part_ml = take(B * H * L.pc * 8);
   L.part_acc = take(B * H * (size_t)(L.pc - 1) * D * 4);
-  L.blockmin = take(B * L.nx_max * 16);
   L.total = off;
   return L;
 }
@@ -498,30 +525,29 @@ extern "C" int tova_decode_step_static(const tova_config* cfg, void* K, void* V,
   }
 
   const int chunk_rows = pick_chunk_rows(*cfg, sd.sm_count);
+  if (chunk_rows < 0) return TOVA_ERR_UNSUPPORTED;
   const StaticLayout lay = make_static_layout(*cfg, chunk_rows);
   if (lay.total > STATIC_SCRATCH_BYTES) return TOVA_ERR_STATIC_LIMIT;
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   unsigned char* base = sd.scratch;
   const size_t B = cfg->batch;
-  // tickets and status must start at zero; the array keeps the previous call's contents
-  if (cudaMemsetAsync(base + lay.control, 0, B * 8 + 8, st) != cudaSuccess) return TOVA_ERR_CUDA;
+  // the status word must start at zero; the array keeps the previous call's contents
+  if (cudaMemsetAsync(base + lay.control, 0, B * 4 + 8, st) != cudaSuccess) return TOVA_ERR_CUDA;
 
   StepParams p{};
   p.K = K;
   p.V = V;
   p.pos = positions;
-  p.counter = reinterpret_cast<unsigned*>(base + lay.control);
-  p.len = reinterpret_cast<int32_t*>(base + lay.control + B * 4);
-  p.status = reinterpret_cast<int32_t*>(base + lay.control + B * 8);
+  p.len = reinterpret_cast<int32_t*>(base + lay.control);
+  p.status = reinterpret_cast<int32_t*>(base + lay.control + B * 4);
   p.cur_pos = p.status + 1;
   p.logits = reinterpret_cast<float*>(base + lay.logits);
   p.part_ml = reinterpret_cast<float2*>(base + lay.part_ml);
   p.part_acc = reinterpret_cast<float*>(base + lay.part_acc);
-  p.blockmin = reinterpret_cast<float4*>(base + lay.blockmin);
   p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.evicted = evicted_pos; p.pos_t = pos;
   p.ld = lay.ld; p.pc = lay.pc;
-  fill_geometry(p, *cfg, n_live, chunk_rows, sd.sm_count, lay.nx_max);
+  fill_geometry(p, *cfg, n_live, chunk_rows);
   const float scale = cfg->sm_scale == 0.f ? 1.f / std::sqrt((float)cfg->head_dim) : cfg->sm_scale;
   p.scale2 = scale * 1.4426950408889634f;
 

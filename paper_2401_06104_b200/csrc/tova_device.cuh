@@ -88,6 +88,16 @@ __device__ __forceinline__ void pdl_launch_dependents() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// Cluster barrier, split in its two halves: a CTA that only needs to publish
+// (stores into a peer's shared memory) arrives and leaves; the reader waits.
+// Every thread of every CTA of the cluster must arrive exactly once.
+__device__ __forceinline__ void cluster_arrive_release() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait_acquire() {
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // 16 bytes of storage -> floats (8 bf16 or 4 fp32).
 template <typename T>
 struct Vec16;

@@ -16,14 +16,20 @@
 // weights are exp2(s2 - max2).
 #pragma once
 
+#include <cooperative_groups.h>
+
 #include "tova_device.cuh"
 
 namespace tova {
 
-constexpr int TILE_ROWS = 32;       // cache rows per pipeline stage of the split kernel
+constexpr int TILE_ROWS = 16;       // cache rows per pipeline stage of the split kernel
 constexpr int SPLIT_BUFFERS = 3;    // tile buffers of a split warp's ring (K and V tiles alternate)
 constexpr int MAX_UNIT_HEADS = 8;   // query heads one split warp carries
-constexpr int COMBINE_THREADS = 128;
+constexpr int COMBINE_THREADS_SMALL = 256;  // combine CTA size when many CTAs are in flight
+constexpr int COMBINE_THREADS_LARGE = 512;  // ... when the batch is small: more loads in flight per sequence
+constexpr int COMBINE_ROW_STAGE_BYTES = 16 * 1024;  // new-token rows (k and v) staged in shared memory up to this size
+constexpr int COMBINE_CLUSTER_MAX = 8;  // CTAs per sequence in the combine kernel (portable cluster size)
+constexpr int MIN_CHUNK_ROWS = 32;      // smallest chunk the scratch is sized for
 
 struct StepParams {
   // state
@@ -35,8 +41,6 @@ struct StepParams {
   float* logits;      // [B,H,ld]   base-2 logits of candidates 0..n (n = the new token)
   float2* part_ml;    // [B,H,pc]   (max2, sum) per chunk; entry n_chunks = the new token
   float* part_acc;    // [B,H,pc-1,D] un-normalised weighted V sums per chunk
-  float4* blockmin;   // [B,nx_max] (lowest mean weight, its candidate index, its position, -)
-  unsigned* counter;  // [B] tickets of the combine CTAs
   int32_t* status;    // [1]
   int32_t* cur_pos;   // [1] position of the token being processed (set by the split kernel)
   // this step
@@ -52,8 +56,9 @@ struct StepParams {
   int32_t n_chunks;   // ceil(n / chunk_rows)
   int32_t chunk_rows; // rows per split warp, a multiple of TILE_ROWS
   int32_t hgroups;    // ceil(G / heads per split warp)
-  int32_t nx;         // combine CTAs per sequence
-  int32_t cand_per_cta;  // candidates scored per combine CTA (<= COMBINE_THREADS)
+  int32_t nx;         // combine CTAs per sequence = cluster size (1..COMBINE_CLUSTER_MAX)
+  int32_t cand_per_cta;  // candidates scored per combine CTA
+  int32_t combine_threads;  // COMBINE_THREADS_SMALL or COMBINE_THREADS_LARGE
   int32_t do_evict;   // n == cap and the policy is on
   float scale2;       // sm_scale * log2(e)
 };
@@ -63,27 +68,28 @@ struct StepParams {
 // ---------------------------------------------------------------------------
 // grid = (max(n_chunks,1), Hkv*hgroups, B), block = one warp.  The warp owns
 // rows [c*chunk_rows, +chunk_rows) of one KV head and up to GU query heads of
-// its group.  The operand tiles K_0 V_0 K_1 V_1 ... (32 rows each) travel through
+// its group.  The operand tiles K_0 V_0 K_1 V_1 ... (16 rows each) travel through
 // a ring of SPLIT_BUFFERS buffers: lane 0 issues the copy of operand tile u+NB
 // into a buffer as soon as the warp has consumed tile u from it, so nothing but
 // this warp ever waits on these barriers.
 // Every lane reads 16 bytes of a row; LPR lanes cover a row, so the warp reads
-// RPW = 32/LPR rows per pass and a tile takes LPR passes.
+// RPW = 32/LPR rows per pass and a tile takes NP = 16/RPW = LPR/2 passes.
 template <typename T, int D, int GU, int GB>
 __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
   constexpr int EPL = Vec16<T>::N;          // elements per lane
   constexpr int RB = D * (int)sizeof(T);    // bytes per row
   constexpr int LPR = RB / 16;              // lanes per row
   constexpr int RPW = 32 / LPR;             // rows per pass
-  constexpr int NP = LPR;                   // passes per tile (RPW * NP = 32)
+  constexpr int NP = TILE_ROWS / RPW;       // passes per tile (= LPR / 2)
   constexpr int TILE_BYTES = TILE_ROWS * RB;
   constexpr int NB = SPLIT_BUFFERS;
   static_assert(LPR >= 8 && LPR <= 32, "row must be 128..512 bytes");
   static_assert(GU % GB == 0, "head block must divide the unit");
+  static_assert(NP * 2 == LPR, "a tile is half as many passes as lanes per row");
 
   extern __shared__ __align__(128) unsigned char smem_raw[];
   unsigned char* ring = smem_raw;                                    // [NB][TILE_BYTES]
-  float* w_p = reinterpret_cast<float*>(smem_raw + NB * TILE_BYTES); // [GU][32] weights of a tile
+  float* w_p = reinterpret_cast<float*>(smem_raw + NB * TILE_BYTES); // [GU][16] weights of a tile
   __shared__ __align__(8) uint64_t bars[NB];
 
   const int lane = threadIdx.x;
@@ -96,7 +102,10 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
   const int row_begin = c * p.chunk_rows;
   const int rows = min(max(p.n - row_begin, 0), p.chunk_rows);
   const int ntiles = (rows + TILE_ROWS - 1) / TILE_ROWS;
-  const int my_row = lig * RPW + sub;                       // tile row this lane ends up owning
+  // After the transposing reduction lanes lig and lig^NP both hold the logit of
+  // tile row (lig % NP) * RPW + sub; the lower one of the pair "owns" it.
+  const int my_row = (lig % NP) * RPW + sub;
+  const bool owner = lig < NP;
 
   if (lane == 0) {
 #pragma unroll
@@ -180,7 +189,7 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
     const unsigned char* kt = ring + (size_t)(uk % NB) * TILE_BYTES;
     const unsigned char* vt = ring + (size_t)(uv % NB) * TILE_BYTES;
 
-    // ---- logits of the tile's 32 rows, GB heads at a time --------------------
+    // ---- logits of the tile's rows, GB heads at a time -------------------------
     if (!warp_wait(&bars[uk % NB], (uint32_t)(uk / NB) & 1u)) { failed = true; break; }
     float s[GU];
 #pragma unroll
@@ -204,7 +213,8 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
       }
 #pragma unroll
       for (int gb = 0; gb < GB; ++gb) {
-        const float v = transpose_reduce<NP>(part[gb], lig) * p.scale2;
+        float v = transpose_reduce<NP>(part[gb], lig % NP);
+        v = (v + __shfl_xor_sync(0xffffffffu, v, NP)) * p.scale2;
         // rows past the live range hold stale shared memory: mask them out
         s[g0 + gb] = (my_row < nvalid) ? v : -INFINITY;
       }
@@ -219,16 +229,17 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
     // ---- online soft-max update, weights of the tile to shared memory --------
 #pragma unroll
     for (int g = 0; g < GU; ++g) {
-      if (g < g_cnt && my_row < nvalid)
+      if (g < g_cnt && owner && my_row < nvalid)
         p.logits[(bh0 + g) * p.ld + row_begin + t * TILE_ROWS + my_row] = s[g];
       const float m_new = fmaxf(m[g], warp_max(s[g]));
       const float corr = exp2_diff(m[g], m_new);
       const float e = exp2_diff(s[g], m_new);
-      l[g] = fmaf(l[g], corr, warp_sum(e));
+      // l stays a per-lane partial sum (rows this lane owns); it is folded once at the end
+      l[g] = fmaf(l[g], corr, owner ? e : 0.f);
       m[g] = m_new;
 #pragma unroll
       for (int k = 0; k < EPL; ++k) acc[g][k] *= corr;
-      w_p[g * 32 + my_row] = e;
+      if (owner) w_p[g * TILE_ROWS + my_row] = e;
     }
     __syncwarp();
 
@@ -242,7 +253,7 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
         Vec16<T>::unpack(*reinterpret_cast<const uint4*>(vt + (size_t)r * RB + lig * 16), vf);
 #pragma unroll
         for (int g = 0; g < GU; ++g) {
-          const float w = w_p[g * 32 + r];
+          const float w = w_p[g * TILE_ROWS + r];
 #pragma unroll
           for (int e = 0; e < EPL; ++e) acc[g][e] = fmaf(w, vf[e], acc[g][e]);
         }
@@ -270,6 +281,7 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
     for (int e = 0; e < EPL; ++e)
 #pragma unroll
       for (int o = LPR; o < 32; o <<= 1) acc[g][e] += __shfl_xor_sync(0xffffffffu, acc[g][e], o);
+    l[g] = warp_sum(l[g]);
     if (g < g_cnt && sub == 0) {
       float* dst = p.part_acc + ((bh0 + g) * (size_t)(p.pc - 1) + c) * D + lig * EPL;
 #pragma unroll
@@ -284,56 +296,146 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
 // ---------------------------------------------------------------------------
 // combine-and-evict kernel
 // ---------------------------------------------------------------------------
-// grid = (nx, B), block = COMBINE_THREADS.  Built for few dependent memory
-// round trips, since the whole step lasts microseconds:
-//   1. every CTA rebuilds each head's global (max2, 1/sum) from the chunk
-//      partials (one round trip);
-//   2. CTA x writes its 1/nx share of the H*D attention outputs (Eq. 7), every
-//      thread merging the chunk partials of one (head, dim);
+// grid = (nx, B) with the nx CTAs of a sequence forming one thread-block cluster
+// (nx <= 8), block = CT threads.  The step lasts microseconds, so the
+// kernel is built around dependent memory round trips, not throughput: every
+// global load a thread will need (chunk partials, logits of its candidates,
+// weighted V sums of its output element, the candidate's position, the words of
+// the new token's row) is issued up front into registers, in one round trip.
+//   1. each CTA rebuilds every head's global (max2, 1/sum) from the partials;
+//   2. CTA x writes its 1/nx share of the H*D attention outputs (Eq. 7);
 //   3. CTA x scores candidates [x*cand_per_cta, +cand_per_cta): the mean over
-//      heads of the soft-max weights (Algorithm 1).  Threads split the heads of
-//      a candidate HS ways and the partial sums are added in a fixed order;
-//      the CTA leaves its lowest (value, index, position);
-//   4. the last CTA of the sequence to finish (atomic ticket, nobody waits)
-//      takes the overall arg-min - lowest index on ties - and replaces that row
-//      by the new token in K, V and the position table (Eq. 9, in place).
-// smem: float hM[H], hInvL[H], sc[COMBINE_THREADS].
-template <typename T, int D>
-__global__ void __launch_bounds__(COMBINE_THREADS) tova_combine_kernel(const StepParams p) {
+//      heads of the soft-max weights (Algorithm 1), in a fixed order, and sends
+//      its lowest (value, index, position) to CTA 0's shared memory;
+//   4. after one cluster barrier CTA 0 takes the overall arg-min - lowest index
+//      on ties - and replaces that row by the new token in K, V and the position
+//      table (Eq. 9, in place).  No global atomics, no CTA waits on a flag.
+// smem: float2 pml[H][np]; float hM[H], hInvL[H], sc[CT]; then, in
+// CTA 0 only, the new token's k and v rows of all KV heads (bulk-copied in at
+// the start when they fit COMBINE_ROW_STAGE_BYTES each).
+template <typename T, int D, int CT>
+__global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_combine_kernel(const StepParams p) {
+  namespace cg = cooperative_groups;
+  constexpr bool BIG = (CT == COMBINE_THREADS_LARGE);
+  constexpr int ML = BIG ? 4 : 2;    // partial pairs prefetched per thread
+  constexpr int LG = BIG ? 16 : 8;   // logits prefetched per thread
+  constexpr int AC = BIG ? 8 : 4;    // weighted V sums prefetched per thread
   extern __shared__ __align__(16) float csm[];
-  float* hM = csm;                 // [H]
-  float* hInvL = csm + p.H;        // [H]
-  float* sc = csm + 2 * p.H;       // [COMBINE_THREADS] partial head sums
-  __shared__ float red_v[COMBINE_THREADS / 32];
-  __shared__ int red_i[COMBINE_THREADS / 32];
-  __shared__ int red_p[COMBINE_THREADS / 32];
-  __shared__ int s_last;
+  const int np = p.n_chunks + 1;   // partials per head: the chunks, then the new token
+  float2* pml = reinterpret_cast<float2*>(csm);                  // [H][np]
+  float* hM = csm + 2 * (size_t)p.H * np;                        // [H]
+  float* hInvL = hM + p.H;                                       // [H]
+  float* sc = hInvL + p.H;                                       // [CT]
+  unsigned char* row_stage = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(sc + CT) + 15) & ~uintptr_t(15));     // [2][Hkv*D*sizeof(T)]
+  __shared__ __align__(8) uint64_t row_bar;
+  __shared__ float red_v[CT / 32];
+  __shared__ int red_i[CT / 32];
+  __shared__ int red_p[CT / 32];
+  __shared__ float4 best_of[COMBINE_CLUSTER_MAX];  // CTA 0's copy collects every CTA's minimum
+  __shared__ int s_victim;
 
   const int x = blockIdx.x, b = blockIdx.y;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int np = p.n_chunks + 1;  // partials per head: the chunks, then the new token
+
+  // geometry (no memory access)
+  int wp = 1;                      // candidates per pass, a power of two <= CT
+  while (wp < p.cand_per_cta && wp < CT) wp <<= 1;
+  const int hs_n = CT / wp;        // threads sharing one candidate's heads
+  const int jl = tid % wp, hs = tid / wp;
+  const int j_begin = x * p.cand_per_cta;
+  const int j_end = min(j_begin + p.cand_per_cta, p.n + 1);
+  const int items = p.H * D;
+  const int per = (items + p.nx - 1) / p.nx;
+  const int it_end = min(items, (x + 1) * per);
+  const int it0 = x * per + tid;
+  constexpr int RB16 = D * (int)sizeof(T) / 16;  // 16-byte words per row
+  const int row_words = p.Hkv * RB16;
+  const int total_ml = p.H * np;
+  const uint32_t row_bytes = (uint32_t)row_words * 16u;          // all KV heads of one operand
+  const bool staged = (x == 0) && 2 * row_bytes <= (uint32_t)COMBINE_ROW_STAGE_BYTES;
+  if (staged && tid == 0) {
+    mbar_init(&row_bar, 1);
+    mbar_fence_init();
+  }
 
   pdl_wait();
   pdl_launch_dependents();
-  const int pos_t = *p.cur_pos;
+  if (staged && tid == 0) {        // the new token's rows, on their way while everything else happens
+    mbar_expect_tx(&row_bar, 2 * row_bytes);
+    bulk_g2s(row_stage, static_cast<const unsigned char*>(p.k_new) + (size_t)b * row_bytes, row_bytes, &row_bar);
+    bulk_g2s(row_stage + row_bytes, static_cast<const unsigned char*>(p.v_new) + (size_t)b * row_bytes, row_bytes,
+             &row_bar);
+  }
 
-  // ---- 1. global max and sum of every head ------------------------------------
-  for (int h = warp; h < p.H; h += COMBINE_THREADS / 32) {
-    const float2* ml = p.part_ml + ((size_t)b * p.H + h) * p.pc;
-    float M = -INFINITY, L = 0.f;
-    if (np <= 32) {
-      const float2 e = (lane < np) ? ml[lane] : make_float2(-INFINITY, 0.f);
-      M = warp_max(e.x);
-      L = warp_sum(e.y * exp2_diff(e.x, M));
-    } else {
-      for (int i = lane; i < np; i += 32) M = fmaxf(M, ml[i].x);
-      M = warp_max(M);
-      for (int i = lane; i < np; i += 32) {
-        const float2 e = ml[i];
-        L = fmaf(e.y, exp2_diff(e.x, M), L);
-      }
-      L = warp_sum(L);
+  // ---- 0. every load this thread needs, issued back to back ---------------------
+  const int pos_t = *p.cur_pos;
+  float2 r_ml[ML];
+#pragma unroll
+  for (int u = 0; u < ML; ++u) {
+    const int i = tid + u * CT;
+    r_ml[u] = (i < total_ml) ? p.part_ml[((size_t)b * p.H + i / np) * p.pc + i % np] : make_float2(0.f, 0.f);
+  }
+  float r_lg[LG];
+  int r_pos = pos_t;               // position held by this thread's first candidate
+  {
+    const int j = j_begin + jl;
+    const bool live = p.do_evict && j < j_end;
+    const float* lg = p.logits + (size_t)b * p.H * p.ld + j;
+#pragma unroll
+    for (int u = 0; u < LG; ++u) {
+      const int h = hs + u * hs_n;
+      r_lg[u] = (live && h < p.H) ? lg[(size_t)h * p.ld] : 0.f;
     }
+    if (live && hs == 0 && j < p.cap) r_pos = p.pos[(size_t)b * p.cap + j];
+  }
+  float r_acc[AC];
+  float r_vn = 0.f;
+  if (it0 < it_end) {
+    const int h = it0 / D, d = it0 % D;
+    const float* acc = p.part_acc + ((size_t)b * p.H + h) * (size_t)(p.pc - 1) * D + d;
+#pragma unroll
+    for (int u = 0; u < AC; ++u) r_acc[u] = (u < p.n_chunks) ? acc[(size_t)u * D] : 0.f;
+    r_vn = (float)static_cast<const T*>(p.v_new)[((size_t)b * p.Hkv + h / p.G) * D + d];
+  } else {
+#pragma unroll
+    for (int u = 0; u < AC; ++u) r_acc[u] = 0.f;
+  }
+
+  // Writes the new token's k and v into row `slot` of every KV head (CTA 0 only).
+  auto insert_row = [&](int slot) {
+    bool from_smem = staged;
+    if (staged && !mbar_wait_bounded(&row_bar, 0)) {
+      from_smem = false;           // fall back to reading the rows again
+      if (tid == 0) atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
+    }
+    const uint4* ks = from_smem ? reinterpret_cast<const uint4*>(row_stage)
+                                : static_cast<const uint4*>(p.k_new) + (size_t)b * row_words;
+    const uint4* vs = from_smem ? reinterpret_cast<const uint4*>(row_stage + row_bytes)
+                                : static_cast<const uint4*>(p.v_new) + (size_t)b * row_words;
+    for (int i = tid; i < row_words; i += CT) {
+      const size_t dst = (((size_t)b * p.Hkv + i / RB16) * p.cap + slot) * RB16 + i % RB16;
+      static_cast<uint4*>(p.K)[dst] = ks[i];
+      static_cast<uint4*>(p.V)[dst] = vs[i];
+    }
+  };
+
+  // ---- 1. partials to shared memory, global max and sum of every head ------------
+#pragma unroll
+  for (int u = 0; u < ML; ++u) {
+    const int i = tid + u * CT;
+    if (i < total_ml) pml[i] = r_ml[u];
+  }
+  for (int i = tid + ML * CT; i < total_ml; i += CT)
+    pml[i] = p.part_ml[((size_t)b * p.H + i / np) * p.pc + i % np];
+  __syncthreads();
+  for (int h = warp; h < p.H; h += CT / 32) {
+    const float2* ml = pml + (size_t)h * np;
+    float M = -INFINITY, L = 0.f;
+    for (int i = lane; i < np; i += 32) M = fmaxf(M, ml[i].x);
+    M = warp_max(M);
+    for (int i = lane; i < np; i += 32) L = fmaf(ml[i].y, exp2_diff(ml[i].x, M), L);
+    L = warp_sum(L);
     if (lane == 0) {
       hM[h] = M;
       hInvL[h] = 1.f / L;
@@ -341,39 +443,34 @@ __global__ void __launch_bounds__(COMBINE_THREADS) tova_combine_kernel(const Ste
   }
   __syncthreads();
 
-  // ---- 2. this CTA's share of the attention output -----------------------------
-  {
-    const int items = p.H * D;
-    const int per = (items + p.nx - 1) / p.nx;
-    const int end = min(items, (x + 1) * per);
-    for (int it = x * per + tid; it < end; it += COMBINE_THREADS) {
-      const int h = it / D, d = it % D;
-      const size_t bh = (size_t)b * p.H + h;
-      const float2* ml = p.part_ml + bh * p.pc;
-      const float* acc = p.part_acc + bh * (size_t)(p.pc - 1) * D + d;
-      const float M = hM[h], iL = hInvL[h];
-      float o = 0.f;
-#pragma unroll 4
+  // ---- 2. this CTA's share of the attention output --------------------------------
+  for (int it = it0; it < it_end; it += CT) {
+    const int h = it / D, d = it % D;
+    const size_t bh = (size_t)b * p.H + h;
+    const float2* ml = pml + (size_t)h * np;
+    const float* acc = p.part_acc + bh * (size_t)(p.pc - 1) * D + d;
+    const float M = hM[h];
+    float o = 0.f;
+    if (it == it0) {
+#pragma unroll
+      for (int u = 0; u < AC; ++u)
+        if (u < p.n_chunks) o = fmaf(r_acc[u], exp2_diff(ml[u].x, M), o);
+#pragma unroll 8
+      for (int i = AC; i < p.n_chunks; ++i) o = fmaf(acc[(size_t)i * D], exp2_diff(ml[i].x, M), o);
+      o = fmaf(r_vn, exp2_diff(ml[p.n_chunks].x, M), o);
+    } else {
+#pragma unroll 8
       for (int i = 0; i < p.n_chunks; ++i) o = fmaf(acc[(size_t)i * D], exp2_diff(ml[i].x, M), o);
-      const T* vn = static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + h / p.G) * D;
-      o = fmaf((float)vn[d], exp2_diff(ml[p.n_chunks].x, M), o);
-      p.out[bh * D + d] = o * iL;
+      const float vn = (float)static_cast<const T*>(p.v_new)[((size_t)b * p.Hkv + h / p.G) * D + d];
+      o = fmaf(vn, exp2_diff(ml[p.n_chunks].x, M), o);
     }
+    p.out[bh * D + d] = o * hInvL[h];
   }
-
-  constexpr int RB16 = D * (int)sizeof(T) / 16;  // 16-byte words per row
-  const int row_words = p.Hkv * RB16;
 
   if (!p.do_evict) {
     // g(t) = min(t, k) not yet reached: the new token takes the next free row.
     if (x == 0) {
-      for (int i = tid; i < row_words; i += COMBINE_THREADS) {
-        const int kvh = i / RB16, wd = i % RB16;
-        const size_t dst = (((size_t)b * p.Hkv + kvh) * p.cap + p.n) * RB16 + wd;
-        const size_t src = ((size_t)b * p.Hkv + kvh) * RB16 + wd;
-        static_cast<uint4*>(p.K)[dst] = static_cast<const uint4*>(p.k_new)[src];
-        static_cast<uint4*>(p.V)[dst] = static_cast<const uint4*>(p.v_new)[src];
-      }
+      insert_row(p.n);
       if (tid == 0) {
         p.pos[(size_t)b * p.cap + p.n] = pos_t;
         p.len[b] = p.n + 1;
@@ -383,31 +480,48 @@ __global__ void __launch_bounds__(COMBINE_THREADS) tova_combine_kernel(const Ste
     return;
   }
 
-  // ---- 3. head-averaged weight of this CTA's candidates ------------------------
-  // wp = cand_per_cta rounded up to a power of two; thread = (candidate jl, head slice hs)
-  int wp = 1;
-  while (wp < p.cand_per_cta) wp <<= 1;
-  const int hs_n = COMBINE_THREADS / wp;
-  const int jl = tid % wp, hs = tid / wp;
-  const int j = x * p.cand_per_cta + jl;
-  const bool live = (jl < p.cand_per_cta) && (j <= p.n);
-  float a = 0.f;
-  if (live) {
-    const float* lg = p.logits + (size_t)b * p.H * p.ld + j;
-#pragma unroll 4
-    for (int h = hs; h < p.H; h += hs_n) a = fmaf(exp2f(lg[(size_t)h * p.ld] - hM[h]), hInvL[h], a);
-  }
-  sc[tid] = a;
-  int cpos = pos_t;  // position held by the candidate (the new token holds pos_t)
-  if (hs == 0 && live && j < p.cap) cpos = p.pos[(size_t)b * p.cap + j];
-  __syncthreads();
+  // ---- 3. head-averaged weight of this CTA's candidates ---------------------------
+  // thread = (candidate jl of a pass, head slice hs); passes of wp candidates
   float val = INFINITY;
   int idx = 0x7fffffff;
-  if (hs == 0 && live) {
-    float tot = 0.f;
-    for (int k = 0; k < hs_n; ++k) tot += sc[k * wp + jl];
-    val = tot * (1.f / (float)p.H);
-    idx = j;
+  int cpos = pos_t;                // position held by the best candidate (the new token holds pos_t)
+  const float inv_h = 1.f / (float)p.H;
+  for (int j0 = j_begin; j0 < j_end; j0 += wp) {
+    const int j = j0 + jl;
+    const bool live = j < j_end;
+    float a = 0.f;
+    if (live) {
+      const float* lg = p.logits + (size_t)b * p.H * p.ld + j;
+      if (j0 == j_begin) {
+#pragma unroll
+        for (int u = 0; u < LG; ++u) {
+          const int h = hs + u * hs_n;
+          if (h < p.H) a = fmaf(exp2f(r_lg[u] - hM[h]), hInvL[h], a);
+        }
+#pragma unroll 8
+        for (int h = hs + LG * hs_n; h < p.H; h += hs_n) a = fmaf(exp2f(lg[(size_t)h * p.ld] - hM[h]), hInvL[h], a);
+      } else {
+#pragma unroll 16
+        for (int h = hs; h < p.H; h += hs_n) a = fmaf(exp2f(lg[(size_t)h * p.ld] - hM[h]), hInvL[h], a);
+      }
+    }
+    if (hs_n > 1) {                // uniform over the CTA
+      sc[tid] = a;
+      __syncthreads();
+      if (hs == 0) {
+        a = 0.f;
+        for (int k = 0; k < hs_n; ++k) a += sc[k * wp + jl];
+      }
+      __syncthreads();
+    }
+    if (hs == 0 && live) {
+      const float v = a * inv_h;
+      if (v < val) {               // passes go up in j: strict < keeps the lowest index
+        val = v;
+        idx = j;
+        cpos = (j0 == j_begin) ? r_pos : ((j < p.cap) ? p.pos[(size_t)b * p.cap + j] : pos_t);
+      }
+    }
   }
   // lowest (value, index) of the block
 #pragma unroll
@@ -419,26 +533,25 @@ __global__ void __launch_bounds__(COMBINE_THREADS) tova_combine_kernel(const Ste
   }
   if (lane == 0) { red_v[warp] = val; red_i[warp] = idx; red_p[warp] = cpos; }
   __syncthreads();
+  cg::cluster_group cluster = cg::this_cluster();
   if (tid == 0) {
-    for (int w = 1; w < COMBINE_THREADS / 32; ++w)
+    for (int w = 1; w < CT / 32; ++w)
       if (red_v[w] < val || (red_v[w] == val && red_i[w] < idx)) { val = red_v[w]; idx = red_i[w]; cpos = red_p[w]; }
-    p.blockmin[(size_t)b * p.nx + x] = make_float4(val, __int_as_float(idx), __int_as_float(cpos), 0.f);
-    __threadfence();
-    const unsigned t = atomicAdd(p.counter + b, 1u);
-    s_last = (t == (unsigned)p.nx - 1u);
+    // into CTA 0's shared memory (distributed shared memory store)
+    *cluster.map_shared_rank(&best_of[x], 0) = make_float4(val, __int_as_float(idx), __int_as_float(cpos), 0.f);
   }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
 
-  // ---- 4. last CTA of the sequence: arg-min over blocks, evict, insert ---------
+  // ---- 4. one cluster barrier; CTA 0 takes the arg-min, evicts, inserts -----------
+  __syncwarp();
+  cluster_arrive_release();        // orders the store above before the barrier completes
+  if (x != 0) return;              // peers are done: nobody reads their shared memory
+  cluster_wait_acquire();
   if (warp == 0) {
     float bv = INFINITY;
     int bi = 0x7fffffff, bp = pos_t;
-    for (int i = lane; i < p.nx; i += 32) {
-      const float4 e = __ldcg(p.blockmin + (size_t)b * p.nx + i);
-      const int ci = __float_as_int(e.y);
-      if (e.x < bv || (e.x == bv && ci < bi)) { bv = e.x; bi = ci; bp = __float_as_int(e.z); }
+    if (lane < p.nx) {
+      const float4 e = best_of[lane];
+      bv = e.x; bi = __float_as_int(e.y); bp = __float_as_int(e.z);
     }
 #pragma unroll
     for (int o = 16; o >= 1; o >>= 1) {
@@ -449,31 +562,23 @@ __global__ void __launch_bounds__(COMBINE_THREADS) tova_combine_kernel(const Ste
     }
     if (lane == 0) {
       if (bi < 0 || bi > p.cap) { atomicExch(p.status, DEV_ERR_BAD_VICTIM); bi = p.cap; bp = pos_t; }
-      red_i[0] = bi;
-      p.counter[b] = 0;  // ready for the next step
+      s_victim = bi;
       if (bi < p.cap) p.pos[(size_t)b * p.cap + bi] = pos_t;
       if (p.evicted) p.evicted[b] = bp;  // the new token's own position if it dropped itself
     }
   }
   __syncthreads();
-  const int victim = red_i[0];
-  if (victim < p.cap) {
-    for (int i = tid; i < row_words; i += COMBINE_THREADS) {
-      const int kvh = i / RB16, wd = i % RB16;
-      const size_t dst = (((size_t)b * p.Hkv + kvh) * p.cap + victim) * RB16 + wd;
-      const size_t src = ((size_t)b * p.Hkv + kvh) * RB16 + wd;
-      static_cast<uint4*>(p.K)[dst] = static_cast<const uint4*>(p.k_new)[src];
-      static_cast<uint4*>(p.V)[dst] = static_cast<const uint4*>(p.v_new)[src];
-    }
-  }
+  const int victim = s_victim;
+  if (victim < p.cap) insert_row(victim);
+  else if (staged) mbar_wait_bounded(&row_bar, 0);  // the staged copy must land before the CTA leaves
 }
 
-// Empty state at init: length 0, positions -1, counters and status 0.
-__global__ void tova_init_kernel(int32_t* pos, int32_t* len, unsigned* counter, int32_t* status,
-                                 int32_t* cur_pos, int B, int cap) {
+// Empty state at init: length 0, positions -1, status 0.
+__global__ void tova_init_kernel(int32_t* pos, int32_t* len, int32_t* status, int32_t* cur_pos, int B,
+                                 int cap) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < (size_t)B * cap) pos[i] = -1;
-  if (i < (size_t)B) { len[i] = 0; counter[i] = 0; }
+  if (i < (size_t)B) len[i] = 0;
   if (i == 0) { *status = 0; *cur_pos = -1; }
 }
 
