@@ -153,7 +153,9 @@ const char* tova_strerror(int status);
  * memory that every GPU context loading the library holds until it exits.
  *
  *   cfg                          shape, dtype, scale, policy (as for tova_cache_init)
- *   K, V [B,Hkv,capacity,D]      the caller's state, updated in place
+ *   K, V [B,Hkv,capacity,D]      the caller's state, updated in place (zero it before
+ *                                the first token: rows not yet written are read with
+ *                                weight zero and must hold finite numbers)
  *   positions [B,capacity] int32 slot table, updated in place (caller sets
  *                                unused slots to -1 before the first token)
  *   n_live                       rows each sequence holds before this token,

@@ -9,8 +9,10 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <type_traits>
 
 #include "tova_kernels.cuh"
+#include "tova_split_mma.cuh"
 
 namespace {
 
@@ -73,6 +75,8 @@ Layout make_layout(const tova_config& c) {
 
 struct tova_cache {
   tova_config cfg;
+  CUtensorMap map_k, map_v;  // tiled views of K and V for the tensor-core split kernel
+  bool use_mma;
   Layout lay;
   unsigned char* base;
   int32_t len;          // rows per sequence (host mirror; sequences move in lock step)
@@ -88,12 +92,23 @@ namespace {
 
 using tova::StepParams;
 
+// The tensor-core split kernel serves bf16 states whose query group is a real
+// contraction (G >= 4 rows of the 16-row MMA tile); everything else - MHA above
+// all, which does one flop per byte - runs on the plain ALUs.
+inline bool wants_mma(const tova_config& cfg) {
+  return cfg.dtype == TOVA_DTYPE_BF16 && cfg.n_q_heads / cfg.n_kv_heads >= 4;
+}
+
 // Heads one split warp carries (GU) and heads per pass over a tile (GB).
-inline int unit_heads(int G) { return G <= 1 ? 1 : G == 2 ? 2 : G <= 4 ? 4 : tova::MAX_UNIT_HEADS; }
+inline int unit_heads_alu(int G) { return G <= 1 ? 1 : G == 2 ? 2 : G <= 4 ? 4 : tova::MAX_UNIT_HEADS; }
+inline int unit_heads(const tova_config& cfg) {
+  return wants_mma(cfg) ? tova::MMA_UNIT_HEADS : unit_heads_alu(cfg.n_q_heads / cfg.n_kv_heads);
+}
 
 inline size_t split_smem_bytes(const tova_config& cfg) {
   const size_t rb = (size_t)cfg.head_dim * (cfg.dtype == TOVA_DTYPE_BF16 ? 2 : 4);
-  const int gu = unit_heads(cfg.n_q_heads / cfg.n_kv_heads);
+  if (wants_mma(cfg)) return (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + 1024;
+  const int gu = unit_heads(cfg);
   return (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + sizeof(float) * gu * tova::TILE_ROWS;
 }
 
@@ -126,7 +141,7 @@ cudaError_t launch_split(int dev, const StepParams& p, dim3 grid, cudaStream_t s
 template <typename T, int D>
 cudaError_t launch_split_g(int dev, int G, const StepParams& p, dim3 grid, cudaStream_t st) {
   constexpr bool wide = (D * sizeof(T) == 512);  // fp32, D = 128: 32 partial sums per head and lane
-  switch (unit_heads(G)) {
+  switch (unit_heads_alu(G)) {
     case 1: return launch_split<T, D, 1, 1>(dev, p, grid, st);
     case 2: return launch_split<T, D, 2, wide ? 1 : 2>(dev, p, grid, st);
     case 4: return launch_split<T, D, 4, wide ? 1 : 4>(dev, p, grid, st);
@@ -184,10 +199,42 @@ cudaError_t launch_combine(int dev, const StepParams& p, cudaStream_t st) {
              : launch_combine_ct<T, D, tova::COMBINE_THREADS_SMALL>(dev, p, st);
 }
 
+template <int D>
+cudaError_t launch_split_mma(int dev, const StepParams& p, const CUtensorMap& mk, const CUtensorMap& mv, dim3 grid,
+                             cudaStream_t st) {
+  const size_t smem = (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * D * 2 + 1024;
+  auto kern = tova::tova_split_mma_kernel<D>;
+  static bool attr_set[64] = {};
+  if (!attr_set[dev & 63]) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+    if (e != cudaSuccess) return e;
+    attr_set[dev & 63] = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, p, mk, mv);
+}
+
 template <typename T, int D>
 cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st) {
   dim3 grid(p.n_chunks > 0 ? p.n_chunks : 1, p.Hkv * p.hgroups, p.B);
-  cudaError_t e = launch_split_g<T, D>(c->device, p.G, p, grid, st);
+  cudaError_t e;
+  if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+    e = c->use_mma ? launch_split_mma<D>(c->device, p, c->map_k, c->map_v, grid, st)
+                   : launch_split_g<T, D>(c->device, p.G, p, grid, st);
+  } else {
+    e = launch_split_g<T, D>(c->device, p.G, p, grid, st);
+  }
   if (e != cudaSuccess) return e;
   e = launch_combine<T, D>(c->device, p, st);
   if (e != cudaSuccess) return e;
@@ -206,7 +253,7 @@ int pick_chunk_rows(const tova_config& cfg, int sm_count) {
   if (per_sm < 1) per_sm = 1;
   const long long slots = per_sm * sm_count;
   const int G = cfg.n_q_heads / cfg.n_kv_heads;
-  const long long hgroups = (G + unit_heads(G) - 1) / unit_heads(G);
+  const long long hgroups = (G + unit_heads(cfg) - 1) / unit_heads(cfg);
   const long long pairs = (long long)cfg.batch * cfg.n_kv_heads * hgroups;
   long long best_cost = -1;
   int best = -1;  // no chunk size keeps the combine kernel's shared memory within its limit
@@ -230,7 +277,7 @@ void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows)
   p.n = n;
   p.chunk_rows = chunk_rows;
   p.n_chunks = (n + chunk_rows - 1) / chunk_rows;
-  p.hgroups = (p.G + unit_heads(p.G) - 1) / unit_heads(p.G);
+  p.hgroups = (p.G + unit_heads(cfg) - 1) / unit_heads(cfg);
   p.do_evict = (n == cfg.capacity) ? 1 : 0;
   // Combine CTAs per sequence (one cluster).  A small batch gets 512-thread CTAs
   // (more loads in flight per sequence, one CTA per SM is enough); a large one
@@ -291,6 +338,34 @@ int check_step_args(const tova_cache* c, const void* q, const void* k, const voi
 
 }  // namespace
 
+// Tiled view of a [B*Hkv*capacity, D] bf16 matrix for the tensor-core split
+// kernel: boxes of 16 rows x 64 columns (128 bytes) with the 128-byte swizzle.
+// The driver's encoder is looked up through the runtime, so the library has no
+// link-time dependency on the driver.
+int encode_state_map(CUtensorMap* map, void* base, const tova_config& cfg) {
+  typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static encode_fn fn = nullptr;
+  if (!fn) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !sym)
+      return TOVA_ERR_CUDA;
+    fn = reinterpret_cast<encode_fn>(sym);
+  }
+  const cuuint64_t rows = (cuuint64_t)cfg.batch * cfg.n_kv_heads * cfg.capacity;
+  const cuuint64_t dims[2] = {(cuuint64_t)cfg.head_dim, rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cfg.head_dim * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)tova::TILE_ROWS};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? TOVA_OK : TOVA_ERR_CUDA;
+}
+
 // ---------------------------------------------------------------------------
 // C ABI
 // ---------------------------------------------------------------------------
@@ -332,8 +407,25 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   c->scale2 = c->cfg.sm_scale * 1.4426950408889634f;
   c->elem = cfg->dtype == TOVA_DTYPE_BF16 ? 2 : 4;
   c->row_bytes = c->elem * cfg->head_dim;
+  c->use_mma = wants_mma(*cfg);
+  if (c->use_mma) {
+    if ((long long)cfg->batch * cfg->n_kv_heads * cfg->capacity >= (1LL << 31)) { delete c; return TOVA_ERR_BAD_SHAPE; }
+    if (encode_state_map(&c->map_k, c->base + lay.K, *cfg) != TOVA_OK ||
+        encode_state_map(&c->map_v, c->base + lay.V, *cfg) != TOVA_OK) {
+      delete c;
+      return TOVA_ERR_CUDA;
+    }
+  }
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // Rows that were never written are still read as part of 16-row tiles (their
+  // weight is zero): they must hold finite numbers.
+  const size_t kv_bytes = (size_t)cfg->batch * cfg->n_kv_heads * cfg->capacity * c->row_bytes;
+  if (cudaMemsetAsync(c->base + lay.K, 0, kv_bytes, st) != cudaSuccess ||
+      cudaMemsetAsync(c->base + lay.V, 0, kv_bytes, st) != cudaSuccess) {
+    delete c;
+    return TOVA_ERR_CUDA;
+  }
   const size_t n = (size_t)cfg->batch * cfg->capacity;
   const int threads = 256;
   const unsigned blocks = (unsigned)((n + threads - 1) / threads);
@@ -551,8 +643,14 @@ extern "C" int tova_decode_step_static(const tova_config* cfg, void* K, void* V,
   const float scale = cfg->sm_scale == 0.f ? 1.f / std::sqrt((float)cfg->head_dim) : cfg->sm_scale;
   p.scale2 = scale * 1.4426950408889634f;
 
-  tova_cache shim{};  // launch_step only reads the device and counts launches
+  tova_cache shim{};  // launch_step reads the device, the tensor maps and counts launches
   shim.device = dev;
+  shim.use_mma = wants_mma(*cfg);
+  if (shim.use_mma) {
+    if ((long long)cfg->batch * cfg->n_kv_heads * cfg->capacity >= (1LL << 31)) return TOVA_ERR_BAD_SHAPE;
+    if (encode_state_map(&shim.map_k, K, *cfg) != TOVA_OK || encode_state_map(&shim.map_v, V, *cfg) != TOVA_OK)
+      return TOVA_ERR_CUDA;
+  }
   cudaError_t e;
   if (cfg->dtype == TOVA_DTYPE_BF16) {
     e = cfg->head_dim == 128 ? launch_step<__nv_bfloat16, 128>(&shim, p, st)

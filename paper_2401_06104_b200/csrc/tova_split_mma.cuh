@@ -1,0 +1,293 @@
+// Split kernel for grouped-query attention on tensor cores (bf16 state).
+//
+// With G >= 4 query heads sharing a KV head, the logits of a tile are a real
+// dense contraction S[heads, rows] = q[heads, D] . K[rows, D]^T, and so is the
+// weighted sum O[heads, D] = P[heads, rows] . V[rows, D] (Eq. 4, Eq. 7).  One
+// warp per (sequence, KV head, chunk) runs them as m16n8k16 bf16 MMAs with fp32
+// accumulation: the M = 16 rows of the MMA are up to 16 heads of the group.
+//   - K/V tiles of 16 rows arrive through tiled TMA copies (tensor maps with the
+//     128-byte swizzle), so that ldmatrix reads them without bank conflicts;
+//   - products of bf16 inputs are exact in fp32, so the logits match an fp32
+//     evaluation up to summation order;
+//   - the soft-max weights are split into two bf16 terms (p = hi + lo, 16
+//     significant bits) before they multiply V, which keeps the output within
+//     the tolerance an fp32 weight would give.
+// Same scratch outputs as the generic split kernel: logits, one (max, sum,
+// weighted V sum) partial per head and chunk.
+#pragma once
+
+#include <cuda.h>
+
+#include "tova_kernels.cuh"
+
+namespace tova {
+
+constexpr int MMA_UNIT_HEADS = 16;  // query heads one MMA split warp carries
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_addr(dst)),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_addr(bar))
+      : "memory");
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+
+// D += A (16x16, row) * B (16x8, col), bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// (x, y) -> bf16x2 with x in the low half; and the rounding remainders.
+__device__ __forceinline__ void split_hi_lo(float x, float y, uint32_t& hi, uint32_t& lo) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(x - __low2float(h), y - __high2float(h));
+  hi = *reinterpret_cast<const uint32_t*>(&h);
+  lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+
+// Byte offset of the 16-byte chunk `chunk` (0..D/8-1) of row `row` (0..15) in
+// a tile stored as D/64 boxes of [16 rows][128 bytes] with the 128-byte swizzle.
+__device__ __forceinline__ uint32_t swz(int row, int chunk) {
+  return (uint32_t)((chunk >> 3) * (TILE_ROWS * 128) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+}
+
+// grid = (max(n_chunks,1), Hkv*hgroups, B), block = one warp.
+template <int D>
+__global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
+                                                            const __grid_constant__ CUtensorMap map_k,
+                                                            const __grid_constant__ CUtensorMap map_v) {
+  using T = __nv_bfloat16;
+  constexpr int RB = D * 2;
+  constexpr int TILE_BYTES = TILE_ROWS * RB;   // 2 KiB (D=64) or 4 KiB (D=128): a multiple of the swizzle period
+  constexpr int NBOX = D / 64;
+  constexpr int NB = SPLIT_BUFFERS;
+  constexpr int KS = D / 16;                   // k-steps of q.K^T, and pairs of n-tiles of P.V
+  constexpr int EPL = 8, LPR = RB / 16;
+
+  extern __shared__ unsigned char smem_raw[];
+  // the swizzle is a function of the shared-memory address: tiles start on 1 KiB boundaries
+  unsigned char* ring = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+  __shared__ __align__(8) uint64_t bars[NB];
+
+  const int lane = threadIdx.x;
+  const int qrow = lane >> 2, qcol = (lane & 3) * 2;   // fragment coordinates of this lane
+  const int c = blockIdx.x, b = blockIdx.z;
+  const int kvh = blockIdx.y / p.hgroups, hg = blockIdx.y % p.hgroups;
+  const int g_begin = hg * MMA_UNIT_HEADS;
+  const int g_cnt = min(MMA_UNIT_HEADS, p.G - g_begin);
+  const bool two = g_cnt > 8;                           // rows 8..15 of the MMA hold heads
+  const int row_begin = c * p.chunk_rows;
+  const int rows = min(max(p.n - row_begin, 0), p.chunk_rows);
+  const int ntiles = (rows + TILE_ROWS - 1) / TILE_ROWS;
+
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < NB; ++s) mbar_init(&bars[s], 1);
+    mbar_fence_init();
+  }
+  __syncwarp();
+
+  pdl_wait();
+  pdl_launch_dependents();
+
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0)
+    *p.cur_pos = (p.pos_t < 0) ? *p.cur_pos + 1 : p.pos_t;
+
+  const int y0 = ((b * p.Hkv + kvh) * p.cap) + row_begin;   // first row of the chunk in the [rows, D] view
+  const int n_ops = 2 * ntiles;                             // u = 2t: K_t, u = 2t+1: V_t
+  auto issue = [&](int u) {                                 // lane 0 only
+    uint64_t* bar = &bars[u % NB];
+    unsigned char* dst = ring + (size_t)(u % NB) * TILE_BYTES;
+    mbar_expect_tx(bar, TILE_BYTES);                        // a tiled copy always delivers the whole box
+#pragma unroll
+    for (int bx = 0; bx < NBOX; ++bx)
+      tma_load_2d(dst + bx * (TILE_ROWS * 128), (u & 1) ? &map_v : &map_k, bx * 64, y0 + (u >> 1) * TILE_ROWS, bar);
+  };
+  if (lane == 0) {
+    for (int u = 0; u < min(NB, n_ops); ++u) issue(u);
+  }
+
+  const T* qbase = static_cast<const T*>(p.q) + ((size_t)b * p.H + (size_t)kvh * p.G + g_begin) * D;
+  const size_t bh0 = (size_t)b * p.H + (size_t)kvh * p.G + g_begin;
+
+  // The new token (candidate n): its logit per head, on the plain ALUs.
+  if (c == 0) {
+    const int lig = lane % LPR;
+    const T* kn = static_cast<const T*>(p.k_new) + ((size_t)b * p.Hkv + kvh) * D;
+    float kf[EPL];
+    Vec16<T>::unpack(*reinterpret_cast<const uint4*>(kn + lig * EPL), kf);
+    for (int g = 0; g < g_cnt; ++g) {
+      float qf[EPL];
+      Vec16<T>::unpack(*reinterpret_cast<const uint4*>(qbase + (size_t)g * D + lig * EPL), qf);
+      float s = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) s = fmaf(qf[e], kf[e], s);
+#pragma unroll
+      for (int o = LPR / 2; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      s *= p.scale2;
+      if (lane == 0) {
+        p.logits[(bh0 + g) * p.ld + p.n] = s;
+        p.part_ml[(bh0 + g) * p.pc + p.n_chunks] = make_float2(s, 1.f);
+      }
+    }
+  }
+  if (ntiles == 0) return;
+
+  // q as the A operand: rows = heads (zero beyond the group), 16 columns per k-step
+  uint32_t qa[KS][4];
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) {
+    const int d = ks * 16 + qcol;
+    const uint32_t* r0 = reinterpret_cast<const uint32_t*>(qbase + (size_t)qrow * D + d);
+    const uint32_t* r1 = reinterpret_cast<const uint32_t*>(qbase + (size_t)(qrow + 8) * D + d);
+    qa[ks][0] = (qrow < g_cnt) ? r0[0] : 0u;
+    qa[ks][1] = (qrow + 8 < g_cnt) ? r1[0] : 0u;
+    qa[ks][2] = (qrow < g_cnt) ? r0[4] : 0u;      // d + 8
+    qa[ks][3] = (qrow + 8 < g_cnt) ? r1[4] : 0u;
+  }
+
+  float o[2 * KS][4];   // O[heads, D]: n-tile j covers d = 8j..8j+7
+#pragma unroll
+  for (int j = 0; j < 2 * KS; ++j)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) o[j][e] = 0.f;
+  float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};   // [0]: head qrow, [1]: head qrow + 8
+
+  // ldmatrix lane roles: lane supplies the address of row (lane % 8) of matrix (lane / 8)
+  const int lm_r = lane & 7, lm_m = lane >> 3;
+  const uint32_t ring_addr = smem_addr(ring);
+
+  bool failed = false;
+  int t = 0;
+  for (; t < ntiles; ++t) {
+    const int uk = 2 * t, uv = 2 * t + 1;
+    const int nvalid = min(TILE_ROWS, rows - t * TILE_ROWS);
+    const uint32_t kt = ring_addr + (uint32_t)(uk % NB) * TILE_BYTES;
+    const uint32_t vt = ring_addr + (uint32_t)(uv % NB) * TILE_BYTES;
+
+    // ---- S = q . K^T for the tile's 16 rows (two n-tiles of 8 rows) -------------
+    if (!warp_wait(&bars[uk % NB], (uint32_t)(uk / NB) & 1u)) { failed = true; break; }
+    float s[2][4];
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      // matrices: (rows 0-7, d0..7) (rows 0-7, d0+8..15) (rows 8-15, d0..7) (rows 8-15, d0+8..15)
+      uint32_t kb[4];
+      ldmatrix_x4(kb, kt + swz(lm_r + 8 * (lm_m >> 1), ks * 2 + (lm_m & 1)));
+      mma_bf16(s[0], qa[ks], kb[0], kb[1]);
+      mma_bf16(s[1], qa[ks], kb[2], kb[3]);
+    }
+    __syncwarp();
+    if (lane == 0 && uk + NB < n_ops) {
+      fence_proxy_async_smem();
+      issue(uk + NB);
+    }
+
+    // ---- online soft-max on the fragments ----------------------------------------
+    // lane holds, for head row qrow (+8): columns nt*8 + qcol + {0,1}
+    uint32_t p_hi[4], p_lo[4];
+#pragma unroll
+    for (int rr = 0; rr < 2; ++rr) {
+      if (rr == 1 && !two) {
+        p_hi[1] = p_hi[3] = p_lo[1] = p_lo[3] = 0u;
+        continue;
+      }
+      const int head = qrow + 8 * rr;
+      float v[4];
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int col = nt * 8 + qcol + e;
+          v[nt * 2 + e] = (col < nvalid) ? s[nt][rr * 2 + e] * p.scale2 : -INFINITY;
+        }
+      if (head < g_cnt) {
+        float* lg = p.logits + (bh0 + head) * p.ld + row_begin + t * TILE_ROWS;
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int col = nt * 8 + qcol + e;
+            if (col < nvalid) lg[col] = v[nt * 2 + e];
+          }
+      }
+      float mx = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3]));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const float m_new = fmaxf(m[rr], mx);
+      const float corr = exp2_diff(m[rr], m_new);
+      float e4[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) e4[i] = exp2_diff(v[i], m_new);
+      l[rr] = fmaf(l[rr], corr, (e4[0] + e4[1]) + (e4[2] + e4[3]));   // per-lane partial, folded at the end
+      m[rr] = m_new;
+#pragma unroll
+      for (int j = 0; j < 2 * KS; ++j) {
+        o[j][rr * 2] *= corr;
+        o[j][rr * 2 + 1] *= corr;
+      }
+      // P as the A operand of P.V: a0/a2 <- n-tile 0, a1/a3 rows + 8; a2,a3 <- n-tile 1
+      split_hi_lo(e4[0], e4[1], p_hi[rr], p_lo[rr]);
+      split_hi_lo(e4[2], e4[3], p_hi[2 + rr], p_lo[2 + rr]);
+    }
+
+    // ---- O += P . V ------------------------------------------------------------------
+    if (!warp_wait(&bars[uv % NB], (uint32_t)(uv / NB) & 1u)) { failed = true; break; }
+#pragma unroll
+    for (int jj = 0; jj < KS; ++jj) {
+      // matrices: (rows 0-7, d0..7) (rows 8-15, d0..7) (rows 0-7, d0+8..15) (rows 8-15, d0+8..15), transposed
+      uint32_t vb[4];
+      ldmatrix_x4_trans(vb, vt + swz(lm_r + 8 * (lm_m & 1), jj * 2 + (lm_m >> 1)));
+      mma_bf16(o[2 * jj], p_hi, vb[0], vb[1]);
+      mma_bf16(o[2 * jj], p_lo, vb[0], vb[1]);
+      mma_bf16(o[2 * jj + 1], p_hi, vb[2], vb[3]);
+      mma_bf16(o[2 * jj + 1], p_lo, vb[2], vb[3]);
+    }
+    __syncwarp();
+    if (lane == 0 && uv + NB < n_ops) {
+      fence_proxy_async_smem();
+      issue(uv + NB);
+    }
+  }
+
+  if (failed) {
+    for (int u = 2 * t; u < min(2 * t + NB, n_ops); ++u) warp_wait(&bars[u % NB], (uint32_t)(u / NB) & 1u);
+    if (lane == 0) atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
+    return;
+  }
+
+  // ---- chunk partial: (max, sum) and the un-normalised weighted V sums ------------------
+#pragma unroll
+  for (int rr = 0; rr < 2; ++rr) {
+    const int head = qrow + 8 * rr;
+    float lsum = l[rr];
+    lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+    lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+    if (head < g_cnt) {
+      float* dst = p.part_acc + ((bh0 + head) * (size_t)(p.pc - 1) + c) * D + qcol;
+#pragma unroll
+      for (int j = 0; j < 2 * KS; ++j)
+        *reinterpret_cast<float2*>(dst + j * 8) = make_float2(o[j][rr * 2], o[j][rr * 2 + 1]);
+      if ((lane & 3) == 0) p.part_ml[(bh0 + head) * p.pc + c] = make_float2(m[rr], lsum);
+    }
+  }
+}
+
+}  // namespace tova
