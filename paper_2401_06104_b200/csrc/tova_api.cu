@@ -153,7 +153,7 @@ cudaError_t launch_split_g(int dev, int G, const StepParams& p, dim3 grid, cudaS
 // sequence, per-head max and 1/sum, one float per thread, and the new token's
 // rows when they are small enough to be staged.
 inline size_t combine_smem_bytes(int H, int n_partials, int threads, size_t row_bytes) {
-  size_t b = sizeof(float) * (2 * (size_t)H * n_partials + 2 * (size_t)H + threads) + 16;
+  size_t b = sizeof(float) * (2 * (size_t)H * n_partials + 3 * (size_t)H + threads) + 16;
   if (2 * row_bytes <= (size_t)tova::COMBINE_ROW_STAGE_BYTES) b += 2 * row_bytes;
   return b;
 }

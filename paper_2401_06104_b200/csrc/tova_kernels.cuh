@@ -310,7 +310,7 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
 //   4. after one cluster barrier CTA 0 takes the overall arg-min - lowest index
 //      on ties - and replaces that row by the new token in K, V and the position
 //      table (Eq. 9, in place).  No global atomics, no CTA waits on a flag.
-// smem: float2 pml[H][np]; float hM[H], hInvL[H], sc[CT]; then, in
+// smem: float2 pml[H][np]; float hM[H], hInvL[H], hLc[H], sc[CT]; then, in
 // CTA 0 only, the new token's k and v rows of all KV heads (bulk-copied in at
 // the start when they fit COMBINE_ROW_STAGE_BYTES each).
 template <typename T, int D, int CT>
@@ -325,7 +325,8 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
   float2* pml = reinterpret_cast<float2*>(csm);                  // [H][np]
   float* hM = csm + 2 * (size_t)p.H * np;                        // [H]
   float* hInvL = hM + p.H;                                       // [H]
-  float* sc = hInvL + p.H;                                       // [CT]
+  float* hLc = hInvL + p.H;                                      // [H] -max2 - log2(sum * H)
+  float* sc = hLc + p.H;                                         // [CT]
   unsigned char* row_stage = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(sc + CT) + 15) & ~uintptr_t(15));     // [2][Hkv*D*sizeof(T)]
   __shared__ __align__(8) uint64_t row_bar;
@@ -345,10 +346,16 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
   const int jl = tid % wp, hs = tid / wp;
   const int j_begin = x * p.cand_per_cta;
   const int j_end = min(j_begin + p.cand_per_cta, p.n + 1);
+  // When a victim is due, CTA 0 is on the critical path (arg-min, insert): if
+  // the output merge is light (few chunks), the output elements are shared among
+  // its peers and written after they arrive at the cluster barrier.
+  const bool late_out = p.do_evict && p.nx > 1 && p.n_chunks <= AC;   // only when the merge is light
+  const int out_ctas = late_out ? p.nx - 1 : p.nx;
+  const int out_x = late_out ? x - 1 : x;      // -1: no share
   const int items = p.H * D;
-  const int per = (items + p.nx - 1) / p.nx;
-  const int it_end = min(items, (x + 1) * per);
-  const int it0 = x * per + tid;
+  const int per = (items + out_ctas - 1) / out_ctas;
+  const int it_end = out_x < 0 ? 0 : min(items, (out_x + 1) * per);
+  const int it0 = out_x < 0 ? 0 : out_x * per + tid;
   constexpr int RB16 = D * (int)sizeof(T) / 16;  // 16-byte words per row
   const int row_words = p.Hkv * RB16;
   const int total_ml = p.H * np;
@@ -429,21 +436,32 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
   for (int i = tid + ML * CT; i < total_ml; i += CT)
     pml[i] = p.part_ml[((size_t)b * p.H + i / np) * p.pc + i % np];
   __syncthreads();
-  for (int h = warp; h < p.H; h += CT / 32) {
-    const float2* ml = pml + (size_t)h * np;
-    float M = -INFINITY, L = 0.f;
-    for (int i = lane; i < np; i += 32) M = fmaxf(M, ml[i].x);
-    M = warp_max(M);
-    for (int i = lane; i < np; i += 32) L = fmaf(ml[i].y, exp2_diff(ml[i].x, M), L);
-    L = warp_sum(L);
-    if (lane == 0) {
-      hM[h] = M;
-      hInvL[h] = 1.f / L;
+  {
+    // a group of lph lanes per head, at most 8 partials per lane
+    int lph = 1;
+    while (lph < 32 && lph * 8 < np) lph <<= 1;
+    const int hpp = CT / lph;                      // heads per pass
+    const int sub_l = tid % lph;
+    for (int h0 = 0; h0 < p.H; h0 += hpp) {        // uniform trip count: the shuffles need whole warps
+      const int h = h0 + tid / lph;
+      const bool hv = h < p.H;
+      const float2* ml = pml + (size_t)(hv ? h : 0) * np;
+      float M = -INFINITY, L = 0.f;
+      for (int i = sub_l; i < np; i += lph) M = fmaxf(M, ml[i].x);
+      for (int o = lph >> 1; o >= 1; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+      for (int i = sub_l; i < np; i += lph) L = fmaf(ml[i].y, exp2_diff(ml[i].x, M), L);
+      for (int o = lph >> 1; o >= 1; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+      if (hv && sub_l == 0) {
+        hM[h] = M;
+        hInvL[h] = 1.f / L;
+        hLc[h] = -M - log2f(L * (float)p.H);
+      }
     }
   }
   __syncthreads();
 
   // ---- 2. this CTA's share of the attention output --------------------------------
+  auto write_outputs = [&]() {
   for (int it = it0; it < it_end; it += CT) {
     const int h = it / D, d = it % D;
     const size_t bh = (size_t)b * p.H + h;
@@ -466,6 +484,8 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
     }
     p.out[bh * D + d] = o * hInvL[h];
   }
+  };
+  if (!late_out) write_outputs();
 
   if (!p.do_evict) {
     // g(t) = min(t, k) not yet reached: the new token takes the next free row.
@@ -485,7 +505,6 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
   float val = INFINITY;
   int idx = 0x7fffffff;
   int cpos = pos_t;                // position held by the best candidate (the new token holds pos_t)
-  const float inv_h = 1.f / (float)p.H;
   for (int j0 = j_begin; j0 < j_end; j0 += wp) {
     const int j = j0 + jl;
     const bool live = j < j_end;
@@ -496,13 +515,13 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
 #pragma unroll
         for (int u = 0; u < LG; ++u) {
           const int h = hs + u * hs_n;
-          if (h < p.H) a = fmaf(exp2f(r_lg[u] - hM[h]), hInvL[h], a);
+          if (h < p.H) a += exp2f(r_lg[u] + hLc[h]);
         }
 #pragma unroll 8
-        for (int h = hs + LG * hs_n; h < p.H; h += hs_n) a = fmaf(exp2f(lg[(size_t)h * p.ld] - hM[h]), hInvL[h], a);
+        for (int h = hs + LG * hs_n; h < p.H; h += hs_n) a += exp2f(lg[(size_t)h * p.ld] + hLc[h]);
       } else {
 #pragma unroll 16
-        for (int h = hs; h < p.H; h += hs_n) a = fmaf(exp2f(lg[(size_t)h * p.ld] - hM[h]), hInvL[h], a);
+        for (int h = hs; h < p.H; h += hs_n) a += exp2f(lg[(size_t)h * p.ld] + hLc[h]);
       }
     }
     if (hs_n > 1) {                // uniform over the CTA
@@ -515,7 +534,7 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
       __syncthreads();
     }
     if (hs == 0 && live) {
-      const float v = a * inv_h;
+      const float v = a;             // the 1/H of the mean is folded into hLc
       if (v < val) {               // passes go up in j: strict < keeps the lowest index
         val = v;
         idx = j;
@@ -544,7 +563,10 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
   // ---- 4. one cluster barrier; CTA 0 takes the arg-min, evicts, inserts -----------
   __syncwarp();
   cluster_arrive_release();        // orders the store above before the barrier completes
-  if (x != 0) return;              // peers are done: nobody reads their shared memory
+  if (x != 0) {                    // peers: nobody reads their shared memory; their outputs are off the critical path
+    if (late_out) write_outputs();
+    return;
+  }
   cluster_wait_acquire();
   if (warp == 0) {
     float bv = INFINITY;
