@@ -21,7 +21,7 @@ inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 struct Layout {
-  size_t K, V, pos, len, logits, part_ml, part_acc, status, cur_pos;
+  size_t K, V, pos, len, last_slot, logits, part_ml, part_acc, status, cur_pos;
   size_t st_q, st_k, st_v, st_out, st_ev;  // staging for host-buffer calls
   size_t total;
   int ld, pc;
@@ -57,6 +57,7 @@ Layout make_layout(const tova_config& c) {
   L.V = take(B * Hkv * cap * D * E);
   L.pos = take(B * cap * 4);
   L.len = take(B * 4);
+  L.last_slot = take(B * 4);
   L.logits = take(B * H * L.ld * 4);
   L.part_ml = take(B * H * L.pc * 8);
   L.part_acc = take(B * H * (size_t)(L.pc - 1) * D * 4);
@@ -315,6 +316,7 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
   p.part_acc = reinterpret_cast<float*>(base + c->lay.part_acc);
   p.status = reinterpret_cast<int32_t*>(base + c->lay.status);
   p.cur_pos = reinterpret_cast<int32_t*>(base + c->lay.cur_pos);
+  p.last_slot = reinterpret_cast<int32_t*>(base + c->lay.last_slot);
   p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.evicted = evicted_pos; p.pos_t = pos;
   p.ld = c->lay.ld; p.pc = c->lay.pc;
   fill_geometry(p, cfg, n, c->chunk_rows);
@@ -431,6 +433,7 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   const unsigned blocks = (unsigned)((n + threads - 1) / threads);
   tova::tova_init_kernel<<<blocks, threads, 0, st>>>(
       reinterpret_cast<int32_t*>(c->base + lay.pos), reinterpret_cast<int32_t*>(c->base + lay.len),
+      reinterpret_cast<int32_t*>(c->base + lay.last_slot),
       reinterpret_cast<int32_t*>(c->base + lay.status),
       reinterpret_cast<int32_t*>(c->base + lay.cur_pos), cfg->batch, cfg->capacity);
   if (cudaGetLastError() != cudaSuccess) { delete c; return TOVA_ERR_CUDA; }

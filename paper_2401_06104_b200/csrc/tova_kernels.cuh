@@ -43,6 +43,7 @@ struct StepParams {
   float* part_acc;    // [B,H,pc-1,D] un-normalised weighted V sums per chunk
   int32_t* status;    // [1]
   int32_t* cur_pos;   // [1] position of the token being processed (set by the split kernel)
+  int32_t* last_slot; // [B] slot the previous step's token went to (-1: none), or null: no early prefetch
   // this step
   const void* q;      // [B,H,D]
   const void* k_new;  // [B,Hkv,D]
@@ -114,14 +115,6 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
   }
   __syncwarp();
 
-  // Nothing above touches global memory; below we read what earlier kernels in
-  // the stream wrote.
-  pdl_wait();
-  pdl_launch_dependents();
-
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0)
-    *p.cur_pos = (p.pos_t < 0) ? *p.cur_pos + 1 : p.pos_t;
-
   const unsigned char* k_src =
       static_cast<const unsigned char*>(p.K) + (((size_t)b * p.Hkv + kvh) * p.cap + row_begin) * RB;
   const unsigned char* v_src =
@@ -136,9 +129,41 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
     bulk_g2s(ring + (size_t)(u % NB) * TILE_BYTES, ((u & 1) ? v_src : k_src) + (size_t)t * TILE_BYTES, bytes,
              bar);
   };
-  if (lane == 0) {
+  // Early prefetch.  The previous step's combine kernel may still be running:
+  // the only thing it writes to the state is one row per sequence (the slot its
+  // token went to, recorded in last_slot).  Every other row is final, so the
+  // first tiles can be fetched now, before the dependency wait; if the one row
+  // in question lies in them, it is fetched again after the wait (patch below).
+  const bool early = p.last_slot != nullptr;
+  if (early && lane == 0) {
     for (int u = 0; u < min(NB, n_ops); ++u) issue(u);
   }
+
+  // Nothing above reads global memory through this thread; below we read what
+  // earlier kernels in the stream wrote.
+  pdl_wait();
+  pdl_launch_dependents();
+
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0)
+    *p.cur_pos = (p.pos_t < 0) ? *p.cur_pos + 1 : p.pos_t;
+  if (!early && lane == 0) {
+    for (int u = 0; u < min(NB, n_ops); ++u) issue(u);
+  }
+  int patch_row = -1;              // row of this chunk that must be fetched again, if any
+  if (early) {
+    const int ls = __ldcg(p.last_slot + b);
+    if (ls >= row_begin && ls < row_begin + rows) patch_row = ls - row_begin;
+  }
+  // Re-fetches row patch_row of operand tile u (already landed) from global memory.
+  auto patch = [&](int u, unsigned char* tile, const unsigned char* src) {
+    const int t = u >> 1;
+    if (patch_row >= 0 && u < NB && patch_row / TILE_ROWS == t) {
+      if (lane < LPR)
+        *reinterpret_cast<uint4*>(tile + (size_t)(patch_row % TILE_ROWS) * RB + lane * 16) =
+            __ldcg(reinterpret_cast<const uint4*>(src + (size_t)patch_row * RB) + lane);
+      __syncwarp();
+    }
+  };
 
   const T* qbase = static_cast<const T*>(p.q) + ((size_t)b * p.H + (size_t)kvh * p.G + g_begin) * D;
   const size_t bh0 = (size_t)b * p.H + (size_t)kvh * p.G + g_begin;
@@ -186,11 +211,12 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
   for (; t < ntiles; ++t) {
     const int uk = 2 * t, uv = 2 * t + 1;
     const int nvalid = min(TILE_ROWS, rows - t * TILE_ROWS);
-    const unsigned char* kt = ring + (size_t)(uk % NB) * TILE_BYTES;
-    const unsigned char* vt = ring + (size_t)(uv % NB) * TILE_BYTES;
+    unsigned char* kt = ring + (size_t)(uk % NB) * TILE_BYTES;
+    unsigned char* vt = ring + (size_t)(uv % NB) * TILE_BYTES;
 
     // ---- logits of the tile's rows, GB heads at a time -------------------------
     if (!warp_wait(&bars[uk % NB], (uint32_t)(uk / NB) & 1u)) { failed = true; break; }
+    patch(uk, kt, k_src);
     float s[GU];
 #pragma unroll
     for (int g0 = 0; g0 < GU; g0 += GB) {
@@ -245,6 +271,7 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
 
     // ---- weighted V sum --------------------------------------------------------
     if (!warp_wait(&bars[uv % NB], (uint32_t)(uv / NB) & 1u)) { failed = true; break; }
+    patch(uv, vt, v_src);
 #pragma unroll
     for (int i = 0; i < NP; ++i) {
       const int r = i * RPW + sub;
@@ -494,6 +521,7 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
       if (tid == 0) {
         p.pos[(size_t)b * p.cap + p.n] = pos_t;
         p.len[b] = p.n + 1;
+        if (p.last_slot) p.last_slot[b] = p.n;
         if (p.evicted) p.evicted[b] = -1;
       }
     }
@@ -586,6 +614,7 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
       if (bi < 0 || bi > p.cap) { atomicExch(p.status, DEV_ERR_BAD_VICTIM); bi = p.cap; bp = pos_t; }
       s_victim = bi;
       if (bi < p.cap) p.pos[(size_t)b * p.cap + bi] = pos_t;
+      if (p.last_slot) p.last_slot[b] = (bi < p.cap) ? bi : -1;
       if (p.evicted) p.evicted[b] = bp;  // the new token's own position if it dropped itself
     }
   }
@@ -596,11 +625,11 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
 }
 
 // Empty state at init: length 0, positions -1, status 0.
-__global__ void tova_init_kernel(int32_t* pos, int32_t* len, int32_t* status, int32_t* cur_pos, int B,
-                                 int cap) {
+__global__ void tova_init_kernel(int32_t* pos, int32_t* len, int32_t* last_slot, int32_t* status,
+                                 int32_t* cur_pos, int B, int cap) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < (size_t)B * cap) pos[i] = -1;
-  if (i < (size_t)B) len[i] = 0;
+  if (i < (size_t)B) { len[i] = 0; last_slot[i] = -1; }
   if (i == 0) { *status = 0; *cur_pos = -1; }
 }
 

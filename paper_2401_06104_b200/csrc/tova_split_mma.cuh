@@ -101,12 +101,6 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
   }
   __syncwarp();
 
-  pdl_wait();
-  pdl_launch_dependents();
-
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0)
-    *p.cur_pos = (p.pos_t < 0) ? *p.cur_pos + 1 : p.pos_t;
-
   const int y0 = ((b * p.Hkv + kvh) * p.cap) + row_begin;   // first row of the chunk in the [rows, D] view
   const int n_ops = 2 * ntiles;                             // u = 2t: K_t, u = 2t+1: V_t
   auto issue = [&](int u) {                                 // lane 0 only
@@ -117,9 +111,39 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
     for (int bx = 0; bx < NBOX; ++bx)
       tma_load_2d(dst + bx * (TILE_ROWS * 128), (u & 1) ? &map_v : &map_k, bx * 64, y0 + (u >> 1) * TILE_ROWS, bar);
   };
-  if (lane == 0) {
+  // Early prefetch before the dependency wait: only the row the previous step's
+  // token went to (last_slot) can still change; it is fetched again after the
+  // wait if it lies in the tiles requested here.
+  const bool early = p.last_slot != nullptr;
+  if (early && lane == 0) {
     for (int u = 0; u < min(NB, n_ops); ++u) issue(u);
   }
+
+  pdl_wait();
+  pdl_launch_dependents();
+
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0)
+    *p.cur_pos = (p.pos_t < 0) ? *p.cur_pos + 1 : p.pos_t;
+  if (!early && lane == 0) {
+    for (int u = 0; u < min(NB, n_ops); ++u) issue(u);
+  }
+  int patch_row = -1;
+  if (early) {
+    const int ls = __ldcg(p.last_slot + b);
+    if (ls >= row_begin && ls < row_begin + rows) patch_row = ls - row_begin;
+  }
+  const unsigned char* k_rows = static_cast<const unsigned char*>(p.K) + (size_t)y0 * RB;
+  const unsigned char* v_rows = static_cast<const unsigned char*>(p.V) + (size_t)y0 * RB;
+  // Re-fetches row patch_row of operand tile u (already landed) into the swizzled tile.
+  auto patch = [&](int u, const unsigned char* src) {
+    if (patch_row >= 0 && u < NB && patch_row / TILE_ROWS == (u >> 1)) {
+      if (lane < LPR) {
+        const uint4 w = __ldcg(reinterpret_cast<const uint4*>(src + (size_t)patch_row * RB) + lane);
+        *reinterpret_cast<uint4*>(ring + (size_t)(u % NB) * TILE_BYTES + swz(patch_row % TILE_ROWS, lane)) = w;
+      }
+      __syncwarp();
+    }
+  };
 
   const T* qbase = static_cast<const T*>(p.q) + ((size_t)b * p.H + (size_t)kvh * p.G + g_begin) * D;
   const size_t bh0 = (size_t)b * p.H + (size_t)kvh * p.G + g_begin;
@@ -181,6 +205,7 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
 
     // ---- S = q . K^T for the tile's 16 rows (two n-tiles of 8 rows) -------------
     if (!warp_wait(&bars[uk % NB], (uint32_t)(uk / NB) & 1u)) { failed = true; break; }
+    patch(uk, k_rows);
     float s[2][4];
 #pragma unroll
     for (int nt = 0; nt < 2; ++nt)
@@ -250,6 +275,7 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
 
     // ---- O += P . V ------------------------------------------------------------------
     if (!warp_wait(&bars[uv % NB], (uint32_t)(uv / NB) & 1u)) { failed = true; break; }
+    patch(uv, v_rows);
 #pragma unroll
     for (int jj = 0; jj < KS; ++jj) {
       // matrices: (rows 0-7, d0..7) (rows 8-15, d0..7) (rows 0-7, d0+8..15) (rows 8-15, d0+8..15), transposed
