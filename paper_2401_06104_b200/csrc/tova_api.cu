@@ -200,11 +200,11 @@ cudaError_t launch_combine(int dev, const StepParams& p, cudaStream_t st) {
              : launch_combine_ct<T, D, tova::COMBINE_THREADS_SMALL>(dev, p, st);
 }
 
-template <int D>
-cudaError_t launch_split_mma(int dev, const StepParams& p, const CUtensorMap& mk, const CUtensorMap& mv, dim3 grid,
-                             cudaStream_t st) {
+template <int D, bool TWO>
+cudaError_t launch_split_mma_t(int dev, const StepParams& p, const CUtensorMap& mk, const CUtensorMap& mv, dim3 grid,
+                               cudaStream_t st) {
   const size_t smem = (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * D * 2 + 1024;
-  auto kern = tova::tova_split_mma_kernel<D>;
+  auto kern = tova::tova_split_mma_kernel<D, TWO>;
   static bool attr_set[64] = {};
   if (!attr_set[dev & 63]) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -224,6 +224,13 @@ cudaError_t launch_split_mma(int dev, const StepParams& p, const CUtensorMap& mk
   cfg.attrs = at;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kern, p, mk, mv);
+}
+
+template <int D>
+cudaError_t launch_split_mma(int dev, const StepParams& p, const CUtensorMap& mk, const CUtensorMap& mv, dim3 grid,
+                             cudaStream_t st) {
+  return p.G > 8 ? launch_split_mma_t<D, true>(dev, p, mk, mv, grid, st)
+                 : launch_split_mma_t<D, false>(dev, p, mk, mv, grid, st);
 }
 
 template <typename T, int D>
@@ -250,6 +257,10 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st) {
 int pick_chunk_rows(const tova_config& cfg, int sm_count) {
   const size_t smem = split_smem_bytes(cfg) + 1024 /* per-CTA reserve */ + 64;
   long long per_sm = (long long)(227 * 1024) / (long long)smem;
+  // registers bound the resident warps too (figures from ptxas for these kernels)
+  const int G0 = cfg.n_q_heads / cfg.n_kv_heads;
+  const long long by_regs = wants_mma(cfg) ? (G0 > 8 ? 12 : 16) : (G0 <= 1 ? 28 : G0 == 2 ? 16 : G0 <= 4 ? 12 : 8);
+  if (per_sm > by_regs) per_sm = by_regs;
   if (per_sm > 32) per_sm = 32;
   if (per_sm < 1) per_sm = 1;
   const long long slots = per_sm * sm_count;

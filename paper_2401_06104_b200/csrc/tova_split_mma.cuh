@@ -51,6 +51,16 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// The same with rows 8..15 of A all zero (at most 8 heads in the group): only
+// the upper half of the accumulator tile is kept, which halves the registers.
+__device__ __forceinline__ void mma_bf16_top(float (&d)[2], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+  float z0, z1;
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%10,%10};"
+      : "+f"(d[0]), "+f"(d[1]), "=f"(z0), "=f"(z1)
+      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.f));
+}
+
 // (x, y) -> bf16x2 with x in the low half; and the rounding remainders.
 __device__ __forceinline__ void split_hi_lo(float x, float y, uint32_t& hi, uint32_t& lo) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
@@ -66,7 +76,8 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
 }
 
 // grid = (max(n_chunks,1), Hkv*hgroups, B), block = one warp.
-template <int D>
+// TWO: the group has more than 8 heads, rows 8..15 of the MMA tile are in use.
+template <int D, bool TWO>
 __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
                                                             const __grid_constant__ CUtensorMap map_k,
                                                             const __grid_constant__ CUtensorMap map_v) {
@@ -89,7 +100,7 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
   const int kvh = blockIdx.y / p.hgroups, hg = blockIdx.y % p.hgroups;
   const int g_begin = hg * MMA_UNIT_HEADS;
   const int g_cnt = min(MMA_UNIT_HEADS, p.G - g_begin);
-  const bool two = g_cnt > 8;                           // rows 8..15 of the MMA hold heads
+  constexpr int R = TWO ? 2 : 1;                        // 8-row halves of the MMA tile that hold heads
   const int row_begin = c * p.chunk_rows;
   const int rows = min(max(p.n - row_begin, 0), p.chunk_rows);
   const int ntiles = (rows + TILE_ROWS - 1) / TILE_ROWS;
@@ -172,24 +183,32 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
   if (ntiles == 0) return;
 
   // q as the A operand: rows = heads (zero beyond the group), 16 columns per k-step
-  uint32_t qa[KS][4];
+  // fragment registers a0..a3 when TWO, else only a0 and a2 (a1 = a3 = 0)
+  uint32_t qa[KS][2 * R];
 #pragma unroll
   for (int ks = 0; ks < KS; ++ks) {
     const int d = ks * 16 + qcol;
     const uint32_t* r0 = reinterpret_cast<const uint32_t*>(qbase + (size_t)qrow * D + d);
     const uint32_t* r1 = reinterpret_cast<const uint32_t*>(qbase + (size_t)(qrow + 8) * D + d);
-    qa[ks][0] = (qrow < g_cnt) ? r0[0] : 0u;
-    qa[ks][1] = (qrow + 8 < g_cnt) ? r1[0] : 0u;
-    qa[ks][2] = (qrow < g_cnt) ? r0[4] : 0u;      // d + 8
-    qa[ks][3] = (qrow + 8 < g_cnt) ? r1[4] : 0u;
+    if constexpr (TWO) {
+      qa[ks][0] = (qrow < g_cnt) ? r0[0] : 0u;
+      qa[ks][1] = (qrow + 8 < g_cnt) ? r1[0] : 0u;
+      qa[ks][2] = (qrow < g_cnt) ? r0[4] : 0u;      // d + 8
+      qa[ks][3] = (qrow + 8 < g_cnt) ? r1[4] : 0u;
+    } else {
+      qa[ks][0] = (qrow < g_cnt) ? r0[0] : 0u;
+      qa[ks][1] = (qrow < g_cnt) ? r0[4] : 0u;      // d + 8
+    }
   }
 
-  float o[2 * KS][4];   // O[heads, D]: n-tile j covers d = 8j..8j+7
+  float o[2 * KS][2 * R];   // O[heads, D]: n-tile j covers d = 8j..8j+7
 #pragma unroll
   for (int j = 0; j < 2 * KS; ++j)
 #pragma unroll
-    for (int e = 0; e < 4; ++e) o[j][e] = 0.f;
-  float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};   // [0]: head qrow, [1]: head qrow + 8
+    for (int e = 0; e < 2 * R; ++e) o[j][e] = 0.f;
+  float m[R], l[R];   // [0]: head qrow, [1]: head qrow + 8
+#pragma unroll
+  for (int rr = 0; rr < R; ++rr) { m[rr] = -INFINITY; l[rr] = 0.f; }
 
   // ldmatrix lane roles: lane supplies the address of row (lane % 8) of matrix (lane / 8)
   const int lm_r = lane & 7, lm_m = lane >> 3;
@@ -206,18 +225,23 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
     // ---- S = q . K^T for the tile's 16 rows (two n-tiles of 8 rows) -------------
     if (!warp_wait(&bars[uk % NB], (uint32_t)(uk / NB) & 1u)) { failed = true; break; }
     patch(uk, k_rows);
-    float s[2][4];
+    float s[2][2 * R];
 #pragma unroll
     for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
+      for (int e = 0; e < 2 * R; ++e) s[nt][e] = 0.f;
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
       // matrices: (rows 0-7, d0..7) (rows 0-7, d0+8..15) (rows 8-15, d0..7) (rows 8-15, d0+8..15)
       uint32_t kb[4];
       ldmatrix_x4(kb, kt + swz(lm_r + 8 * (lm_m >> 1), ks * 2 + (lm_m & 1)));
-      mma_bf16(s[0], qa[ks], kb[0], kb[1]);
-      mma_bf16(s[1], qa[ks], kb[2], kb[3]);
+      if constexpr (TWO) {
+        mma_bf16(s[0], qa[ks], kb[0], kb[1]);
+        mma_bf16(s[1], qa[ks], kb[2], kb[3]);
+      } else {
+        mma_bf16_top(s[0], qa[ks][0], qa[ks][1], kb[0], kb[1]);
+        mma_bf16_top(s[1], qa[ks][0], qa[ks][1], kb[2], kb[3]);
+      }
     }
     __syncwarp();
     if (lane == 0 && uk + NB < n_ops) {
@@ -227,13 +251,9 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
 
     // ---- online soft-max on the fragments ----------------------------------------
     // lane holds, for head row qrow (+8): columns nt*8 + qcol + {0,1}
-    uint32_t p_hi[4], p_lo[4];
+    uint32_t p_hi[2 * R], p_lo[2 * R];   // a0..a3 when TWO, else a0 and a2
 #pragma unroll
-    for (int rr = 0; rr < 2; ++rr) {
-      if (rr == 1 && !two) {
-        p_hi[1] = p_hi[3] = p_lo[1] = p_lo[3] = 0u;
-        continue;
-      }
+    for (int rr = 0; rr < R; ++rr) {
       const int head = qrow + 8 * rr;
       float v[4];
 #pragma unroll
@@ -269,8 +289,8 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
         o[j][rr * 2 + 1] *= corr;
       }
       // P as the A operand of P.V: a0/a2 <- n-tile 0, a1/a3 rows + 8; a2,a3 <- n-tile 1
-      split_hi_lo(e4[0], e4[1], p_hi[rr], p_lo[rr]);
-      split_hi_lo(e4[2], e4[3], p_hi[2 + rr], p_lo[2 + rr]);
+      split_hi_lo(e4[0], e4[1], p_hi[TWO ? rr : 0], p_lo[TWO ? rr : 0]);
+      split_hi_lo(e4[2], e4[3], p_hi[TWO ? 2 + rr : 1], p_lo[TWO ? 2 + rr : 1]);
     }
 
     // ---- O += P . V ------------------------------------------------------------------
@@ -281,10 +301,17 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
       // matrices: (rows 0-7, d0..7) (rows 8-15, d0..7) (rows 0-7, d0+8..15) (rows 8-15, d0+8..15), transposed
       uint32_t vb[4];
       ldmatrix_x4_trans(vb, vt + swz(lm_r + 8 * (lm_m & 1), jj * 2 + (lm_m >> 1)));
-      mma_bf16(o[2 * jj], p_hi, vb[0], vb[1]);
-      mma_bf16(o[2 * jj], p_lo, vb[0], vb[1]);
-      mma_bf16(o[2 * jj + 1], p_hi, vb[2], vb[3]);
-      mma_bf16(o[2 * jj + 1], p_lo, vb[2], vb[3]);
+      if constexpr (TWO) {
+        mma_bf16(o[2 * jj], p_hi, vb[0], vb[1]);
+        mma_bf16(o[2 * jj], p_lo, vb[0], vb[1]);
+        mma_bf16(o[2 * jj + 1], p_hi, vb[2], vb[3]);
+        mma_bf16(o[2 * jj + 1], p_lo, vb[2], vb[3]);
+      } else {
+        mma_bf16_top(o[2 * jj], p_hi[0], p_hi[1], vb[0], vb[1]);
+        mma_bf16_top(o[2 * jj], p_lo[0], p_lo[1], vb[0], vb[1]);
+        mma_bf16_top(o[2 * jj + 1], p_hi[0], p_hi[1], vb[2], vb[3]);
+        mma_bf16_top(o[2 * jj + 1], p_lo[0], p_lo[1], vb[2], vb[3]);
+      }
     }
     __syncwarp();
     if (lane == 0 && uv + NB < n_ops) {
@@ -301,7 +328,7 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
 
   // ---- chunk partial: (max, sum) and the un-normalised weighted V sums ------------------
 #pragma unroll
-  for (int rr = 0; rr < 2; ++rr) {
+  for (int rr = 0; rr < R; ++rr) {
     const int head = qrow + 8 * rr;
     float lsum = l[rr];
     lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
