@@ -121,13 +121,14 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
       static_cast<const unsigned char*>(p.V) + (((size_t)b * p.Hkv + kvh) * p.cap + row_begin) * RB;
 
   const int n_ops = 2 * ntiles;        // operand tiles: u = 2t is K_t, u = 2t+1 is V_t
+  const uint64_t stream_policy = l2_policy_evict_first();
   auto issue = [&](int u) {            // lane 0 only
     const int t = u >> 1;
     const uint32_t bytes = (uint32_t)min(TILE_ROWS, rows - t * TILE_ROWS) * RB;
     uint64_t* bar = &bars[u % NB];
     mbar_expect_tx(bar, bytes);
-    bulk_g2s(ring + (size_t)(u % NB) * TILE_BYTES, ((u & 1) ? v_src : k_src) + (size_t)t * TILE_BYTES, bytes,
-             bar);
+    bulk_g2s_hint(ring + (size_t)(u % NB) * TILE_BYTES, ((u & 1) ? v_src : k_src) + (size_t)t * TILE_BYTES, bytes,
+                  bar, stream_policy);
   };
   // Early prefetch.  The previous step's combine kernel may still be running:
   // the only thing it writes to the state is one row per sequence (the slot its

@@ -24,11 +24,12 @@ namespace tova {
 
 constexpr int MMA_UNIT_HEADS = 16;  // query heads one MMA split warp carries
 
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar,
+                                            uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-          smem_addr(dst)),
-      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_addr(bar))
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, "
+      "%3}], [%4], %5;" ::"r"(smem_addr(dst)),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_addr(bar)), "l"(policy)
       : "memory");
 }
 
@@ -114,13 +115,15 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
 
   const int y0 = ((b * p.Hkv + kvh) * p.cap) + row_begin;   // first row of the chunk in the [rows, D] view
   const int n_ops = 2 * ntiles;                             // u = 2t: K_t, u = 2t+1: V_t
+  const uint64_t stream_policy = l2_policy_evict_first();   // K/V rows are read once per step
   auto issue = [&](int u) {                                 // lane 0 only
     uint64_t* bar = &bars[u % NB];
     unsigned char* dst = ring + (size_t)(u % NB) * TILE_BYTES;
     mbar_expect_tx(bar, TILE_BYTES);                        // a tiled copy always delivers the whole box
 #pragma unroll
     for (int bx = 0; bx < NBOX; ++bx)
-      tma_load_2d(dst + bx * (TILE_ROWS * 128), (u & 1) ? &map_v : &map_k, bx * 64, y0 + (u >> 1) * TILE_ROWS, bar);
+      tma_load_2d(dst + bx * (TILE_ROWS * 128), (u & 1) ? &map_v : &map_k, bx * 64, y0 + (u >> 1) * TILE_ROWS, bar,
+                  stream_policy);
   };
   // Early prefetch before the dependency wait: only the row the previous step's
   // token went to (last_slot) can still change; it is fetched again after the
