@@ -153,21 +153,23 @@ cudaError_t launch_split_g(int dev, int G, const StepParams& p, dim3 grid, cudaS
 // Dynamic shared memory of the combine kernel: all (max, sum) partials of a
 // sequence, per-head max and 1/sum, one float per thread, and the new token's
 // rows when they are small enough to be staged.
-inline size_t combine_smem_bytes(int H, int n_partials, int threads, size_t row_bytes) {
+inline size_t combine_smem_bytes(int H, int n_partials, int threads, size_t row_bytes, size_t logit_bytes) {
   size_t b = sizeof(float) * (2 * (size_t)H * n_partials + 3 * (size_t)H + threads) + 16;
   if (2 * row_bytes <= (size_t)tova::COMBINE_ROW_STAGE_BYTES) b += 2 * row_bytes;
-  return b;
+  return b + logit_bytes;
 }
-constexpr size_t COMBINE_SMEM_LIMIT = 160 * 1024;
+constexpr size_t COMBINE_SMEM_LIMIT = 200 * 1024;   // opt-in maximum of the combine kernel
+constexpr size_t COMBINE_BASE_LIMIT = 100 * 1024;   // partials + rows; staged logits come on top
 // upper bound used when choosing chunk sizes (largest CTA, rows staged)
 inline size_t combine_smem_bound(int H, int n_partials) {
-  return combine_smem_bytes(H, n_partials, tova::COMBINE_THREADS_LARGE, 0) + tova::COMBINE_ROW_STAGE_BYTES;
+  return combine_smem_bytes(H, n_partials, tova::COMBINE_THREADS_LARGE, 0, 0) + tova::COMBINE_ROW_STAGE_BYTES;
 }
 
 template <typename T, int D, int CT>
 cudaError_t launch_combine_ct(int dev, const StepParams& p, cudaStream_t st) {
   const size_t row_bytes = (size_t)p.Hkv * D * sizeof(T);
-  const size_t smem = combine_smem_bytes(p.H, p.n_chunks + 1, CT, row_bytes);
+  const size_t logit_bytes = p.stage_logits ? (size_t)p.H * p.cand_per_cta * sizeof(float) : 0;
+  const size_t smem = combine_smem_bytes(p.H, p.n_chunks + 1, CT, row_bytes, logit_bytes);
   auto kern = tova::tova_combine_kernel<T, D, CT>;
   static bool attr_set[64] = {};
   if (!attr_set[dev & 63]) {
@@ -275,7 +277,7 @@ int pick_chunk_rows(const tova_config& cfg, int sm_count) {
     const long long rounds = (units + slots - 1) / slots;
     const long long rows = cr < cfg.capacity ? cr : cfg.capacity;
     const long long cost = rounds * (rows + 24);
-    if (combine_smem_bound(cfg.n_q_heads, (int)chunks + 1) > COMBINE_SMEM_LIMIT) continue;
+    if (combine_smem_bound(cfg.n_q_heads, (int)chunks + 1) > COMBINE_BASE_LIMIT) continue;
     if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best = cr; }
     if (cr >= cfg.capacity) break;
   }
@@ -308,7 +310,13 @@ void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows)
   if (nx < 1) nx = 1;
   p.combine_threads = ct;
   p.nx = nx;
-  p.cand_per_cta = (n + 1 + nx - 1) / nx;
+  p.cand_per_cta = ((n + 1 + nx - 1) / nx + 3) / 4 * 4;   // a multiple of 4: 16-byte aligned blocks of logits
+  // Stage a CTA's logits through shared memory (bulk copies) only when a thread
+  // would otherwise need several dependent batches of loads for them.
+  const long long per_thread = (long long)cfg.n_q_heads * p.cand_per_cta / ct;
+  p.stage_logits =
+      p.do_evict && per_thread > 3 * lg &&
+      (size_t)cfg.n_q_heads * p.cand_per_cta * sizeof(float) <= (size_t)tova::COMBINE_LOGIT_STAGE_BYTES;
 }
 
 int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_t pos, float* out,
@@ -458,7 +466,7 @@ int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows) {
   if (rows == 0) { c->chunk_rows = pick_chunk_rows(c->cfg, c->sm_count); return TOVA_OK; }  // fits: init checked
   if (rows < tova::MIN_CHUNK_ROWS || rows > 8192 || rows % tova::MIN_CHUNK_ROWS != 0) return TOVA_ERR_BAD_SHAPE;
   const int chunks = (c->cfg.capacity + rows - 1) / rows;
-  if (combine_smem_bound(c->cfg.n_q_heads, chunks + 1) > COMBINE_SMEM_LIMIT) return TOVA_ERR_BAD_SHAPE;
+  if (combine_smem_bound(c->cfg.n_q_heads, chunks + 1) > COMBINE_BASE_LIMIT) return TOVA_ERR_BAD_SHAPE;
   c->chunk_rows = rows;
   return TOVA_OK;
 }

@@ -27,6 +27,7 @@ constexpr int SPLIT_BUFFERS = 3;    // tile buffers of a split warp's ring (K an
 constexpr int MAX_UNIT_HEADS = 8;   // query heads one split warp carries
 constexpr int COMBINE_THREADS_SMALL = 256;  // combine CTA size when many CTAs are in flight
 constexpr int COMBINE_THREADS_LARGE = 512;  // ... when the batch is small: more loads in flight per sequence
+constexpr int COMBINE_LOGIT_STAGE_BYTES = 96 * 1024;  // a combine CTA's [H][candidates] logits, staged if they fit
 constexpr int COMBINE_ROW_STAGE_BYTES = 16 * 1024;  // new-token rows (k and v) staged in shared memory up to this size
 constexpr int COMBINE_CLUSTER_MAX = 8;  // CTAs per sequence in the combine kernel (portable cluster size)
 constexpr int MIN_CHUNK_ROWS = 32;      // smallest chunk the scratch is sized for
@@ -60,6 +61,7 @@ struct StepParams {
   int32_t nx;         // combine CTAs per sequence = cluster size (1..COMBINE_CLUSTER_MAX)
   int32_t cand_per_cta;  // candidates scored per combine CTA
   int32_t combine_threads;  // COMBINE_THREADS_SMALL or COMBINE_THREADS_LARGE
+  int32_t stage_logits;     // combine CTAs bulk-copy their block of logits to shared memory
   int32_t do_evict;   // n == cap and the policy is on
   float scale2;       // sm_scale * log2(e)
 };
@@ -340,7 +342,9 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
 //      table (Eq. 9, in place).  No global atomics, no CTA waits on a flag.
 // smem: float2 pml[H][np]; float hM[H], hInvL[H], hLc[H], sc[CT]; then, in
 // CTA 0 only, the new token's k and v rows of all KV heads (bulk-copied in at
-// the start when they fit COMBINE_ROW_STAGE_BYTES each).
+// the start when they fit COMBINE_ROW_STAGE_BYTES); then the CTA's
+// [H][cand_per_cta] block of logits (bulk-copied in at the start when the host
+// says it fits).
 template <typename T, int D, int CT>
 __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_combine_kernel(const StepParams p) {
   namespace cg = cooperative_groups;
@@ -358,6 +362,7 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
   unsigned char* row_stage = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(sc + CT) + 15) & ~uintptr_t(15));     // [2][Hkv*D*sizeof(T)]
   __shared__ __align__(8) uint64_t row_bar;
+  __shared__ __align__(8) uint64_t lg_bar;
   __shared__ float red_v[CT / 32];
   __shared__ int red_i[CT / 32];
   __shared__ int red_p[CT / 32];
@@ -389,10 +394,17 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
   const int total_ml = p.H * np;
   const uint32_t row_bytes = (uint32_t)row_words * 16u;          // all KV heads of one operand
   const bool staged = (x == 0) && 2 * row_bytes <= (uint32_t)COMBINE_ROW_STAGE_BYTES;
-  if (staged && tid == 0) {
+  // staged logits: rows of cand_per_cta floats (a multiple of 4), one per head
+  float* lg_stage = reinterpret_cast<float*>(
+      row_stage + (2 * row_bytes <= (uint32_t)COMBINE_ROW_STAGE_BYTES ? 2 * row_bytes : 0));
+  const int lg_cols = max(min(p.cand_per_cta, p.ld - j_begin), 0);   // floats per head row actually copied
+  const bool lg_staged = p.do_evict && p.stage_logits && lg_cols > 0;
+  if (tid == 0) {
     mbar_init(&row_bar, 1);
+    mbar_init(&lg_bar, 1);
     mbar_fence_init();
   }
+  __syncthreads();
 
   pdl_wait();
   pdl_launch_dependents();
@@ -401,6 +413,13 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
     bulk_g2s(row_stage, static_cast<const unsigned char*>(p.k_new) + (size_t)b * row_bytes, row_bytes, &row_bar);
     bulk_g2s(row_stage + row_bytes, static_cast<const unsigned char*>(p.v_new) + (size_t)b * row_bytes, row_bytes,
              &row_bar);
+  }
+  if (lg_staged && warp == 1) {    // this CTA's block of logits: one bulk copy per head
+    if (lane == 0) mbar_expect_tx(&lg_bar, (uint32_t)p.H * (uint32_t)lg_cols * 4u);
+    __syncwarp();
+    for (int h = lane; h < p.H; h += 32)
+      bulk_g2s(lg_stage + (size_t)h * p.cand_per_cta, p.logits + ((size_t)b * p.H + h) * p.ld + j_begin,
+               (uint32_t)lg_cols * 4u, &lg_bar);
   }
 
   // ---- 0. every load this thread needs, issued back to back ---------------------
@@ -420,7 +439,7 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
 #pragma unroll
     for (int u = 0; u < LG; ++u) {
       const int h = hs + u * hs_n;
-      r_lg[u] = (live && h < p.H) ? lg[(size_t)h * p.ld] : 0.f;
+      r_lg[u] = (live && !lg_staged && h < p.H) ? lg[(size_t)h * p.ld] : 0.f;
     }
     if (live && hs == 0 && j < p.cap) r_pos = p.pos[(size_t)b * p.cap + j];
   }
@@ -534,13 +553,22 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_
   float val = INFINITY;
   int idx = 0x7fffffff;
   int cpos = pos_t;                // position held by the best candidate (the new token holds pos_t)
+  bool lg_ok = true;
+  if (lg_staged && !mbar_wait_bounded(&lg_bar, 0)) {
+    lg_ok = false;                 // read the logits from global memory instead
+    if (tid == 0) atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
+  }
   for (int j0 = j_begin; j0 < j_end; j0 += wp) {
     const int j = j0 + jl;
     const bool live = j < j_end;
     float a = 0.f;
     if (live) {
       const float* lg = p.logits + (size_t)b * p.H * p.ld + j;
-      if (j0 == j_begin) {
+      if (lg_staged && lg_ok) {
+        const float* sl = lg_stage + (j - j_begin);
+#pragma unroll 8
+        for (int h = hs; h < p.H; h += hs_n) a += exp2f(sl[(size_t)h * p.cand_per_cta] + hLc[h]);
+      } else if (j0 == j_begin && !lg_staged) {
 #pragma unroll
         for (int u = 0; u < LG; ++u) {
           const int h = hs + u * hs_n;
