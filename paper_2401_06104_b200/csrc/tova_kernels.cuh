@@ -61,6 +61,7 @@ struct StepParams {
   int32_t nx;         // combine CTAs per sequence = cluster size (1..COMBINE_CLUSTER_MAX)
   int32_t cand_per_cta;  // candidates scored per combine CTA
   int32_t combine_threads;  // COMBINE_THREADS_SMALL or COMBINE_THREADS_LARGE
+  int32_t combine_deep;     // deep register prefetch variant (small batches)
   int32_t stage_logits;     // combine CTAs bulk-copy their block of logits to shared memory
   int32_t do_evict;   // n == cap and the policy is on
   float scale2;       // sm_scale * log2(e)
@@ -345,10 +346,11 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
 // the start when they fit COMBINE_ROW_STAGE_BYTES); then the CTA's
 // [H][cand_per_cta] block of logits (bulk-copied in at the start when the host
 // says it fits).
-template <typename T, int D, int CT>
-__global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 1) tova_combine_kernel(const StepParams p) {
+// BIG: deep register prefetch (one CTA per SM); otherwise 64 registers per thread.
+template <typename T, int D, int CT, bool BIG>
+__global__ void __launch_bounds__(CT, BIG ? 1 : (CT == COMBINE_THREADS_SMALL ? 4 : 2))
+    tova_combine_kernel(const StepParams p) {
   namespace cg = cooperative_groups;
-  constexpr bool BIG = (CT == COMBINE_THREADS_LARGE);
   constexpr int ML = BIG ? 4 : 2;    // partial pairs prefetched per thread
   constexpr int LG = BIG ? 16 : 8;   // logits prefetched per thread
   constexpr int AC = BIG ? 8 : 4;    // weighted V sums prefetched per thread
