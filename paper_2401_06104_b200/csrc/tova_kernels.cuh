@@ -353,7 +353,7 @@ __global__ void __launch_bounds__(CT, BIG ? 1 : (CT == COMBINE_THREADS_SMALL ? 4
   namespace cg = cooperative_groups;
   constexpr int ML = BIG ? 4 : 2;    // partial pairs prefetched per thread
   constexpr int LG = BIG ? 16 : 8;   // logits prefetched per thread
-  constexpr int AC = BIG ? 8 : 4;    // weighted V sums prefetched per thread
+  constexpr int AC = BIG ? 8 : 2;    // weighted V sums (float4) prefetched per thread
   extern __shared__ __align__(16) float csm[];
   const int np = p.n_chunks + 1;   // partials per head: the chunks, then the new token
   float2* pml = reinterpret_cast<float2*>(csm);                  // [H][np]
@@ -384,13 +384,18 @@ __global__ void __launch_bounds__(CT, BIG ? 1 : (CT == COMBINE_THREADS_SMALL ? 4
   // When a victim is due, CTA 0 is on the critical path (arg-min, insert): if
   // the output merge is light (few chunks), the output elements are shared among
   // its peers and written after they arrive at the cluster barrier.
-  const bool late_out = p.do_evict && p.nx > 1 && p.n_chunks <= AC;   // only when the merge is light
+  const bool late_out = p.do_evict && p.nx > 1 && p.n_chunks <= 8;   // only when the merge is light
   const int out_ctas = late_out ? p.nx - 1 : p.nx;
   const int out_x = late_out ? x - 1 : x;      // -1: no share
-  const int items = p.H * D;
-  const int per = (items + out_ctas - 1) / out_ctas;
-  const int it_end = out_x < 0 ? 0 : min(items, (out_x + 1) * per);
-  const int it0 = out_x < 0 ? 0 : out_x * per + tid;
+  // Output work item = (head, 4 consecutive dims, slice of the chunks): S lanes
+  // next to each other share an output quad, each merging every S-th chunk with
+  // 16-byte loads; their sums are folded by shuffles.
+  const int items4 = p.H * (D / 4);
+  const int out_threads = out_ctas * CT;
+  int S = 1;
+  while (S < 32 && 2 * S * items4 <= out_threads && 2 * S <= p.n_chunks) S <<= 1;
+  const int work = items4 * S;                 // a multiple of 32 whenever S > 1
+  const int g0 = out_x < 0 ? work : out_x * CT + tid;
   constexpr int RB16 = D * (int)sizeof(T) / 16;  // 16-byte words per row
   const int row_words = p.Hkv * RB16;
   const int total_ml = p.H * np;
@@ -445,17 +450,19 @@ __global__ void __launch_bounds__(CT, BIG ? 1 : (CT == COMBINE_THREADS_SMALL ? 4
     }
     if (live && hs == 0 && j < p.cap) r_pos = p.pos[(size_t)b * p.cap + j];
   }
-  float r_acc[AC];
-  float r_vn = 0.f;
-  if (it0 < it_end) {
-    const int h = it0 / D, d = it0 % D;
-    const float* acc = p.part_acc + ((size_t)b * p.H + h) * (size_t)(p.pc - 1) * D + d;
+  float4 r_acc[AC];
+  if (g0 < work) {
+    const int it = g0 / S, cs = g0 % S;
+    const int h = it / (D / 4), d4 = it % (D / 4);
+    const float4* acc = reinterpret_cast<const float4*>(p.part_acc + ((size_t)b * p.H + h) * (size_t)(p.pc - 1) * D) + d4;
 #pragma unroll
-    for (int u = 0; u < AC; ++u) r_acc[u] = (u < p.n_chunks) ? acc[(size_t)u * D] : 0.f;
-    r_vn = (float)static_cast<const T*>(p.v_new)[((size_t)b * p.Hkv + h / p.G) * D + d];
+    for (int u = 0; u < AC; ++u) {
+      const int i = cs + u * S;
+      r_acc[u] = (i < p.n_chunks) ? acc[(size_t)i * (D / 4)] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
   } else {
 #pragma unroll
-    for (int u = 0; u < AC; ++u) r_acc[u] = 0.f;
+    for (int u = 0; u < AC; ++u) r_acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
 
   // Writes the new token's k and v into row `slot` of every KV head (CTA 0 only).
@@ -511,28 +518,44 @@ __global__ void __launch_bounds__(CT, BIG ? 1 : (CT == COMBINE_THREADS_SMALL ? 4
 
   // ---- 2. this CTA's share of the attention output --------------------------------
   auto write_outputs = [&]() {
-  for (int it = it0; it < it_end; it += CT) {
-    const int h = it / D, d = it % D;
-    const size_t bh = (size_t)b * p.H + h;
-    const float2* ml = pml + (size_t)h * np;
-    const float* acc = p.part_acc + bh * (size_t)(p.pc - 1) * D + d;
-    const float M = hM[h];
-    float o = 0.f;
-    if (it == it0) {
+    for (int g = g0; g < work; g += out_threads) {   // whole warps run the same trips (see `work`)
+      const int it = g / S, cs = g % S;
+      const int h = it / (D / 4), d4 = it % (D / 4);
+      const size_t bh = (size_t)b * p.H + h;
+      const float2* ml = pml + (size_t)h * np;
+      const float4* acc = reinterpret_cast<const float4*>(p.part_acc + bh * (size_t)(p.pc - 1) * D) + d4;
+      const float M = hM[h];
+      float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+      int i = cs;
+      if (g == g0) {
 #pragma unroll
-      for (int u = 0; u < AC; ++u)
-        if (u < p.n_chunks) o = fmaf(r_acc[u], exp2_diff(ml[u].x, M), o);
-#pragma unroll 8
-      for (int i = AC; i < p.n_chunks; ++i) o = fmaf(acc[(size_t)i * D], exp2_diff(ml[i].x, M), o);
-      o = fmaf(r_vn, exp2_diff(ml[p.n_chunks].x, M), o);
-    } else {
-#pragma unroll 8
-      for (int i = 0; i < p.n_chunks; ++i) o = fmaf(acc[(size_t)i * D], exp2_diff(ml[i].x, M), o);
-      const float vn = (float)static_cast<const T*>(p.v_new)[((size_t)b * p.Hkv + h / p.G) * D + d];
-      o = fmaf(vn, exp2_diff(ml[p.n_chunks].x, M), o);
+        for (int u = 0; u < AC; ++u) {
+          if (i < p.n_chunks) {
+            const float w = exp2_diff(ml[i].x, M);
+            o.x = fmaf(r_acc[u].x, w, o.x); o.y = fmaf(r_acc[u].y, w, o.y);
+            o.z = fmaf(r_acc[u].z, w, o.z); o.w = fmaf(r_acc[u].w, w, o.w);
+          }
+          i += S;
+        }
+      }
+#pragma unroll 4
+      for (; i < p.n_chunks; i += S) {
+        const float4 a = acc[(size_t)i * (D / 4)];
+        const float w = exp2_diff(ml[i].x, M);
+        o.x = fmaf(a.x, w, o.x); o.y = fmaf(a.y, w, o.y); o.z = fmaf(a.z, w, o.z); o.w = fmaf(a.w, w, o.w);
+      }
+      for (int off = S >> 1; off >= 1; off >>= 1) {
+        o.x += __shfl_xor_sync(0xffffffffu, o.x, off); o.y += __shfl_xor_sync(0xffffffffu, o.y, off);
+        o.z += __shfl_xor_sync(0xffffffffu, o.z, off); o.w += __shfl_xor_sync(0xffffffffu, o.w, off);
+      }
+      if (cs == 0) {
+        const T* vn = static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + h / p.G) * D + d4 * 4;
+        const float w = exp2_diff(ml[p.n_chunks].x, M), iL = hInvL[h];
+        o.x = fmaf((float)vn[0], w, o.x) * iL; o.y = fmaf((float)vn[1], w, o.y) * iL;
+        o.z = fmaf((float)vn[2], w, o.z) * iL; o.w = fmaf((float)vn[3], w, o.w) * iL;
+        reinterpret_cast<float4*>(p.out + bh * D)[d4] = o;
+      }
     }
-    p.out[bh * D + d] = o * hInvL[h];
-  }
   };
   if (!late_out) write_outputs();
 
