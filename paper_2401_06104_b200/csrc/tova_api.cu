@@ -165,12 +165,12 @@ inline size_t combine_smem_bound(int H, int n_partials) {
   return combine_smem_bytes(H, n_partials, tova::COMBINE_THREADS_LARGE, 0, 0) + tova::COMBINE_ROW_STAGE_BYTES;
 }
 
-template <typename T, int D, int CT, bool BIG>
+template <typename T, int D, int CT>
 cudaError_t launch_combine_ct(int dev, const StepParams& p, cudaStream_t st) {
   const size_t row_bytes = (size_t)p.Hkv * D * sizeof(T);
   const size_t logit_bytes = p.stage_logits ? (size_t)p.H * p.cand_per_cta * sizeof(float) : 0;
   const size_t smem = combine_smem_bytes(p.H, p.n_chunks + 1, CT, row_bytes, logit_bytes);
-  auto kern = tova::tova_combine_kernel<T, D, CT, BIG>;
+  auto kern = tova::tova_combine_kernel<T, D, CT>;
   static bool attr_set[64] = {};
   if (!attr_set[dev & 63]) {
     cudaError_t e =
@@ -197,10 +197,9 @@ cudaError_t launch_combine_ct(int dev, const StepParams& p, cudaStream_t st) {
 
 template <typename T, int D>
 cudaError_t launch_combine(int dev, const StepParams& p, cudaStream_t st) {
-  if (p.combine_threads == tova::COMBINE_THREADS_LARGE)
-    return p.combine_deep ? launch_combine_ct<T, D, tova::COMBINE_THREADS_LARGE, true>(dev, p, st)
-                          : launch_combine_ct<T, D, tova::COMBINE_THREADS_LARGE, false>(dev, p, st);
-  return launch_combine_ct<T, D, tova::COMBINE_THREADS_SMALL, false>(dev, p, st);
+  return p.combine_threads == tova::COMBINE_THREADS_LARGE
+             ? launch_combine_ct<T, D, tova::COMBINE_THREADS_LARGE>(dev, p, st)
+             : launch_combine_ct<T, D, tova::COMBINE_THREADS_SMALL>(dev, p, st);
 }
 
 template <int D, bool TWO>
@@ -294,24 +293,20 @@ void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows)
   p.n_chunks = (n + chunk_rows - 1) / chunk_rows;
   p.hgroups = (p.G + unit_heads(cfg) - 1) / unit_heads(cfg);
   p.do_evict = (n == cfg.capacity) ? 1 : 0;
-  // Combine CTAs per sequence (one cluster).  A small batch gets 512-thread CTAs
-  // with a deep register prefetch (one CTA per SM is enough), a medium one
-  // 512-thread CTAs with a light prefetch (two per SM), a large one 256-thread
-  // CTAs (four per SM).  Per thread: about one output element and at most LG
-  // logits per pass.
+  // Combine CTAs per sequence (one cluster): 512-thread CTAs (two per SM)
+  // while they all fit on the GPU at once, else 256-thread CTAs (four per SM).
+  // Per thread: about one output quad and at most 8 logits per pass.
   const int sm_guess = 148;
-  const long long ctas = (long long)cfg.batch * tova::COMBINE_CLUSTER_MAX;
-  const bool deep = ctas <= sm_guess;                  // 512 threads, deep prefetch, one CTA per SM
-  const bool wide = !deep && ctas <= 2 * sm_guess;     // 512 threads, light prefetch, two CTAs per SM
-  const int ct = (deep || wide) ? tova::COMBINE_THREADS_LARGE : tova::COMBINE_THREADS_SMALL;
-  const int lg = deep ? 16 : 8;
-  p.combine_deep = deep ? 1 : 0;
+  const int cl_max = tova::COMBINE_CLUSTER_MAX;
+  const long long ctas = (long long)cfg.batch * cl_max;
+  const int ct = ctas <= 2 * sm_guess ? tova::COMBINE_THREADS_LARGE : tova::COMBINE_THREADS_SMALL;
+  const int lg = 8;
   const long long items = (long long)cfg.n_q_heads * cfg.head_dim;
   int nx = (int)((items + ct - 1) / ct);
   const long long score_loads = (long long)(n + 1) * cfg.n_q_heads;
   const int by_scores = (int)((score_loads + (long long)lg * ct - 1) / ((long long)lg * ct));
   if (p.do_evict && nx < by_scores) nx = by_scores;
-  if (nx > tova::COMBINE_CLUSTER_MAX) nx = tova::COMBINE_CLUSTER_MAX;
+  if (nx > cl_max) nx = cl_max;
   if (nx < 1) nx = 1;
   p.combine_threads = ct;
   p.nx = nx;

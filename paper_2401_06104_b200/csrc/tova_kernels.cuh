@@ -29,7 +29,8 @@ constexpr int COMBINE_THREADS_SMALL = 256;  // combine CTA size when many CTAs a
 constexpr int COMBINE_THREADS_LARGE = 512;  // ... when the batch is small: more loads in flight per sequence
 constexpr int COMBINE_LOGIT_STAGE_BYTES = 96 * 1024;  // a combine CTA's [H][candidates] logits, staged if they fit
 constexpr int COMBINE_ROW_STAGE_BYTES = 16 * 1024;  // new-token rows (k and v) staged in shared memory up to this size
-constexpr int COMBINE_CLUSTER_MAX = 8;  // CTAs per sequence in the combine kernel (portable cluster size)
+constexpr int COMBINE_CLUSTER_MAX = 8;  // CTAs per sequence in the combine kernel (portable cluster size;
+                                        // clusters of 16 were measured slower)
 constexpr int MIN_CHUNK_ROWS = 32;      // smallest chunk the scratch is sized for
 
 struct StepParams {
@@ -61,7 +62,6 @@ struct StepParams {
   int32_t nx;         // combine CTAs per sequence = cluster size (1..COMBINE_CLUSTER_MAX)
   int32_t cand_per_cta;  // candidates scored per combine CTA
   int32_t combine_threads;  // COMBINE_THREADS_SMALL or COMBINE_THREADS_LARGE
-  int32_t combine_deep;     // deep register prefetch variant (small batches)
   int32_t stage_logits;     // combine CTAs bulk-copy their block of logits to shared memory
   int32_t do_evict;   // n == cap and the policy is on
   float scale2;       // sm_scale * log2(e)
@@ -346,11 +346,11 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
 // the start when they fit COMBINE_ROW_STAGE_BYTES); then the CTA's
 // [H][cand_per_cta] block of logits (bulk-copied in at the start when the host
 // says it fits).
-// BIG: deep register prefetch (one CTA per SM); otherwise 64 registers per thread.
-template <typename T, int D, int CT, bool BIG>
-__global__ void __launch_bounds__(CT, BIG ? 1 : (CT == COMBINE_THREADS_SMALL ? 4 : 2))
-    tova_combine_kernel(const StepParams p) {
+// 64 registers per thread: CTAs of the next kernel can share the SM with them.
+template <typename T, int D, int CT>
+__global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_combine_kernel(const StepParams p) {
   namespace cg = cooperative_groups;
+  constexpr bool BIG = false;
   constexpr int ML = BIG ? 4 : 2;    // partial pairs prefetched per thread
   constexpr int LG = BIG ? 16 : 8;   // logits prefetched per thread
   constexpr int AC = BIG ? 8 : 2;    // weighted V sums (float4) prefetched per thread
