@@ -43,6 +43,8 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="independent layer caches to rotate over (0 = auto)")
     ap.add_argument("--chunk-rows", type=int, default=0)
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of CUDA graphs")
+    ap.add_argument("--no-deferred", action="store_true",
+                    help="pick the victim on the caller's stream instead of overlapping it with the next layer's step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
@@ -229,7 +231,9 @@ def run_ours(args):
     w = pick_workload(args)
     B, H, Hkv, D, cap = w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity
     step_bytes = w.step_bytes()
-    L = args.layers or max(1, -(-WORKING_SET // step_bytes))
+    # at least two layers: consecutive steps then belong to different caches, as in a model
+    L = args.layers or max(2, -(-WORKING_SET // step_bytes))
+    deferred = not args.no_deferred and L >= 2
     ring = W.tokens(w, 0, RING)                                   # seeded, host
     dq, dk, dv = (tova.to_device(a, w.dtype, dev) for a in ring)
 
@@ -253,6 +257,13 @@ def run_ours(args):
     torch.cuda.synchronize()
     for c in caches:
         assert c.tova_cache_len() == cap
+        if deferred:
+            c.tova_cache_set_deferred_eviction(True)
+
+    def join_all():
+        if deferred:
+            for c in caches:
+                c.tova_cache_join()
 
     counter = [0]
 
@@ -267,6 +278,7 @@ def run_ours(args):
             counter[0] += 1
 
     run_direct(min(64, max(args.warmup, 3)))                      # sets function attributes before capture
+    join_all()
     torch.cuda.synchronize()
 
     graph, G = None, 0
@@ -280,6 +292,7 @@ def run_ours(args):
             with torch.cuda.graph(graph):
                 for j in range(G):
                     step(base + j)
+                join_all()                                        # side streams rejoin before the capture ends
             launch_mode = "cuda_graph"
         except Exception as e:  # pragma: no cover
             print(f"bench.py: graph capture failed ({e}); launching from the host", file=sys.stderr)
@@ -292,6 +305,7 @@ def run_ours(args):
                 graph.replay()
             n = n % G
         run_direct(n)
+        join_all()
 
     launches_before = sum(c.tova_cache_launches() for c in caches)
     run(max(args.warmup, 3))
@@ -362,6 +376,8 @@ def run_ours(args):
         "config": workload_config(w, {
             "layers_rotated": L, "working_set_bytes": L * step_bytes, "l2": "inputs larger than L2",
             "launch": launch_mode, "graph_steps": G, "bytes_per_step": step_bytes,
+            "eviction": "deferred to the cache's side stream, overlaps the next layer's step" if deferred
+                        else "on the caller's stream",
             "parallelism": "replicas only" if world > 1 else "single GPU"}),
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                      "traffic": recorded_traffic(w, step_bytes), "peak_kind": peak_kind,
@@ -369,7 +385,7 @@ def run_ours(args):
                      "note": "algorithmic bytes (K/V read + one slot written) / whole-step time (split + combine kernels)"},
         "cpu_baseline": cpu,
         "e2e": e2e,
-        "gpu_launches": 2 * args.steps,
+        "gpu_launches": (3 if deferred else 2) * args.steps,
         "clocks": clocks,
     }
     print(json.dumps(line))

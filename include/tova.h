@@ -121,6 +121,29 @@ int tova_decode_step_host(tova_cache* c, const void* q_host, const void* k_host,
 int tova_cache_read(const tova_cache* c, int32_t* len, int32_t* positions, void* k_out,
                     void* v_out, int32_t* status, void* cuda_stream);
 
+/* Deferred eviction (off by default).  The attention output of a step is what
+ * the rest of a model waits for; which row is dropped (Algorithm 1) only has
+ * to be settled before the SAME cache sees its next token, a whole model pass
+ * later.  With on != 0, tova_decode_step enqueues attention and output on the
+ * caller's stream, while the head average, the arg-min and the in-place insert
+ * run on a stream the cache owns and overlap whatever the caller enqueues
+ * next (normally the next layer's step).  Consequences for the caller:
+ *   - `out` is ready in stream order as before; `evicted_pos`, and the state as
+ *     tova_cache_read sees it, are ready only after tova_cache_join;
+ *   - the next tova_decode_step / tova_prefill on this cache waits for the
+ *     pending eviction by itself; the k and v buffers may be reused at once
+ *     (the library keeps copies), `evicted_pos` must stay valid until the join;
+ *   - when capturing a CUDA graph, call tova_cache_join on the capturing
+ *     stream for every cache before the capture ends, and have no eviction
+ *     pending when it begins.
+ * Results are identical to the default mode.  tova_prefill and
+ * tova_decode_step_host always run undeferred.  Switching off with an eviction
+ * pending is refused (TOVA_ERR_BAD_SHAPE): join first. */
+int tova_cache_set_deferred_eviction(tova_cache* c, int32_t on);
+
+/* Make `cuda_stream` wait for this cache's pending deferred eviction, if any. */
+int tova_cache_join(tova_cache* c, void* cuda_stream);
+
 /* Tuning: rows of the state one warp of the streaming kernel covers (a multiple
  * of 32 up to 8192; 0 restores the automatic choice made at init).  Results do
  * not depend on it beyond floating-point summation order. */

@@ -58,6 +58,10 @@ def lib() -> ctypes.CDLL:
         L.tova_cache_read.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.tova_cache_set_chunk_rows.restype = ctypes.c_int
         L.tova_cache_set_chunk_rows.argtypes = [vp, i32]
+        L.tova_cache_set_deferred_eviction.restype = ctypes.c_int
+        L.tova_cache_set_deferred_eviction.argtypes = [vp, i32]
+        L.tova_cache_join.restype = ctypes.c_int
+        L.tova_cache_join.argtypes = [vp, vp]
         L.tova_cache_len.restype = i32
         L.tova_cache_len.argtypes = [vp]
         L.tova_cache_launches.restype = i64
@@ -153,6 +157,13 @@ class TovaCache:
 
     def tova_cache_set_chunk_rows(self, rows: int) -> None:
         _check(lib().tova_cache_set_chunk_rows(self._h, int(rows)), "tova_cache_set_chunk_rows")
+
+    def tova_cache_set_deferred_eviction(self, on: bool) -> None:
+        _check(lib().tova_cache_set_deferred_eviction(self._h, 1 if on else 0),
+               "tova_cache_set_deferred_eviction")
+
+    def tova_cache_join(self, stream=None) -> None:
+        _check(lib().tova_cache_join(self._h, _stream(stream)), "tova_cache_join")
 
     def tova_cache_len(self) -> int:
         return int(lib().tova_cache_len(self._h))

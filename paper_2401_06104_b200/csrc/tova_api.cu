@@ -23,6 +23,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 struct Layout {
   size_t K, V, pos, len, last_slot, logits, part_ml, part_acc, status, cur_pos;
   size_t st_q, st_k, st_v, st_out, st_ev;  // staging for host-buffer calls
+  size_t df_k, df_v;                       // the new token's rows kept for a deferred eviction
   size_t total;
   int ld, pc;
 };
@@ -68,6 +69,8 @@ Layout make_layout(const tova_config& c) {
   L.st_v = take(B * Hkv * D * E);
   L.st_out = take(B * H * D * 4);
   L.st_ev = take(B * 4);
+  L.df_k = take(B * Hkv * D * E);
+  L.df_v = take(B * Hkv * D * E);
   L.total = off;
   return L;
 }
@@ -78,6 +81,10 @@ struct tova_cache {
   tova_config cfg;
   CUtensorMap map_k, map_v;  // tiled views of K and V for the tensor-core split kernel
   bool use_mma;
+  // deferred eviction: victim choice and insert run on a side stream, overlapping later work
+  bool deferred, pending;
+  cudaStream_t side;
+  cudaEvent_t ev_fork, ev_join;
   Layout lay;
   unsigned char* base;
   int32_t len;          // rows per sequence (host mirror; sequences move in lock step)
@@ -166,7 +173,7 @@ inline size_t combine_smem_bound(int H, int n_partials) {
 }
 
 template <typename T, int D, int CT>
-cudaError_t launch_combine_ct(int dev, const StepParams& p, cudaStream_t st) {
+cudaError_t launch_combine_ct(int dev, const StepParams& p, cudaStream_t st, bool use_pdl) {
   const size_t row_bytes = (size_t)p.Hkv * D * sizeof(T);
   const size_t logit_bytes = p.stage_logits ? (size_t)p.H * p.cand_per_cta * sizeof(float) : 0;
   const size_t smem = combine_smem_bytes(p.H, p.n_chunks + 1, CT, row_bytes, logit_bytes);
@@ -184,22 +191,29 @@ cudaError_t launch_combine_ct(int dev, const StepParams& p, cudaStream_t st) {
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute at[2];
-  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[0].val.programmaticStreamSerializationAllowed = 1;
-  at[1].id = cudaLaunchAttributeClusterDimension;  // the CTAs of one sequence form a cluster
-  at[1].val.clusterDim.x = p.nx;
-  at[1].val.clusterDim.y = 1;
-  at[1].val.clusterDim.z = 1;
+  int na = 0;
+  if (use_pdl) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  if (p.mode != tova::COMBINE_OUTPUTS) {  // the CTAs of one sequence form a cluster (needed to pick the victim)
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = p.nx;
+    at[na].val.clusterDim.y = 1;
+    at[na].val.clusterDim.z = 1;
+    ++na;
+  }
   cfg.attrs = at;
-  cfg.numAttrs = 2;
+  cfg.numAttrs = na;
   return cudaLaunchKernelEx(&cfg, kern, p);
 }
 
 template <typename T, int D>
-cudaError_t launch_combine(int dev, const StepParams& p, cudaStream_t st) {
+cudaError_t launch_combine(int dev, const StepParams& p, cudaStream_t st, bool use_pdl = true) {
   return p.combine_threads == tova::COMBINE_THREADS_LARGE
-             ? launch_combine_ct<T, D, tova::COMBINE_THREADS_LARGE>(dev, p, st)
-             : launch_combine_ct<T, D, tova::COMBINE_THREADS_SMALL>(dev, p, st);
+             ? launch_combine_ct<T, D, tova::COMBINE_THREADS_LARGE>(dev, p, st, use_pdl)
+             : launch_combine_ct<T, D, tova::COMBINE_THREADS_SMALL>(dev, p, st, use_pdl);
 }
 
 template <int D, bool TWO>
@@ -236,9 +250,14 @@ cudaError_t launch_split_mma(int dev, const StepParams& p, const CUtensorMap& mk
 }
 
 template <typename T, int D>
-cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st) {
+cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, bool defer) {
   dim3 grid(p.n_chunks > 0 ? p.n_chunks : 1, p.Hkv * p.hgroups, p.B);
   cudaError_t e;
+  if (c->pending) {  // the previous token's deferred insert must land before the state is read
+    e = cudaStreamWaitEvent(st, c->ev_join, 0);
+    if (e != cudaSuccess) return e;
+    c->pending = false;
+  }
   if constexpr (std::is_same<T, __nv_bfloat16>::value) {
     e = c->use_mma ? launch_split_mma<D>(c->device, p, c->map_k, c->map_v, grid, st)
                    : launch_split_g<T, D>(c->device, p.G, p, grid, st);
@@ -246,9 +265,33 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st) {
     e = launch_split_g<T, D>(c->device, p.G, p, grid, st);
   }
   if (e != cudaSuccess) return e;
-  e = launch_combine<T, D>(c->device, p, st);
+  if (!defer) {
+    e = launch_combine<T, D>(c->device, p, st);
+    if (e != cudaSuccess) return e;
+    c->launches += 2;
+    return cudaSuccess;
+  }
+  // Deferred eviction: the outputs (what the caller's next kernels need) come
+  // from a launch on the caller's stream; victim choice and insert follow on the
+  // side stream and overlap whatever the caller enqueues next.
+  StepParams pa = p;
+  pa.mode = tova::COMBINE_OUTPUTS;
+  pa.k_stage = c->base + c->lay.df_k;
+  pa.v_stage = c->base + c->lay.df_v;
+  pa.stage_logits = 0;
+  e = launch_combine<T, D>(c->device, pa, st);
   if (e != cudaSuccess) return e;
-  c->launches += 2;
+  if ((e = cudaEventRecord(c->ev_fork, st)) != cudaSuccess) return e;
+  if ((e = cudaStreamWaitEvent(c->side, c->ev_fork, 0)) != cudaSuccess) return e;
+  StepParams pb = p;
+  pb.mode = tova::COMBINE_EVICT;
+  pb.k_new = pa.k_stage;
+  pb.v_new = pa.v_stage;
+  e = launch_combine<T, D>(c->device, pb, c->side, /*use_pdl=*/false);
+  if (e != cudaSuccess) return e;
+  if ((e = cudaEventRecord(c->ev_join, c->side)) != cudaSuccess) return e;
+  c->pending = true;
+  c->launches += 3;
   return cudaSuccess;
 }
 
@@ -320,7 +363,7 @@ void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows)
 }
 
 int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_t pos, float* out,
-              int32_t* evicted_pos, cudaStream_t st) {
+              int32_t* evicted_pos, cudaStream_t st, bool allow_defer = true) {
   const tova_config& cfg = c->cfg;
   const int n = c->len;
   if (n >= cfg.capacity && !cfg.evict) return TOVA_ERR_FULL;
@@ -341,10 +384,12 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
   fill_geometry(p, cfg, n, c->chunk_rows);
   p.scale2 = c->scale2;
   cudaError_t e;
+  const bool defer = c->deferred && allow_defer;
   if (cfg.dtype == TOVA_DTYPE_BF16) {
-    e = cfg.head_dim == 128 ? launch_step<__nv_bfloat16, 128>(c, p, st) : launch_step<__nv_bfloat16, 64>(c, p, st);
+    e = cfg.head_dim == 128 ? launch_step<__nv_bfloat16, 128>(c, p, st, defer)
+                            : launch_step<__nv_bfloat16, 64>(c, p, st, defer);
   } else {
-    e = cfg.head_dim == 128 ? launch_step<float, 128>(c, p, st) : launch_step<float, 64>(c, p, st);
+    e = cfg.head_dim == 128 ? launch_step<float, 128>(c, p, st, defer) : launch_step<float, 64>(c, p, st, defer);
   }
   if (e != cudaSuccess) return TOVA_ERR_CUDA;
   if (c->len < cfg.capacity) c->len += 1;
@@ -428,6 +473,10 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   c->scale2 = c->cfg.sm_scale * 1.4426950408889634f;
   c->elem = cfg->dtype == TOVA_DTYPE_BF16 ? 2 : 4;
   c->row_bytes = c->elem * cfg->head_dim;
+  c->deferred = false;
+  c->pending = false;
+  c->side = nullptr;
+  c->ev_fork = c->ev_join = nullptr;
   c->use_mma = wants_mma(*cfg);
   if (c->use_mma) {
     if ((long long)cfg->batch * cfg->n_kv_heads * cfg->capacity >= (1LL << 31)) { delete c; return TOVA_ERR_BAD_SHAPE; }
@@ -495,7 +544,8 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
                    static_cast<const unsigned char*>(v) + t * kv_stride,
                    first_pos < 0 ? first_pos : first_pos + t,
                    out ? out + (size_t)t * B * H * D : scratch_out,
-                   evicted_pos ? evicted_pos + (size_t)t * B : nullptr, static_cast<cudaStream_t>(cuda_stream));
+                   evicted_pos ? evicted_pos + (size_t)t * B : nullptr, static_cast<cudaStream_t>(cuda_stream),
+                   /*allow_defer=*/false);  // consecutive tokens of one cache cannot overlap anyway
     if (rc != TOVA_OK) return rc;
   }
   return TOVA_OK;
@@ -514,7 +564,7 @@ int tova_decode_step_host(tova_cache* c, const void* q_host, const void* k_host,
     return TOVA_ERR_CUDA;
   int rc = step_impl(c, base + c->lay.st_q, base + c->lay.st_k, base + c->lay.st_v, pos,
                      reinterpret_cast<float*>(base + c->lay.st_out),
-                     reinterpret_cast<int32_t*>(base + c->lay.st_ev), st);
+                     reinterpret_cast<int32_t*>(base + c->lay.st_ev), st, /*allow_defer=*/false);
   if (rc != TOVA_OK) return rc;
   if (cudaMemcpyAsync(out_host, base + c->lay.st_out, ob, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return TOVA_ERR_CUDA;
@@ -525,9 +575,34 @@ int tova_decode_step_host(tova_cache* c, const void* q_host, const void* k_host,
   return TOVA_OK;
 }
 
-int tova_cache_read(const tova_cache* c, int32_t* len, int32_t* positions, void* k_out, void* v_out,
-                    int32_t* status, void* cuda_stream) {
+int tova_cache_join(tova_cache* c, void* cuda_stream) {
   if (!c) return TOVA_ERR_NULL;
+  if (c->pending) {
+    if (cudaStreamWaitEvent(static_cast<cudaStream_t>(cuda_stream), c->ev_join, 0) != cudaSuccess)
+      return TOVA_ERR_CUDA;
+    c->pending = false;
+  }
+  return TOVA_OK;
+}
+
+int tova_cache_set_deferred_eviction(tova_cache* c, int32_t on) {
+  if (!c) return TOVA_ERR_NULL;
+  if (on && !c->side) {
+    if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess)
+      return TOVA_ERR_CUDA;
+  }
+  if (!on && c->pending) return TOVA_ERR_BAD_SHAPE;  // join first
+  c->deferred = on != 0;
+  return TOVA_OK;
+}
+
+int tova_cache_read(const tova_cache* c_in, int32_t* len, int32_t* positions, void* k_out, void* v_out,
+                    int32_t* status, void* cuda_stream) {
+  if (!c_in) return TOVA_ERR_NULL;
+  tova_cache* c = const_cast<tova_cache*>(c_in);  // joining a deferred eviction updates host bookkeeping only
+  if (tova_cache_join(c, cuda_stream) != TOVA_OK) return TOVA_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const size_t B = c->cfg.batch, Hkv = c->cfg.n_kv_heads, cap = c->cfg.capacity;
   const size_t kvb = B * Hkv * cap * c->row_bytes;
@@ -547,6 +622,12 @@ int64_t tova_cache_launches(const tova_cache* c) { return c ? c->launches : -1; 
 
 int tova_cache_destroy(tova_cache* c) {
   if (!c) return TOVA_ERR_NULL;
+  if (c->side) {
+    cudaStreamSynchronize(c->side);
+    cudaEventDestroy(c->ev_fork);
+    cudaEventDestroy(c->ev_join);
+    cudaStreamDestroy(c->side);
+  }
   delete c;
   return TOVA_OK;
 }
@@ -675,10 +756,11 @@ extern "C" int tova_decode_step_static(const tova_config* cfg, void* K, void* V,
   }
   cudaError_t e;
   if (cfg->dtype == TOVA_DTYPE_BF16) {
-    e = cfg->head_dim == 128 ? launch_step<__nv_bfloat16, 128>(&shim, p, st)
-                             : launch_step<__nv_bfloat16, 64>(&shim, p, st);
+    e = cfg->head_dim == 128 ? launch_step<__nv_bfloat16, 128>(&shim, p, st, false)
+                             : launch_step<__nv_bfloat16, 64>(&shim, p, st, false);
   } else {
-    e = cfg->head_dim == 128 ? launch_step<float, 128>(&shim, p, st) : launch_step<float, 64>(&shim, p, st);
+    e = cfg->head_dim == 128 ? launch_step<float, 128>(&shim, p, st, false)
+                             : launch_step<float, 64>(&shim, p, st, false);
   }
   return e == cudaSuccess ? TOVA_OK : TOVA_ERR_CUDA;
 }

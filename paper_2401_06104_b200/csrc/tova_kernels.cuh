@@ -32,6 +32,7 @@ constexpr int COMBINE_ROW_STAGE_BYTES = 16 * 1024;  // new-token rows (k and v) 
 constexpr int COMBINE_CLUSTER_MAX = 8;  // CTAs per sequence in the combine kernel (portable cluster size;
                                         // clusters of 16 were measured slower)
 constexpr int MIN_CHUNK_ROWS = 32;      // smallest chunk the scratch is sized for
+enum : int { COMBINE_ALL = 0, COMBINE_OUTPUTS = 1, COMBINE_EVICT = 2 };  // StepParams::mode
 
 struct StepParams {
   // state
@@ -64,6 +65,9 @@ struct StepParams {
   int32_t combine_threads;  // COMBINE_THREADS_SMALL or COMBINE_THREADS_LARGE
   int32_t stage_logits;     // combine CTAs bulk-copy their block of logits to shared memory
   int32_t do_evict;   // n == cap and the policy is on
+  int32_t mode;       // combine kernel: 0 whole step, 1 outputs only, 2 victim + insert only
+  void* k_stage;      // [B,Hkv,D] mode 1: copies of the new token's rows for a later mode-2 launch
+  void* v_stage;
   float scale2;       // sm_scale * log2(e)
 };
 
@@ -384,7 +388,8 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
   // When a victim is due, CTA 0 is on the critical path (arg-min, insert): if
   // the output merge is light (few chunks), the output elements are shared among
   // its peers and written after they arrive at the cluster barrier.
-  const bool late_out = p.do_evict && p.nx > 1 && p.n_chunks <= 8;   // only when the merge is light
+  const bool score = p.do_evict && p.mode != COMBINE_OUTPUTS;        // this launch picks a victim
+  const bool late_out = score && p.mode == COMBINE_ALL && p.nx > 1 && p.n_chunks <= 8;   // only when the merge is light
   const int out_ctas = late_out ? p.nx - 1 : p.nx;
   const int out_x = late_out ? x - 1 : x;      // -1: no share
   // Output work item = (head, 4 consecutive dims, slice of the chunks): S lanes
@@ -395,17 +400,17 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
   int S = 1;
   while (S < 32 && 2 * S * items4 <= out_threads && 2 * S <= p.n_chunks) S <<= 1;
   const int work = items4 * S;                 // a multiple of 32 whenever S > 1
-  const int g0 = out_x < 0 ? work : out_x * CT + tid;
+  const int g0 = (out_x < 0 || p.mode == COMBINE_EVICT) ? work : out_x * CT + tid;
   constexpr int RB16 = D * (int)sizeof(T) / 16;  // 16-byte words per row
   const int row_words = p.Hkv * RB16;
   const int total_ml = p.H * np;
   const uint32_t row_bytes = (uint32_t)row_words * 16u;          // all KV heads of one operand
-  const bool staged = (x == 0) && 2 * row_bytes <= (uint32_t)COMBINE_ROW_STAGE_BYTES;
+  const bool staged = (x == 0) && p.mode != COMBINE_OUTPUTS && 2 * row_bytes <= (uint32_t)COMBINE_ROW_STAGE_BYTES;
   // staged logits: rows of cand_per_cta floats (a multiple of 4), one per head
   float* lg_stage = reinterpret_cast<float*>(
       row_stage + (2 * row_bytes <= (uint32_t)COMBINE_ROW_STAGE_BYTES ? 2 * row_bytes : 0));
   const int lg_cols = max(min(p.cand_per_cta, p.ld - j_begin), 0);   // floats per head row actually copied
-  const bool lg_staged = p.do_evict && p.stage_logits && lg_cols > 0;
+  const bool lg_staged = score && p.stage_logits && lg_cols > 0;
   if (tid == 0) {
     mbar_init(&row_bar, 1);
     mbar_init(&lg_bar, 1);
@@ -441,7 +446,7 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
   int r_pos = pos_t;               // position held by this thread's first candidate
   {
     const int j = j_begin + jl;
-    const bool live = p.do_evict && j < j_end;
+    const bool live = score && j < j_end;
     const float* lg = p.logits + (size_t)b * p.H * p.ld + j;
 #pragma unroll
     for (int u = 0; u < LG; ++u) {
@@ -557,7 +562,21 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
       }
     }
   };
-  if (!late_out) write_outputs();
+  if (!late_out) write_outputs();   // no work in COMBINE_EVICT mode (g0 = work)
+
+  if (p.mode == COMBINE_OUTPUTS) {
+    // The victim is chosen by a later launch, possibly after the caller has
+    // reused its k/v buffers: keep copies of the new token's rows.
+    if (x == 0) {
+      for (int i = tid; i < row_words; i += CT) {
+        static_cast<uint4*>(p.k_stage)[(size_t)b * row_words + i] =
+            static_cast<const uint4*>(p.k_new)[(size_t)b * row_words + i];
+        static_cast<uint4*>(p.v_stage)[(size_t)b * row_words + i] =
+            static_cast<const uint4*>(p.v_new)[(size_t)b * row_words + i];
+      }
+    }
+    return;
+  }
 
   if (!p.do_evict) {
     // g(t) = min(t, k) not yet reached: the new token takes the next free row.

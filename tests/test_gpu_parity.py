@@ -169,3 +169,36 @@ def test_step_argument_errors():
     with pytest.raises(tova.TovaError):
         c.tova_cache_set_chunk_rows(48)
     assert c.tova_cache_len() == 0
+
+
+def test_deferred_eviction_gives_identical_results():
+    """Eviction on the cache's side stream, two caches taking turns like the
+    layers of a model: same outputs, dropped positions and state as the default."""
+    w = LLAMA.scaled(batch=2, n_q_heads=8, n_kv_heads=4, capacity=90)
+    T = 220
+    streams = [W.tokens(w, 0, T, layer=l) for l in range(2)]
+    ref = [make_cache(w) for _ in range(2)]
+    dfr = [make_cache(w) for _ in range(2)]
+    for c in dfr:
+        c.tova_cache_set_deferred_eviction(True)
+    dev = [[tova.to_device(a, w.dtype) for a in s] for s in streams]
+    shape = (T, w.batch, w.n_q_heads, w.head_dim)
+    o_ref = [torch.empty(shape, device="cuda:0") for _ in range(2)]
+    o_dfr = [torch.empty(shape, device="cuda:0") for _ in range(2)]
+    e_ref = [torch.full((T, w.batch), -7, dtype=torch.int32, device="cuda:0") for _ in range(2)]
+    e_dfr = [torch.full((T, w.batch), -7, dtype=torch.int32, device="cuda:0") for _ in range(2)]
+    for t in range(T):
+        for l in range(2):
+            q, k, v = dev[l]
+            ref[l].tova_decode_step(q[t], k[t], v[t], t, o_ref[l][t], e_ref[l][t])
+            dfr[l].tova_decode_step(q[t], k[t], v[t], t, o_dfr[l][t], e_dfr[l][t])
+    for c in dfr:
+        c.tova_cache_join()
+    torch.cuda.synchronize()
+    for l in range(2):
+        assert torch.equal(o_ref[l], o_dfr[l]) and torch.equal(e_ref[l], e_dfr[l])
+        a, b = ref[l].tova_cache_read(want_kv=True), dfr[l].tova_cache_read(want_kv=True)
+        assert a["status"] == 0 and b["status"] == 0
+        for key in ("len", "positions", "K", "V"):
+            assert torch.equal(a[key], b[key]), key
+        assert dfr[l].tova_cache_launches() == 1 + 3 * T
