@@ -43,6 +43,7 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="independent layer caches to rotate over (0 = auto)")
     ap.add_argument("--chunk-rows", type=int, default=0)
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of CUDA graphs")
+    ap.add_argument("--deferred", action="store_true", help="force deferred eviction on")
     ap.add_argument("--no-deferred", action="store_true",
                     help="pick the victim on the caller's stream instead of overlapping it with the next layer's step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -233,7 +234,10 @@ def run_ours(args):
     step_bytes = w.step_bytes()
     # at least two layers: consecutive steps then belong to different caches, as in a model
     L = args.layers or max(2, -(-WORKING_SET // step_bytes))
-    deferred = not args.no_deferred and L >= 2
+    # Deferred eviction pays when the combine kernel leaves SMs free for the next layer's
+    # streaming kernel (small batch: at most one combine CTA per SM) or is long enough to be
+    # worth hiding (large capacity); in between it only competes for the same SMs.
+    deferred = (not args.no_deferred and L >= 2 and (B * 8 <= 148 or cap >= 4096)) or args.deferred
     ring = W.tokens(w, 0, RING)                                   # seeded, host
     dq, dk, dv = (tova.to_device(a, w.dtype, dev) for a in ring)
 
