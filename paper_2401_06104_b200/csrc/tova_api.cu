@@ -296,9 +296,13 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, boo
 }
 
 // Rows of the state per split warp.  Every SM holds `per_sm` split warps at a
-// time (shared memory bound); warps beyond one full set wait for a free slot,
-// so the choice trades rounds against per-warp fixed cost (launch, first copy,
-// partial write: about 24 rows' worth).
+// time (shared memory and registers).  Measured on B200 over the model-shaped
+// workloads: 128-row chunks are best whenever they give at least ~0.8 warps per
+// slot (several rounds of short warps beat one round of long ones: the tail
+// is shorter and the load spreads better); with fewer, 64-row chunks double
+// the warps; 32-row chunks lose more in the combine kernel (twice the
+// partials) than they gain.  Larger chunks only where the combine kernel's
+// shared memory would not hold all partials of a sequence.
 int pick_chunk_rows(const tova_config& cfg, int sm_count) {
   const size_t smem = split_smem_bytes(cfg) + 1024 /* per-CTA reserve */ + 64;
   long long per_sm = (long long)(227 * 1024) / (long long)smem;
@@ -309,22 +313,15 @@ int pick_chunk_rows(const tova_config& cfg, int sm_count) {
   if (per_sm > 32) per_sm = 32;
   if (per_sm < 1) per_sm = 1;
   const long long slots = per_sm * sm_count;
-  const int G = cfg.n_q_heads / cfg.n_kv_heads;
-  const long long hgroups = (G + unit_heads(cfg) - 1) / unit_heads(cfg);
+  const long long hgroups = (G0 + unit_heads(cfg) - 1) / unit_heads(cfg);
   const long long pairs = (long long)cfg.batch * cfg.n_kv_heads * hgroups;
-  long long best_cost = -1;
-  int best = -1;  // no chunk size keeps the combine kernel's shared memory within its limit
-  for (int cr = tova::MIN_CHUNK_ROWS; cr <= 8192; cr *= 2) {
-    const long long chunks = (cfg.capacity + (long long)cr - 1) / cr;
-    const long long units = pairs * chunks;
-    const long long rounds = (units + slots - 1) / slots;
-    const long long rows = cr < cfg.capacity ? cr : cfg.capacity;
-    const long long cost = rounds * (rows + 24);
-    if (combine_smem_bound(cfg.n_q_heads, (int)chunks + 1) > COMBINE_BASE_LIMIT) continue;
-    if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best = cr; }
-    if (cr >= cfg.capacity) break;
-  }
-  return best;
+  auto units = [&](int cr) { return pairs * ((cfg.capacity + (long long)cr - 1) / cr); };
+  int cr = 128;
+  if (10 * units(128) < 8 * slots) cr = 64;
+  if (cr == 64 && cfg.capacity <= 256 && 10 * units(64) < 8 * slots) cr = 32;  // short states: partials are few anyway
+  while (cr <= 8192 && combine_smem_bound(cfg.n_q_heads, (int)((cfg.capacity + cr - 1) / cr) + 1) > COMBINE_BASE_LIMIT)
+    cr *= 2;
+  return cr <= 8192 ? cr : -1;  // -1: no chunk size keeps the combine kernel's shared memory within its limit
 }
 
 // Launch geometry of one step for n live rows.
