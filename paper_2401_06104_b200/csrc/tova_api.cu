@@ -172,12 +172,12 @@ inline size_t combine_smem_bound(int H, int n_partials) {
   return combine_smem_bytes(H, n_partials, tova::COMBINE_THREADS_LARGE, 0, 0) + tova::COMBINE_ROW_STAGE_BYTES;
 }
 
-template <typename T, int D, int CT>
+template <typename T, int D, int CT, int MODE>
 cudaError_t launch_combine_ct(int dev, const StepParams& p, cudaStream_t st, bool use_pdl) {
   const size_t row_bytes = (size_t)p.Hkv * D * sizeof(T);
   const size_t logit_bytes = p.stage_logits ? (size_t)p.H * p.cand_per_cta * sizeof(float) : 0;
   const size_t smem = combine_smem_bytes(p.H, p.n_chunks + 1, CT, row_bytes, logit_bytes);
-  auto kern = tova::tova_combine_kernel<T, D, CT>;
+  auto kern = tova::tova_combine_kernel<T, D, CT, MODE>;
   static bool attr_set[64] = {};
   if (!attr_set[dev & 63]) {
     cudaError_t e =
@@ -197,7 +197,7 @@ cudaError_t launch_combine_ct(int dev, const StepParams& p, cudaStream_t st, boo
     at[na].val.programmaticStreamSerializationAllowed = 1;
     ++na;
   }
-  if (p.mode != tova::COMBINE_OUTPUTS) {  // the CTAs of one sequence form a cluster (needed to pick the victim)
+  if (MODE != tova::COMBINE_OUTPUTS) {  // the CTAs of one sequence form a cluster (needed to pick the victim)
     at[na].id = cudaLaunchAttributeClusterDimension;
     at[na].val.clusterDim.x = p.nx;
     at[na].val.clusterDim.y = 1;
@@ -211,9 +211,19 @@ cudaError_t launch_combine_ct(int dev, const StepParams& p, cudaStream_t st, boo
 
 template <typename T, int D>
 cudaError_t launch_combine(int dev, const StepParams& p, cudaStream_t st, bool use_pdl = true) {
-  return p.combine_threads == tova::COMBINE_THREADS_LARGE
-             ? launch_combine_ct<T, D, tova::COMBINE_THREADS_LARGE>(dev, p, st, use_pdl)
-             : launch_combine_ct<T, D, tova::COMBINE_THREADS_SMALL>(dev, p, st, use_pdl);
+  constexpr int CL = tova::COMBINE_THREADS_LARGE, CS = tova::COMBINE_THREADS_SMALL;
+  const bool large = p.combine_threads == CL;
+  switch (p.mode) {
+    case tova::COMBINE_OUTPUTS:
+      return large ? launch_combine_ct<T, D, CL, tova::COMBINE_OUTPUTS>(dev, p, st, use_pdl)
+                   : launch_combine_ct<T, D, CS, tova::COMBINE_OUTPUTS>(dev, p, st, use_pdl);
+    case tova::COMBINE_EVICT:
+      return large ? launch_combine_ct<T, D, CL, tova::COMBINE_EVICT>(dev, p, st, use_pdl)
+                   : launch_combine_ct<T, D, CS, tova::COMBINE_EVICT>(dev, p, st, use_pdl);
+    default:
+      return large ? launch_combine_ct<T, D, CL, tova::COMBINE_ALL>(dev, p, st, use_pdl)
+                   : launch_combine_ct<T, D, CS, tova::COMBINE_ALL>(dev, p, st, use_pdl);
+  }
 }
 
 template <int D, bool TWO>

@@ -351,7 +351,10 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
 // [H][cand_per_cta] block of logits (bulk-copied in at the start when the host
 // says it fits).
 // 64 registers per thread: CTAs of the next kernel can share the SM with them.
-template <typename T, int D, int CT>
+// MODE (COMBINE_ALL / COMBINE_OUTPUTS / COMBINE_EVICT) is a template parameter:
+// with warm data the kernel stalls mostly on instruction fetch, so every launch
+// should carry only the code it runs.
+template <typename T, int D, int CT, int MODE>
 __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_combine_kernel(const StepParams p) {
   namespace cg = cooperative_groups;
   constexpr bool BIG = false;
@@ -388,8 +391,8 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
   // When a victim is due, CTA 0 is on the critical path (arg-min, insert): if
   // the output merge is light (few chunks), the output elements are shared among
   // its peers and written after they arrive at the cluster barrier.
-  const bool score = p.do_evict && p.mode != COMBINE_OUTPUTS;        // this launch picks a victim
-  const bool late_out = score && p.mode == COMBINE_ALL && p.nx > 1 && p.n_chunks <= 8;   // only when the merge is light
+  const bool score = p.do_evict && MODE != COMBINE_OUTPUTS;          // this launch picks a victim
+  const bool late_out = score && MODE == COMBINE_ALL && p.nx > 1 && p.n_chunks <= 8;   // only when the merge is light
   const int out_ctas = late_out ? p.nx - 1 : p.nx;
   const int out_x = late_out ? x - 1 : x;      // -1: no share
   // Output work item = (head, 4 consecutive dims, slice of the chunks): S lanes
@@ -400,12 +403,12 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
   int S = 1;
   while (S < 32 && 2 * S * items4 <= out_threads && 2 * S <= p.n_chunks) S <<= 1;
   const int work = items4 * S;                 // a multiple of 32 whenever S > 1
-  const int g0 = (out_x < 0 || p.mode == COMBINE_EVICT) ? work : out_x * CT + tid;
+  const int g0 = (out_x < 0 || MODE == COMBINE_EVICT) ? work : out_x * CT + tid;
   constexpr int RB16 = D * (int)sizeof(T) / 16;  // 16-byte words per row
   const int row_words = p.Hkv * RB16;
   const int total_ml = p.H * np;
   const uint32_t row_bytes = (uint32_t)row_words * 16u;          // all KV heads of one operand
-  const bool staged = (x == 0) && p.mode != COMBINE_OUTPUTS && 2 * row_bytes <= (uint32_t)COMBINE_ROW_STAGE_BYTES;
+  const bool staged = (x == 0) && MODE != COMBINE_OUTPUTS && 2 * row_bytes <= (uint32_t)COMBINE_ROW_STAGE_BYTES;
   // staged logits: rows of cand_per_cta floats (a multiple of 4), one per head
   float* lg_stage = reinterpret_cast<float*>(
       row_stage + (2 * row_bytes <= (uint32_t)COMBINE_ROW_STAGE_BYTES ? 2 * row_bytes : 0));
@@ -456,7 +459,7 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
     if (live && hs == 0 && j < p.cap) r_pos = p.pos[(size_t)b * p.cap + j];
   }
   float4 r_acc[AC];
-  if (g0 < work) {
+  if (MODE != COMBINE_EVICT && g0 < work) {
     const int it = g0 / S, cs = g0 % S;
     const int h = it / (D / 4), d4 = it % (D / 4);
     const float4* acc = reinterpret_cast<const float4*>(p.part_acc + ((size_t)b * p.H + h) * (size_t)(p.pc - 1) * D) + d4;
@@ -510,12 +513,12 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
       float M = -INFINITY, L = 0.f;
       for (int i = sub_l; i < np; i += lph) M = fmaxf(M, ml[i].x);
       for (int o = lph >> 1; o >= 1; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-      for (int i = sub_l; i < np; i += lph) L = fmaf(ml[i].y, exp2_diff(ml[i].x, M), L);
+      for (int i = sub_l; i < np; i += lph) L = fmaf(ml[i].y, exp2f(ml[i].x - M), L);   // M is finite: the new token's partial is
       for (int o = lph >> 1; o >= 1; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
       if (hv && sub_l == 0) {
         hM[h] = M;
-        hInvL[h] = 1.f / L;
-        hLc[h] = -M - log2f(L * (float)p.H);
+        hInvL[h] = __frcp_rn(L);
+        hLc[h] = -M - __log2f(L * (float)p.H);
       }
     }
   }
@@ -536,7 +539,7 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
 #pragma unroll
         for (int u = 0; u < AC; ++u) {
           if (i < p.n_chunks) {
-            const float w = exp2_diff(ml[i].x, M);
+            const float w = exp2f(ml[i].x - M);
             o.x = fmaf(r_acc[u].x, w, o.x); o.y = fmaf(r_acc[u].y, w, o.y);
             o.z = fmaf(r_acc[u].z, w, o.z); o.w = fmaf(r_acc[u].w, w, o.w);
           }
@@ -546,7 +549,7 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
 #pragma unroll 4
       for (; i < p.n_chunks; i += S) {
         const float4 a = acc[(size_t)i * (D / 4)];
-        const float w = exp2_diff(ml[i].x, M);
+        const float w = exp2f(ml[i].x - M);
         o.x = fmaf(a.x, w, o.x); o.y = fmaf(a.y, w, o.y); o.z = fmaf(a.z, w, o.z); o.w = fmaf(a.w, w, o.w);
       }
       for (int off = S >> 1; off >= 1; off >>= 1) {
@@ -555,16 +558,16 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
       }
       if (cs == 0) {
         const T* vn = static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + h / p.G) * D + d4 * 4;
-        const float w = exp2_diff(ml[p.n_chunks].x, M), iL = hInvL[h];
+        const float w = exp2f(ml[p.n_chunks].x - M), iL = hInvL[h];
         o.x = fmaf((float)vn[0], w, o.x) * iL; o.y = fmaf((float)vn[1], w, o.y) * iL;
         o.z = fmaf((float)vn[2], w, o.z) * iL; o.w = fmaf((float)vn[3], w, o.w) * iL;
         reinterpret_cast<float4*>(p.out + bh * D)[d4] = o;
       }
     }
   };
-  if (!late_out) write_outputs();   // no work in COMBINE_EVICT mode (g0 = work)
+  if (MODE != COMBINE_EVICT && !late_out) write_outputs();
 
-  if (p.mode == COMBINE_OUTPUTS) {
+  if (MODE == COMBINE_OUTPUTS) {
     // The victim is chosen by a later launch, possibly after the caller has
     // reused its k/v buffers: keep copies of the new token's rows.
     if (x == 0) {
@@ -618,10 +621,10 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
           const int h = hs + u * hs_n;
           if (h < p.H) a += exp2f(r_lg[u] + hLc[h]);
         }
-#pragma unroll 8
+#pragma unroll 4
         for (int h = hs + LG * hs_n; h < p.H; h += hs_n) a += exp2f(lg[(size_t)h * p.ld] + hLc[h]);
       } else {
-#pragma unroll 16
+#pragma unroll 4
         for (int h = hs; h < p.H; h += hs_n) a += exp2f(lg[(size_t)h * p.ld] + hLc[h]);
       }
     }
@@ -665,7 +668,7 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
   __syncwarp();
   cluster_arrive_release();        // orders the store above before the barrier completes
   if (x != 0) {                    // peers: nobody reads their shared memory; their outputs are off the critical path
-    if (late_out) write_outputs();
+    if (MODE == COMBINE_ALL && late_out) write_outputs();
     return;
   }
   cluster_wait_acquire();
