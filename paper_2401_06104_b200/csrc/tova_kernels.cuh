@@ -382,10 +382,12 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   // geometry (no memory access)
-  int wp = 1;                      // candidates per pass, a power of two <= CT
-  while (wp < p.cand_per_cta && wp < CT) wp <<= 1;
-  const int hs_n = CT / wp;        // threads sharing one candidate's heads
-  const int jl = tid % wp, hs = tid / wp;
+  // (all the divisors below are powers of two: shifts and masks, no integer division)
+  int lg_wp = 0;                   // wp = candidates per pass, a power of two <= CT
+  while ((1 << lg_wp) < p.cand_per_cta && (1 << lg_wp) < CT) ++lg_wp;
+  const int wp = 1 << lg_wp;
+  const int hs_n = CT >> lg_wp;    // threads sharing one candidate's heads
+  const int jl = tid & (wp - 1), hs = tid >> lg_wp;
   const int j_begin = x * p.cand_per_cta;
   const int j_end = min(j_begin + p.cand_per_cta, p.n + 1);
   // When a victim is due, CTA 0 is on the critical path (arg-min, insert): if
@@ -400,13 +402,16 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
   // 16-byte loads; their sums are folded by shuffles.
   const int items4 = p.H * (D / 4);
   const int out_threads = out_ctas * CT;
-  int S = 1;
-  while (S < 32 && 2 * S * items4 <= out_threads && 2 * S <= p.n_chunks) S <<= 1;
+  int lg_S = 0;
+  while ((2 << lg_S) <= 32 && (2 << lg_S) * items4 <= out_threads && (2 << lg_S) <= p.n_chunks) ++lg_S;
+  const int S = 1 << lg_S;
   const int work = items4 * S;                 // a multiple of 32 whenever S > 1
   const int g0 = (out_x < 0 || MODE == COMBINE_EVICT) ? work : out_x * CT + tid;
   constexpr int RB16 = D * (int)sizeof(T) / 16;  // 16-byte words per row
   const int row_words = p.Hkv * RB16;
-  const int total_ml = p.H * np;
+  int lg_np = 0;                   // partials per head rounded up to a power of two: thread i -> (i >> lg_np, i & mask)
+  while ((1 << lg_np) < np) ++lg_np;
+  const int total_ml = p.H << lg_np;
   const uint32_t row_bytes = (uint32_t)row_words * 16u;          // all KV heads of one operand
   const bool staged = (x == 0) && MODE != COMBINE_OUTPUTS && 2 * row_bytes <= (uint32_t)COMBINE_ROW_STAGE_BYTES;
   // staged logits: rows of cand_per_cta floats (a multiple of 4), one per head
@@ -443,7 +448,8 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
 #pragma unroll
   for (int u = 0; u < ML; ++u) {
     const int i = tid + u * CT;
-    r_ml[u] = (i < total_ml) ? p.part_ml[((size_t)b * p.H + i / np) * p.pc + i % np] : make_float2(0.f, 0.f);
+    const int h = i >> lg_np, cc = i & ((1 << lg_np) - 1);
+    r_ml[u] = (i < total_ml && cc < np) ? p.part_ml[((size_t)b * p.H + h) * p.pc + cc] : make_float2(0.f, 0.f);
   }
   float r_lg[LG];
   int r_pos = pos_t;               // position held by this thread's first candidate
@@ -460,7 +466,7 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
   }
   float4 r_acc[AC];
   if (MODE != COMBINE_EVICT && g0 < work) {
-    const int it = g0 / S, cs = g0 % S;
+    const int it = g0 >> lg_S, cs = g0 & (S - 1);
     const int h = it / (D / 4), d4 = it % (D / 4);
     const float4* acc = reinterpret_cast<const float4*>(p.part_acc + ((size_t)b * p.H + h) * (size_t)(p.pc - 1) * D) + d4;
 #pragma unroll
@@ -495,19 +501,23 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
 #pragma unroll
   for (int u = 0; u < ML; ++u) {
     const int i = tid + u * CT;
-    if (i < total_ml) pml[i] = r_ml[u];
+    const int h = i >> lg_np, cc = i & ((1 << lg_np) - 1);
+    if (i < total_ml && cc < np) pml[h * np + cc] = r_ml[u];
   }
-  for (int i = tid + ML * CT; i < total_ml; i += CT)
-    pml[i] = p.part_ml[((size_t)b * p.H + i / np) * p.pc + i % np];
+  for (int i = tid + ML * CT; i < total_ml; i += CT) {
+    const int h = i >> lg_np, cc = i & ((1 << lg_np) - 1);
+    if (cc < np) pml[h * np + cc] = p.part_ml[((size_t)b * p.H + h) * p.pc + cc];
+  }
   __syncthreads();
   {
     // a group of lph lanes per head, at most 8 partials per lane
-    int lph = 1;
-    while (lph < 32 && lph * 8 < np) lph <<= 1;
-    const int hpp = CT / lph;                      // heads per pass
-    const int sub_l = tid % lph;
+    int lg_lph = 0;
+    while ((1 << lg_lph) < 32 && (8 << lg_lph) < np) ++lg_lph;
+    const int lph = 1 << lg_lph;
+    const int hpp = CT >> lg_lph;                  // heads per pass
+    const int sub_l = tid & (lph - 1);
     for (int h0 = 0; h0 < p.H; h0 += hpp) {        // uniform trip count: the shuffles need whole warps
-      const int h = h0 + tid / lph;
+      const int h = h0 + (tid >> lg_lph);
       const bool hv = h < p.H;
       const float2* ml = pml + (size_t)(hv ? h : 0) * np;
       float M = -INFINITY, L = 0.f;
@@ -527,7 +537,7 @@ __global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_
   // ---- 2. this CTA's share of the attention output --------------------------------
   auto write_outputs = [&]() {
     for (int g = g0; g < work; g += out_threads) {   // whole warps run the same trips (see `work`)
-      const int it = g / S, cs = g % S;
+      const int it = g >> lg_S, cs = g & (S - 1);
       const int h = it / (D / 4), d4 = it % (D / 4);
       const size_t bh = (size_t)b * p.H + h;
       const float2* ml = pml + (size_t)h * np;
