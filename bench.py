@@ -281,7 +281,10 @@ def run_ours(args):
             step(counter[0])
             counter[0] += 1
 
-    run_direct(min(64, max(args.warmup, 3)))                      # sets function attributes before capture
+    l0 = sum(c.tova_cache_launches() for c in caches)
+    n_direct = min(64, max(args.warmup, 3))
+    run_direct(n_direct)                                          # sets function attributes before capture
+    launches_per_step = (sum(c.tova_cache_launches() for c in caches) - l0) // n_direct
     join_all()
     torch.cuda.synchronize()
 
@@ -389,7 +392,7 @@ def run_ours(args):
                      "note": "algorithmic bytes (K/V read + one slot written) / whole-step time (split + combine kernels)"},
         "cpu_baseline": cpu,
         "e2e": e2e,
-        "gpu_launches": (3 if deferred else 2) * args.steps,
+        "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks,
     }
     print(json.dumps(line))
