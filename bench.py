@@ -233,7 +233,7 @@ def run_ours(args):
     B, H, Hkv, D, cap = w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity
     step_bytes = w.step_bytes()
     # at least two layers: consecutive steps then belong to different caches, as in a model
-    L = args.layers or max(2, -(-WORKING_SET // step_bytes))
+    L = args.layers or min(64, max(2, -(-WORKING_SET // step_bytes)))
     # Deferred eviction pays when the combine kernel leaves SMs free for the next layer's
     # streaming kernel (small batch: at most one combine CTA per SM) or is long enough to be
     # worth hiding (large capacity); in between it only competes for the same SMs.
@@ -381,7 +381,7 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": workload_config(w, {
-            "layers_rotated": L, "working_set_bytes": L * step_bytes, "l2": "inputs larger than L2",
+            "layers_rotated": L, "working_set_bytes": L * step_bytes, "l2": "inputs larger than L2" if L * step_bytes > 2 * 126e6 else "working set near or below L2 size",
             "launch": launch_mode, "graph_steps": G, "bytes_per_step": step_bytes,
             "eviction": "deferred to the cache's side stream, overlaps the next layer's step" if deferred
                         else "on the caller's stream",
