@@ -212,6 +212,17 @@ def recorded_traffic(w, layers_bytes_per_step):
         return None
 
 
+def max_over_ranks(x: float, device) -> float:
+    """Max of a host number over all ranks (1 rank: the number itself)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -329,11 +340,7 @@ def run_ours(args):
     clocks = sampler.stop()
     if world > 1:
         dist.barrier()
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), dev)
     for c in caches:
         assert c.tova_cache_read()["status"] == 0, "a kernel reported a failed check"
 
@@ -359,11 +366,7 @@ def run_ours(args):
             r = (i // L + 29 * (i % L)) % RING
             caches[i % L].tova_decode_step_host(hq[r], hk[r], hv[r], -1, hout, hev)
         torch.cuda.synchronize()
-        dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = max_over_ranks(time.perf_counter() - t0, dev)
         e2e = {"value": world * B * n_e / dt, "unit": UNIT, "steps": n_e,
                "h2d_bytes_per_step": int(hq[0].nbytes + hk[0].nbytes + hv[0].nbytes),
                "d2h_bytes_per_step": int(hout.nbytes + hev.nbytes)}
