@@ -245,10 +245,7 @@ def run_ours(args):
     step_bytes = w.step_bytes()
     # at least two layers: consecutive steps then belong to different caches, as in a model
     L = args.layers or min(64, max(2, -(-WORKING_SET // step_bytes)))
-    # Deferred eviction pays when the combine kernel leaves SMs free for the next layer's
-    # streaming kernel (small batch: at most one combine CTA per SM) or is long enough to be
-    # worth hiding (large capacity); in between it only competes for the same SMs.
-    deferred = (not args.no_deferred and L >= 2 and (B * 8 <= 148 or cap >= 4096)) or args.deferred
+    deferred = (not args.no_deferred and L >= 2) or args.deferred
     ring = W.tokens(w, 0, RING)                                   # seeded, host
     dq, dk, dv = (tova.to_device(a, w.dtype, dev) for a in ring)
 

@@ -211,13 +211,14 @@ cudaError_t launch_combine_ct(int dev, const StepParams& p, cudaStream_t st, boo
 
 template <typename T, int D>
 cudaError_t launch_combine(int dev, const StepParams& p, cudaStream_t st, bool use_pdl = true) {
-  constexpr int CL = tova::COMBINE_THREADS_LARGE, CS = tova::COMBINE_THREADS_SMALL;
+  constexpr int CL = tova::COMBINE_THREADS_LARGE, CS = tova::COMBINE_THREADS_SMALL, CY = tova::COMBINE_THREADS_TINY;
   const bool large = p.combine_threads == CL;
   switch (p.mode) {
     case tova::COMBINE_OUTPUTS:
       return large ? launch_combine_ct<T, D, CL, tova::COMBINE_OUTPUTS>(dev, p, st, use_pdl)
                    : launch_combine_ct<T, D, CS, tova::COMBINE_OUTPUTS>(dev, p, st, use_pdl);
     case tova::COMBINE_EVICT:
+      if (p.combine_threads == CY) return launch_combine_ct<T, D, CY, tova::COMBINE_EVICT>(dev, p, st, use_pdl);
       return large ? launch_combine_ct<T, D, CL, tova::COMBINE_EVICT>(dev, p, st, use_pdl)
                    : launch_combine_ct<T, D, CS, tova::COMBINE_EVICT>(dev, p, st, use_pdl);
     default:
@@ -259,6 +260,8 @@ cudaError_t launch_split_mma(int dev, const StepParams& p, const CUtensorMap& mk
                  : launch_split_mma_t<D, false>(dev, p, mk, mv, grid, st);
 }
 
+void set_combine_threads(StepParams& p, int ct);
+
 template <typename T, int D>
 cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, bool defer) {
   dim3 grid(p.n_chunks > 0 ? p.n_chunks : 1, p.Hkv * p.hgroups, p.B);
@@ -288,6 +291,9 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, boo
   pa.mode = tova::COMBINE_OUTPUTS;
   pa.k_stage = c->base + c->lay.df_k;
   pa.v_stage = c->base + c->lay.df_v;
+  // Outputs-only launch: half-size CTAs once the batch would otherwise fill the
+  // register files and keep the next split kernel from becoming resident early.
+  if ((long long)p.B * p.nx > 148) set_combine_threads(pa, tova::COMBINE_THREADS_SMALL);
   pa.stage_logits = 0;
   e = launch_combine<T, D>(c->device, pa, st);
   if (e != cudaSuccess) return e;
@@ -297,6 +303,10 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, boo
   pb.mode = tova::COMBINE_EVICT;
   pb.k_new = pa.k_stage;
   pb.v_new = pa.v_stage;
+  // Victim + insert launch: off the critical path, so small CTAs that fit beside
+  // the next layer's split warps (128 threads unless that means long serial scoring).
+  set_combine_threads(pb, (long long)p.H * p.cand_per_cta / tova::COMBINE_THREADS_TINY <= 40
+                              ? tova::COMBINE_THREADS_TINY : tova::COMBINE_THREADS_SMALL);
   e = launch_combine<T, D>(c->device, pb, c->side, /*use_pdl=*/false);
   if (e != cudaSuccess) return e;
   if ((e = cudaEventRecord(c->ev_join, c->side)) != cudaSuccess) return e;
@@ -334,6 +344,16 @@ int pick_chunk_rows(const tova_config& cfg, int sm_count) {
   return cr <= 8192 ? cr : -1;  // -1: no chunk size keeps the combine kernel's shared memory within its limit
 }
 
+// CTA size of a combine launch, and with it whether a CTA's logits are staged
+// through shared memory (bulk copies): only when a thread would otherwise need
+// several dependent batches of loads for them.
+void set_combine_threads(StepParams& p, int ct) {
+  p.combine_threads = ct;
+  const long long per_thread = (long long)p.H * p.cand_per_cta / ct;
+  p.stage_logits = p.do_evict && per_thread > 3 * 8 &&
+                   (size_t)p.H * p.cand_per_cta * sizeof(float) <= (size_t)tova::COMBINE_LOGIT_STAGE_BYTES;
+}
+
 // Launch geometry of one step for n live rows.
 void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows) {
   p.B = cfg.batch; p.H = cfg.n_q_heads; p.Hkv = cfg.n_kv_heads; p.G = cfg.n_q_heads / cfg.n_kv_heads;
@@ -358,15 +378,9 @@ void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows)
   if (p.do_evict && nx < by_scores) nx = by_scores;
   if (nx > cl_max) nx = cl_max;
   if (nx < 1) nx = 1;
-  p.combine_threads = ct;
   p.nx = nx;
   p.cand_per_cta = ((n + 1 + nx - 1) / nx + 3) / 4 * 4;   // a multiple of 4: 16-byte aligned blocks of logits
-  // Stage a CTA's logits through shared memory (bulk copies) only when a thread
-  // would otherwise need several dependent batches of loads for them.
-  const long long per_thread = (long long)cfg.n_q_heads * p.cand_per_cta / ct;
-  p.stage_logits =
-      p.do_evict && per_thread > 3 * lg &&
-      (size_t)cfg.n_q_heads * p.cand_per_cta * sizeof(float) <= (size_t)tova::COMBINE_LOGIT_STAGE_BYTES;
+  set_combine_threads(p, ct);
 }
 
 int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_t pos, float* out,

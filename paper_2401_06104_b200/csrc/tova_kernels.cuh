@@ -25,6 +25,7 @@ namespace tova {
 constexpr int TILE_ROWS = 16;       // cache rows per pipeline stage of the split kernel
 constexpr int SPLIT_BUFFERS = 3;    // tile buffers of a split warp's ring (K and V tiles alternate)
 constexpr int MAX_UNIT_HEADS = 8;   // query heads one split warp carries
+constexpr int COMBINE_THREADS_TINY = 128;   // deferred victim/insert launches: small enough to slip in beside split warps
 constexpr int COMBINE_THREADS_SMALL = 256;  // combine CTA size when many CTAs are in flight
 constexpr int COMBINE_THREADS_LARGE = 512;  // ... when the batch is small: more loads in flight per sequence
 constexpr int COMBINE_LOGIT_STAGE_BYTES = 96 * 1024;  // a combine CTA's [H][candidates] logits, staged if they fit
@@ -62,7 +63,7 @@ struct StepParams {
   int32_t hgroups;    // ceil(G / heads per split warp)
   int32_t nx;         // combine CTAs per sequence = cluster size (1..COMBINE_CLUSTER_MAX)
   int32_t cand_per_cta;  // candidates scored per combine CTA
-  int32_t combine_threads;  // COMBINE_THREADS_SMALL or COMBINE_THREADS_LARGE
+  int32_t combine_threads;  // COMBINE_THREADS_TINY, _SMALL or _LARGE
   int32_t stage_logits;     // combine CTAs bulk-copy their block of logits to shared memory
   int32_t do_evict;   // n == cap and the policy is on
   int32_t mode;       // combine kernel: 0 whole step, 1 outputs only, 2 victim + insert only
@@ -355,7 +356,7 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
 // with warm data the kernel stalls mostly on instruction fetch, so every launch
 // should carry only the code it runs.
 template <typename T, int D, int CT, int MODE>
-__global__ void __launch_bounds__(CT, CT == COMBINE_THREADS_SMALL ? 4 : 2) tova_combine_kernel(const StepParams p) {
+__global__ void __launch_bounds__(CT, 1024 / CT) tova_combine_kernel(const StepParams p) {
   namespace cg = cooperative_groups;
   constexpr bool BIG = false;
   constexpr int ML = BIG ? 4 : 2;    // partial pairs prefetched per thread
