@@ -43,6 +43,8 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="independent layer caches to rotate over (0 = auto)")
     ap.add_argument("--chunk-rows", type=int, default=0)
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of CUDA graphs")
+    ap.add_argument("--no-fused-merge", action="store_true",
+                    help="merge the chunk partials through global memory even where a cluster could")
     ap.add_argument("--deferred", action="store_true", help="force deferred eviction on")
     ap.add_argument("--no-deferred", action="store_true",
                     help="pick the victim on the caller's stream instead of overlapping it with the next layer's step")
@@ -254,6 +256,8 @@ def run_ours(args):
         c = tova.TovaCache(B, H, Hkv, D, cap, dtype=w.dtype, device=dev)
         if args.chunk_rows:
             c.tova_cache_set_chunk_rows(args.chunk_rows)
+        if args.no_fused_merge:
+            c.tova_cache_set_fused_merge(False)
         caches.append(c)
     outs = torch.empty(L, B, H, D, dtype=torch.float32, device=dev)
     evs = torch.empty(L, B, dtype=torch.int32, device=dev)

@@ -149,6 +149,16 @@ int tova_cache_join(tova_cache* c, void* cuda_stream);
  * not depend on it beyond floating-point summation order. */
 int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows);
 
+/* Tuning: where the per-chunk partial results of a head are merged into the
+ * attention output (Eq. 7 evaluated chunk by chunk).  on (default): when the
+ * state splits into at most 8 chunks, the streaming warps of a head group are
+ * launched as one thread-block cluster and merge through distributed shared
+ * memory, so the outputs are final when the streaming kernel ends.  off: the
+ * partials go through global memory to the second kernel.  Larger chunk counts
+ * always take the second route.  Results do not depend on it beyond
+ * floating-point summation order.  Returns TOVA_ERR_NULL for a null handle. */
+int tova_cache_set_fused_merge(tova_cache* c, int32_t on);
+
 /* Rows each sequence holds now, min(tokens fed, capacity) = g(t) of Section
  * 3.3, tracked on the host (sequences advance in lock step). */
 int32_t tova_cache_len(const tova_cache* c);

@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.tova_cache_read.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.tova_cache_set_chunk_rows.restype = ctypes.c_int
         L.tova_cache_set_chunk_rows.argtypes = [vp, i32]
+        L.tova_cache_set_fused_merge.restype = ctypes.c_int
+        L.tova_cache_set_fused_merge.argtypes = [vp, i32]
         L.tova_cache_set_deferred_eviction.restype = ctypes.c_int
         L.tova_cache_set_deferred_eviction.argtypes = [vp, i32]
         L.tova_cache_join.restype = ctypes.c_int
@@ -157,6 +159,9 @@ class TovaCache:
 
     def tova_cache_set_chunk_rows(self, rows: int) -> None:
         _check(lib().tova_cache_set_chunk_rows(self._h, int(rows)), "tova_cache_set_chunk_rows")
+
+    def tova_cache_set_fused_merge(self, on: bool) -> None:
+        _check(lib().tova_cache_set_fused_merge(self._h, 1 if on else 0), "tova_cache_set_fused_merge")
 
     def tova_cache_set_deferred_eviction(self, on: bool) -> None:
         _check(lib().tova_cache_set_deferred_eviction(self._h, 1 if on else 0),

@@ -21,7 +21,7 @@ inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 struct Layout {
-  size_t K, V, pos, len, last_slot, logits, part_ml, part_acc, status, cur_pos;
+  size_t K, V, pos, len, last_slot, logits, part_ml, part_acc, head_ml, status, cur_pos;
   size_t st_q, st_k, st_v, st_out, st_ev;  // staging for host-buffer calls
   size_t df_k, df_v;                       // the new token's rows kept for a deferred eviction
   size_t total;
@@ -62,6 +62,7 @@ Layout make_layout(const tova_config& c) {
   L.logits = take(B * H * L.ld * 4);
   L.part_ml = take(B * H * L.pc * 8);
   L.part_acc = take(B * H * (size_t)(L.pc - 1) * D * 4);
+  L.head_ml = take(B * H * 8);
   L.status = take(4);
   L.cur_pos = take(4);
   L.st_q = take(B * H * D * E);
@@ -81,6 +82,7 @@ struct tova_cache {
   tova_config cfg;
   CUtensorMap map_k, map_v;  // tiled views of K and V for the tensor-core split kernel
   bool use_mma;
+  bool fuse_merge;      // the split warps of a head group form a cluster and merge the outputs themselves
   // deferred eviction: victim choice and insert run on a side stream, overlapping later work
   bool deferred, pending;
   cudaStream_t side;
@@ -117,17 +119,31 @@ inline size_t split_smem_bytes(const tova_config& cfg) {
   const size_t rb = (size_t)cfg.head_dim * (cfg.dtype == TOVA_DTYPE_BF16 ? 2 : 4);
   if (wants_mma(cfg)) return (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + 1024;
   const int gu = unit_heads(cfg);
-  return (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + sizeof(float) * gu * tova::TILE_ROWS;
+  return ((size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + sizeof(float) * gu * tova::TILE_ROWS + 127) / 128 * 128;
 }
 
-template <typename T, int D, int GU, int GB>
-cudaError_t launch_split(int dev, const StepParams& p, dim3 grid, cudaStream_t st) {
+// Merge inside the split kernel: the warps of a head group's chunks form one CTA.
+inline void split_launch_shape(const StepParams& p, dim3& grid, dim3& block) {
+  block = dim3(32);
+  if (p.fuse_out) {
+    block.y = grid.x;
+    grid.x = 1;
+  }
+}
+
+template <typename T, int D, int GU, int GB, bool FUSED>
+cudaError_t launch_split_f(int dev, const StepParams& p, dim3 grid, cudaStream_t st) {
   const size_t rb = (size_t)D * sizeof(T);
-  const size_t smem = (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + sizeof(float) * GU * tova::TILE_ROWS;
-  auto kern = tova::tova_split_kernel<T, D, GU, GB>;
+  const size_t warp_smem =
+      ((size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + sizeof(float) * GU * tova::TILE_ROWS + 127) / 128 * 128;
+  dim3 block;
+  split_launch_shape(p, grid, block);
+  const size_t smem = warp_smem * block.y;
+  auto kern = tova::tova_split_kernel<T, D, GU, GB, FUSED>;
   static bool attr_set[64] = {};  // per instantiation and device: the attribute is per function
   if (!attr_set[dev & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)(warp_smem * tova::SPLIT_MERGE_MAX_WARPS));
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     if (e != cudaSuccess) return e;
@@ -135,7 +151,7 @@ cudaError_t launch_split(int dev, const StepParams& p, dim3 grid, cudaStream_t s
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = grid;
-  cfg.blockDim = dim3(32);
+  cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute at[1];
@@ -144,6 +160,12 @@ cudaError_t launch_split(int dev, const StepParams& p, dim3 grid, cudaStream_t s
   cfg.attrs = at;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
+template <typename T, int D, int GU, int GB>
+cudaError_t launch_split(int dev, const StepParams& p, dim3 grid, cudaStream_t st) {
+  return p.fuse_out ? launch_split_f<T, D, GU, GB, true>(dev, p, grid, st)
+                    : launch_split_f<T, D, GU, GB, false>(dev, p, grid, st);
 }
 
 template <typename T, int D>
@@ -227,14 +249,18 @@ cudaError_t launch_combine(int dev, const StepParams& p, cudaStream_t st, bool u
   }
 }
 
-template <int D, bool TWO>
+template <int D, bool TWO, bool FUSED>
 cudaError_t launch_split_mma_t(int dev, const StepParams& p, const CUtensorMap& mk, const CUtensorMap& mv, dim3 grid,
                                cudaStream_t st) {
-  const size_t smem = (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * D * 2 + 1024;
-  auto kern = tova::tova_split_mma_kernel<D, TWO>;
+  const size_t warp_smem = (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * D * 2;
+  dim3 block;
+  split_launch_shape(p, grid, block);
+  const size_t smem = warp_smem * block.y + 1024;
+  auto kern = tova::tova_split_mma_kernel<D, TWO, FUSED>;
   static bool attr_set[64] = {};
   if (!attr_set[dev & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)(warp_smem * tova::SPLIT_MERGE_MAX_WARPS + 1024));
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     if (e != cudaSuccess) return e;
@@ -242,7 +268,7 @@ cudaError_t launch_split_mma_t(int dev, const StepParams& p, const CUtensorMap& 
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = grid;
-  cfg.blockDim = dim3(32);
+  cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute at[1];
@@ -256,8 +282,11 @@ cudaError_t launch_split_mma_t(int dev, const StepParams& p, const CUtensorMap& 
 template <int D>
 cudaError_t launch_split_mma(int dev, const StepParams& p, const CUtensorMap& mk, const CUtensorMap& mv, dim3 grid,
                              cudaStream_t st) {
-  return p.G > 8 ? launch_split_mma_t<D, true>(dev, p, mk, mv, grid, st)
-                 : launch_split_mma_t<D, false>(dev, p, mk, mv, grid, st);
+  if (p.fuse_out)
+    return p.G > 8 ? launch_split_mma_t<D, true, true>(dev, p, mk, mv, grid, st)
+                   : launch_split_mma_t<D, false, true>(dev, p, mk, mv, grid, st);
+  return p.G > 8 ? launch_split_mma_t<D, true, false>(dev, p, mk, mv, grid, st)
+                 : launch_split_mma_t<D, false, false>(dev, p, mk, mv, grid, st);
 }
 
 void set_combine_threads(StepParams& p, int ct);
@@ -278,6 +307,31 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, boo
     e = launch_split_g<T, D>(c->device, p.G, p, grid, st);
   }
   if (e != cudaSuccess) return e;
+  if (p.fuse_out) {
+    // The split kernel has written the outputs; what is left is the victim and
+    // the insert, on the caller's stream or (deferred) on the side stream.
+    StepParams pb = p;
+    pb.mode = tova::COMBINE_EVICT;
+    if (!defer) {
+      e = launch_combine<T, D>(c->device, pb, st);
+      if (e != cudaSuccess) return e;
+      c->launches += 2;
+      return cudaSuccess;
+    }
+    if ((e = cudaEventRecord(c->ev_fork, st)) != cudaSuccess) return e;
+    if ((e = cudaStreamWaitEvent(c->side, c->ev_fork, 0)) != cudaSuccess) return e;
+    pb.k_new = p.k_stage;
+    pb.v_new = p.v_stage;
+    pb.k_stage = pb.v_stage = nullptr;
+    set_combine_threads(pb, (long long)p.H * p.cand_per_cta / tova::COMBINE_THREADS_TINY <= 40
+                                ? tova::COMBINE_THREADS_TINY : tova::COMBINE_THREADS_SMALL);
+    e = launch_combine<T, D>(c->device, pb, c->side, /*use_pdl=*/false);
+    if (e != cudaSuccess) return e;
+    if ((e = cudaEventRecord(c->ev_join, c->side)) != cudaSuccess) return e;
+    c->pending = true;
+    c->launches += 2;
+    return cudaSuccess;
+  }
   if (!defer) {
     e = launch_combine<T, D>(c->device, p, st);
     if (e != cudaSuccess) return e;
@@ -406,6 +460,12 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
   p.scale2 = c->scale2;
   cudaError_t e;
   const bool defer = c->deferred && allow_defer;
+  p.head_ml = reinterpret_cast<float2*>(base + c->lay.head_ml);
+  p.fuse_out = (c->fuse_merge && (cfg.capacity + c->chunk_rows - 1) / c->chunk_rows <= tova::SPLIT_MERGE_MAX_WARPS) ? 1 : 0;
+  if (p.fuse_out && defer) {   // the split kernel keeps copies of the new token's rows for the later insert
+    p.k_stage = base + c->lay.df_k;
+    p.v_stage = base + c->lay.df_v;
+  }
   if (cfg.dtype == TOVA_DTYPE_BF16) {
     e = cfg.head_dim == 128 ? launch_step<__nv_bfloat16, 128>(c, p, st, defer)
                             : launch_step<__nv_bfloat16, 64>(c, p, st, defer);
@@ -494,6 +554,7 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   c->scale2 = c->cfg.sm_scale * 1.4426950408889634f;
   c->elem = cfg->dtype == TOVA_DTYPE_BF16 ? 2 : 4;
   c->row_bytes = c->elem * cfg->head_dim;
+  c->fuse_merge = true;
   c->deferred = false;
   c->pending = false;
   c->side = nullptr;
@@ -538,6 +599,12 @@ int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows) {
   const int chunks = (c->cfg.capacity + rows - 1) / rows;
   if (combine_smem_bound(c->cfg.n_q_heads, chunks + 1) > COMBINE_BASE_LIMIT) return TOVA_ERR_BAD_SHAPE;
   c->chunk_rows = rows;
+  return TOVA_OK;
+}
+
+int tova_cache_set_fused_merge(tova_cache* c, int32_t on) {
+  if (!c) return TOVA_ERR_NULL;
+  c->fuse_merge = on != 0;
   return TOVA_OK;
 }
 

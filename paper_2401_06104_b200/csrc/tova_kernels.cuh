@@ -48,6 +48,7 @@ struct StepParams {
   int32_t* status;    // [1]
   int32_t* cur_pos;   // [1] position of the token being processed (set by the split kernel)
   int32_t* last_slot; // [B] slot the previous step's token went to (-1: none), or null: no early prefetch
+  float2* head_ml;    // [B,H] final (max2, sum) of every head, written with the outputs when fuse_out
   // this step
   const void* q;      // [B,H,D]
   const void* k_new;  // [B,Hkv,D]
@@ -66,11 +67,82 @@ struct StepParams {
   int32_t combine_threads;  // COMBINE_THREADS_TINY, _SMALL or _LARGE
   int32_t stage_logits;     // combine CTAs bulk-copy their block of logits to shared memory
   int32_t do_evict;   // n == cap and the policy is on
+  int32_t fuse_out;   // the split kernel's warps of a (sequence, KV head, head group) form a cluster and write
+                      // the outputs themselves; the combine kernel then only picks the victim
   int32_t mode;       // combine kernel: 0 whole step, 1 outputs only, 2 victim + insert only
   void* k_stage;      // [B,Hkv,D] mode 1: copies of the new token's rows for a later mode-2 launch
   void* v_stage;
   float scale2;       // sm_scale * log2(e)
 };
+
+// ---------------------------------------------------------------------------
+// output merge inside the split kernels (fuse_out)
+// ---------------------------------------------------------------------------
+// With at most SPLIT_MERGE_MAX_WARPS chunks, the split warps of one (sequence,
+// KV head, head group) are launched as ONE CTA (blockDim = (32, n_chunks)):
+// every warp still streams its own chunk through its own ring of buffers, then
+// leaves its soft-max partial in shared memory where its tiles were; after one
+// CTA barrier all threads merge the group's output quads - chunks in ascending
+// order, then the new token (Eq. 7) - and write the final outputs and each
+// head's (max2, sum).  No partial crosses global memory and no second kernel
+// stands between the streaming and the caller's next kernel.
+//
+// Partial of a warp: per head D+4 floats: acc[D], max2, sum, -, -.  Warp 0
+// also holds snew[g], the new token's logit per head.
+constexpr int PART_STRIDE_EXTRA = 4;
+constexpr int SPLIT_MERGE_MAX_WARPS = 8;
+
+template <int D>
+__device__ __forceinline__ void empty_partial(float* part, int heads, int lane) {
+  for (int i = lane; i < heads * (D + PART_STRIDE_EXTRA); i += 32)
+    part[i] = (i % (D + PART_STRIDE_EXTRA) == D) ? -INFINITY : 0.f;
+}
+
+// part0 / snew: warp 0's partial and new-token logits; warp w's partial lies
+// warp_stride floats further per warp.  Called by every warp of the CTA.
+template <typename T, int D>
+__device__ __noinline__ void block_merge_outputs(float* out, float2* head_ml, const T* v_new_row, const float* part0,
+                                                 int warp_stride, const float* snew, size_t bh0, int g_cnt) {
+  constexpr int PS = D + PART_STRIDE_EXTRA;
+  constexpr int NW = SPLIT_MERGE_MAX_WARPS;
+  const int nw = (int)blockDim.y;
+  const int tid = (int)(threadIdx.y * 32 + threadIdx.x);
+  __syncthreads();                             // every warp's partial is in shared memory
+  const int items = g_cnt * (D / 4);           // output quads of the group
+  for (int it = tid; it < items; it += nw * 32) {
+    const int g = it / (D / 4), d4 = it % (D / 4);
+    const float s_new = snew[g];
+    float mr[NW], lr[NW];
+    float M = s_new;
+#pragma unroll
+    for (int r = 0; r < NW; ++r) {
+      if (r < nw) {
+        mr[r] = part0[r * warp_stride + g * PS + D];
+        lr[r] = part0[r * warp_stride + g * PS + D + 1];
+        M = fmaxf(M, mr[r]);
+      }
+    }
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
+#pragma unroll
+    for (int r = 0; r < NW; ++r) {
+      if (r < nw) {
+        const float w = exp2_diff(mr[r], M);
+        const float4 a = *reinterpret_cast<const float4*>(part0 + r * warp_stride + g * PS + d4 * 4);
+        o.x = fmaf(a.x, w, o.x); o.y = fmaf(a.y, w, o.y); o.z = fmaf(a.z, w, o.z); o.w = fmaf(a.w, w, o.w);
+        L = fmaf(lr[r], w, L);
+      }
+    }
+    const float wn = exp2f(s_new - M);
+    L += wn;
+    const T* vn = v_new_row + d4 * 4;
+    const float iL = 1.f / L;
+    o.x = fmaf((float)vn[0], wn, o.x) * iL; o.y = fmaf((float)vn[1], wn, o.y) * iL;
+    o.z = fmaf((float)vn[2], wn, o.z) * iL; o.w = fmaf((float)vn[3], wn, o.w) * iL;
+    reinterpret_cast<float4*>(out + (bh0 + g) * D)[d4] = o;
+    if (d4 == 0) head_ml[bh0 + g] = make_float2(M, L);
+  }
+}
 
 // ---------------------------------------------------------------------------
 // split kernel
@@ -83,8 +155,8 @@ struct StepParams {
 // this warp ever waits on these barriers.
 // Every lane reads 16 bytes of a row; LPR lanes cover a row, so the warp reads
 // RPW = 32/LPR rows per pass and a tile takes NP = 16/RPW = LPR/2 passes.
-template <typename T, int D, int GU, int GB>
-__global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
+template <typename T, int D, int GU, int GB, bool FUSED>
+__global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32) tova_split_kernel(const StepParams p) {
   constexpr int EPL = Vec16<T>::N;          // elements per lane
   constexpr int RB = D * (int)sizeof(T);    // bytes per row
   constexpr int LPR = RB / 16;              // lanes per row
@@ -96,15 +168,27 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
   static_assert(GU % GB == 0, "head block must divide the unit");
   static_assert(NP * 2 == LPR, "a tile is half as many passes as lanes per row");
 
-  extern __shared__ __align__(128) unsigned char smem_raw[];
+  // per warp: the ring and the weights of a tile, rounded up to 128 bytes
+  constexpr int WARP_SMEM = (NB * TILE_BYTES + GU * TILE_ROWS * (int)sizeof(float) + 127) / 128 * 128;
+  extern __shared__ __align__(128) unsigned char smem_all[];
+  const int wib = FUSED ? threadIdx.y : 0;  // warp in block (FUSED: one CTA per head group, one warp per chunk)
+  unsigned char* smem_raw = smem_all + (size_t)wib * WARP_SMEM;
   unsigned char* ring = smem_raw;                                    // [NB][TILE_BYTES]
   float* w_p = reinterpret_cast<float*>(smem_raw + NB * TILE_BYTES); // [GU][16] weights of a tile
-  __shared__ __align__(8) uint64_t bars[NB];
+  // fuse_out: once all tiles are consumed the ring holds this warp's partial [GU][D+4]
+  // and (rank 0) the new token's logits [GU]
+  float* part = reinterpret_cast<float*>(ring);
+  float* snew = part + GU * (D + PART_STRIDE_EXTRA);
+  static_assert((GU * (D + PART_STRIDE_EXTRA) + GU) * sizeof(float) <= (size_t)NB * TILE_BYTES, "partial fits the ring");
+  __shared__ __align__(8) uint64_t bars_all[SPLIT_MERGE_MAX_WARPS][NB];
+  uint64_t* bars = bars_all[wib];
+  const float* part0 = reinterpret_cast<const float*>(smem_all);    // warp 0's partial and new-token logits
+  const float* snew0 = part0 + GU * (D + PART_STRIDE_EXTRA);
 
   const int lane = threadIdx.x;
   const int lig = lane % LPR;   // lane in row group
   const int sub = lane / LPR;   // which of the RPW rows of a pass
-  const int c = blockIdx.x, b = blockIdx.z;
+  const int c = FUSED ? wib : (int)blockIdx.x, b = blockIdx.z;
   const int kvh = blockIdx.y / p.hgroups, hg = blockIdx.y % p.hgroups;
   const int g_begin = hg * GU;
   const int g_cnt = min(GU, p.G - g_begin);                 // real heads of this unit
@@ -153,7 +237,7 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
   pdl_wait();
   pdl_launch_dependents();
 
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0)
+  if (c == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0)
     *p.cur_pos = (p.pos_t < 0) ? *p.cur_pos + 1 : p.pos_t;
   if (!early && lane == 0) {
     for (int u = 0; u < min(NB, n_ops); ++u) issue(u);
@@ -179,6 +263,7 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
 
   // The new token (candidate n): its logit per head, by the warp of chunk 0
   // while its first copies are in flight.
+  float s_new = 0.f;           // lane g keeps head g's logit of the new token (fuse_out)
   if (c == 0) {
     const T* kn = static_cast<const T*>(p.k_new) + ((size_t)b * p.Hkv + kvh) * D;
     float kf[EPL];
@@ -192,13 +277,27 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
 #pragma unroll
       for (int o = LPR / 2; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
       s *= p.scale2;
+      if (lane == g) s_new = s;
       if (lane == 0) {
         p.logits[(bh0 + g) * p.ld + p.n] = s;
-        p.part_ml[(bh0 + g) * p.pc + p.n_chunks] = make_float2(s, 1.f);
+        if (!FUSED) p.part_ml[(bh0 + g) * p.pc + p.n_chunks] = make_float2(s, 1.f);
       }
     }
+    if (FUSED && p.k_stage && hg == 0 && lane < LPR) {  // copies for a deferred eviction (the caller may reuse k and v)
+      const size_t w16 = ((size_t)b * p.Hkv + kvh) * LPR + lane;
+      static_cast<uint4*>(p.k_stage)[w16] = static_cast<const uint4*>(p.k_new)[w16];
+      static_cast<uint4*>(p.v_stage)[w16] = static_cast<const uint4*>(p.v_new)[w16];
+    }
   }
-  if (ntiles == 0) return;  // empty state: only the new token exists
+  if (ntiles == 0) {          // empty state: only the new token exists
+    if (FUSED) {
+      empty_partial<D>(part, GU, lane);
+      if (lane < GU) snew[lane] = s_new;
+      block_merge_outputs<T, D>(p.out, p.head_ml, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0,
+                                WARP_SMEM / 4, snew0, bh0, g_cnt);
+    }
+    return;
+  }
 
   // q of the unit's heads, kept packed (16 bytes per head and lane)
   uint4 qpk[GU];
@@ -307,9 +406,17 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
     // shared memory is released, and report.
     for (int u = 2 * t; u < min(2 * t + NB, n_ops); ++u) warp_wait(&bars[u % NB], (uint32_t)(u / NB) & 1u);
     if (lane == 0) atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
+    if (FUSED) {           // the other warps wait at the CTA barrier: join them with an empty partial
+      empty_partial<D>(part, GU, lane);
+      if (lane < GU) snew[lane] = s_new;
+      block_merge_outputs<T, D>(p.out, p.head_ml, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0,
+                                WARP_SMEM / 4, snew0, bh0, g_cnt);
+    }
     return;
   }
 
+  __syncwarp();                 // fuse_out: the partial goes where the tiles were
+  if (FUSED && lane < GU) snew[lane] = s_new;
   // ---- fold the RPW row groups of the warp, write the chunk partial -----------
 #pragma unroll
   for (int g = 0; g < GU; ++g) {
@@ -319,13 +426,23 @@ __global__ void __launch_bounds__(32) tova_split_kernel(const StepParams p) {
       for (int o = LPR; o < 32; o <<= 1) acc[g][e] += __shfl_xor_sync(0xffffffffu, acc[g][e], o);
     l[g] = warp_sum(l[g]);
     if (g < g_cnt && sub == 0) {
-      float* dst = p.part_acc + ((bh0 + g) * (size_t)(p.pc - 1) + c) * D + lig * EPL;
+      float* dst = FUSED ? part + g * (D + PART_STRIDE_EXTRA) + lig * EPL
+                              : p.part_acc + ((bh0 + g) * (size_t)(p.pc - 1) + c) * D + lig * EPL;
 #pragma unroll
       for (int e = 0; e < EPL; e += 4)
         *reinterpret_cast<float4*>(dst + e) = make_float4(acc[g][e], acc[g][e + 1], acc[g][e + 2], acc[g][e + 3]);
-      if (lane == 0) p.part_ml[(bh0 + g) * p.pc + c] = make_float2(m[g], l[g]);
+      if (lane == 0) {
+        if (FUSED) {
+          part[g * (D + PART_STRIDE_EXTRA) + D] = m[g];
+          part[g * (D + PART_STRIDE_EXTRA) + D + 1] = l[g];
+        } else {
+          p.part_ml[(bh0 + g) * p.pc + c] = make_float2(m[g], l[g]);
+        }
+      }
     }
   }
+  if (FUSED) block_merge_outputs<T, D>(p.out, p.head_ml, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0,
+                                WARP_SMEM / 4, snew0, bh0, g_cnt);
 }
 
 
@@ -407,7 +524,8 @@ __global__ void __launch_bounds__(CT, 1024 / CT) tova_combine_kernel(const StepP
   while ((2 << lg_S) <= 32 && (2 << lg_S) * items4 <= out_threads && (2 << lg_S) <= p.n_chunks) ++lg_S;
   const int S = 1 << lg_S;
   const int work = items4 * S;                 // a multiple of 32 whenever S > 1
-  const int g0 = (out_x < 0 || MODE == COMBINE_EVICT) ? work : out_x * CT + tid;
+  const bool fused = p.fuse_out != 0;          // outputs and per-head (max, sum) already came from the split kernel
+  const int g0 = (out_x < 0 || MODE == COMBINE_EVICT || fused) ? work : out_x * CT + tid;
   constexpr int RB16 = D * (int)sizeof(T) / 16;  // 16-byte words per row
   const int row_words = p.Hkv * RB16;
   int lg_np = 0;                   // partials per head rounded up to a power of two: thread i -> (i >> lg_np, i & mask)
@@ -450,7 +568,8 @@ __global__ void __launch_bounds__(CT, 1024 / CT) tova_combine_kernel(const StepP
   for (int u = 0; u < ML; ++u) {
     const int i = tid + u * CT;
     const int h = i >> lg_np, cc = i & ((1 << lg_np) - 1);
-    r_ml[u] = (i < total_ml && cc < np) ? p.part_ml[((size_t)b * p.H + h) * p.pc + cc] : make_float2(0.f, 0.f);
+    r_ml[u] = (!fused && i < total_ml && cc < np) ? p.part_ml[((size_t)b * p.H + h) * p.pc + cc]
+                                                  : make_float2(0.f, 0.f);
   }
   float r_lg[LG];
   int r_pos = pos_t;               // position held by this thread's first candidate
@@ -498,42 +617,52 @@ __global__ void __launch_bounds__(CT, 1024 / CT) tova_combine_kernel(const StepP
     }
   };
 
-  // ---- 1. partials to shared memory, global max and sum of every head ------------
+  // ---- 1. global max and sum of every head ---------------------------------------------
+  if (fused) {
+    for (int h = tid; h < p.H; h += CT) {
+      const float2 e = p.head_ml[(size_t)b * p.H + h];
+      hM[h] = e.x;
+      hInvL[h] = __frcp_rn(e.y);
+      hLc[h] = -e.x - __log2f(e.y * (float)p.H);
+    }
+    __syncthreads();
+  } else {
 #pragma unroll
-  for (int u = 0; u < ML; ++u) {
-    const int i = tid + u * CT;
-    const int h = i >> lg_np, cc = i & ((1 << lg_np) - 1);
-    if (i < total_ml && cc < np) pml[h * np + cc] = r_ml[u];
-  }
-  for (int i = tid + ML * CT; i < total_ml; i += CT) {
-    const int h = i >> lg_np, cc = i & ((1 << lg_np) - 1);
-    if (cc < np) pml[h * np + cc] = p.part_ml[((size_t)b * p.H + h) * p.pc + cc];
-  }
-  __syncthreads();
-  {
-    // a group of lph lanes per head, at most 8 partials per lane
-    int lg_lph = 0;
-    while ((1 << lg_lph) < 32 && (8 << lg_lph) < np) ++lg_lph;
-    const int lph = 1 << lg_lph;
-    const int hpp = CT >> lg_lph;                  // heads per pass
-    const int sub_l = tid & (lph - 1);
-    for (int h0 = 0; h0 < p.H; h0 += hpp) {        // uniform trip count: the shuffles need whole warps
-      const int h = h0 + (tid >> lg_lph);
-      const bool hv = h < p.H;
-      const float2* ml = pml + (size_t)(hv ? h : 0) * np;
-      float M = -INFINITY, L = 0.f;
-      for (int i = sub_l; i < np; i += lph) M = fmaxf(M, ml[i].x);
-      for (int o = lph >> 1; o >= 1; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-      for (int i = sub_l; i < np; i += lph) L = fmaf(ml[i].y, exp2f(ml[i].x - M), L);   // M is finite: the new token's partial is
-      for (int o = lph >> 1; o >= 1; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
-      if (hv && sub_l == 0) {
-        hM[h] = M;
-        hInvL[h] = __frcp_rn(L);
-        hLc[h] = -M - __log2f(L * (float)p.H);
+    for (int u = 0; u < ML; ++u) {
+      const int i = tid + u * CT;
+      const int h = i >> lg_np, cc = i & ((1 << lg_np) - 1);
+      if (i < total_ml && cc < np) pml[h * np + cc] = r_ml[u];
+    }
+    for (int i = tid + ML * CT; i < total_ml; i += CT) {
+      const int h = i >> lg_np, cc = i & ((1 << lg_np) - 1);
+      if (cc < np) pml[h * np + cc] = p.part_ml[((size_t)b * p.H + h) * p.pc + cc];
+    }
+    __syncthreads();
+    {
+      // a group of lph lanes per head, at most 8 partials per lane
+      int lg_lph = 0;
+      while ((1 << lg_lph) < 32 && (8 << lg_lph) < np) ++lg_lph;
+      const int lph = 1 << lg_lph;
+      const int hpp = CT >> lg_lph;                  // heads per pass
+      const int sub_l = tid & (lph - 1);
+      for (int h0 = 0; h0 < p.H; h0 += hpp) {        // uniform trip count: the shuffles need whole warps
+        const int h = h0 + (tid >> lg_lph);
+        const bool hv = h < p.H;
+        const float2* ml = pml + (size_t)(hv ? h : 0) * np;
+        float M = -INFINITY, L = 0.f;
+        for (int i = sub_l; i < np; i += lph) M = fmaxf(M, ml[i].x);
+        for (int o = lph >> 1; o >= 1; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        for (int i = sub_l; i < np; i += lph) L = fmaf(ml[i].y, exp2f(ml[i].x - M), L);   // M is finite: the new token's partial is
+        for (int o = lph >> 1; o >= 1; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+        if (hv && sub_l == 0) {
+          hM[h] = M;
+          hInvL[h] = __frcp_rn(L);
+          hLc[h] = -M - __log2f(L * (float)p.H);
+        }
       }
     }
+    __syncthreads();
   }
-  __syncthreads();
 
   // ---- 2. this CTA's share of the attention output --------------------------------
   auto write_outputs = [&]() {

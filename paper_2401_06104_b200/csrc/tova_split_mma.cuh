@@ -78,8 +78,8 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
 
 // grid = (max(n_chunks,1), Hkv*hgroups, B), block = one warp.
 // TWO: the group has more than 8 heads, rows 8..15 of the MMA tile are in use.
-template <int D, bool TWO>
-__global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
+template <int D, bool TWO, bool FUSED>
+__global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED ? (TWO ? 1 : 2) : 0) tova_split_mma_kernel(const StepParams p,
                                                             const __grid_constant__ CUtensorMap map_k,
                                                             const __grid_constant__ CUtensorMap map_v) {
   using T = __nv_bfloat16;
@@ -92,12 +92,24 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
 
   extern __shared__ unsigned char smem_raw[];
   // the swizzle is a function of the shared-memory address: tiles start on 1 KiB boundaries
-  unsigned char* ring = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
-  __shared__ __align__(8) uint64_t bars[NB];
+  constexpr int WARP_SMEM = NB * TILE_BYTES;   // per warp; a multiple of 1 KiB
+  const int wib = FUSED ? threadIdx.y : 0;     // warp in block (FUSED: one CTA per head group, one warp per chunk)
+  unsigned char* ring0 = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+  unsigned char* ring = ring0 + (size_t)wib * WARP_SMEM;
+  __shared__ __align__(8) uint64_t bars_all[SPLIT_MERGE_MAX_WARPS][NB];
+  uint64_t* bars = bars_all[wib];
+  const float* part0 = reinterpret_cast<const float*>(ring0);      // warp 0's partial and new-token logits
+  const float* snew0 = part0 + MMA_UNIT_HEADS * (D + PART_STRIDE_EXTRA);
+  // fuse_out: once all tiles are consumed the ring holds this warp's partial
+  // [MMA_UNIT_HEADS][D+4] and (rank 0) the new token's logits
+  float* part = reinterpret_cast<float*>(ring);
+  float* snew = part + MMA_UNIT_HEADS * (D + PART_STRIDE_EXTRA);
+  static_assert((MMA_UNIT_HEADS * (D + PART_STRIDE_EXTRA) + MMA_UNIT_HEADS) * sizeof(float) <= (size_t)NB * TILE_BYTES,
+                "partial fits the ring");
 
   const int lane = threadIdx.x;
   const int qrow = lane >> 2, qcol = (lane & 3) * 2;   // fragment coordinates of this lane
-  const int c = blockIdx.x, b = blockIdx.z;
+  const int c = FUSED ? wib : (int)blockIdx.x, b = blockIdx.z;
   const int kvh = blockIdx.y / p.hgroups, hg = blockIdx.y % p.hgroups;
   const int g_begin = hg * MMA_UNIT_HEADS;
   const int g_cnt = min(MMA_UNIT_HEADS, p.G - g_begin);
@@ -136,7 +148,7 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
   pdl_wait();
   pdl_launch_dependents();
 
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0)
+  if (c == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0)
     *p.cur_pos = (p.pos_t < 0) ? *p.cur_pos + 1 : p.pos_t;
   if (!early && lane == 0) {
     for (int u = 0; u < min(NB, n_ops); ++u) issue(u);
@@ -163,6 +175,7 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
   const size_t bh0 = (size_t)b * p.H + (size_t)kvh * p.G + g_begin;
 
   // The new token (candidate n): its logit per head, on the plain ALUs.
+  float s_new = 0.f;           // lane g keeps head g's logit (fuse_out)
   if (c == 0) {
     const int lig = lane % LPR;
     const T* kn = static_cast<const T*>(p.k_new) + ((size_t)b * p.Hkv + kvh) * D;
@@ -177,13 +190,27 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
 #pragma unroll
       for (int o = LPR / 2; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
       s *= p.scale2;
+      if (lane == g) s_new = s;
       if (lane == 0) {
         p.logits[(bh0 + g) * p.ld + p.n] = s;
-        p.part_ml[(bh0 + g) * p.pc + p.n_chunks] = make_float2(s, 1.f);
+        if (!FUSED) p.part_ml[(bh0 + g) * p.pc + p.n_chunks] = make_float2(s, 1.f);
       }
     }
+    if (FUSED && p.k_stage && hg == 0 && lane < LPR) {  // copies for a deferred eviction
+      const size_t w16 = ((size_t)b * p.Hkv + kvh) * LPR + lane;
+      static_cast<uint4*>(p.k_stage)[w16] = static_cast<const uint4*>(p.k_new)[w16];
+      static_cast<uint4*>(p.v_stage)[w16] = static_cast<const uint4*>(p.v_new)[w16];
+    }
   }
-  if (ntiles == 0) return;
+  if (ntiles == 0) {
+    if (FUSED) {
+      empty_partial<D>(part, MMA_UNIT_HEADS, lane);
+      if (lane < MMA_UNIT_HEADS) snew[lane] = s_new;
+      block_merge_outputs<T, D>(p.out, p.head_ml, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0,
+                                WARP_SMEM / 4, snew0, bh0, g_cnt);
+    }
+    return;
+  }
 
   // q as the A operand: rows = heads (zero beyond the group), 16 columns per k-step
   // fragment registers a0..a3 when TWO, else only a0 and a2 (a1 = a3 = 0)
@@ -326,10 +353,18 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
   if (failed) {
     for (int u = 2 * t; u < min(2 * t + NB, n_ops); ++u) warp_wait(&bars[u % NB], (uint32_t)(u / NB) & 1u);
     if (lane == 0) atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
+    if (FUSED) {           // the other warps wait at the CTA barrier: join them with an empty partial
+      empty_partial<D>(part, MMA_UNIT_HEADS, lane);
+      if (lane < MMA_UNIT_HEADS) snew[lane] = s_new;
+      block_merge_outputs<T, D>(p.out, p.head_ml, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0,
+                                WARP_SMEM / 4, snew0, bh0, g_cnt);
+    }
     return;
   }
 
   // ---- chunk partial: (max, sum) and the un-normalised weighted V sums ------------------
+  __syncwarp();                 // fuse_out: the partial goes where the tiles were
+  if (FUSED && lane < MMA_UNIT_HEADS) snew[lane] = s_new;
 #pragma unroll
   for (int rr = 0; rr < R; ++rr) {
     const int head = qrow + 8 * rr;
@@ -337,13 +372,23 @@ __global__ void __launch_bounds__(32) tova_split_mma_kernel(const StepParams p,
     lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
     lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
     if (head < g_cnt) {
-      float* dst = p.part_acc + ((bh0 + head) * (size_t)(p.pc - 1) + c) * D + qcol;
+      float* dst = FUSED ? part + head * (D + PART_STRIDE_EXTRA) + qcol
+                              : p.part_acc + ((bh0 + head) * (size_t)(p.pc - 1) + c) * D + qcol;
 #pragma unroll
       for (int j = 0; j < 2 * KS; ++j)
         *reinterpret_cast<float2*>(dst + j * 8) = make_float2(o[j][rr * 2], o[j][rr * 2 + 1]);
-      if ((lane & 3) == 0) p.part_ml[(bh0 + head) * p.pc + c] = make_float2(m[rr], lsum);
+      if ((lane & 3) == 0) {
+        if (FUSED) {
+          part[head * (D + PART_STRIDE_EXTRA) + D] = m[rr];
+          part[head * (D + PART_STRIDE_EXTRA) + D + 1] = lsum;
+        } else {
+          p.part_ml[(bh0 + head) * p.pc + c] = make_float2(m[rr], lsum);
+        }
+      }
     }
   }
+  if (FUSED) block_merge_outputs<T, D>(p.out, p.head_ml, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0,
+                                WARP_SMEM / 4, snew0, bh0, g_cnt);
 }
 
 }  // namespace tova

@@ -53,12 +53,28 @@ def test_tiny_reference_config_full_stream(name):
           f"max_err {rep.max_err:.2e} max_gap {rep.max_gap:.2e}")
 
 
+@pytest.mark.parametrize("fused", [True, False])
 @pytest.mark.parametrize("chunk_rows", [0, 32, 64, 96, 128, 256, 1024])
-def test_llama_shape_reduced_every_chunk_size(chunk_rows):
-    """bf16 MHA, capacity 203: several tiles plus a ragged tail at every chunk size."""
+def test_llama_shape_reduced_every_chunk_size(chunk_rows, fused):
+    """bf16 MHA, capacity 203: several tiles plus a ragged tail at every chunk
+    size, with the partials merged inside the streaming kernel (clusters of 1 to
+    7 warps) and through global memory."""
     w = LLAMA.scaled(batch=2, n_q_heads=6, n_kv_heads=6, capacity=203)
-    rep = run_lockstep(w, 460, chunk_rows=chunk_rows, block=50)
+    rep = run_lockstep(w, 460, chunk_rows=chunk_rows, block=50, fused_merge=fused)
     assert rep.evictions == 2 * (460 - 203)
+
+
+@pytest.mark.parametrize("H,Hkv", [(6, 6), (8, 2), (16, 1)])
+def test_more_chunks_than_a_cluster_holds(H, Hkv):
+    """Capacity 300 in 32-row chunks: 10 chunks, beyond the 8 a cluster merges,
+    so the partials take the global-memory route even with the fused merge on;
+    and 8 chunks exactly (capacity 256), the largest cluster."""
+    w = LLAMA.scaled(batch=2, n_q_heads=H, n_kv_heads=Hkv, capacity=300)
+    rep = run_lockstep(w, 300 + 120, chunk_rows=32, block=60)
+    assert rep.evictions == 2 * 120
+    w = LLAMA.scaled(batch=2, n_q_heads=H, n_kv_heads=Hkv, capacity=256)
+    rep = run_lockstep(w, 256 + 100, chunk_rows=32, block=60)
+    assert rep.evictions == 2 * 100
 
 
 @pytest.mark.parametrize("H,Hkv,D,dtype,cap,B", [
@@ -72,9 +88,10 @@ def test_llama_shape_reduced_every_chunk_size(chunk_rows):
     (2, 1, 128, W.DTYPE_BF16, 1, 2),        # capacity 1: every step evicts
     (4, 4, 128, W.DTYPE_BF16, 33, 1),       # one row past a tile
 ])
-def test_head_layouts_and_dtypes(H, Hkv, D, dtype, cap, B):
+@pytest.mark.parametrize("fused", [True, False])
+def test_head_layouts_and_dtypes(H, Hkv, D, dtype, cap, B, fused):
     w = MISTRAL.scaled(batch=B, n_q_heads=H, n_kv_heads=Hkv, head_dim=D, dtype=dtype, capacity=cap)
-    rep = run_lockstep(w, cap + 150, block=40)
+    rep = run_lockstep(w, cap + 150, block=40, fused_merge=fused)
     assert rep.evictions == B * 150
 
 
@@ -171,14 +188,17 @@ def test_step_argument_errors():
     assert c.tova_cache_len() == 0
 
 
-def test_deferred_eviction_gives_identical_results():
+@pytest.mark.parametrize("fused", [True, False])
+def test_deferred_eviction_gives_identical_results(fused):
     """Eviction on the cache's side stream, two caches taking turns like the
-    layers of a model: same outputs, dropped positions and state as the default."""
+    layers of a model: same outputs, dropped positions and state as the default.
+    Launches per step: streaming kernel + eviction kernel, plus the outputs-only
+    kernel when the partials are merged through global memory."""
     w = LLAMA.scaled(batch=2, n_q_heads=8, n_kv_heads=4, capacity=90)
     T = 220
     streams = [W.tokens(w, 0, T, layer=l) for l in range(2)]
-    ref = [make_cache(w) for _ in range(2)]
-    dfr = [make_cache(w) for _ in range(2)]
+    ref = [make_cache(w, fused_merge=fused) for _ in range(2)]
+    dfr = [make_cache(w, fused_merge=fused) for _ in range(2)]
     for c in dfr:
         c.tova_cache_set_deferred_eviction(True)
     dev = [[tova.to_device(a, w.dtype) for a in s] for s in streams]
@@ -201,4 +221,4 @@ def test_deferred_eviction_gives_identical_results():
         assert a["status"] == 0 and b["status"] == 0
         for key in ("len", "positions", "K", "V"):
             assert torch.equal(a[key], b[key]), key
-        assert dfr[l].tova_cache_launches() == 1 + 3 * T
+        assert dfr[l].tova_cache_launches() == 1 + (2 if fused else 3) * T
