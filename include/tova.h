@@ -151,11 +151,11 @@ int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows);
 
 /* Tuning: where the per-chunk partial results of a head are merged into the
  * attention output (Eq. 7 evaluated chunk by chunk).  on (default): when the
- * state splits into at most 8 chunks, the streaming warps of a head group are
- * launched as one thread-block cluster and merge through distributed shared
- * memory, so the outputs are final when the streaming kernel ends.  off: the
- * partials go through global memory to the second kernel.  Larger chunk counts
- * always take the second route.  Results do not depend on it beyond
+ * state splits into at most 8 chunks, the streaming warps of a head group run
+ * as one thread block and merge through shared memory, so the outputs are
+ * final when the streaming kernel ends.  off: the partials go through global
+ * memory to the second kernel.  Larger chunk counts always take the second
+ * route.  Results do not depend on it beyond
  * floating-point summation order.  Returns TOVA_ERR_NULL for a null handle. */
 int tova_cache_set_fused_merge(tova_cache* c, int32_t on);
 

@@ -82,7 +82,7 @@ struct tova_cache {
   tova_config cfg;
   CUtensorMap map_k, map_v;  // tiled views of K and V for the tensor-core split kernel
   bool use_mma;
-  bool fuse_merge;      // the split warps of a head group form a cluster and merge the outputs themselves
+  bool fuse_merge;      // the split warps of a head group form one CTA and merge the outputs themselves
   // deferred eviction: victim choice and insert run on a side stream, overlapping later work
   bool deferred, pending;
   cudaStream_t side;
