@@ -1,10 +1,15 @@
 // Split kernel for grouped-query attention on tensor cores (bf16 state).
 //
 // With G >= 4 query heads sharing a KV head, the logits of a tile are a real
-// dense contraction S[heads, rows] = q[heads, D] . K[rows, D]^T, and so is the
-// weighted sum O[heads, D] = P[heads, rows] . V[rows, D] (Eq. 4, Eq. 7).  One
-// warp per (sequence, KV head, chunk) runs them as m16n8k16 bf16 MMAs with fp32
-// accumulation: the M = 16 rows of the MMA are up to 16 heads of the group.
+// dense contraction and so is the weighted sum (Eq. 4, Eq. 7).  One warp per
+// (sequence, KV head, chunk) runs them as m16n8k16 bf16 MMAs with fp32
+// accumulation, in the transposed form that keeps the MMA tile full:
+//   S^T[rows, heads] = K[rows, D] . q^T[D, heads]      M = the tile's 16 rows, N = 8 heads
+//   O^T[D, heads]   += V^T[D, rows] . P^T[rows, heads] M = 16 of the D columns, N = 8 heads
+// (a second N tile when the group has more than 8 heads).  K and V^T are the A
+// operands, read from shared memory with ldmatrix (V transposed on the way);
+// q^T stays in registers; P^T goes from the accumulator layout of S^T to the
+// B-operand layout with four 8x8 warp transposes (movmatrix) per tile.
 //   - K/V tiles of 16 rows arrive through tiled TMA copies (tensor maps with the
 //     128-byte swizzle), so that ldmatrix reads them without bank conflicts;
 //   - products of bf16 inputs are exact in fp32, so the logits match an fp32
@@ -52,14 +57,12 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// The same with rows 8..15 of A all zero (at most 8 heads in the group): only
-// the upper half of the accumulator tile is kept, which halves the registers.
-__device__ __forceinline__ void mma_bf16_top(float (&d)[2], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-  float z0, z1;
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%10,%10};"
-      : "+f"(d[0]), "+f"(d[1]), "=f"(z0), "=f"(z1)
-      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.f));
+// Transposes an 8x8 matrix of 16-bit elements held one row pair per lane (lane = 4*row + col/2):
+// afterwards the lane holds elements (2(lane%4), lane/4) and (2(lane%4)+1, lane/4) of the input.
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
 }
 
 // (x, y) -> bf16x2 with x in the low half; and the rounding remainders.
@@ -212,33 +215,37 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
     return;
   }
 
-  // q as the A operand: rows = heads (zero beyond the group), 16 columns per k-step
-  // fragment registers a0..a3 when TWO, else only a0 and a2 (a1 = a3 = 0)
-  uint32_t qa[KS][2 * R];
+  // q^T as the B operand of S^T = K . q^T: column n of the MMA tile is head n
+  // (heads beyond the group are zero), 16 of the D values per k-step.
+  // qb[ks][2*nh + {0,1}]: head-tile nh (heads 8nh..8nh+7), d = 16ks + qcol (+8)
+  uint32_t qb[KS][2 * R];
 #pragma unroll
   for (int ks = 0; ks < KS; ++ks) {
     const int d = ks * 16 + qcol;
-    const uint32_t* r0 = reinterpret_cast<const uint32_t*>(qbase + (size_t)qrow * D + d);
-    const uint32_t* r1 = reinterpret_cast<const uint32_t*>(qbase + (size_t)(qrow + 8) * D + d);
-    if constexpr (TWO) {
-      qa[ks][0] = (qrow < g_cnt) ? r0[0] : 0u;
-      qa[ks][1] = (qrow + 8 < g_cnt) ? r1[0] : 0u;
-      qa[ks][2] = (qrow < g_cnt) ? r0[4] : 0u;      // d + 8
-      qa[ks][3] = (qrow + 8 < g_cnt) ? r1[4] : 0u;
-    } else {
-      qa[ks][0] = (qrow < g_cnt) ? r0[0] : 0u;
-      qa[ks][1] = (qrow < g_cnt) ? r0[4] : 0u;      // d + 8
+#pragma unroll
+    for (int nh = 0; nh < R; ++nh) {
+      const int head = qrow + 8 * nh;
+      const uint32_t* r = reinterpret_cast<const uint32_t*>(qbase + (size_t)head * D + d);
+      qb[ks][2 * nh] = (head < g_cnt) ? r[0] : 0u;
+      qb[ks][2 * nh + 1] = (head < g_cnt) ? r[4] : 0u;   // d + 8
     }
   }
 
-  float o[2 * KS][2 * R];   // O[heads, D]: n-tile j covers d = 8j..8j+7
+  // O^T[D, heads]: accumulator tile (nh, mt) covers d = 16mt..16mt+15 of heads 8nh..8nh+7;
+  // this lane holds d = 16mt + qrow (+8) of heads 8nh + qcol, qcol + 1
+  float o[R][KS][4];
 #pragma unroll
-  for (int j = 0; j < 2 * KS; ++j)
+  for (int nh = 0; nh < R; ++nh)
 #pragma unroll
-    for (int e = 0; e < 2 * R; ++e) o[j][e] = 0.f;
-  float m[R], l[R];   // [0]: head qrow, [1]: head qrow + 8
+    for (int mt = 0; mt < KS; ++mt)
 #pragma unroll
-  for (int rr = 0; rr < R; ++rr) { m[rr] = -INFINITY; l[rr] = 0.f; }
+      for (int e = 0; e < 4; ++e) o[nh][mt][e] = 0.f;
+  float m[R][2], l[R][2];   // heads 8nh + qcol + {0,1}
+#pragma unroll
+  for (int nh = 0; nh < R; ++nh) {
+    m[nh][0] = m[nh][1] = -INFINITY;
+    l[nh][0] = l[nh][1] = 0.f;
+  }
 
   // ldmatrix lane roles: lane supplies the address of row (lane % 8) of matrix (lane / 8)
   const int lm_r = lane & 7, lm_m = lane >> 3;
@@ -252,26 +259,21 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
     const uint32_t kt = ring_addr + (uint32_t)(uk % NB) * TILE_BYTES;
     const uint32_t vt = ring_addr + (uint32_t)(uv % NB) * TILE_BYTES;
 
-    // ---- S = q . K^T for the tile's 16 rows (two n-tiles of 8 rows) -------------
+    // ---- S^T = K . q^T: the tile's 16 rows are the M rows of the MMA -------------
     if (!warp_wait(&bars[uk % NB], (uint32_t)(uk / NB) & 1u)) { failed = true; break; }
     patch(uk, k_rows);
-    float s[2][2 * R];
+    float s[R][4];    // rows qrow (e = 0,1) and qrow + 8 (e = 2,3) of heads 8nh + qcol + (e & 1)
 #pragma unroll
-    for (int nt = 0; nt < 2; ++nt)
+    for (int nh = 0; nh < R; ++nh)
 #pragma unroll
-      for (int e = 0; e < 2 * R; ++e) s[nt][e] = 0.f;
+      for (int e = 0; e < 4; ++e) s[nh][e] = 0.f;
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
-      // matrices: (rows 0-7, d0..7) (rows 0-7, d0+8..15) (rows 8-15, d0..7) (rows 8-15, d0+8..15)
-      uint32_t kb[4];
-      ldmatrix_x4(kb, kt + swz(lm_r + 8 * (lm_m >> 1), ks * 2 + (lm_m & 1)));
-      if constexpr (TWO) {
-        mma_bf16(s[0], qa[ks], kb[0], kb[1]);
-        mma_bf16(s[1], qa[ks], kb[2], kb[3]);
-      } else {
-        mma_bf16_top(s[0], qa[ks][0], qa[ks][1], kb[0], kb[1]);
-        mma_bf16_top(s[1], qa[ks][0], qa[ks][1], kb[2], kb[3]);
-      }
+      // A fragment: (rows 0-7, d0..7) (rows 8-15, d0..7) (rows 0-7, d0+8..15) (rows 8-15, d0+8..15)
+      uint32_t ka[4];
+      ldmatrix_x4(ka, kt + swz(lm_r + 8 * (lm_m & 1), ks * 2 + (lm_m >> 1)));
+#pragma unroll
+      for (int nh = 0; nh < R; ++nh) mma_bf16(s[nh], ka, qb[ks][2 * nh], qb[ks][2 * nh + 1]);
     }
     __syncwarp();
     if (lane == 0 && uk + NB < n_ops) {
@@ -280,67 +282,65 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
     }
 
     // ---- online soft-max on the fragments ----------------------------------------
-    // lane holds, for head row qrow (+8): columns nt*8 + qcol + {0,1}
-    uint32_t p_hi[2 * R], p_lo[2 * R];   // a0..a3 when TWO, else a0 and a2
+    const bool row_lo = qrow < nvalid, row_hi = qrow + 8 < nvalid;
+    uint32_t pb_hi[R][2], pb_lo[R][2];   // P^T as the B operand of O^T += V^T . P^T: rows 2(lane%4)+{0,1} (+8), head lane/4
 #pragma unroll
-    for (int rr = 0; rr < R; ++rr) {
-      const int head = qrow + 8 * rr;
+    for (int nh = 0; nh < R; ++nh) {
       float v[4];
 #pragma unroll
-      for (int nt = 0; nt < 2; ++nt)
+      for (int e = 0; e < 4; ++e) v[e] = ((e < 2) ? row_lo : row_hi) ? s[nh][e] * p.scale2 : -INFINITY;
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int col = nt * 8 + qcol + e;
-          v[nt * 2 + e] = (col < nvalid) ? s[nt][rr * 2 + e] * p.scale2 : -INFINITY;
+      for (int hh = 0; hh < 2; ++hh) {
+        const int head = 8 * nh + qcol + hh;
+        if (head < g_cnt) {
+          float* lg = p.logits + (bh0 + head) * p.ld + row_begin + t * TILE_ROWS + qrow;
+          if (row_lo) lg[0] = v[hh];
+          if (row_hi) lg[8] = v[2 + hh];
         }
-      if (head < g_cnt) {
-        float* lg = p.logits + (bh0 + head) * p.ld + row_begin + t * TILE_ROWS;
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int col = nt * 8 + qcol + e;
-            if (col < nvalid) lg[col] = v[nt * 2 + e];
-          }
       }
-      float mx = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3]));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-      const float m_new = fmaxf(m[rr], mx);
-      const float corr = exp2_diff(m[rr], m_new);
       float e4[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) e4[i] = exp2_diff(v[i], m_new);
-      l[rr] = fmaf(l[rr], corr, (e4[0] + e4[1]) + (e4[2] + e4[3]));   // per-lane partial, folded at the end
-      m[rr] = m_new;
+      for (int hh = 0; hh < 2; ++hh) {
+        float mx = fmaxf(v[hh], v[2 + hh]);
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+        const float m_new = fmaxf(m[nh][hh], mx);
+        const float corr = exp2_diff(m[nh][hh], m_new);
+        e4[hh] = exp2_diff(v[hh], m_new);
+        e4[2 + hh] = exp2_diff(v[2 + hh], m_new);
+        l[nh][hh] = fmaf(l[nh][hh], corr, e4[hh] + e4[2 + hh]);   // per-lane partial, folded at the end
+        m[nh][hh] = m_new;
 #pragma unroll
-      for (int j = 0; j < 2 * KS; ++j) {
-        o[j][rr * 2] *= corr;
-        o[j][rr * 2 + 1] *= corr;
+        for (int mt = 0; mt < KS; ++mt) {
+          o[nh][mt][hh] *= corr;
+          o[nh][mt][2 + hh] *= corr;
+        }
       }
-      // P as the A operand of P.V: a0/a2 <- n-tile 0, a1/a3 rows + 8; a2,a3 <- n-tile 1
-      split_hi_lo(e4[0], e4[1], p_hi[TWO ? rr : 0], p_lo[TWO ? rr : 0]);
-      split_hi_lo(e4[2], e4[3], p_hi[TWO ? 2 + rr : 1], p_lo[TWO ? 2 + rr : 1]);
+      // weights as two bf16 terms, then from the accumulator layout (row = lane/4, heads
+      // 2(lane%4)+{0,1}) to the B-operand layout (rows 2(lane%4)+{0,1}, head = lane/4)
+      uint32_t hi0, lo0, hi1, lo1;
+      split_hi_lo(e4[0], e4[1], hi0, lo0);   // rows 0-7
+      split_hi_lo(e4[2], e4[3], hi1, lo1);   // rows 8-15
+      pb_hi[nh][0] = movmatrix_trans(hi0);
+      pb_hi[nh][1] = movmatrix_trans(hi1);
+      pb_lo[nh][0] = movmatrix_trans(lo0);
+      pb_lo[nh][1] = movmatrix_trans(lo1);
     }
 
-    // ---- O += P . V ------------------------------------------------------------------
+    // ---- O^T += V^T . P^T ----------------------------------------------------------------
     if (!warp_wait(&bars[uv % NB], (uint32_t)(uv / NB) & 1u)) { failed = true; break; }
     patch(uv, v_rows);
 #pragma unroll
-    for (int jj = 0; jj < KS; ++jj) {
-      // matrices: (rows 0-7, d0..7) (rows 8-15, d0..7) (rows 0-7, d0+8..15) (rows 8-15, d0+8..15), transposed
-      uint32_t vb[4];
-      ldmatrix_x4_trans(vb, vt + swz(lm_r + 8 * (lm_m & 1), jj * 2 + (lm_m >> 1)));
-      if constexpr (TWO) {
-        mma_bf16(o[2 * jj], p_hi, vb[0], vb[1]);
-        mma_bf16(o[2 * jj], p_lo, vb[0], vb[1]);
-        mma_bf16(o[2 * jj + 1], p_hi, vb[2], vb[3]);
-        mma_bf16(o[2 * jj + 1], p_lo, vb[2], vb[3]);
-      } else {
-        mma_bf16_top(o[2 * jj], p_hi[0], p_hi[1], vb[0], vb[1]);
-        mma_bf16_top(o[2 * jj], p_lo[0], p_lo[1], vb[0], vb[1]);
-        mma_bf16_top(o[2 * jj + 1], p_hi[0], p_hi[1], vb[2], vb[3]);
-        mma_bf16_top(o[2 * jj + 1], p_lo[0], p_lo[1], vb[2], vb[3]);
+    for (int mt = 0; mt < KS; ++mt) {
+      // A fragment of V^T (d rows, tile-row columns), transposing loads:
+      // (rows 0-7, d0..7) (rows 0-7, d0+8..15) (rows 8-15, d0..7) (rows 8-15, d0+8..15)
+      uint32_t va[4];
+      ldmatrix_x4_trans(va, vt + swz(lm_r + 8 * (lm_m >> 1), mt * 2 + (lm_m & 1)));
+#pragma unroll
+      for (int nh = 0; nh < R; ++nh) {
+        mma_bf16(o[nh][mt], va, pb_hi[nh][0], pb_hi[nh][1]);
+        mma_bf16(o[nh][mt], va, pb_lo[nh][0], pb_lo[nh][1]);
       }
     }
     __syncwarp();
@@ -366,27 +366,32 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
   __syncwarp();                 // fuse_out: the partial goes where the tiles were
   if (FUSED && lane < MMA_UNIT_HEADS) snew[lane] = s_new;
 #pragma unroll
-  for (int rr = 0; rr < R; ++rr) {
-    const int head = qrow + 8 * rr;
-    float lsum = l[rr];
-    lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
-    lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
-    if (head < g_cnt) {
-      float* dst = FUSED ? part + head * (D + PART_STRIDE_EXTRA) + qcol
-                              : p.part_acc + ((bh0 + head) * (size_t)(p.pc - 1) + c) * D + qcol;
+  for (int nh = 0; nh < R; ++nh)
 #pragma unroll
-      for (int j = 0; j < 2 * KS; ++j)
-        *reinterpret_cast<float2*>(dst + j * 8) = make_float2(o[j][rr * 2], o[j][rr * 2 + 1]);
-      if ((lane & 3) == 0) {
-        if (FUSED) {
-          part[head * (D + PART_STRIDE_EXTRA) + D] = m[rr];
-          part[head * (D + PART_STRIDE_EXTRA) + D + 1] = lsum;
-        } else {
-          p.part_ml[(bh0 + head) * p.pc + c] = make_float2(m[rr], lsum);
+    for (int hh = 0; hh < 2; ++hh) {
+      const int head = 8 * nh + qcol + hh;
+      float lsum = l[nh][hh];
+      lsum += __shfl_xor_sync(0xffffffffu, lsum, 4);
+      lsum += __shfl_xor_sync(0xffffffffu, lsum, 8);
+      lsum += __shfl_xor_sync(0xffffffffu, lsum, 16);
+      if (head < g_cnt) {
+        float* dst = FUSED ? part + head * (D + PART_STRIDE_EXTRA) + qrow
+                           : p.part_acc + ((bh0 + head) * (size_t)(p.pc - 1) + c) * D + qrow;
+#pragma unroll
+        for (int mt = 0; mt < KS; ++mt) {
+          dst[mt * 16] = o[nh][mt][hh];
+          dst[mt * 16 + 8] = o[nh][mt][2 + hh];
+        }
+        if (qrow == 0) {
+          if (FUSED) {
+            part[head * (D + PART_STRIDE_EXTRA) + D] = m[nh][hh];
+            part[head * (D + PART_STRIDE_EXTRA) + D + 1] = lsum;
+          } else {
+            p.part_ml[(bh0 + head) * p.pc + c] = make_float2(m[nh][hh], lsum);
+          }
         }
       }
     }
-  }
   if (FUSED) block_merge_outputs<T, D>(p.out, p.head_ml, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0,
                                 WARP_SMEM / 4, snew0, bh0, g_cnt);
 }
