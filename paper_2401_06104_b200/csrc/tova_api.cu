@@ -122,13 +122,29 @@ inline size_t split_smem_bytes(const tova_config& cfg) {
   return ((size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + sizeof(float) * gu * tova::TILE_ROWS + 127) / 128 * 128;
 }
 
-// Merge inside the split kernel: the warps of a head group's chunks form one CTA.
+// Merge inside the split kernel: the warps of a head group's chunks form one CTA
+// of up to 8 warps, or merge_ctas such CTAs in a cluster along x.
 inline void split_launch_shape(const StepParams& p, dim3& grid, dim3& block) {
   block = dim3(32);
   if (p.fuse_out) {
-    block.y = grid.x;
-    grid.x = 1;
+    block.y = (grid.x + p.merge_ctas - 1) / p.merge_ctas;
+    grid.x = p.merge_ctas;
   }
+}
+// Launch attributes of a split kernel: programmatic dependent launch, plus the cluster when CTAs merge across.
+inline int split_launch_attrs(const StepParams& p, cudaLaunchAttribute* at) {
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  if (!p.fuse_out || p.merge_ctas <= 1) return 1;
+  at[1].id = cudaLaunchAttributeClusterDimension;
+  at[1].val.clusterDim.x = p.merge_ctas;
+  at[1].val.clusterDim.y = 1;
+  at[1].val.clusterDim.z = 1;
+  return 2;
+}
+// Shared memory behind the rings for a CTA's merged partial (cluster merge only).
+inline size_t cluster_partial_bytes(const StepParams& p, int heads, int D) {
+  return (p.fuse_out && p.merge_ctas > 1) ? sizeof(float) * heads * (D + tova::PART_STRIDE_EXTRA) : 0;
 }
 
 template <typename T, int D, int GU, int GB, bool FUSED>
@@ -138,12 +154,13 @@ cudaError_t launch_split_f(int dev, const StepParams& p, dim3 grid, cudaStream_t
       ((size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * rb + sizeof(float) * GU * tova::TILE_ROWS + 127) / 128 * 128;
   dim3 block;
   split_launch_shape(p, grid, block);
-  const size_t smem = warp_smem * block.y;
+  const size_t smem = warp_smem * block.y + cluster_partial_bytes(p, GU, D);
   auto kern = tova::tova_split_kernel<T, D, GU, GB, FUSED>;
   static bool attr_set[64] = {};  // per instantiation and device: the attribute is per function
   if (!attr_set[dev & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)(warp_smem * tova::SPLIT_MERGE_MAX_WARPS));
+    cudaError_t e = cudaFuncSetAttribute(
+        kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        (int)(warp_smem * tova::SPLIT_MERGE_MAX_WARPS + sizeof(float) * GU * (D + tova::PART_STRIDE_EXTRA)));
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     if (e != cudaSuccess) return e;
@@ -154,11 +171,9 @@ cudaError_t launch_split_f(int dev, const StepParams& p, dim3 grid, cudaStream_t
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute at[2];
   cfg.attrs = at;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = split_launch_attrs(p, at);
   return cudaLaunchKernelEx(&cfg, kern, p);
 }
 
@@ -255,12 +270,14 @@ cudaError_t launch_split_mma_t(int dev, const StepParams& p, const CUtensorMap& 
   const size_t warp_smem = (size_t)tova::SPLIT_BUFFERS * tova::TILE_ROWS * D * 2;
   dim3 block;
   split_launch_shape(p, grid, block);
-  const size_t smem = warp_smem * block.y + 1024;
+  const size_t smem = warp_smem * block.y + 1024 + cluster_partial_bytes(p, tova::MMA_UNIT_HEADS, D);
   auto kern = tova::tova_split_mma_kernel<D, TWO, FUSED>;
   static bool attr_set[64] = {};
   if (!attr_set[dev & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)(warp_smem * tova::SPLIT_MERGE_MAX_WARPS + 1024));
+    cudaError_t e = cudaFuncSetAttribute(
+        kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        (int)(warp_smem * tova::SPLIT_MERGE_MAX_WARPS + 1024 +
+              sizeof(float) * tova::MMA_UNIT_HEADS * (D + tova::PART_STRIDE_EXTRA)));
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     if (e != cudaSuccess) return e;
@@ -271,11 +288,9 @@ cudaError_t launch_split_mma_t(int dev, const StepParams& p, const CUtensorMap& 
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute at[2];
   cfg.attrs = at;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = split_launch_attrs(p, at);
   return cudaLaunchKernelEx(&cfg, kern, p, mk, mv);
 }
 
@@ -398,6 +413,21 @@ int pick_chunk_rows(const tova_config& cfg, int sm_count) {
   return cr <= 8192 ? cr : -1;  // -1: no chunk size keeps the combine kernel's shared memory within its limit
 }
 
+// Whether the split kernel merges the chunk partials itself: always when one CTA
+// of 8 warps covers the state; with up to 8 such CTAs per head group (a
+// cluster) only while all CTAs of the launch are resident at once - beyond
+// that single-warp CTAs, which the hardware hands out one by one, stream better.
+bool fused_merge_fits(const tova_config& cfg, int chunk_rows, int sm_count) {
+  const int chunks = (cfg.capacity + chunk_rows - 1) / chunk_rows;
+  if (chunks <= tova::SPLIT_MERGE_MAX_WARPS) return true;
+  if (chunks > tova::SPLIT_MERGE_MAX_WARPS * tova::COMBINE_CLUSTER_MAX) return false;
+  const int G = cfg.n_q_heads / cfg.n_kv_heads;
+  const long long hgroups = (G + unit_heads(cfg) - 1) / unit_heads(cfg);
+  const long long ctas = (long long)cfg.batch * cfg.n_kv_heads * hgroups *
+                         ((chunks + tova::SPLIT_MERGE_MAX_WARPS - 1) / tova::SPLIT_MERGE_MAX_WARPS);
+  return ctas <= 2LL * sm_count;
+}
+
 // CTA size of a combine launch, and with it whether a CTA's logits are staged
 // through shared memory (bulk copies): only when a thread would otherwise need
 // several dependent batches of loads for them.
@@ -461,7 +491,9 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
   cudaError_t e;
   const bool defer = c->deferred && allow_defer;
   p.head_ml = reinterpret_cast<float2*>(base + c->lay.head_ml);
-  p.fuse_out = (c->fuse_merge && (cfg.capacity + c->chunk_rows - 1) / c->chunk_rows <= tova::SPLIT_MERGE_MAX_WARPS) ? 1 : 0;
+  p.fuse_out = (c->fuse_merge && fused_merge_fits(cfg, c->chunk_rows, c->sm_count)) ? 1 : 0;
+  p.merge_ctas = p.fuse_out ? (p.n_chunks + tova::SPLIT_MERGE_MAX_WARPS - 1) / tova::SPLIT_MERGE_MAX_WARPS : 1;
+  if (p.merge_ctas < 1) p.merge_ctas = 1;
   if (p.fuse_out && defer) {   // the split kernel keeps copies of the new token's rows for the later insert
     p.k_stage = base + c->lay.df_k;
     p.v_stage = base + c->lay.df_v;

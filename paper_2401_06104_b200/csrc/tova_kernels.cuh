@@ -69,6 +69,7 @@ struct StepParams {
   int32_t do_evict;   // n == cap and the policy is on
   int32_t fuse_out;   // the split kernel's warps of a (sequence, KV head, head group) form a cluster and write
                       // the outputs themselves; the combine kernel then only picks the victim
+  int32_t merge_ctas; // fuse_out: CTAs (of up to 8 warps = chunks) per head group; > 1: they form a cluster (x)
   int32_t mode;       // combine kernel: 0 whole step, 1 outputs only, 2 victim + insert only
   void* k_stage;      // [B,Hkv,D] mode 1: copies of the new token's rows for a later mode-2 launch
   void* v_stage;
@@ -144,6 +145,107 @@ __device__ __noinline__ void block_merge_outputs(float* out, float2* head_ml, co
   }
 }
 
+// The same across a thread-block cluster, for states of up to 8 x 8 chunks: the
+// CTAs that share a head group (cluster dimension x, CTA r streams chunks 8r ..
+// 8r+7) first merge their own warps' partials into one partial per head
+// (`cpart`, shared memory of their own), meet at a cluster barrier, and then
+// split the output quads among all threads of the cluster, each reading the
+// CTAs' partials through distributed shared memory.  CTA 0's warp 0 holds the
+// new token's logits.  Nobody leaves before the second cluster barrier: a peer
+// may still be reading its shared memory.
+template <typename T, int D>
+__device__ __noinline__ void cluster_merge_outputs(float* out, float2* head_ml, const T* v_new_row, const float* part0,
+                                                   int warp_stride, float* snew0, float* cpart, size_t bh0,
+                                                   int g_cnt) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cl = cg::this_cluster();
+  constexpr int PS = D + PART_STRIDE_EXTRA;
+  constexpr int NW = SPLIT_MERGE_MAX_WARPS;
+  const int nw = (int)blockDim.y, nthreads = nw * 32;
+  const int tid = (int)(threadIdx.y * 32 + threadIdx.x);
+  const int ncta = (int)cl.num_blocks(), rank = (int)cl.block_rank();
+  const int items = g_cnt * (D / 4);           // output quads of the group
+  __syncthreads();                             // every warp's partial is in shared memory
+  for (int it = tid; it < items; it += nthreads) {
+    const int g = it / (D / 4), d4 = it % (D / 4);
+    float mr[NW], lr[NW];
+    float M = -INFINITY;
+#pragma unroll
+    for (int r = 0; r < NW; ++r) {
+      if (r < nw) {
+        mr[r] = part0[r * warp_stride + g * PS + D];
+        lr[r] = part0[r * warp_stride + g * PS + D + 1];
+        M = fmaxf(M, mr[r]);
+      }
+    }
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
+#pragma unroll
+    for (int r = 0; r < NW; ++r) {
+      if (r < nw) {
+        const float w = exp2_diff(mr[r], M);
+        const float4 a = *reinterpret_cast<const float4*>(part0 + r * warp_stride + g * PS + d4 * 4);
+        o.x = fmaf(a.x, w, o.x); o.y = fmaf(a.y, w, o.y); o.z = fmaf(a.z, w, o.z); o.w = fmaf(a.w, w, o.w);
+        L = fmaf(lr[r], w, L);
+      }
+    }
+    *reinterpret_cast<float4*>(cpart + g * PS + d4 * 4) = o;
+    if (d4 == 0) {
+      cpart[g * PS + D] = M;
+      cpart[g * PS + D + 1] = L;
+    }
+  }
+  cl.sync();                                   // every CTA's partial is in its shared memory
+  const float* rp[COMBINE_CLUSTER_MAX];
+#pragma unroll
+  for (int r = 0; r < COMBINE_CLUSTER_MAX; ++r) rp[r] = cl.map_shared_rank(cpart, r < ncta ? r : 0);
+  const float* rs = cl.map_shared_rank(snew0, 0);
+  for (int it = rank * nthreads + tid; it < items; it += ncta * nthreads) {
+    const int g = it / (D / 4), d4 = it % (D / 4);
+    const float s_new = rs[g];
+    float mr[COMBINE_CLUSTER_MAX], lr[COMBINE_CLUSTER_MAX];
+    float M = s_new;
+#pragma unroll
+    for (int r = 0; r < COMBINE_CLUSTER_MAX; ++r) {
+      if (r < ncta) {
+        mr[r] = rp[r][g * PS + D];
+        lr[r] = rp[r][g * PS + D + 1];
+        M = fmaxf(M, mr[r]);
+      }
+    }
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
+#pragma unroll
+    for (int r = 0; r < COMBINE_CLUSTER_MAX; ++r) {
+      if (r < ncta) {
+        const float w = exp2_diff(mr[r], M);
+        const float4 a = *reinterpret_cast<const float4*>(rp[r] + g * PS + d4 * 4);
+        o.x = fmaf(a.x, w, o.x); o.y = fmaf(a.y, w, o.y); o.z = fmaf(a.z, w, o.z); o.w = fmaf(a.w, w, o.w);
+        L = fmaf(lr[r], w, L);
+      }
+    }
+    const float wn = exp2f(s_new - M);
+    L += wn;
+    const T* vn = v_new_row + d4 * 4;
+    const float iL = 1.f / L;
+    o.x = fmaf((float)vn[0], wn, o.x) * iL; o.y = fmaf((float)vn[1], wn, o.y) * iL;
+    o.z = fmaf((float)vn[2], wn, o.z) * iL; o.w = fmaf((float)vn[3], wn, o.w) * iL;
+    reinterpret_cast<float4*>(out + (bh0 + g) * D)[d4] = o;
+    if (d4 == 0) head_ml[bh0 + g] = make_float2(M, L);
+  }
+  cl.sync();
+}
+
+// One CTA per head group, or a cluster of them (merge_ctas > 1).
+template <typename T, int D>
+__device__ __forceinline__ void fused_merge(const StepParams& p, const T* v_new_row, const float* part0, int warp_stride,
+                                            float* snew0, float* cpart, size_t bh0, int g_cnt) {
+  if (p.merge_ctas > 1)
+    cluster_merge_outputs<T, D>(p.out, p.head_ml, v_new_row, part0, warp_stride, snew0, cpart, bh0, g_cnt);
+  else
+    block_merge_outputs<T, D>(p.out, p.head_ml, v_new_row, part0, warp_stride, snew0, bh0, g_cnt);
+}
+
 // ---------------------------------------------------------------------------
 // split kernel
 // ---------------------------------------------------------------------------
@@ -183,12 +285,14 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32) tova_
   __shared__ __align__(8) uint64_t bars_all[SPLIT_MERGE_MAX_WARPS][NB];
   uint64_t* bars = bars_all[wib];
   const float* part0 = reinterpret_cast<const float*>(smem_all);    // warp 0's partial and new-token logits
-  const float* snew0 = part0 + GU * (D + PART_STRIDE_EXTRA);
+  float* snew0 = reinterpret_cast<float*>(smem_all) + GU * (D + PART_STRIDE_EXTRA);
+  // merge_ctas > 1: this CTA's merged partial, behind the rings
+  float* cpart = reinterpret_cast<float*>(smem_all + (size_t)(FUSED ? blockDim.y : 1) * WARP_SMEM);
 
   const int lane = threadIdx.x;
   const int lig = lane % LPR;   // lane in row group
   const int sub = lane / LPR;   // which of the RPW rows of a pass
-  const int c = FUSED ? wib : (int)blockIdx.x, b = blockIdx.z;
+  const int c = FUSED ? (int)(blockIdx.x * blockDim.y) + wib : (int)blockIdx.x, b = blockIdx.z;
   const int kvh = blockIdx.y / p.hgroups, hg = blockIdx.y % p.hgroups;
   const int g_begin = hg * GU;
   const int g_cnt = min(GU, p.G - g_begin);                 // real heads of this unit
@@ -293,8 +397,8 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32) tova_
     if (FUSED) {
       empty_partial<D>(part, GU, lane);
       if (lane < GU) snew[lane] = s_new;
-      block_merge_outputs<T, D>(p.out, p.head_ml, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0,
-                                WARP_SMEM / 4, snew0, bh0, g_cnt);
+      fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew0,
+                        cpart, bh0, g_cnt);
     }
     return;
   }
@@ -409,8 +513,8 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32) tova_
     if (FUSED) {           // the other warps wait at the CTA barrier: join them with an empty partial
       empty_partial<D>(part, GU, lane);
       if (lane < GU) snew[lane] = s_new;
-      block_merge_outputs<T, D>(p.out, p.head_ml, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0,
-                                WARP_SMEM / 4, snew0, bh0, g_cnt);
+      fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew0,
+                        cpart, bh0, g_cnt);
     }
     return;
   }
@@ -441,8 +545,8 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32) tova_
       }
     }
   }
-  if (FUSED) block_merge_outputs<T, D>(p.out, p.head_ml, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0,
-                                WARP_SMEM / 4, snew0, bh0, g_cnt);
+  if (FUSED) fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew0,
+                        cpart, bh0, g_cnt);
 }
 
 

@@ -102,7 +102,9 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
   __shared__ __align__(8) uint64_t bars_all[SPLIT_MERGE_MAX_WARPS][NB];
   uint64_t* bars = bars_all[wib];
   const float* part0 = reinterpret_cast<const float*>(ring0);      // warp 0's partial and new-token logits
-  const float* snew0 = part0 + MMA_UNIT_HEADS * (D + PART_STRIDE_EXTRA);
+  float* snew0 = reinterpret_cast<float*>(ring0) + MMA_UNIT_HEADS * (D + PART_STRIDE_EXTRA);
+  // merge_ctas > 1: this CTA's merged partial, behind the rings
+  float* cpart = reinterpret_cast<float*>(ring0 + (size_t)(FUSED ? blockDim.y : 1) * WARP_SMEM);
   // fuse_out: once all tiles are consumed the ring holds this warp's partial
   // [MMA_UNIT_HEADS][D+4] and (rank 0) the new token's logits
   float* part = reinterpret_cast<float*>(ring);
@@ -112,7 +114,7 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
 
   const int lane = threadIdx.x;
   const int qrow = lane >> 2, qcol = (lane & 3) * 2;   // fragment coordinates of this lane
-  const int c = FUSED ? wib : (int)blockIdx.x, b = blockIdx.z;
+  const int c = FUSED ? (int)(blockIdx.x * blockDim.y) + wib : (int)blockIdx.x, b = blockIdx.z;
   const int kvh = blockIdx.y / p.hgroups, hg = blockIdx.y % p.hgroups;
   const int g_begin = hg * MMA_UNIT_HEADS;
   const int g_cnt = min(MMA_UNIT_HEADS, p.G - g_begin);
@@ -209,8 +211,8 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
     if (FUSED) {
       empty_partial<D>(part, MMA_UNIT_HEADS, lane);
       if (lane < MMA_UNIT_HEADS) snew[lane] = s_new;
-      block_merge_outputs<T, D>(p.out, p.head_ml, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0,
-                                WARP_SMEM / 4, snew0, bh0, g_cnt);
+      fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew0,
+                        cpart, bh0, g_cnt);
     }
     return;
   }
@@ -356,8 +358,8 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
     if (FUSED) {           // the other warps wait at the CTA barrier: join them with an empty partial
       empty_partial<D>(part, MMA_UNIT_HEADS, lane);
       if (lane < MMA_UNIT_HEADS) snew[lane] = s_new;
-      block_merge_outputs<T, D>(p.out, p.head_ml, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0,
-                                WARP_SMEM / 4, snew0, bh0, g_cnt);
+      fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew0,
+                        cpart, bh0, g_cnt);
     }
     return;
   }
@@ -392,8 +394,8 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
         }
       }
     }
-  if (FUSED) block_merge_outputs<T, D>(p.out, p.head_ml, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0,
-                                WARP_SMEM / 4, snew0, bh0, g_cnt);
+  if (FUSED) fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew0,
+                        cpart, bh0, g_cnt);
 }
 
 }  // namespace tova

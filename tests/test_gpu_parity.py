@@ -65,16 +65,26 @@ def test_llama_shape_reduced_every_chunk_size(chunk_rows, fused):
 
 
 @pytest.mark.parametrize("H,Hkv", [(6, 6), (8, 2), (16, 1)])
-def test_more_chunks_than_a_cluster_holds(H, Hkv):
-    """Capacity 300 in 32-row chunks: 10 chunks, beyond the 8 a cluster merges,
-    so the partials take the global-memory route even with the fused merge on;
-    and 8 chunks exactly (capacity 256), the largest cluster."""
+def test_head_groups_spanning_several_ctas(H, Hkv):
+    """Capacity 300 in 32-row chunks: 10 chunks, i.e. two CTAs of 5 warps per head
+    group that merge across a cluster (1 to 2 CTAs while the state fills); and 8
+    chunks exactly (capacity 256), the largest single CTA."""
     w = LLAMA.scaled(batch=2, n_q_heads=H, n_kv_heads=Hkv, capacity=300)
     rep = run_lockstep(w, 300 + 120, chunk_rows=32, block=60)
     assert rep.evictions == 2 * 120
     w = LLAMA.scaled(batch=2, n_q_heads=H, n_kv_heads=Hkv, capacity=256)
     rep = run_lockstep(w, 256 + 100, chunk_rows=32, block=60)
     assert rep.evictions == 2 * 100
+
+
+@pytest.mark.parametrize("H,Hkv,cap", [(4, 4, 2040), (8, 2, 1500), (2, 2, 2100)])
+def test_cluster_sizes_up_to_eight_and_beyond(H, Hkv, cap):
+    """32-row chunks: 64 chunks (8 CTAs x 8 warps, the largest cluster), 47 chunks
+    (6 CTAs, ragged), and 66 chunks, which no cluster holds: partials through
+    global memory although the fused merge is on."""
+    w = LLAMA.scaled(batch=1, n_q_heads=H, n_kv_heads=Hkv, capacity=cap)
+    rep = run_lockstep(w, cap + 40, chunk_rows=32, block=64, direct_fill=True, check_state_every=8)
+    assert rep.evictions == 40
 
 
 @pytest.mark.parametrize("H,Hkv,D,dtype,cap,B", [
