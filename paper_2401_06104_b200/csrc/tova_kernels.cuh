@@ -648,6 +648,11 @@ __global__ void __launch_bounds__(CT, 1024 / CT) tova_combine_kernel(const StepP
     mbar_fence_init();
   }
   __syncthreads();
+  // The block minima travel to CTA 0 through distributed shared memory, which
+  // may only be touched once its CTA runs: the CTAs of a cluster are resident
+  // together but need not start together.  Everybody reports in here (without
+  // waiting) and checks that all have done so just before that store.
+  if (score) cluster_arrive_release();
 
   pdl_wait();
   pdl_launch_dependents();
@@ -901,6 +906,7 @@ __global__ void __launch_bounds__(CT, 1024 / CT) tova_combine_kernel(const StepP
   if (lane == 0) { red_v[warp] = val; red_i[warp] = idx; red_p[warp] = cpos; }
   __syncthreads();
   cg::cluster_group cluster = cg::this_cluster();
+  cluster_wait_acquire();          // every CTA of the cluster has started (arrival at kernel entry)
   if (tid == 0) {
     for (int w = 1; w < CT / 32; ++w)
       if (red_v[w] < val || (red_v[w] == val && red_i[w] < idx)) { val = red_v[w]; idx = red_i[w]; cpos = red_p[w]; }
