@@ -280,12 +280,11 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32) tova_
   // fuse_out: once all tiles are consumed the ring holds this warp's partial [GU][D+4]
   // and (rank 0) the new token's logits [GU]
   float* part = reinterpret_cast<float*>(ring);
-  float* snew = part + GU * (D + PART_STRIDE_EXTRA);
   static_assert((GU * (D + PART_STRIDE_EXTRA) + GU) * sizeof(float) <= (size_t)NB * TILE_BYTES, "partial fits the ring");
   __shared__ __align__(8) uint64_t bars_all[SPLIT_MERGE_MAX_WARPS][NB];
   uint64_t* bars = bars_all[wib];
-  const float* part0 = reinterpret_cast<const float*>(smem_all);    // warp 0's partial and new-token logits
-  float* snew0 = reinterpret_cast<float*>(smem_all) + GU * (D + PART_STRIDE_EXTRA);
+  const float* part0 = reinterpret_cast<const float*>(smem_all);    // warp 0's partial
+  __shared__ float snew_s[MAX_UNIT_HEADS];                          // the new token's logit per head (chunk 0's warp)
   // merge_ctas > 1: this CTA's merged partial, behind the rings
   float* cpart = reinterpret_cast<float*>(smem_all + (size_t)(FUSED ? blockDim.y : 1) * WARP_SMEM);
 
@@ -346,11 +345,22 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32) tova_
   if (!early && lane == 0) {
     for (int u = 0; u < min(NB, n_ops); ++u) issue(u);
   }
+  // Every global load of the prologue is issued before the first one is used:
+  // the row that may have changed, q of the unit's heads (kept packed, 16 bytes
+  // per head and lane) and, for chunk 0's warp, the new token's key.
+  const T* qbase = static_cast<const T*>(p.q) + ((size_t)b * p.H + (size_t)kvh * p.G + g_begin) * D;
+  const size_t bh0 = (size_t)b * p.H + (size_t)kvh * p.G + g_begin;
+  const int ls = early ? __ldcg(p.last_slot + b) : -1;
+  uint4 qpk[GU];
+#pragma unroll
+  for (int g = 0; g < GU; ++g)
+    qpk[g] = *reinterpret_cast<const uint4*>(qbase + (size_t)min(g, g_cnt - 1) * D + lig * EPL);
+  uint4 knw = make_uint4(0u, 0u, 0u, 0u);
+  if (c == 0)
+    knw = *reinterpret_cast<const uint4*>(static_cast<const T*>(p.k_new) + ((size_t)b * p.Hkv + kvh) * D + lig * EPL);
+
   int patch_row = -1;              // row of this chunk that must be fetched again, if any
-  if (early) {
-    const int ls = __ldcg(p.last_slot + b);
-    if (ls >= row_begin && ls < row_begin + rows) patch_row = ls - row_begin;
-  }
+  if (ls >= row_begin && ls < row_begin + rows) patch_row = ls - row_begin;
   // Re-fetches row patch_row of operand tile u (already landed) from global memory.
   auto patch = [&](int u, unsigned char* tile, const unsigned char* src) {
     const int t = u >> 1;
@@ -362,29 +372,27 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32) tova_
     }
   };
 
-  const T* qbase = static_cast<const T*>(p.q) + ((size_t)b * p.H + (size_t)kvh * p.G + g_begin) * D;
-  const size_t bh0 = (size_t)b * p.H + (size_t)kvh * p.G + g_begin;
-
   // The new token (candidate n): its logit per head, by the warp of chunk 0
   // while its first copies are in flight.
-  float s_new = 0.f;           // lane g keeps head g's logit of the new token (fuse_out)
   if (c == 0) {
-    const T* kn = static_cast<const T*>(p.k_new) + ((size_t)b * p.Hkv + kvh) * D;
     float kf[EPL];
-    Vec16<T>::unpack(*reinterpret_cast<const uint4*>(kn + lig * EPL), kf);
-    for (int g = 0; g < g_cnt; ++g) {
-      float qf[EPL];
-      Vec16<T>::unpack(*reinterpret_cast<const uint4*>(qbase + (size_t)g * D + lig * EPL), qf);
-      float s = 0.f;
+    Vec16<T>::unpack(knw, kf);
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) s = fmaf(qf[e], kf[e], s);
+    for (int g = 0; g < GU; ++g) {
+      if (g < g_cnt) {
+        float qf[EPL];
+        Vec16<T>::unpack(qpk[g], qf);
+        float s = 0.f;
 #pragma unroll
-      for (int o = LPR / 2; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-      s *= p.scale2;
-      if (lane == g) s_new = s;
-      if (lane == 0) {
-        p.logits[(bh0 + g) * p.ld + p.n] = s;
-        if (!FUSED) p.part_ml[(bh0 + g) * p.pc + p.n_chunks] = make_float2(s, 1.f);
+        for (int e = 0; e < EPL; ++e) s = fmaf(qf[e], kf[e], s);
+#pragma unroll
+        for (int o = LPR / 2; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        s *= p.scale2;
+        if (lane == 0) {
+          p.logits[(bh0 + g) * p.ld + p.n] = s;
+          if (FUSED) snew_s[g] = s;
+          else p.part_ml[(bh0 + g) * p.pc + p.n_chunks] = make_float2(s, 1.f);
+        }
       }
     }
     if (FUSED && p.k_stage && hg == 0 && lane < LPR) {  // copies for a deferred eviction (the caller may reuse k and v)
@@ -396,18 +404,12 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32) tova_
   if (ntiles == 0) {          // empty state: only the new token exists
     if (FUSED) {
       empty_partial<D>(part, GU, lane);
-      if (lane < GU) snew[lane] = s_new;
-      fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew0,
+      fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew_s,
                         cpart, bh0, g_cnt);
     }
     return;
   }
 
-  // q of the unit's heads, kept packed (16 bytes per head and lane)
-  uint4 qpk[GU];
-#pragma unroll
-  for (int g = 0; g < GU; ++g)
-    qpk[g] = *reinterpret_cast<const uint4*>(qbase + (size_t)min(g, g_cnt - 1) * D + lig * EPL);
 
   float m[GU], l[GU], acc[GU][EPL];
 #pragma unroll
@@ -512,15 +514,13 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32) tova_
     if (lane == 0) atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
     if (FUSED) {           // the other warps wait at the CTA barrier: join them with an empty partial
       empty_partial<D>(part, GU, lane);
-      if (lane < GU) snew[lane] = s_new;
-      fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew0,
+      fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew_s,
                         cpart, bh0, g_cnt);
     }
     return;
   }
 
   __syncwarp();                 // fuse_out: the partial goes where the tiles were
-  if (FUSED && lane < GU) snew[lane] = s_new;
   // ---- fold the RPW row groups of the warp, write the chunk partial -----------
 #pragma unroll
   for (int g = 0; g < GU; ++g) {
@@ -545,7 +545,7 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32) tova_
       }
     }
   }
-  if (FUSED) fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew0,
+  if (FUSED) fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew_s,
                         cpart, bh0, g_cnt);
 }
 

@@ -101,14 +101,13 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
   unsigned char* ring = ring0 + (size_t)wib * WARP_SMEM;
   __shared__ __align__(8) uint64_t bars_all[SPLIT_MERGE_MAX_WARPS][NB];
   uint64_t* bars = bars_all[wib];
-  const float* part0 = reinterpret_cast<const float*>(ring0);      // warp 0's partial and new-token logits
-  float* snew0 = reinterpret_cast<float*>(ring0) + MMA_UNIT_HEADS * (D + PART_STRIDE_EXTRA);
+  const float* part0 = reinterpret_cast<const float*>(ring0);      // warp 0's partial
+  __shared__ float snew_s[MMA_UNIT_HEADS];                         // the new token's logit per head (chunk 0's warp)
   // merge_ctas > 1: this CTA's merged partial, behind the rings
   float* cpart = reinterpret_cast<float*>(ring0 + (size_t)(FUSED ? blockDim.y : 1) * WARP_SMEM);
   // fuse_out: once all tiles are consumed the ring holds this warp's partial
   // [MMA_UNIT_HEADS][D+4] and (rank 0) the new token's logits
   float* part = reinterpret_cast<float*>(ring);
-  float* snew = part + MMA_UNIT_HEADS * (D + PART_STRIDE_EXTRA);
   static_assert((MMA_UNIT_HEADS * (D + PART_STRIDE_EXTRA) + MMA_UNIT_HEADS) * sizeof(float) <= (size_t)NB * TILE_BYTES,
                 "partial fits the ring");
 
@@ -158,11 +157,41 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
   if (!early && lane == 0) {
     for (int u = 0; u < min(NB, n_ops); ++u) issue(u);
   }
-  int patch_row = -1;
-  if (early) {
-    const int ls = __ldcg(p.last_slot + b);
-    if (ls >= row_begin && ls < row_begin + rows) patch_row = ls - row_begin;
+  // Every global load of the prologue is issued before the first one is used:
+  // the row that may have changed, q^T (the B operand of S^T = K . q^T) and, for
+  // chunk 0's warp, the new token's key and the q rows in the layout of its dot products.
+  const T* qbase = static_cast<const T*>(p.q) + ((size_t)b * p.H + (size_t)kvh * p.G + g_begin) * D;
+  const size_t bh0 = (size_t)b * p.H + (size_t)kvh * p.G + g_begin;
+  const int ls = early ? __ldcg(p.last_slot + b) : -1;
+  // q^T: column n of the MMA tile is head n (heads beyond the group are zero), 16 of the D values per k-step.
+  // qb[ks][2*nh + {0,1}]: head-tile nh (heads 8nh..8nh+7), d = 16ks + qcol (+8)
+  uint32_t qb[KS][2 * R];
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) {
+    const int d = ks * 16 + qcol;
+#pragma unroll
+    for (int nh = 0; nh < R; ++nh) {
+      const int head = qrow + 8 * nh;
+      const uint32_t* r = reinterpret_cast<const uint32_t*>(qbase + (size_t)head * D + d);
+      qb[ks][2 * nh] = (head < g_cnt) ? r[0] : 0u;
+      qb[ks][2 * nh + 1] = (head < g_cnt) ? r[4] : 0u;   // d + 8
+    }
   }
+  constexpr int HPP = 32 / LPR;                       // heads per pass of the new token's dot products
+  constexpr int NPASS = (TWO ? 16 : 8) / HPP;
+  const int lig = lane % LPR, hsub = lane / LPR;
+  uint4 knw = make_uint4(0u, 0u, 0u, 0u), qw[NPASS];
+  if (c == 0) {
+    knw = *reinterpret_cast<const uint4*>(static_cast<const T*>(p.k_new) + ((size_t)b * p.Hkv + kvh) * D + lig * EPL);
+#pragma unroll
+    for (int ps = 0; ps < NPASS; ++ps) {
+      const int g = ps * HPP + hsub;
+      qw[ps] = *reinterpret_cast<const uint4*>(qbase + (size_t)min(g, g_cnt - 1) * D + lig * EPL);
+    }
+  }
+
+  int patch_row = -1;
+  if (ls >= row_begin && ls < row_begin + rows) patch_row = ls - row_begin;
   const unsigned char* k_rows = static_cast<const unsigned char*>(p.K) + (size_t)y0 * RB;
   const unsigned char* v_rows = static_cast<const unsigned char*>(p.V) + (size_t)y0 * RB;
   // Re-fetches row patch_row of operand tile u (already landed) into the swizzled tile.
@@ -176,29 +205,27 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
     }
   };
 
-  const T* qbase = static_cast<const T*>(p.q) + ((size_t)b * p.H + (size_t)kvh * p.G + g_begin) * D;
-  const size_t bh0 = (size_t)b * p.H + (size_t)kvh * p.G + g_begin;
-
-  // The new token (candidate n): its logit per head, on the plain ALUs.
-  float s_new = 0.f;           // lane g keeps head g's logit (fuse_out)
+  // The new token (candidate n): its logit per head, on the plain ALUs, HPP heads per pass.
   if (c == 0) {
-    const int lig = lane % LPR;
-    const T* kn = static_cast<const T*>(p.k_new) + ((size_t)b * p.Hkv + kvh) * D;
     float kf[EPL];
-    Vec16<T>::unpack(*reinterpret_cast<const uint4*>(kn + lig * EPL), kf);
-    for (int g = 0; g < g_cnt; ++g) {
-      float qf[EPL];
-      Vec16<T>::unpack(*reinterpret_cast<const uint4*>(qbase + (size_t)g * D + lig * EPL), qf);
-      float s = 0.f;
+    Vec16<T>::unpack(knw, kf);
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) s = fmaf(qf[e], kf[e], s);
+    for (int ps = 0; ps < NPASS; ++ps) {
+      if (ps * HPP < g_cnt) {
+        const int g = ps * HPP + hsub;
+        float qf[EPL];
+        Vec16<T>::unpack(qw[ps], qf);
+        float s = 0.f;
 #pragma unroll
-      for (int o = LPR / 2; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-      s *= p.scale2;
-      if (lane == g) s_new = s;
-      if (lane == 0) {
-        p.logits[(bh0 + g) * p.ld + p.n] = s;
-        if (!FUSED) p.part_ml[(bh0 + g) * p.pc + p.n_chunks] = make_float2(s, 1.f);
+        for (int e = 0; e < EPL; ++e) s = fmaf(qf[e], kf[e], s);
+#pragma unroll
+        for (int o = LPR / 2; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        s *= p.scale2;
+        if (lig == 0 && g < g_cnt) {
+          p.logits[(bh0 + g) * p.ld + p.n] = s;
+          if (FUSED) snew_s[g] = s;
+          else p.part_ml[(bh0 + g) * p.pc + p.n_chunks] = make_float2(s, 1.f);
+        }
       }
     }
     if (FUSED && p.k_stage && hg == 0 && lane < LPR) {  // copies for a deferred eviction
@@ -210,27 +237,10 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
   if (ntiles == 0) {
     if (FUSED) {
       empty_partial<D>(part, MMA_UNIT_HEADS, lane);
-      if (lane < MMA_UNIT_HEADS) snew[lane] = s_new;
-      fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew0,
+      fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew_s,
                         cpart, bh0, g_cnt);
     }
     return;
-  }
-
-  // q^T as the B operand of S^T = K . q^T: column n of the MMA tile is head n
-  // (heads beyond the group are zero), 16 of the D values per k-step.
-  // qb[ks][2*nh + {0,1}]: head-tile nh (heads 8nh..8nh+7), d = 16ks + qcol (+8)
-  uint32_t qb[KS][2 * R];
-#pragma unroll
-  for (int ks = 0; ks < KS; ++ks) {
-    const int d = ks * 16 + qcol;
-#pragma unroll
-    for (int nh = 0; nh < R; ++nh) {
-      const int head = qrow + 8 * nh;
-      const uint32_t* r = reinterpret_cast<const uint32_t*>(qbase + (size_t)head * D + d);
-      qb[ks][2 * nh] = (head < g_cnt) ? r[0] : 0u;
-      qb[ks][2 * nh + 1] = (head < g_cnt) ? r[4] : 0u;   // d + 8
-    }
   }
 
   // O^T[D, heads]: accumulator tile (nh, mt) covers d = 16mt..16mt+15 of heads 8nh..8nh+7;
@@ -357,8 +367,7 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
     if (lane == 0) atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
     if (FUSED) {           // the other warps wait at the CTA barrier: join them with an empty partial
       empty_partial<D>(part, MMA_UNIT_HEADS, lane);
-      if (lane < MMA_UNIT_HEADS) snew[lane] = s_new;
-      fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew0,
+      fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew_s,
                         cpart, bh0, g_cnt);
     }
     return;
@@ -366,7 +375,6 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
 
   // ---- chunk partial: (max, sum) and the un-normalised weighted V sums ------------------
   __syncwarp();                 // fuse_out: the partial goes where the tiles were
-  if (FUSED && lane < MMA_UNIT_HEADS) snew[lane] = s_new;
 #pragma unroll
   for (int nh = 0; nh < R; ++nh)
 #pragma unroll
@@ -394,7 +402,7 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
         }
       }
     }
-  if (FUSED) fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew0,
+  if (FUSED) fused_merge<T, D>(p, static_cast<const T*>(p.v_new) + ((size_t)b * p.Hkv + kvh) * D, part0, WARP_SMEM / 4, snew_s,
                         cpart, bh0, g_cnt);
 }
 
