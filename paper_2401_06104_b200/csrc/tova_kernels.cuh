@@ -99,6 +99,22 @@ __device__ __forceinline__ void empty_partial(float* part, int heads, int lane) 
     part[i] = (i % (D + PART_STRIDE_EXTRA) == D) ? -INFINITY : 0.f;
 }
 
+// Four consecutive elements of the new token's value row, as floats.
+template <typename T>
+__device__ __forceinline__ float4 load_quad(const T* src) {
+  return make_float4((float)src[0], (float)src[1], (float)src[2], (float)src[3]);
+}
+template <>
+__device__ __forceinline__ float4 load_quad<float>(const float* src) {
+  return *reinterpret_cast<const float4*>(src);
+}
+template <>
+__device__ __forceinline__ float4 load_quad<__nv_bfloat16>(const __nv_bfloat16* src) {
+  const uint2 w = *reinterpret_cast<const uint2*>(src);   // 8-byte aligned: the quad starts at a multiple of 4 elements
+  return make_float4(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u), __uint_as_float(w.y << 16),
+                     __uint_as_float(w.y & 0xffff0000u));
+}
+
 // part0 / snew: warp 0's partial and new-token logits; warp w's partial lies
 // warp_stride floats further per warp.  Called by every warp of the CTA.
 template <typename T, int D>
@@ -108,10 +124,14 @@ __device__ __noinline__ void block_merge_outputs(float* out, float2* head_ml, co
   constexpr int NW = SPLIT_MERGE_MAX_WARPS;
   const int nw = (int)blockDim.y;
   const int tid = (int)(threadIdx.y * 32 + threadIdx.x);
-  __syncthreads();                             // every warp's partial is in shared memory
   const int items = g_cnt * (D / 4);           // output quads of the group
+  // the new token's value for this thread's first quad: on its way before the barrier
+  float4 vq = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (tid < items) vq = load_quad<T>(v_new_row + (tid % (D / 4)) * 4);
+  __syncthreads();                             // every warp's partial is in shared memory
   for (int it = tid; it < items; it += nw * 32) {
     const int g = it / (D / 4), d4 = it % (D / 4);
+    if (it != tid) vq = load_quad<T>(v_new_row + d4 * 4);
     const float s_new = snew[g];
     float mr[NW], lr[NW];
     float M = s_new;
@@ -136,10 +156,9 @@ __device__ __noinline__ void block_merge_outputs(float* out, float2* head_ml, co
     }
     const float wn = exp2f(s_new - M);
     L += wn;
-    const T* vn = v_new_row + d4 * 4;
     const float iL = 1.f / L;
-    o.x = fmaf((float)vn[0], wn, o.x) * iL; o.y = fmaf((float)vn[1], wn, o.y) * iL;
-    o.z = fmaf((float)vn[2], wn, o.z) * iL; o.w = fmaf((float)vn[3], wn, o.w) * iL;
+    o.x = fmaf(vq.x, wn, o.x) * iL; o.y = fmaf(vq.y, wn, o.y) * iL;
+    o.z = fmaf(vq.z, wn, o.z) * iL; o.w = fmaf(vq.w, wn, o.w) * iL;
     reinterpret_cast<float4*>(out + (bh0 + g) * D)[d4] = o;
     if (d4 == 0) head_ml[bh0 + g] = make_float2(M, L);
   }
@@ -165,6 +184,10 @@ __device__ __noinline__ void cluster_merge_outputs(float* out, float2* head_ml, 
   const int tid = (int)(threadIdx.y * 32 + threadIdx.x);
   const int ncta = (int)cl.num_blocks(), rank = (int)cl.block_rank();
   const int items = g_cnt * (D / 4);           // output quads of the group
+  // the new token's value for this thread's first quad of the second stage: on its way before the barriers
+  const int it0 = rank * nthreads + tid;
+  float4 vq = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (it0 < items) vq = load_quad<T>(v_new_row + (it0 % (D / 4)) * 4);
   __syncthreads();                             // every warp's partial is in shared memory
   for (int it = tid; it < items; it += nthreads) {
     const int g = it / (D / 4), d4 = it % (D / 4);
@@ -200,8 +223,9 @@ __device__ __noinline__ void cluster_merge_outputs(float* out, float2* head_ml, 
 #pragma unroll
   for (int r = 0; r < COMBINE_CLUSTER_MAX; ++r) rp[r] = cl.map_shared_rank(cpart, r < ncta ? r : 0);
   const float* rs = cl.map_shared_rank(snew0, 0);
-  for (int it = rank * nthreads + tid; it < items; it += ncta * nthreads) {
+  for (int it = it0; it < items; it += ncta * nthreads) {
     const int g = it / (D / 4), d4 = it % (D / 4);
+    if (it != it0) vq = load_quad<T>(v_new_row + d4 * 4);
     const float s_new = rs[g];
     float mr[COMBINE_CLUSTER_MAX], lr[COMBINE_CLUSTER_MAX];
     float M = s_new;
@@ -226,10 +250,9 @@ __device__ __noinline__ void cluster_merge_outputs(float* out, float2* head_ml, 
     }
     const float wn = exp2f(s_new - M);
     L += wn;
-    const T* vn = v_new_row + d4 * 4;
     const float iL = 1.f / L;
-    o.x = fmaf((float)vn[0], wn, o.x) * iL; o.y = fmaf((float)vn[1], wn, o.y) * iL;
-    o.z = fmaf((float)vn[2], wn, o.z) * iL; o.w = fmaf((float)vn[3], wn, o.w) * iL;
+    o.x = fmaf(vq.x, wn, o.x) * iL; o.y = fmaf(vq.y, wn, o.y) * iL;
+    o.z = fmaf(vq.z, wn, o.z) * iL; o.w = fmaf(vq.w, wn, o.w) * iL;
     reinterpret_cast<float4*>(out + (bh0 + g) * D)[d4] = o;
     if (d4 == 0) head_ml[bh0 + g] = make_float2(M, L);
   }
