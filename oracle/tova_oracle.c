@@ -28,6 +28,16 @@
  *   - the state is kept in place: the new token takes the victim's row, so
  *     row order is not position order; positions travel with the rows.
  *
+ * Other compression policies of the paper, selectable per call (Section 4.1
+ * and the ablation in the appendix, Table "lm_ablation"):
+ *   - Window: first in, first out - when the state is over capacity the row
+ *     holding the earliest position is deleted; the attention weights play no
+ *     part;
+ *   - "+i" (Window+i, TOVA+i): rows holding the first i positions (0..i-1) are
+ *     never deleted; the policy picks among the others.
+ * The layer output does not depend on the policy (it is computed before the
+ * deletion).
+ *
  * Precision: every operation is carried out in REAL (float for the parity
  * checker, double for the reference the float build is itself checked with).
  * Sums run in ascending index order; the soft-max divides (no reciprocal).
@@ -36,7 +46,10 @@
  * on tiny states, library causal attention when k >= stream length, the
  * size invariant len_t = min(t, k), a hand-worked 3-row example in exact
  * rational arithmetic, an order-preserving restatement of Algorithm 1, and
- * permutation / shift invariances.
+ * permutation / shift invariances.  Window and "+i": the closed form of the
+ * retained positions (the first i and the most recent k-i), hand-worked
+ * traces of the 3-row example, "+0" equal to the plain policy, and the
+ * invariant that a protected position is never reported as dropped.
  */
 #include <math.h>
 #include <stdlib.h>
@@ -65,11 +78,17 @@ static REAL real_exp(REAL x) { return sizeof(REAL) == 4 ? (REAL)expf((float)x) :
  *   evicted_pos out  position dropped; -1 when nothing was dropped
  *   victim   out     candidate index dropped (cap = the new token), -1 if none
  *   argmin   out     the arg-min itself (differs from victim only when forced), -1 if none
- *   gap      out     mean[dropped] - min(mean) (0 unless forced differs)
+ *   gap      out     mean[dropped] - min(mean) (0 unless forced differs); under the
+ *                    Window policy 0 if the forced row holds the earliest
+ *                    droppable position, else 1; 1e30 if a protected row is forced
+ *   policy, keep_first  which row goes once the state is over capacity (see top)
  *   mean_out out     [cap+1] head-averaged weights, or NULL
  *   work     scratch [H+1][cap+1] REAL (weights per head, then their mean)
  */
-static void step_one(int H, int Hkv, int D, int cap, REAL scale,
+#define POLICY_TOVA 0
+#define POLICY_WINDOW 1
+
+static void step_one(int H, int Hkv, int D, int cap, REAL scale, int policy, int keep_first,
                      int *len, int *pos, REAL *K, REAL *V,
                      const REAL *q, const REAL *k_new, const REAL *v_new,
                      int pos_t, int forced,
@@ -122,22 +141,35 @@ static void step_one(int H, int Hkv, int D, int cap, REAL scale,
         return;
     }
 
-    /* Average the last query's weights over the heads, take the arg-min
-     * (Algorithm 1), lowest index on ties. */
+    /* Average the last query's weights over the heads (Algorithm 1). */
     REAL *mean = work + (size_t)H * ld;
-    int jmin = 0;
     for (int j = 0; j < m; ++j) {
         REAL a = 0;
         for (int h = 0; h < H; ++h) a += work[(size_t)h * ld + j];
         mean[j] = a / (REAL)H;
-        if (mean[j] < mean[jmin]) jmin = j;
     }
     if (mean_out) for (int j = 0; j < m; ++j) mean_out[j] = mean[j];
+    /* The row to delete, among those not holding one of the first keep_first
+     * positions: lowest average (TOVA, Algorithm 1) or earliest position
+     * (Window, Section 4.1); lowest index on ties. */
+    int jmin = -1;
+    for (int j = 0; j < m; ++j) {
+        const int pj = (j < n) ? pos[j] : pos_t;
+        if (pj < keep_first) continue;
+        if (jmin < 0) { jmin = j; continue; }
+        const int pmin = (jmin < n) ? pos[jmin] : pos_t;
+        if (policy == POLICY_WINDOW ? (pj < pmin) : (mean[j] < mean[jmin])) jmin = j;
+    }
+    if (jmin < 0) jmin = n;      /* every row is protected: the new token cannot stay */
     int drop = jmin;
     *argmin = jmin;
     if (forced >= 0 && forced < m) {
         drop = forced;
-        *gap = mean[drop] - mean[jmin];
+        const int pd = (drop < n) ? pos[drop] : pos_t;
+        const int pmin = (jmin < n) ? pos[jmin] : pos_t;
+        if (pd < keep_first && drop != jmin) *gap = (REAL)1e30;
+        else if (policy == POLICY_WINDOW) *gap = (pd == pmin) ? (REAL)0 : (REAL)1;
+        else *gap = mean[drop] - mean[jmin];
     }
 
     /* Delete row `drop` from K and V (Eq. 9): in place, the new token takes
@@ -163,14 +195,15 @@ static void step_one(int H, int Hkv, int D, int cap, REAL scale,
  * mean_out [B][cap+1] or NULL.  Sequences are spread over `nthreads` threads;
  * nothing else is parallel.  Returns 0, or -1 on a bad argument.
  */
-int tova_oracle_step(int B, int H, int Hkv, int D, int cap, REAL scale,
-                     int *len, int *pos, REAL *K, REAL *V,
-                     const REAL *q, const REAL *k_new, const REAL *v_new,
-                     int pos_t, const int *forced,
-                     REAL *out, int *evicted_pos, int *victim, int *argmin, REAL *gap,
-                     REAL *mean_out, int nthreads)
+int tova_oracle_step_policy(int B, int H, int Hkv, int D, int cap, REAL scale, int policy, int keep_first,
+                            int *len, int *pos, REAL *K, REAL *V,
+                            const REAL *q, const REAL *k_new, const REAL *v_new,
+                            int pos_t, const int *forced,
+                            REAL *out, int *evicted_pos, int *victim, int *argmin, REAL *gap,
+                            REAL *mean_out, int nthreads)
 {
     if (B < 1 || H < 1 || Hkv < 1 || D < 1 || cap < 1 || H % Hkv != 0) return -1;
+    if ((policy != POLICY_TOVA && policy != POLICY_WINDOW) || keep_first < 0) return -1;
     const size_t ld = (size_t)cap + 1;
     if (nthreads < 1) nthreads = 1;
     int bad = 0;
@@ -181,7 +214,7 @@ int tova_oracle_step(int B, int H, int Hkv, int D, int cap, REAL scale,
         REAL *work = (REAL *)malloc(sizeof(REAL) * (size_t)(H + 1) * ld);
         if (!work) { bad = 1; continue; }
         if (len[b] < 0 || len[b] > cap) { bad = 1; free(work); continue; }
-        step_one(H, Hkv, D, cap, scale,
+        step_one(H, Hkv, D, cap, scale, policy, keep_first,
                  len + b, pos + (size_t)b * cap,
                  K + (size_t)b * Hkv * cap * D, V + (size_t)b * Hkv * cap * D,
                  q + (size_t)b * H * D, k_new + (size_t)b * Hkv * D, v_new + (size_t)b * Hkv * D,
@@ -191,6 +224,18 @@ int tova_oracle_step(int B, int H, int Hkv, int D, int cap, REAL scale,
         free(work);
     }
     return bad ? -1 : 0;
+}
+
+/* The TOVA policy with no protected positions (the paper's method as is). */
+int tova_oracle_step(int B, int H, int Hkv, int D, int cap, REAL scale,
+                     int *len, int *pos, REAL *K, REAL *V,
+                     const REAL *q, const REAL *k_new, const REAL *v_new,
+                     int pos_t, const int *forced,
+                     REAL *out, int *evicted_pos, int *victim, int *argmin, REAL *gap,
+                     REAL *mean_out, int nthreads)
+{
+    return tova_oracle_step_policy(B, H, Hkv, D, cap, scale, POLICY_TOVA, 0, len, pos, K, V, q, k_new, v_new,
+                                   pos_t, forced, out, evicted_pos, victim, argmin, gap, mean_out, nthreads);
 }
 
 int tova_oracle_real_bytes(void) { return (int)sizeof(REAL); }

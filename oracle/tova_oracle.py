@@ -38,6 +38,7 @@ def _lib(precision: str):
         tag = {"f32": "f32", "f64": "f64"}[precision]
         lib = ctypes.CDLL(os.path.join(_HERE, f"libtova_oracle_{tag}.so"))
         lib.tova_oracle_step.restype = ctypes.c_int
+        lib.tova_oracle_step_policy.restype = ctypes.c_int
         lib.tova_oracle_real_bytes.restype = ctypes.c_int
         lib.tova_oracle_max_threads.restype = ctypes.c_int
         _LIBS[precision] = lib
@@ -61,7 +62,7 @@ class OracleCache:
 
     def __init__(self, batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
                  capacity: int, sm_scale: float = 0.0, precision: str = "f32",
-                 threads: Optional[int] = None):
+                 threads: Optional[int] = None, policy: str = "tova", keep_first: int = 0):
         if n_q_heads % n_kv_heads:
             raise ValueError("n_q_heads must be a multiple of n_kv_heads")
         self.B, self.H, self.Hkv, self.D, self.cap = batch, n_q_heads, n_kv_heads, head_dim, capacity
@@ -72,6 +73,8 @@ class OracleCache:
         self.lib = _lib(precision)
         assert self.lib.tova_oracle_real_bytes() == np.dtype(self.real).itemsize
         self.threads = threads or host_threads()
+        self.policy = {"tova": 0, "window": 1}[policy]   # Section 4 / Section 4.1
+        self.keep_first = int(keep_first)                  # "+i": positions 0..i-1 are never dropped
         self.len = np.zeros(batch, np.int32)
         self.pos = np.full((batch, capacity), -1, np.int32)
         self.K = np.zeros((batch, n_kv_heads, capacity, head_dim), self.real)
@@ -95,9 +98,9 @@ class OracleCache:
         gap = np.zeros(B, self.real)
         mean = np.zeros((B, cap + 1), self.real) if want_mean else None
         f = None if forced is None else np.ascontiguousarray(forced, np.int32)
-        rc = self.lib.tova_oracle_step(
+        rc = self.lib.tova_oracle_step_policy(
             ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D),
-            ctypes.c_int(cap), self.creal(self.scale),
+            ctypes.c_int(cap), self.creal(self.scale), ctypes.c_int(self.policy), ctypes.c_int(self.keep_first),
             _ptr(self.len), _ptr(self.pos), _ptr(self.K), _ptr(self.V),
             _ptr(q), _ptr(k_new), _ptr(v_new), ctypes.c_int(int(pos_t)), _ptr(f),
             _ptr(out), _ptr(ev), _ptr(victim), _ptr(argmin), _ptr(gap), _ptr(mean),

@@ -339,3 +339,119 @@ def test_memory_model_matches_table_1():
     from paper_2401_06104_b200 import workloads as W
     w = W.WORKLOADS["llama2_7b_layer"]
     assert w.step_bytes() == 8 * (per_token // 32) * 512 + 8 * (per_token // 32)
+
+
+# ----------------------------------------------------------------------------
+# 9. the other compression policies: Window, Window+i, TOVA+i (Section 4.1 and
+#    the appendix ablation)
+# ----------------------------------------------------------------------------
+POLICY_GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "hand_worked_3slot_policies.txt")
+
+
+def parse_policy_golden():
+    traces, cur = [], None
+    for line in open(POLICY_GOLDEN):
+        f = line.split()
+        if not f or f[0].startswith("#"):
+            continue
+        if f[0] == "trace":
+            cur = (f[1], int(f[2]), [])
+            traces.append(cur)
+        elif f[0] == "step":
+            cur[2].append((int(f[1]), int(f[2]), [int(x) for x in f[3].split(",")], Fraction(f[4]), Fraction(f[5])))
+    return traces
+
+
+def test_policy_traces_are_consistent_in_exact_arithmetic():
+    """The fixture follows from the definitions in exact rational arithmetic."""
+    toks, _ = parse_golden()
+    cap = 3
+    for policy, keep, steps in parse_policy_golden():
+        rows = []
+        for (t, ev, rows_after, o0, o1) in steps:
+            cand = rows + [t]
+            outs, probs = [], []
+            for h in range(2):
+                a = [Fraction(toks[p][2 * h]) for p in cand]
+                v = [Fraction(toks[p][2 * h + 1]) for p in cand]
+                tot = sum(a)
+                probs.append([x / tot for x in a])
+                outs.append(sum(x / tot * vv for x, vv in zip(a, v)))
+            assert outs == [o0, o1], (policy, keep, t)
+            if len(cand) <= cap:
+                rows = cand
+                assert ev == -1
+            else:
+                free = [i for i in range(len(cand)) if cand[i] >= keep]
+                if policy == "window":
+                    j = min(free, key=lambda i: (cand[i], i))
+                else:
+                    mean = [(probs[0][i] + probs[1][i]) / 2 for i in range(len(cand))]
+                    j = min(free, key=lambda i: (mean[i], i))
+                assert cand[j] == ev, (policy, keep, t)
+                if j < cap:
+                    rows[j] = t
+            assert rows + [-1] * (cap - len(rows)) == rows_after, (policy, keep, t)
+
+
+@pytest.mark.parametrize("precision", ["f32", "f64"])
+def test_checker_reproduces_policy_traces(precision):
+    toks, _ = parse_golden()
+    for policy, keep, steps in parse_policy_golden():
+        c = OracleCache(1, 2, 2, 1, 3, sm_scale=1.0, precision=precision, policy=policy, keep_first=keep)
+        for (t, ev, rows_after, o0, o1) in steps:
+            q = np.ones((1, 2, 1))
+            a0, v0, a1, v1 = toks[t]
+            k = np.array([[[np.log(a0)], [np.log(a1)]]])
+            v = np.array([[[float(v0)], [float(v1)]]])
+            out, evp, victim, argmin, gap, _ = c.step(q, k, v, t)
+            assert evp[0] == ev, (policy, keep, t)
+            assert list(c.pos[0]) == rows_after, (policy, keep, t)
+            tol = 2e-5 if precision == "f32" else 1e-12
+            assert abs(out[0, 0, 0] - float(o0)) < tol and abs(out[0, 1, 0] - float(o1)) < tol
+
+
+@pytest.mark.parametrize("cap,keep,T", [(8, 0, 50), (8, 1, 50), (16, 4, 90), (5, 4, 30)])
+def test_window_policy_closed_form(cap, keep, T):
+    """Window(+i) keeps exactly the first i and the most recent k - i positions,
+    whatever the inputs (Section 4.1); each step drops the earliest of the rest."""
+    H, Hkv, D = 4, 2, 8
+    q, k, v = random_stream(7, T, H, Hkv, D)
+    c = OracleCache(1, H, Hkv, D, cap, precision="f64", policy="window", keep_first=keep)
+    for t in range(T):
+        out, evp, *_ = c.step(q[t][None], k[t][None], v[t][None], t)
+        held = sorted(int(p) for p in c.pos[0] if p >= 0)
+        if t + 1 <= cap:
+            assert held == list(range(t + 1)) and evp[0] == -1
+        else:
+            assert held == list(range(keep)) + list(range(t + 1 - (cap - keep), t + 1))
+            assert evp[0] == t - (cap - keep)
+
+
+def test_plus_zero_is_the_plain_policy_and_protected_rows_stay():
+    H, Hkv, D, cap, T = 4, 2, 16, 6, 80
+    q, k, v = random_stream(11, T, H, Hkv, D, std=1.5)
+    plain = OracleCache(1, H, Hkv, D, cap, precision="f64")
+    plus0 = OracleCache(1, H, Hkv, D, cap, precision="f64", policy="tova", keep_first=0)
+    plus3 = OracleCache(1, H, Hkv, D, cap, precision="f64", policy="tova", keep_first=3)
+    rows3 = []
+    scale = 1.0 / np.sqrt(D)
+    for t in range(T):
+        a = plain.step(q[t][None], k[t][None], v[t][None], t)
+        b = plus0.step(q[t][None], k[t][None], v[t][None], t)
+        assert a[1][0] == b[1][0] and np.array_equal(plain.pos, plus0.pos) and np.array_equal(a[0], b[0])
+        out, evp, victim, argmin, gap, mean = plus3.step(q[t][None], k[t][None], v[t][None], t, want_mean=True)
+        # brute force from the full history: textbook soft-max, mean over heads, arg-min over unprotected rows
+        cand = rows3 + [t]
+        ref_out, probs = attend_over_positions(q, k, v, t, cand, scale, H // Hkv)
+        assert np.abs(out[0] - ref_out).max() < 1e-12
+        if len(cand) <= cap:
+            rows3 = cand
+        else:
+            ref_mean = probs.mean(axis=0)
+            free = [i for i in range(len(cand)) if cand[i] >= 3]
+            j = min(free, key=lambda i: (ref_mean[i], i))
+            assert evp[0] == cand[j] and evp[0] >= 3
+            if j < cap:
+                rows3[j] = t
+        assert {0, 1, 2} <= set(int(p) for p in plus3.pos[0]) or t < 2
