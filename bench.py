@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="independent layer caches to rotate over (0 = auto)")
     ap.add_argument("--chunk-rows", type=int, default=0)
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of CUDA graphs")
+    ap.add_argument("--policy", choices=["tova", "window"], default="tova",
+                    help="which row is dropped once the state is over capacity")
+    ap.add_argument("--keep-first", type=int, default=0, help="the +i of Window+i / TOVA+i")
     ap.add_argument("--no-fused-merge", action="store_true",
                     help="merge the chunk partials through global memory even where a cluster could")
     ap.add_argument("--deferred", action="store_true", help="force deferred eviction on")
@@ -258,6 +261,9 @@ def run_ours(args):
             c.tova_cache_set_chunk_rows(args.chunk_rows)
         if args.no_fused_merge:
             c.tova_cache_set_fused_merge(False)
+        if args.policy != "tova" or args.keep_first:
+            c.tova_cache_set_policy(tova.TOVA_POLICY_WINDOW if args.policy == "window" else tova.TOVA_POLICY_TOVA,
+                                    args.keep_first)
         caches.append(c)
     outs = torch.empty(L, B, H, D, dtype=torch.float32, device=dev)
     evs = torch.empty(L, B, dtype=torch.int32, device=dev)
@@ -387,6 +393,7 @@ def run_ours(args):
         "config": workload_config(w, {
             "layers_rotated": L, "working_set_bytes": L * step_bytes, "l2": "inputs larger than L2" if L * step_bytes > 2 * 126e6 else "working set near or below L2 size",
             "launch": launch_mode, "graph_steps": G, "bytes_per_step": step_bytes,
+            "policy": args.policy + (f"+{args.keep_first}" if args.keep_first else ""),
             "eviction": "deferred to the cache's side stream, overlaps the next layer's step" if deferred
                         else "on the caller's stream",
             "parallelism": "replicas only" if world > 1 else "single GPU"}),

@@ -149,6 +149,24 @@ int tova_cache_join(tova_cache* c, void* cuda_stream);
  * not depend on it beyond floating-point summation order. */
 int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows);
 
+/* Other compression policies of the paper, on the same kernels (only the
+ * choice of the row to drop changes; the attention output never depends on
+ * it):
+ *   policy TOVA_POLICY_TOVA (default)  the row with the lowest head-averaged
+ *          attention weight goes (Section 4, Algorithm 1);
+ *   policy TOVA_POLICY_WINDOW          first in, first out: the row holding the
+ *          earliest position goes (Section 4.1, "Window");
+ *   keep_first = i >= 0                rows holding positions 0..i-1 are never
+ *          dropped: Window+i (Section 4.1) and TOVA+i (appendix ablation).
+ * Allowed only while the state is empty (before the first token) and with
+ * keep_first < capacity, else TOVA_ERR_BAD_SHAPE; an unknown policy gives
+ * TOVA_ERR_UNSUPPORTED.  Positions passed to the step calls must be >= 0 and
+ * distinct for these policies to mean what the paper describes; ties go to the
+ * lowest slot as everywhere.  Not available through tova_decode_step_static. */
+#define TOVA_POLICY_TOVA 0
+#define TOVA_POLICY_WINDOW 1
+int tova_cache_set_policy(tova_cache* c, int32_t policy, int32_t keep_first);
+
 /* Tuning: where the per-chunk partial results of a head are merged into the
  * attention output (Eq. 7 evaluated chunk by chunk).  on (default): when the
  * state splits into at most 8 chunks, the streaming warps of a head group run

@@ -16,6 +16,8 @@ from . import build as _build
 
 TOVA_DTYPE_FP32 = 0
 TOVA_DTYPE_BF16 = 1
+TOVA_POLICY_TOVA = 0
+TOVA_POLICY_WINDOW = 1
 
 
 class TovaError(RuntimeError):
@@ -58,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.tova_cache_read.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.tova_cache_set_chunk_rows.restype = ctypes.c_int
         L.tova_cache_set_chunk_rows.argtypes = [vp, i32]
+        L.tova_cache_set_policy.restype = ctypes.c_int
+        L.tova_cache_set_policy.argtypes = [vp, i32, i32]
         L.tova_cache_set_fused_merge.restype = ctypes.c_int
         L.tova_cache_set_fused_merge.argtypes = [vp, i32]
         L.tova_cache_set_deferred_eviction.restype = ctypes.c_int
@@ -159,6 +163,10 @@ class TovaCache:
 
     def tova_cache_set_chunk_rows(self, rows: int) -> None:
         _check(lib().tova_cache_set_chunk_rows(self._h, int(rows)), "tova_cache_set_chunk_rows")
+
+    def tova_cache_set_policy(self, policy: int, keep_first: int = 0) -> None:
+        """policy: TOVA_POLICY_TOVA (0) or TOVA_POLICY_WINDOW (1); keep_first = i of the "+i" variants."""
+        _check(lib().tova_cache_set_policy(self._h, int(policy), int(keep_first)), "tova_cache_set_policy")
 
     def tova_cache_set_fused_merge(self, on: bool) -> None:
         _check(lib().tova_cache_set_fused_merge(self._h, 1 if on else 0), "tova_cache_set_fused_merge")

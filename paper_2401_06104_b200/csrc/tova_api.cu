@@ -82,6 +82,7 @@ struct tova_cache {
   tova_config cfg;
   CUtensorMap map_k, map_v;  // tiled views of K and V for the tensor-core split kernel
   bool use_mma;
+  int policy, keep_first;  // which row is dropped once the state is over capacity (tova_cache_set_policy)
   bool fuse_merge;      // the split warps of a head group form one CTA and merge the outputs themselves
   // deferred eviction: victim choice and insert run on a side stream, overlapping later work
   bool deferred, pending;
@@ -491,6 +492,8 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
   cudaError_t e;
   const bool defer = c->deferred && allow_defer;
   p.head_ml = reinterpret_cast<float2*>(base + c->lay.head_ml);
+  p.policy = c->policy;
+  p.keep_first = c->keep_first;
   p.fuse_out = (c->fuse_merge && fused_merge_fits(cfg, c->chunk_rows, c->sm_count)) ? 1 : 0;
   p.merge_ctas = p.fuse_out ? (p.n_chunks + tova::SPLIT_MERGE_MAX_WARPS - 1) / tova::SPLIT_MERGE_MAX_WARPS : 1;
   if (p.merge_ctas < 1) p.merge_ctas = 1;
@@ -587,6 +590,8 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   c->elem = cfg->dtype == TOVA_DTYPE_BF16 ? 2 : 4;
   c->row_bytes = c->elem * cfg->head_dim;
   c->fuse_merge = true;
+  c->policy = tova::POLICY_TOVA;
+  c->keep_first = 0;
   c->deferred = false;
   c->pending = false;
   c->side = nullptr;
@@ -631,6 +636,17 @@ int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows) {
   const int chunks = (c->cfg.capacity + rows - 1) / rows;
   if (combine_smem_bound(c->cfg.n_q_heads, chunks + 1) > COMBINE_BASE_LIMIT) return TOVA_ERR_BAD_SHAPE;
   c->chunk_rows = rows;
+  return TOVA_OK;
+}
+
+int tova_cache_set_policy(tova_cache* c, int32_t policy, int32_t keep_first) {
+  if (!c) return TOVA_ERR_NULL;
+  if (policy != TOVA_POLICY_TOVA && policy != TOVA_POLICY_WINDOW) return TOVA_ERR_UNSUPPORTED;
+  // a droppable row must always exist, and Window compares ages that stay below the capacity only if the
+  // state has been under this policy from the start
+  if (keep_first < 0 || keep_first >= c->cfg.capacity || c->len != 0) return TOVA_ERR_BAD_SHAPE;
+  c->policy = policy == TOVA_POLICY_WINDOW ? tova::POLICY_WINDOW : tova::POLICY_TOVA;
+  c->keep_first = keep_first;
   return TOVA_OK;
 }
 

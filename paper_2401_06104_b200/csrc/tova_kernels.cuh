@@ -69,6 +69,9 @@ struct StepParams {
   int32_t do_evict;   // n == cap and the policy is on
   int32_t fuse_out;   // the split kernel's warps of a (sequence, KV head, head group) form a cluster and write
                       // the outputs themselves; the combine kernel then only picks the victim
+  int32_t policy;     // which row goes once the state is over capacity: POLICY_TOVA (lowest head-averaged weight,
+                      // Algorithm 1) or POLICY_WINDOW (earliest position, Section 4.1)
+  int32_t keep_first; // rows holding positions 0..keep_first-1 are never dropped ("+i" variants)
   int32_t merge_ctas; // fuse_out: CTAs (of up to 8 warps = chunks) per head group; > 1: they form a cluster (x)
   int32_t mode;       // combine kernel: 0 whole step, 1 outputs only, 2 victim + insert only
   void* k_stage;      // [B,Hkv,D] mode 1: copies of the new token's rows for a later mode-2 launch
@@ -91,6 +94,7 @@ struct StepParams {
 // Partial of a warp: per head D+4 floats: acc[D], max2, sum, -, -.  Warp 0
 // also holds snew[g], the new token's logit per head.
 constexpr int PART_STRIDE_EXTRA = 4;
+constexpr int POLICY_TOVA = 0, POLICY_WINDOW = 1;
 constexpr int SPLIT_MERGE_MAX_WARPS = 8;
 
 template <int D>
@@ -910,11 +914,20 @@ __global__ void __launch_bounds__(CT, 1024 / CT) tova_combine_kernel(const StepP
       __syncthreads();
     }
     if (hs == 0 && live) {
-      const float v = a;             // the 1/H of the mean is folded into hLc
+      float v = a;                   // the 1/H of the mean is folded into hLc
+      int pj = 0;
+      const bool by_pos = p.policy != POLICY_TOVA || p.keep_first > 0;   // uniform
+      if (by_pos) {                  // the other policies look at the position the candidate holds
+        pj = (j0 == j_begin) ? r_pos : ((j < p.cap) ? p.pos[(size_t)b * p.cap + j] : pos_t);
+        // Window: the earliest position goes.  Ages of droppable rows are below the capacity
+        // (the policy is fixed while the state is empty), so the float is exact.
+        if (p.policy == POLICY_WINDOW) v = (float)(pj - pos_t);
+        if (pj < p.keep_first) v = INFINITY;     // one of the first i token states: never dropped
+      }
       if (v < val) {               // passes go up in j: strict < keeps the lowest index
         val = v;
         idx = j;
-        cpos = (j0 == j_begin) ? r_pos : ((j < p.cap) ? p.pos[(size_t)b * p.cap + j] : pos_t);
+        cpos = by_pos ? pj : ((j0 == j_begin) ? r_pos : ((j < p.cap) ? p.pos[(size_t)b * p.cap + j] : pos_t));
       }
     }
   }

@@ -40,14 +40,19 @@ class ParityReport:
     evicted_log: List[np.ndarray] = field(default_factory=list)
 
 
+POLICIES = {"tova": tova.TOVA_POLICY_TOVA, "window": tova.TOVA_POLICY_WINDOW}
+
+
 def make_cache(w: W.Workload, sm_scale: float = 0.0, evict: bool = True, chunk_rows: int = 0,
-               fused_merge: bool = True):
+               fused_merge: bool = True, policy: str = "tova", keep_first: int = 0):
     c = tova.TovaCache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, dtype=w.dtype,
                        sm_scale=sm_scale, evict=evict)
     if chunk_rows:
         c.tova_cache_set_chunk_rows(chunk_rows)
     if not fused_merge:
         c.tova_cache_set_fused_merge(False)
+    if policy != "tova" or keep_first:
+        c.tova_cache_set_policy(POLICIES[policy], keep_first)
     return c
 
 
@@ -70,7 +75,7 @@ def run_lockstep(w: W.Workload, n_tokens: int, *, seqs: Optional[Sequence[int]] 
                  block: int = 64, use_prefill: bool = True, chunk_rows: int = 0,
                  sm_scale: float = 0.0, layer: int = 0, cache=None, oracle=None,
                  first_pos: int = 0, check_state_every: int = 4, direct_fill: bool = False,
-                 fused_merge: bool = True) -> ParityReport:
+                 fused_merge: bool = True, policy: str = "tova", keep_first: int = 0) -> ParityReport:
     """Feed n_tokens tokens to both sides and compare at every token.
 
     direct_fill: while the state is filling nothing is dropped (Section 3.3), so
@@ -80,9 +85,10 @@ def run_lockstep(w: W.Workload, n_tokens: int, *, seqs: Optional[Sequence[int]] 
     token grows with the state; this keeps capacity-4096 cases affordable)."""
     seqs = list(range(w.batch)) if seqs is None else list(seqs)
     own = cache is None
-    cache = cache or make_cache(w, sm_scale=sm_scale, chunk_rows=chunk_rows, fused_merge=fused_merge)
+    cache = cache or make_cache(w, sm_scale=sm_scale, chunk_rows=chunk_rows, fused_merge=fused_merge,
+                                policy=policy, keep_first=keep_first)
     orc = oracle or OracleCache(len(seqs), w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity,
-                                sm_scale=sm_scale, precision="f32")
+                                sm_scale=sm_scale, precision="f32", policy=policy, keep_first=keep_first)
     tol = out_tol(w)
     rep = ParityReport()
     done = 0

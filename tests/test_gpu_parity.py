@@ -232,3 +232,63 @@ def test_deferred_eviction_gives_identical_results(fused):
         for key in ("len", "positions", "K", "V"):
             assert torch.equal(a[key], b[key]), key
         assert dfr[l].tova_cache_launches() == 1 + (2 if fused else 3) * T
+
+
+# ---------------------------------------------------------------------------
+# other compression policies on the same kernels (Section 4.1, appendix ablation)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("policy,keep", [("window", 0), ("window", 4), ("tova", 1), ("tova", 4)])
+@pytest.mark.parametrize("shape", ["mha", "gqa"])
+def test_policy_variants_against_the_checker(policy, keep, shape):
+    """Window, Window+4, TOVA+1, TOVA+4: dropped positions and slot tables bit-exact,
+    outputs within tolerance; both merge routes (capacity 150: one CTA; chunk 32)."""
+    w = (LLAMA.scaled(batch=2, n_q_heads=6, n_kv_heads=6, capacity=150) if shape == "mha"
+         else MISTRAL.scaled(batch=2, n_q_heads=8, n_kv_heads=2, capacity=150))
+    rep = run_lockstep(w, 150 + 200, block=50, policy=policy, keep_first=keep)
+    assert rep.evictions == 2 * 200
+    held = rep.cache.tova_cache_read()["positions"].numpy()
+    for b in range(2):
+        assert set(range(keep)) <= set(held[b].tolist())
+        if policy == "window":       # closed form: the first i and the most recent k - i positions
+            assert sorted(held[b].tolist()) == list(range(keep)) + list(range(350 - (150 - keep), 350))
+    rep = run_lockstep(w, 150 + 60, block=50, policy=policy, keep_first=keep, fused_merge=False, chunk_rows=32)
+    assert rep.evictions == 2 * 60
+
+
+def test_policy_hand_worked_traces_on_gpu():
+    from test_oracle_pins import parse_policy_golden
+    toks, _ = parse_golden()
+    D = 64
+    for policy, keep, steps in parse_policy_golden():
+        c = tova.TovaCache(1, 2, 2, D, 3, dtype=tova.TOVA_DTYPE_FP32, sm_scale=1.0)
+        c.tova_cache_set_policy({"tova": 0, "window": 1}[policy], keep)
+        out = torch.empty(1, 2, D, device="cuda:0")
+        ev = torch.empty(1, dtype=torch.int32, device="cuda:0")
+        for (t, e, rows_after, o0, o1) in steps:
+            q = np.zeros((1, 2, D), np.float32); q[..., 0] = 1.0
+            k = np.zeros((1, 2, D), np.float32); v = np.zeros((1, 2, D), np.float32)
+            a0, v0, a1, v1 = toks[t]
+            k[0, 0, 0], k[0, 1, 0] = np.log(a0), np.log(a1)
+            v[0, 0, 0], v[0, 1, 0] = v0, v1
+            c.tova_decode_step(*(tova.to_device(a, 0) for a in (q, k, v)), t, out, ev)
+            st = c.tova_cache_read()
+            assert int(ev.item()) == e, (policy, keep, t)
+            assert st["positions"][0].tolist() == rows_after, (policy, keep, t)
+            o = out.cpu().numpy()
+            assert abs(o[0, 0, 0] - float(o0)) < 1e-4 and abs(o[0, 1, 0] - float(o1)) < 1e-4
+
+
+def test_policy_argument_errors():
+    w = LLAMA.scaled(batch=1, n_q_heads=2, n_kv_heads=2, capacity=8)
+    c = make_cache(w)
+    with pytest.raises(tova.TovaError) as e:
+        c.tova_cache_set_policy(7, 0)
+    assert e.value.code == -3
+    for bad in (-1, 8):
+        with pytest.raises(tova.TovaError):
+            c.tova_cache_set_policy(tova.TOVA_POLICY_WINDOW, bad)
+    c.tova_cache_set_policy(tova.TOVA_POLICY_WINDOW, 7)
+    q = torch.zeros(1, 2, 128, dtype=torch.bfloat16, device="cuda:0")
+    c.tova_decode_step(q, q, q, 0, torch.zeros(1, 2, 128, device="cuda:0"))
+    with pytest.raises(tova.TovaError):            # the state is no longer empty
+        c.tova_cache_set_policy(tova.TOVA_POLICY_TOVA, 0)
