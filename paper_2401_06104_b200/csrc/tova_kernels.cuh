@@ -4,13 +4,19 @@
 //                     head, chunk of rows) through a private shared-memory ring
 //                     fed by bulk asynchronous copies, computes the logits of
 //                     the query heads that share the KV head (Eq. 4), keeps an
-//                     online soft-max (max, sum, weighted V sum) per head and
-//                     writes it as the chunk's partial (Eq. 7); every logit is
-//                     kept in an fp32 scratch.
-//   combine kernel  : merges the partials into the attention output, forms the
-//                     head-averaged weights from the kept logits, takes the
-//                     arg-min and overwrites the victim's row with the new
-//                     token (Section 4, Eq. 9, Algorithm 1).
+//                     online soft-max (max, sum, weighted V sum) per head: the
+//                     chunk's partial (Eq. 7); every logit is kept in an fp32
+//                     scratch.  When the state splits into few chunks, the
+//                     warps of a head group run as one CTA (or a cluster of
+//                     CTAs), merge their partials in shared memory and write
+//                     the attention output themselves; otherwise each warp is
+//                     its own CTA and the partials go through global memory.
+//   combine kernel  : merges the partials into the attention output where the
+//                     split kernel has not, forms the head-averaged weights
+//                     from the kept logits, takes the arg-min and overwrites
+//                     the victim's row with the new token (Section 4, Eq. 9,
+//                     Algorithm 1).  The Window and "+i" policies of Section
+//                     4.1 differ only in the score a candidate gets there.
 //
 // Logits are kept in the base-2 domain: s2 = sm_scale * log2(e) * (q . k), so
 // weights are exp2(s2 - max2).
