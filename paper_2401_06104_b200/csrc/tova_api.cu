@@ -398,7 +398,7 @@ int pick_chunk_rows(const tova_config& cfg, int sm_count) {
   long long per_sm = (long long)(227 * 1024) / (long long)smem;
   // registers bound the resident warps too (figures from ptxas for these kernels)
   const int G0 = cfg.n_q_heads / cfg.n_kv_heads;
-  const long long by_regs = wants_mma(cfg) ? (G0 > 8 ? 12 : 16) : (G0 <= 1 ? 28 : G0 == 2 ? 16 : G0 <= 4 ? 12 : 8);
+  const long long by_regs = wants_mma(cfg) ? (G0 > 8 ? 12 : 21) : (G0 <= 1 ? 25 : G0 == 2 ? 16 : G0 <= 4 ? 12 : 8);
   if (per_sm > by_regs) per_sm = by_regs;
   if (per_sm > 32) per_sm = 32;
   if (per_sm < 1) per_sm = 1;
