@@ -106,10 +106,12 @@ int tova_decode_step(tova_cache* c, const void* q, const void* k, const void* v,
 int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int32_t n_tokens,
                  int32_t first_pos, float* out, int32_t* evicted_pos, void* cuda_stream);
 
-/* tova_decode_step with HOST buffers: q, k, v are copied to the device, the
- * step runs, out (and evicted_pos if not NULL) are copied back, all on
- * `cuda_stream`; returns after the stream has been synchronised.  Pinned host
- * memory makes the copies asynchronous, pageable memory works too. */
+/* tova_decode_step with HOST buffers; returns after `cuda_stream` has been
+ * synchronised, when out (and evicted_pos if not NULL) hold the results.
+ * Page-locked buffers (pinned or registered, 16-byte aligned; all of them) are
+ * read and written in place by the kernels, over the bus: no staging copies.
+ * Otherwise (pageable memory) q, k, v are copied to the device, the step runs
+ * and the results are copied back, all on `cuda_stream`. */
 int tova_decode_step_host(tova_cache* c, const void* q_host, const void* k_host,
                           const void* v_host, int32_t pos, float* out_host,
                           int32_t* evicted_pos_host, void* cuda_stream);

@@ -687,10 +687,39 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
   return TOVA_OK;
 }
 
+namespace {
+// The address under which the GPU can read or write a host buffer in place:
+// page-locked (pinned or registered) memory only; null for pageable memory.
+void* device_view_of_host(const void* host) {
+  cudaPointerAttributes a{};
+  if (cudaPointerGetAttributes(&a, host) != cudaSuccess) {
+    (void)cudaGetLastError();   // older runtimes report pageable memory as an error: clear it
+    return nullptr;
+  }
+  if (a.type != cudaMemoryTypeHost || !a.devicePointer || !aligned16(a.devicePointer)) return nullptr;
+  return a.devicePointer;
+}
+}  // namespace
+
 int tova_decode_step_host(tova_cache* c, const void* q_host, const void* k_host, const void* v_host,
                           int32_t pos, float* out_host, int32_t* evicted_pos_host, void* cuda_stream) {
   if (!c || !q_host || !k_host || !v_host || !out_host) return TOVA_ERR_NULL;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // Page-locked buffers: the kernels read q, k, v and write the outputs in place
+  // over the bus; five small copies per step would cost more than the step.
+  {
+    void* dq = device_view_of_host(q_host);
+    void* dk = device_view_of_host(k_host);
+    void* dv = device_view_of_host(v_host);
+    void* dout = device_view_of_host(out_host);
+    void* dev_ev = evicted_pos_host ? device_view_of_host(evicted_pos_host) : nullptr;
+    if (dq && dk && dv && dout && (dev_ev || !evicted_pos_host)) {
+      int rc = step_impl(c, dq, dk, dv, pos, static_cast<float*>(dout), static_cast<int32_t*>(dev_ev), st,
+                         /*allow_defer=*/false);
+      if (rc != TOVA_OK) return rc;
+      return cudaStreamSynchronize(st) == cudaSuccess ? TOVA_OK : TOVA_ERR_CUDA;
+    }
+  }
   const size_t B = c->cfg.batch, H = c->cfg.n_q_heads, Hkv = c->cfg.n_kv_heads, D = c->cfg.head_dim;
   const size_t qb = B * H * D * c->elem, kb = B * Hkv * D * c->elem, ob = B * H * D * sizeof(float);
   unsigned char* base = c->base;

@@ -166,16 +166,20 @@ def test_unbounded_arm_matches_checker_and_reports_full():
     assert e.value.code == -6
 
 
-def test_host_buffer_entry_point_matches_device_path():
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_buffer_entry_point_matches_device_path(pinned):
+    """Page-locked buffers are read and written in place by the kernels, pageable
+    ones go through staging copies: the same results either way."""
     w = LLAMA.scaled(batch=2, n_q_heads=4, n_kv_heads=4, capacity=40)
     T = 90
     q, k, v = W.tokens(w, 0, T)
     dev = make_cache(w)
     o_dev, e_dev = gpu_block(dev, w, q, k, v, 0)
     host = make_cache(w)
-    hq, hk, hv = (torch.from_numpy(a).to(torch.bfloat16).pin_memory() for a in (q, k, v))
-    out = torch.empty(w.batch, w.n_q_heads, w.head_dim, dtype=torch.float32).pin_memory()
-    ev = torch.empty(w.batch, dtype=torch.int32).pin_memory()
+    pin = (lambda x: x.pin_memory()) if pinned else (lambda x: x)
+    hq, hk, hv = (pin(torch.from_numpy(a).to(torch.bfloat16)) for a in (q, k, v))
+    out = pin(torch.empty(w.batch, w.n_q_heads, w.head_dim, dtype=torch.float32))
+    ev = pin(torch.empty(w.batch, dtype=torch.int32))
     for t in range(T):
         host.tova_decode_step_host(hq[t], hk[t], hv[t], t, out, ev)
         assert np.array_equal(out.numpy(), o_dev[t]) and np.array_equal(ev.numpy(), e_dev[t])
