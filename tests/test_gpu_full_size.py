@@ -38,3 +38,79 @@ def test_full_layer_shapes(name, cap, extra, seqs, direct_fill):
     check_all_sequences(rep, w, n)
     print(f"{name} k={cap}: max_err {rep.max_err:.2e} resyncs {rep.resyncs}/{rep.evictions} "
           f"self {rep.self_evictions}")
+
+
+@pytest.mark.parametrize("name,cap", [("llama2_7b_layer", 512), ("mistral_7b_gqa", 1024), ("yi_6b_long", 4096)])
+def test_full_shapes_as_the_benchmark_launches_them(name, cap):
+    """Deferred eviction, two layer caches taking turns, steps replayed from a CUDA
+    graph with positions from the device counter: bit-identical outputs, dropped
+    positions and state to plain stream-ordered steps (which the test above holds
+    against the checker)."""
+    import torch
+    import paper_2401_06104_b200 as tova
+    w = W.WORKLOADS[name].scaled(capacity=cap)
+    L, G, R = 2, 8, 3                      # caches, steps per graph, replays
+    n_fill = cap + 8
+    toks = [W.tokens(w, 0, n_fill + G * R, layer=l) for l in range(L)]
+    dev = [[tova.to_device(a, w.dtype) for a in t] for t in toks]
+    ref = [make_cache(w) for _ in range(L)]
+    dfr = [make_cache(w) for _ in range(L)]
+    for l in range(L):
+        for c in (ref[l], dfr[l]):
+            c.tova_prefill(dev[l][0], dev[l][1], dev[l][2], n_fill, 0, None, None)
+    shape = (G * R, w.batch, w.n_q_heads, w.head_dim)
+    o_ref = [torch.empty(shape, device="cuda:0") for _ in range(L)]
+    e_ref = [torch.full((G * R, w.batch), -7, dtype=torch.int32, device="cuda:0") for _ in range(L)]
+    for t in range(G * R):
+        for l in range(L):
+            q, k, v = (a[n_fill + t] for a in dev[l])
+            ref[l].tova_decode_step(q, k, v, n_fill + t, o_ref[l][t], e_ref[l][t])
+    # the benchmark's way: static input/output buffers, one graph of G steps per cache, replayed
+    for c in dfr:
+        c.tova_cache_set_deferred_eviction(True)
+    sq = [[torch.empty_like(a[:G]) for a in dev[l]] for l in range(L)]
+    so = [torch.empty((G,) + shape[1:], device="cuda:0") for _ in range(L)]
+    se = [torch.full((G, w.batch), -7, dtype=torch.int32, device="cuda:0") for _ in range(L)]
+    o_dfr = [torch.empty(shape, device="cuda:0") for _ in range(L)]
+    e_dfr = [torch.empty((G * R, w.batch), dtype=torch.int32, device="cuda:0") for _ in range(L)]
+
+    def steps():
+        for t in range(G):
+            for l in range(L):
+                dfr[l].tova_decode_step(sq[l][0][t], sq[l][1][t], sq[l][2][t], -1, so[l][t], se[l][t])
+        for c in dfr:
+            c.tova_cache_join()
+
+    def load(r):
+        for l in range(L):
+            for i in range(3):
+                sq[l][i].copy_(dev[l][i][n_fill + r * G: n_fill + (r + 1) * G])
+
+    side = torch.cuda.Stream()
+    load(0)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        steps()                              # replay 0 runs directly (sets function attributes before capture)
+        side.synchronize()
+        for l in range(L):
+            o_dfr[l][:G].copy_(so[l]); e_dfr[l][:G].copy_(se[l])
+        load(1)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            steps()
+    for r in range(1, R):
+        if r > 1:
+            load(r)
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        for l in range(L):
+            o_dfr[l][r * G:(r + 1) * G].copy_(so[l]); e_dfr[l][r * G:(r + 1) * G].copy_(se[l])
+    torch.cuda.synchronize()
+    for l in range(L):
+        assert torch.equal(e_ref[l], e_dfr[l]), f"{name} layer {l}: dropped positions differ"
+        assert torch.equal(o_ref[l], o_dfr[l]), f"{name} layer {l}: outputs differ"
+        a, b = ref[l].tova_cache_read(), dfr[l].tova_cache_read()
+        assert a["status"] == 0 and b["status"] == 0
+        assert torch.equal(a["positions"], b["positions"]) and torch.equal(a["len"], b["len"])
