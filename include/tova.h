@@ -108,8 +108,10 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
 
 /* tova_decode_step with HOST buffers; returns after `cuda_stream` has been
  * synchronised, when out (and evicted_pos if not NULL) hold the results.
- * Page-locked buffers (pinned or registered, 16-byte aligned; all of them) are
- * read and written in place by the kernels, over the bus: no staging copies.
+ * Page-locked buffers (pinned or registered, 16-byte aligned; all of them):
+ * the kernels read q, k, v over the bus (directly, or through one small fetch
+ * kernel when many warps share them) and write the outputs in place - no
+ * copy calls.
  * Otherwise (pageable memory) q, k, v are copied to the device, the step runs
  * and the results are copied back, all on `cuda_stream`. */
 int tova_decode_step_host(tova_cache* c, const void* q_host, const void* k_host,

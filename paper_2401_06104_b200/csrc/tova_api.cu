@@ -705,8 +705,7 @@ int tova_decode_step_host(tova_cache* c, const void* q_host, const void* k_host,
                           int32_t pos, float* out_host, int32_t* evicted_pos_host, void* cuda_stream) {
   if (!c || !q_host || !k_host || !v_host || !out_host) return TOVA_ERR_NULL;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  // Page-locked buffers: the kernels read q, k, v and write the outputs in place
-  // over the bus; five small copies per step would cost more than the step.
+  // Page-locked buffers: no copy calls; five small copies per step would cost more than the step.
   {
     void* dq = device_view_of_host(q_host);
     void* dk = device_view_of_host(k_host);
@@ -714,7 +713,26 @@ int tova_decode_step_host(tova_cache* c, const void* q_host, const void* k_host,
     void* dout = device_view_of_host(out_host);
     void* dev_ev = evicted_pos_host ? device_view_of_host(evicted_pos_host) : nullptr;
     if (dq && dk && dv && dout && (dev_ev || !evicted_pos_host)) {
-      int rc = step_impl(c, dq, dk, dv, pos, static_cast<float*>(dout), static_cast<int32_t*>(dev_ev), st,
+      const size_t B = c->cfg.batch, H = c->cfg.n_q_heads, Hkv = c->cfg.n_kv_heads, D = c->cfg.head_dim;
+      const int nq = (int)(B * H * D * c->elem / 16), nk = (int)(B * Hkv * D * c->elem / 16);
+      unsigned char* base = c->base;
+      const int threads = 256;
+      int blocks = (nq + 2 * nk + threads - 1) / threads;
+      if (blocks > 4 * c->sm_count) blocks = 4 * c->sm_count;
+      // Every output element is written once, in place.  The inputs are read in place too while few warps
+      // share a head group's q (each reads it over the bus: measured faster up to 8 chunks per group);
+      // beyond that one small kernel brings q, k, v across once.
+      const void *sq = dq, *sk = dk, *sv = dv;
+      if ((c->cfg.capacity + c->chunk_rows - 1) / c->chunk_rows > tova::SPLIT_MERGE_MAX_WARPS) {
+        tova::tova_fetch_inputs_kernel<<<blocks, threads, 0, st>>>(
+            reinterpret_cast<uint4*>(base + c->lay.st_q), static_cast<const uint4*>(dq), nq,
+            reinterpret_cast<uint4*>(base + c->lay.st_k), static_cast<const uint4*>(dk),
+            reinterpret_cast<uint4*>(base + c->lay.st_v), static_cast<const uint4*>(dv), nk);
+        if (cudaGetLastError() != cudaSuccess) return TOVA_ERR_CUDA;
+        c->launches += 1;
+        sq = base + c->lay.st_q; sk = base + c->lay.st_k; sv = base + c->lay.st_v;
+      }
+      int rc = step_impl(c, sq, sk, sv, pos, static_cast<float*>(dout), static_cast<int32_t*>(dev_ev), st,
                          /*allow_defer=*/false);
       if (rc != TOVA_OK) return rc;
       return cudaStreamSynchronize(st) == cudaSuccess ? TOVA_OK : TOVA_ERR_CUDA;

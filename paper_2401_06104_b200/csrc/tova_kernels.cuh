@@ -992,6 +992,19 @@ __global__ void __launch_bounds__(CT, 1024 / CT) tova_combine_kernel(const StepP
   else if (staged) mbar_wait_bounded(&row_bar, 0);  // the staged copy must land before the CTA leaves
 }
 
+// Host-buffer steps: q, k and v are fetched from page-locked host memory once,
+// with coalesced 16-byte reads, into device staging (the split kernel's warps
+// would each read q over the bus otherwise).
+__global__ void tova_fetch_inputs_kernel(uint4* dq, const uint4* hq, int nq, uint4* dk, const uint4* hk, uint4* dv,
+                                         const uint4* hv, int nk) {
+  const int stride = gridDim.x * blockDim.x;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nq + 2 * nk; i += stride) {
+    if (i < nq) dq[i] = hq[i];
+    else if (i < nq + nk) dk[i - nq] = hk[i - nq];
+    else dv[i - nq - nk] = hv[i - nq - nk];
+  }
+}
+
 // Empty state at init: length 0, positions -1, status 0.
 __global__ void tova_init_kernel(int32_t* pos, int32_t* len, int32_t* last_slot, int32_t* status,
                                  int32_t* cur_pos, int B, int cap) {
