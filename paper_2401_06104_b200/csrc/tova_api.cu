@@ -416,8 +416,8 @@ int pick_chunk_rows(const tova_config& cfg, int sm_count) {
 
 // Whether the split kernel merges the chunk partials itself: always when one CTA
 // of 8 warps covers the state; with up to 8 such CTAs per head group (a
-// cluster) only while all CTAs of the launch are resident at once - beyond
-// that single-warp CTAs, which the hardware hands out one by one, stream better.
+// cluster) only while the launch is a few waves of CTAs at most - beyond that
+// single-warp CTAs, which the hardware hands out one by one, stream better.
 bool fused_merge_fits(const tova_config& cfg, int chunk_rows, int sm_count) {
   const int chunks = (cfg.capacity + chunk_rows - 1) / chunk_rows;
   if (chunks <= tova::SPLIT_MERGE_MAX_WARPS) return true;
@@ -426,7 +426,9 @@ bool fused_merge_fits(const tova_config& cfg, int chunk_rows, int sm_count) {
   const long long hgroups = (G + unit_heads(cfg) - 1) / unit_heads(cfg);
   const long long ctas = (long long)cfg.batch * cfg.n_kv_heads * hgroups *
                          ((chunks + tova::SPLIT_MERGE_MAX_WARPS - 1) / tova::SPLIT_MERGE_MAX_WARPS);
-  return ctas <= 2LL * sm_count;
+  // measured: the tensor-core kernel keeps gaining from the in-kernel merge up to several waves of CTAs
+  // (mistral k=2048/4096 at batch 32: -7 % / -2 % per step), the ALU kernel only within one resident wave
+  return ctas <= (wants_mma(cfg) ? 8LL : 2LL) * sm_count;
 }
 
 // CTA size of a combine launch, and with it whether a CTA's logits are staged
