@@ -409,6 +409,13 @@ int pick_chunk_rows(const tova_config& cfg, int sm_count) {
   int cr = 128;
   if (10 * units(128) < 8 * slots) cr = 64;
   if (cr == 64 && cfg.capacity <= 256 && 10 * units(64) < 8 * slots) cr = 32;  // short states: partials are few anyway
+  // Tensor-core kernel with at least 1.5 head groups per SM: one CTA of 8 warps per group fills the GPU by
+  // itself, so the state is cut into exactly 8 chunks however long (measured at mistral B=32: k=4096 96.1 ->
+  // 90.2 us, k=2048 even; with fewer groups, or on the ALU kernel, shorter chunks in more CTAs win).
+  if (wants_mma(cfg) && 2 * pairs >= 3LL * sm_count) {
+    const int cr8 = (int)(((cfg.capacity + 7) / 8 + 31) / 32 * 32);
+    if (cr8 > cr) cr = cr8;
+  }
   while (cr <= 8192 && combine_smem_bound(cfg.n_q_heads, (int)((cfg.capacity + cr - 1) / cr) + 1) > COMBINE_BASE_LIMIT)
     cr *= 2;
   return cr <= 8192 ? cr : -1;  // -1: no chunk size keeps the combine kernel's shared memory within its limit
