@@ -262,6 +262,15 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
   // ldmatrix lane roles: lane supplies the address of row (lane % 8) of matrix (lane / 8)
   const int lm_r = lane & 7, lm_m = lane >> 3;
   const uint32_t ring_addr = smem_addr(ring);
+  // swz(row, 2i + c) with this lane's row and c, for the four values of i mod 4, worked out once:
+  // the 16-byte column 2(i mod 4) + c is XORed with row mod 8 = lm_r, and 2(i mod 4) has no bit in
+  // common with c, so the lane-dependent part (c ^ lm_r) << 4 splits off.
+  uint32_t k_ofs[4], v_ofs[4];   // K: row lm_r + 8(lm_m & 1), c = lm_m >> 1;  V: row lm_r + 8(lm_m >> 1), c = lm_m & 1
+#pragma unroll
+  for (int a = 0; a < 4; ++a) {
+    k_ofs[a] = (uint32_t)(lm_r + 8 * (lm_m & 1)) * 128u + ((uint32_t)(a * 32) ^ ((uint32_t)(((lm_m >> 1) ^ lm_r) & 7) << 4));
+    v_ofs[a] = (uint32_t)(lm_r + 8 * (lm_m >> 1)) * 128u + ((uint32_t)(a * 32) ^ ((uint32_t)(((lm_m & 1) ^ lm_r) & 7) << 4));
+  }
 
   bool failed = false;
   int t = 0;
@@ -283,7 +292,7 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
     for (int ks = 0; ks < KS; ++ks) {
       // A fragment: (rows 0-7, d0..7) (rows 8-15, d0..7) (rows 0-7, d0+8..15) (rows 8-15, d0+8..15)
       uint32_t ka[4];
-      ldmatrix_x4(ka, kt + swz(lm_r + 8 * (lm_m & 1), ks * 2 + (lm_m >> 1)));
+      ldmatrix_x4(ka, kt + k_ofs[ks & 3] + (uint32_t)(ks >> 2) * (TILE_ROWS * 128));
 #pragma unroll
       for (int nh = 0; nh < R; ++nh) mma_bf16(s[nh], ka, qb[ks][2 * nh], qb[ks][2 * nh + 1]);
     }
@@ -348,7 +357,7 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
       // A fragment of V^T (d rows, tile-row columns), transposing loads:
       // (rows 0-7, d0..7) (rows 0-7, d0+8..15) (rows 8-15, d0..7) (rows 8-15, d0+8..15)
       uint32_t va[4];
-      ldmatrix_x4_trans(va, vt + swz(lm_r + 8 * (lm_m >> 1), mt * 2 + (lm_m & 1)));
+      ldmatrix_x4_trans(va, vt + v_ofs[mt & 3] + (uint32_t)(mt >> 2) * (TILE_ROWS * 128));
 #pragma unroll
       for (int nh = 0; nh < R; ++nh) {
         mma_bf16(o[nh][mt], va, pb_hi[nh][0], pb_hi[nh][1]);
