@@ -510,8 +510,10 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32) tova_
       // l stays a per-lane partial sum (rows this lane owns); it is folded once at the end
       l[g] = fmaf(l[g], corr, owner ? e : 0.f);
       m[g] = m_new;
+      if (corr != 1.f) {             // warp-uniform (the max is a warp reduction): rare after the first tiles
 #pragma unroll
-      for (int k = 0; k < EPL; ++k) acc[g][k] *= corr;
+        for (int k = 0; k < EPL; ++k) acc[g][k] *= corr;
+      }
       if (owner) w_p[g * TILE_ROWS + my_row] = e;
     }
     __syncwarp();

@@ -332,10 +332,12 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
         e4[2 + hh] = exp2_diff(v[2 + hh], m_new);
         l[nh][hh] = fmaf(l[nh][hh], corr, e4[hh] + e4[2 + hh]);   // per-lane partial, folded at the end
         m[nh][hh] = m_new;
+        if (__any_sync(0xffffffffu, corr != 1.f)) {   // the running max moved for some head: rescale (rare after the first tiles)
 #pragma unroll
-        for (int mt = 0; mt < KS; ++mt) {
-          o[nh][mt][hh] *= corr;
-          o[nh][mt][2 + hh] *= corr;
+          for (int mt = 0; mt < KS; ++mt) {
+            o[nh][mt][hh] *= corr;
+            o[nh][mt][2 + hh] *= corr;
+          }
         }
       }
       // weights as two bf16 terms, then from the accumulator layout (row = lane/4, heads
