@@ -339,7 +339,19 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, boo
     pb.k_new = p.k_stage;
     pb.v_new = p.v_stage;
     pb.k_stage = pb.v_stage = nullptr;
-    set_combine_threads(pb, (long long)p.H * p.cand_per_cta / tova::COMBINE_THREADS_TINY <= 40
+    // Off the critical path, but every CTA of this launch that sits on an SM keeps one of the next split
+    // kernel's 8-warp CTAs from becoming resident there: as few CTAs as about 32 logits per thread allow
+    // (measured at mistral k=256, B=32: 256 -> 96 CTAs, 11.2 -> 10.5 us per step).
+    {
+      const long long score_loads = (long long)(p.n + 1) * p.H;
+      int nx = (int)((score_loads + 32LL * tova::COMBINE_THREADS_TINY - 1) / (32LL * tova::COMBINE_THREADS_TINY));
+      if (nx < 1) nx = 1;
+      if (nx < p.nx && p.do_evict) {
+        pb.nx = nx;
+        pb.cand_per_cta = ((p.n + 1 + nx - 1) / nx + 3) / 4 * 4;
+      }
+    }
+    set_combine_threads(pb, (long long)pb.H * pb.cand_per_cta / tova::COMBINE_THREADS_TINY <= 40
                                 ? tova::COMBINE_THREADS_TINY : tova::COMBINE_THREADS_SMALL);
     e = launch_combine<T, D>(c->device, pb, c->side, /*use_pdl=*/false);
     if (e != cudaSuccess) return e;
