@@ -51,6 +51,10 @@ def parse_args():
     ap.add_argument("--deferred", action="store_true", help="force deferred eviction on")
     ap.add_argument("--no-deferred", action="store_true",
                     help="pick the victim on the caller's stream instead of overlapping it with the next layer's step")
+    ap.add_argument("--prefill", type=int, default=0, metavar="T",
+                    help="time tova_prefill of a T-token prompt into an empty state instead of decode steps "
+                         "(-1: as many tokens as the state holds); a step is one whole prompt")
+    ap.add_argument("--no-bulk-prefill", action="store_true", help="with --prefill: every prompt token takes the decode kernels")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
@@ -412,10 +416,78 @@ def run_ours(args):
     return 0
 
 
+def run_prefill(args):
+    """Prompt processing: one tova_prefill call of T tokens into an empty state per step (a fresh cache each
+    step, so inputs and state are cold).  One GPU.  Roofline of the bulk route: the causal-attention kernel,
+    2*B*H*D*F*(F+1) flops for the F tokens that find a free row, against the measured bf16 GEMM rate."""
+    import torch
+    import paper_2401_06104_b200 as tova
+    from paper_2401_06104_b200 import workloads as W
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the prefill path has no CPU fallback")
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    w = pick_workload(args)
+    B, H, Hkv, D, cap = w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity
+    T = cap if args.prefill < 0 else args.prefill
+    steps, warm = min(args.steps, 8), min(max(args.warmup, 3), 3)
+    q, k, v = (tova.to_device(a, w.dtype, dev) for a in W.tokens(w, 0, T))
+    out = torch.empty(T, B, H, D, dtype=torch.float32, device=dev)
+    ev = torch.empty(T, B, dtype=torch.int32, device=dev)
+    caches = []
+    for _ in range(steps + warm):
+        c = tova.TovaCache(B, H, Hkv, D, cap, dtype=w.dtype, device=dev)
+        if args.no_bulk_prefill:
+            c.tova_cache_set_bulk_prefill(False)
+        caches.append(c)
+    torch.cuda.synchronize()
+    for c in caches[:warm]:
+        c.tova_prefill(q, k, v, T, 0, out, ev)
+    sampler = ClockSampler(0)
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for c in caches[warm:]:
+        c.tova_prefill(q, k, v, T, 0, out, ev)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / steps
+    launches = caches[-1].tova_cache_launches() - 1
+    F = min(T, cap)
+    flops = 2.0 * B * H * D * F * (F + 1)
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            peak, kind = float(json.load(fh)["bf16_tflops"]), "measured"
+    except Exception:
+        peak, kind = 1590.0, "fallback"
+    bulk = (not args.no_bulk_prefill) and w.dtype == W.DTYPE_BF16 and F >= 4
+    line = {
+        "metric": "tova_prefill_tokens_per_s_per_layer", "value": B * T / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+        "steps": steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(w, {"prompt_tokens": T, "tokens_into_free_rows": F,
+                                      "route": "bulk fill + per-token steps" if bulk else "per-token steps",
+                                      "l2": "a fresh cache per step; inputs larger than L2" if q.numel() * 2 > 126e6
+                                            else "a fresh cache per step",
+                                      "parallelism": "single GPU"}),
+        "roofline": ({"bound": "tensor", "achieved": flops / (ms * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
+                      "frac": flops / (ms * 1e-3) / 1e12 / peak, "traffic": None, "peak_kind": kind,
+                      "note": "causal-attention flops of the bulk run / whole prefill time; warp-level MMA kernel"}
+                     if bulk and T == F else None),
+        "cpu_baseline": None, "e2e": None, "gpu_launches": launches * steps, "clocks": clocks,
+    }
+    print(json.dumps(line))
+    return 0
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.prefill:
+        return run_prefill(args)
     return run_ours(args)
 
 

@@ -99,10 +99,22 @@ int tova_decode_step(tova_cache* c, const void* q, const void* k, const void* v,
                      float* out, int32_t* evicted_pos, void* cuda_stream);
 
 /* The same per-token policy run over n_tokens consecutive prompt tokens at
- * positions first_pos, first_pos+1, ...: identical results to n_tokens calls
- * of tova_decode_step.
+ * positions first_pos, first_pos+1, ... (first_pos = TOVA_POS_AUTO continues
+ * from the previous token): the state, the dropped positions and every later
+ * step are identical to n_tokens calls of tova_decode_step.
  *   q [T,B,H,D], k and v [T,B,Hkv,D]; out [T,B,H,D] fp32 or NULL;
- *   evicted_pos [T,B] or NULL. */
+ *   evicted_pos [T,B] or NULL.
+ * Tokens that find a free row are never followed by a deletion (the state
+ * holds g(t) = min(t, k) tokens, Section 3.3; Algorithm 1 returns early while
+ * the cache is within its size), so for them Eq. 6-7 are ordinary causal
+ * attention.  On bf16 states a run of at least 4 such tokens is therefore
+ * processed in bulk - one copy of the rows, one tensor-core causal-attention
+ * kernel (skipped when out is NULL), one small commit kernel - instead of
+ * token by token; its outputs equal the per-token ones up to floating-point
+ * summation order (within the library's output tolerance), everything else
+ * bit for bit.  The tokens that remain once the state is full are processed
+ * one at a time.  tova_cache_set_bulk_prefill(c, 0) forces the per-token
+ * route for all of them (then outputs are bit-identical to decode steps). */
 int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int32_t n_tokens,
                  int32_t first_pos, float* out, int32_t* evicted_pos, void* cuda_stream);
 
@@ -180,6 +192,11 @@ int tova_cache_set_policy(tova_cache* c, int32_t policy, int32_t keep_first);
  * route.  Results do not depend on it beyond
  * floating-point summation order.  Returns TOVA_ERR_NULL for a null handle. */
 int tova_cache_set_fused_merge(tova_cache* c, int32_t on);
+
+/* Bulk processing of the prompt tokens that fill free rows (see tova_prefill;
+ * on by default, used on bf16 states).  on = 0: every prompt token takes the
+ * decode kernels.  Returns TOVA_ERR_NULL for a null handle. */
+int tova_cache_set_bulk_prefill(tova_cache* c, int32_t on);
 
 /* Rows each sequence holds now, min(tokens fed, capacity) = g(t) of Section
  * 3.3, tracked on the host (sequences advance in lock step). */

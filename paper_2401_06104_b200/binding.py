@@ -18,6 +18,7 @@ TOVA_DTYPE_FP32 = 0
 TOVA_DTYPE_BF16 = 1
 TOVA_POLICY_TOVA = 0
 TOVA_POLICY_WINDOW = 1
+TOVA_POS_AUTO = -1       # "the previous token's position + 1"
 
 
 class TovaError(RuntimeError):
@@ -64,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.tova_cache_set_policy.argtypes = [vp, i32, i32]
         L.tova_cache_set_fused_merge.restype = ctypes.c_int
         L.tova_cache_set_fused_merge.argtypes = [vp, i32]
+        L.tova_cache_set_bulk_prefill.restype = ctypes.c_int
+        L.tova_cache_set_bulk_prefill.argtypes = [vp, i32]
         L.tova_cache_set_deferred_eviction.restype = ctypes.c_int
         L.tova_cache_set_deferred_eviction.argtypes = [vp, i32]
         L.tova_cache_join.restype = ctypes.c_int
@@ -170,6 +173,9 @@ class TovaCache:
 
     def tova_cache_set_fused_merge(self, on: bool) -> None:
         _check(lib().tova_cache_set_fused_merge(self._h, 1 if on else 0), "tova_cache_set_fused_merge")
+
+    def tova_cache_set_bulk_prefill(self, on: bool) -> None:
+        _check(lib().tova_cache_set_bulk_prefill(self._h, 1 if on else 0), "tova_cache_set_bulk_prefill")
 
     def tova_cache_set_deferred_eviction(self, on: bool) -> None:
         _check(lib().tova_cache_set_deferred_eviction(self._h, 1 if on else 0),

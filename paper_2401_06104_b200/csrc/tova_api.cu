@@ -1,7 +1,8 @@
 // Host side of the C ABI declared in include/tova.h: argument checks, the
 // layout of the caller-provided device block, launch configuration.  Every
-// step of the decode path runs in the kernels of tova_kernels.cuh; there is no
-// CPU fallback.
+// step of the decode path runs in the kernels of tova_kernels.cuh and
+// tova_split_mma.cuh, the bulk fill of a prompt in those of tova_fill.cuh;
+// there is no CPU fallback.
 #include "../../include/tova.h"
 
 #include <cmath>
@@ -13,6 +14,7 @@
 
 #include "tova_kernels.cuh"
 #include "tova_split_mma.cuh"
+#include "tova_fill.cuh"
 
 namespace {
 
@@ -82,6 +84,8 @@ struct tova_cache {
   tova_config cfg;
   CUtensorMap map_k, map_v;  // tiled views of K and V for the tensor-core split kernel
   bool use_mma;
+  CUtensorMap fill_map_k, fill_map_v;  // the same matrices in boxes of 64 rows, for the bulk fill of a prompt
+  bool fill_maps, bulk_fill;
   int policy, keep_first;  // which row is dropped once the state is over capacity (tova_cache_set_policy)
   bool fuse_merge;      // the split warps of a head group form one CTA and merge the outputs themselves
   // deferred eviction: victim choice and insert run on a side stream, overlapping later work
@@ -533,6 +537,70 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
   return TOVA_OK;
 }
 
+// Shortest run of prompt tokens worth the three launches of the bulk fill.
+constexpr int BULK_FILL_MIN_TOKENS = 4;
+
+template <int D>
+cudaError_t launch_fill_d(tova_cache* c, const tova::FillParams& p, cudaStream_t st) {
+  const size_t chunks = (size_t)p.F * p.B * p.Hkv * (D * 2 / 16);
+  unsigned blocks = (unsigned)((chunks + 255) / 256);
+  const unsigned cap_blocks = (unsigned)c->sm_count * 16u;
+  if (blocks > cap_blocks) blocks = cap_blocks;
+  if (blocks < 1) blocks = 1;
+  tova::tova_fill_rows_kernel<D><<<blocks, 256, 0, st>>>(p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  c->launches += 1;
+  if (p.out) {
+    constexpr size_t smem = 5 * (size_t)tova::FILL_K_ROWS * D * 2 + 1024;
+    static bool configured[64] = {};
+    if (c->device >= 0 && c->device < 64 && !configured[c->device]) {
+      e = cudaFuncSetAttribute(tova::tova_fill_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      configured[c->device] = true;
+    }
+    dim3 grid((p.F + tova::FILL_Q_ROWS - 1) / tova::FILL_Q_ROWS, p.H, p.B);
+    tova::tova_fill_attn_kernel<D><<<grid, tova::FILL_THREADS, smem, st>>>(p, c->fill_map_k, c->fill_map_v);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    c->launches += 1;
+  }
+  // A plain launch after the attention: a later split kernel, which starts fetching rows before its own
+  // dependency wait, can then start only once the copies above have completed.
+  tova::tova_fill_commit_kernel<<<(p.B + 127) / 128, 128, 0, st>>>(p);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  c->launches += 1;
+  return cudaSuccess;
+}
+
+// F tokens into free rows of a bf16 state (len + F <= capacity): rows, positions, causal attention.
+int launch_fill(tova_cache* c, const void* q, const void* k, const void* v, int F, int32_t first_pos, float* out,
+                int32_t* evicted_pos, cudaStream_t st) {
+  if (c->pending) {  // a deferred insert of an earlier token must land first
+    if (cudaStreamWaitEvent(st, c->ev_join, 0) != cudaSuccess) return TOVA_ERR_CUDA;
+    c->pending = false;
+  }
+  tova::FillParams p{};
+  unsigned char* base = c->base;
+  p.K = base + c->lay.K;
+  p.V = base + c->lay.V;
+  p.pos = reinterpret_cast<int32_t*>(base + c->lay.pos);
+  p.len = reinterpret_cast<int32_t*>(base + c->lay.len);
+  p.last_slot = reinterpret_cast<int32_t*>(base + c->lay.last_slot);
+  p.cur_pos = reinterpret_cast<int32_t*>(base + c->lay.cur_pos);
+  p.status = reinterpret_cast<int32_t*>(base + c->lay.status);
+  p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.evicted = evicted_pos;
+  p.B = c->cfg.batch; p.H = c->cfg.n_q_heads; p.Hkv = c->cfg.n_kv_heads; p.G = p.H / p.Hkv;
+  p.cap = c->cfg.capacity;
+  p.n0 = c->len;
+  p.F = F;
+  p.first_pos = first_pos;
+  p.scale2 = c->scale2;
+  const cudaError_t e = c->cfg.head_dim == 128 ? launch_fill_d<128>(c, p, st) : launch_fill_d<64>(c, p, st);
+  if (e != cudaSuccess) return TOVA_ERR_CUDA;
+  c->len += F;
+  return TOVA_OK;
+}
+
 int check_step_args(const tova_cache* c, const void* q, const void* k, const void* v, const void* out) {
   if (!c || !q || !k || !v || !out) return TOVA_ERR_NULL;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return TOVA_ERR_ALIGN;
@@ -545,7 +613,7 @@ int check_step_args(const tova_cache* c, const void* q, const void* k, const voi
 // kernel: boxes of 16 rows x 64 columns (128 bytes) with the 128-byte swizzle.
 // The driver's encoder is looked up through the runtime, so the library has no
 // link-time dependency on the driver.
-int encode_state_map(CUtensorMap* map, void* base, const tova_config& cfg) {
+int encode_state_map(CUtensorMap* map, void* base, const tova_config& cfg, int box_rows = tova::TILE_ROWS) {
   typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -561,7 +629,7 @@ int encode_state_map(CUtensorMap* map, void* base, const tova_config& cfg) {
   const cuuint64_t rows = (cuuint64_t)cfg.batch * cfg.n_kv_heads * cfg.capacity;
   const cuuint64_t dims[2] = {(cuuint64_t)cfg.head_dim, rows};
   const cuuint64_t strides[1] = {(cuuint64_t)cfg.head_dim * 2};
-  const cuuint32_t box[2] = {64, (cuuint32_t)tova::TILE_ROWS};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -626,6 +694,16 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
       return TOVA_ERR_CUDA;
     }
   }
+  // Bulk fill of a prompt (bf16 states): tiled views in boxes of 64 rows.  Where they cannot be had
+  // (a state of fewer rows than one box, 2^31 rows or more) prompts go token by token.
+  c->bulk_fill = true;
+  c->fill_maps = false;
+  {
+    const long long rows = (long long)cfg->batch * cfg->n_kv_heads * cfg->capacity;
+    if (cfg->dtype == TOVA_DTYPE_BF16 && rows >= tova::FILL_K_ROWS && rows < (1LL << 31))
+      c->fill_maps = encode_state_map(&c->fill_map_k, c->base + lay.K, *cfg, tova::FILL_K_ROWS) == TOVA_OK &&
+                     encode_state_map(&c->fill_map_v, c->base + lay.V, *cfg, tova::FILL_K_ROWS) == TOVA_OK;
+  }
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   // Rows that were never written are still read as part of 16-row tiles (their
@@ -671,6 +749,12 @@ int tova_cache_set_policy(tova_cache* c, int32_t policy, int32_t keep_first) {
   return TOVA_OK;
 }
 
+int tova_cache_set_bulk_prefill(tova_cache* c, int32_t on) {
+  if (!c) return TOVA_ERR_NULL;
+  c->bulk_fill = on != 0;
+  return TOVA_OK;
+}
+
 int tova_cache_set_fused_merge(tova_cache* c, int32_t on) {
   if (!c) return TOVA_ERR_NULL;
   c->fuse_merge = on != 0;
@@ -695,7 +779,19 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
   if (!c->cfg.evict && (int64_t)c->len + n_tokens > c->cfg.capacity) return TOVA_ERR_FULL;
   const size_t B = c->cfg.batch, H = c->cfg.n_q_heads, Hkv = c->cfg.n_kv_heads, D = c->cfg.head_dim;
   const size_t q_stride = B * H * D * c->elem, kv_stride = B * Hkv * D * c->elem;
-  for (int32_t t = 0; t < n_tokens; ++t) {
+  int32_t done = 0;
+  // Tokens that fit into free rows are not followed by a deletion (g(t) = min(t, k), Section 3.3):
+  // they are ordinary causal attention and go through the bulk kernels in one piece.
+  {
+    const int room = c->cfg.capacity - c->len;
+    const int F = n_tokens < room ? n_tokens : room;
+    if (c->bulk_fill && c->fill_maps && F >= BULK_FILL_MIN_TOKENS) {
+      rc = launch_fill(c, q, k, v, F, first_pos, out, evicted_pos, static_cast<cudaStream_t>(cuda_stream));
+      if (rc != TOVA_OK) return rc;
+      done = F;
+    }
+  }
+  for (int32_t t = done; t < n_tokens; ++t) {
     rc = step_impl(c, static_cast<const unsigned char*>(q) + t * q_stride,
                    static_cast<const unsigned char*>(k) + t * kv_stride,
                    static_cast<const unsigned char*>(v) + t * kv_stride,

@@ -114,3 +114,39 @@ def test_full_shapes_as_the_benchmark_launches_them(name, cap):
         a, b = ref[l].tova_cache_read(), dfr[l].tova_cache_read()
         assert a["status"] == 0 and b["status"] == 0
         assert torch.equal(a["positions"], b["positions"]) and torch.equal(a["len"], b["len"])
+
+
+@pytest.mark.parametrize("name,cap", [("llama2_7b_layer", 512), ("mistral_7b_gqa", 1024), ("yi_6b_long", 4096)])
+def test_bulk_prefill_full_shapes_on_sampled_tokens(name, cap):
+    """A prompt that fills the whole state in one tova_prefill call (one bulk run: rows copied, one causal-attention
+    launch, one commit).  The state must be the prompt in order; the outputs of sampled (token, sequence) pairs are
+    recomputed by the checker, whose state is written with the tokens before the sampled one."""
+    from oracle.tova_oracle import OracleCache
+    from parity import gpu_block, out_tol
+    w = W.WORKLOADS[name].scaled(capacity=cap)
+    T = cap
+    q, k, v = W.tokens(w, 0, T)
+    cache = make_cache(w)
+    out, ev = gpu_block(cache, w, q, k, v, 0)
+    assert cache.tova_cache_launches() == 1 + 3
+    assert np.all(ev == -1)
+    st = cache.tova_cache_read(want_kv=True)
+    assert st["status"] == 0
+    assert np.all(st["len"].numpy() == cap)
+    assert np.array_equal(st["positions"].numpy(), np.tile(np.arange(cap, dtype=np.int32), (w.batch, 1)))
+    assert np.array_equal(st["K"].float().numpy(), k.transpose(1, 2, 0, 3))
+    assert np.array_equal(st["V"].float().numpy(), v.transpose(1, 2, 0, 3))
+    worst = 0.0
+    for b in sorted({0, w.batch // 2, w.batch - 1}):
+        for t in sorted({0, 1, 15, 16, 63, 64, 65, 127, 128, cap // 2 - 1, cap // 2 + 37, cap - 65, cap - 2, cap - 1}):
+            orc = OracleCache(1, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, precision="f32")
+            orc.K[0, :, :t] = k[:t, b].transpose(1, 0, 2)
+            orc.V[0, :, :t] = v[:t, b].transpose(1, 0, 2)
+            orc.pos[0, :t] = np.arange(t)
+            orc.len[:] = t
+            o, e, *_ = orc.step(q[t, b:b + 1], k[t, b:b + 1], v[t, b:b + 1], t)
+            assert e[0] == -1
+            err = float(np.abs(o[0] - out[t, b]).max())
+            assert err <= out_tol(w), (b, t, err)
+            worst = max(worst, err)
+    print(f"{name} k={cap}: bulk prefill max_err {worst:.2e}")

@@ -112,10 +112,12 @@ def test_yi_shape_reduced_with_periodic_heavy_keys():
 
 
 def test_prefill_equals_decode_steps_bitwise():
+    """Per-token route of tova_prefill (bulk processing off): the same launches as decode steps."""
     w = LLAMA.scaled(batch=2, n_q_heads=8, n_kv_heads=8, capacity=100)
     T = 260
     q, k, v = W.tokens(w, 0, T)
     a, b = make_cache(w), make_cache(w)
+    a.tova_cache_set_bulk_prefill(False)
     oa, ea = gpu_block(a, w, q, k, v, 0, use_prefill=True)
     ob, eb = gpu_block(b, w, q, k, v, 0, use_prefill=False)
     assert np.array_equal(oa, ob) and np.array_equal(ea, eb)
@@ -123,6 +125,57 @@ def test_prefill_equals_decode_steps_bitwise():
     for key in ("len", "positions", "K", "V"):
         assert torch.equal(sa[key], sb[key]), key
     assert a.tova_cache_launches() == b.tova_cache_launches() == 1 + 2 * T
+
+
+@pytest.mark.parametrize("H,Hkv,D,cap,T0,T1", [
+    (8, 8, 128, 300, 200, 330),    # MHA; 4 query tiles with a ragged tail, then a run onto 200 held rows, then full
+    (8, 2, 128, 130, 7, 200),      # GQA; a short run first (one ragged tile), second run crosses tile borders
+    (4, 4, 64, 96, 96, 40),        # D = 64; the run fills the state exactly
+    (16, 1, 128, 257, 3, 254),     # below the bulk threshold first (per-token), then a run from 3 held rows
+])
+def test_bulk_prefill_against_decode_steps(H, Hkv, D, cap, T0, T1):
+    """The bulk route for tokens that fill free rows: state, dropped positions and all later outputs bit-identical
+    to decode steps; outputs of the bulk tokens within the output tolerance (other summation order)."""
+    w = LLAMA.scaled(batch=3, n_q_heads=H, n_kv_heads=Hkv, head_dim=D, capacity=cap)
+    T = T0 + T1
+    q, k, v = W.tokens(w, 0, T)
+    a, b = make_cache(w), make_cache(w)
+    o0, e0 = gpu_block(a, w, q[:T0], k[:T0], v[:T0], 0, use_prefill=True)
+    o1, e1 = gpu_block(a, w, q[T0:], k[T0:], v[T0:], T0, use_prefill=True)
+    oa, ea = np.concatenate([o0, o1]), np.concatenate([e0, e1])
+    ob, eb = gpu_block(b, w, q, k, v, 0, use_prefill=False)
+    assert np.array_equal(ea, eb)
+    fill = min(T, cap)
+    assert np.all(ea[:fill] == -1)
+    assert np.abs(oa[:fill] - ob[:fill]).max() <= out_tol(w)
+    assert np.array_equal(oa[fill:], ob[fill:])
+    sa, sb = a.tova_cache_read(want_kv=True), b.tova_cache_read(want_kv=True)
+    assert sa["status"] == 0
+    for key in ("len", "positions", "K", "V"):
+        assert torch.equal(sa[key], sb[key]), key
+    assert a.tova_cache_launches() < b.tova_cache_launches()
+
+
+def test_bulk_prefill_against_the_checker_with_automatic_positions():
+    """Bulk runs of several query tiles held against the checker token by token; positions continue from
+    the device counter (TOVA_POS_AUTO) across a bulk run and the per-token steps after it."""
+    w = MISTRAL.scaled(batch=2, n_q_heads=8, n_kv_heads=2, capacity=200)
+    rep = run_lockstep(w, 200 + 60, block=150)          # runs of 150 and 50 tokens in bulk, then evictions
+    assert rep.evictions == 2 * 60
+    T = 230
+    q, k, v = W.tokens(w, 0, T)
+    c = make_cache(w)
+    dq, dk, dv = (tova.to_device(x, w.dtype) for x in (q, k, v))
+    ev = torch.empty(T, w.batch, dtype=torch.int32, device="cuda:0")
+    c.tova_prefill(dq[:5], dk[:5], dv[:5], 5, 0, None, ev[:5])                        # position counter starts at 0
+    c.tova_prefill(dq[5:], dk[5:], dv[5:], T - 5, tova.TOVA_POS_AUTO, None, ev[5:])   # no outputs wanted
+    torch.cuda.synchronize()
+    log = ev.cpu().numpy()
+    assert np.array_equal(log, np.concatenate(rep.evicted_log)[:T])
+    st = c.tova_cache_read()
+    held = replay_slot_table(log, w.capacity)
+    for b in range(w.batch):
+        assert set(st["positions"][b].tolist()) == held[b]
 
 
 def test_cached_rows_are_the_inserted_tokens():
@@ -174,7 +227,7 @@ def test_host_buffer_entry_point_matches_device_path(pinned):
     T = 90
     q, k, v = W.tokens(w, 0, T)
     dev = make_cache(w)
-    o_dev, e_dev = gpu_block(dev, w, q, k, v, 0)
+    o_dev, e_dev = gpu_block(dev, w, q, k, v, 0, use_prefill=False)
     host = make_cache(w)
     pin = (lambda x: x.pin_memory()) if pinned else (lambda x: x)
     hq, hk, hv = (pin(torch.from_numpy(a).to(torch.bfloat16)) for a in (q, k, v))
