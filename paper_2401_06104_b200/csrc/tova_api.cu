@@ -552,7 +552,7 @@ cudaError_t launch_fill_d(tova_cache* c, const tova::FillParams& p, cudaStream_t
   if (e != cudaSuccess) return e;
   c->launches += 1;
   if (p.out) {
-    constexpr size_t smem = 5 * (size_t)tova::FILL_K_ROWS * D * 2 + 1024;
+    constexpr size_t smem = 4 * (size_t)tova::FILL_K_ROWS * D * 2 + 1024;
     static bool configured[64] = {};
     if (c->device >= 0 && c->device < 64 && !configured[c->device]) {
       e = cudaFuncSetAttribute(tova::tova_fill_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

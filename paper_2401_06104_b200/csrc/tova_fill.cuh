@@ -100,22 +100,20 @@ __device__ __forceinline__ uint32_t fill_swz(int row, int chunk) {
   return (uint32_t)((chunk >> 3) * (FILL_K_ROWS * 128) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 
-// grid = (ceil(F/64), H, B), block = 128.  Dynamic shared memory: Q tile + 2 x (K tile + V tile) + 1 KiB slack.
+// grid = (ceil(F/64), H, B), block = 128.  Dynamic shared memory: 2 x (K tile + V tile) + 1 KiB slack; three CTAs per SM.
 template <int D>
-__global__ void __launch_bounds__(FILL_THREADS) tova_fill_attn_kernel(const FillParams p,
+__global__ void __launch_bounds__(FILL_THREADS, 3) tova_fill_attn_kernel(const FillParams p,
                                                                       const __grid_constant__ CUtensorMap map_k,
                                                                       const __grid_constant__ CUtensorMap map_v) {
   constexpr int TILE_BYTES = FILL_K_ROWS * D * 2;  // 8 KiB (D=64) or 16 KiB (D=128)
   constexpr int BOXES = D / 64;
   constexpr int KS = D / 16;                       // k-steps of Q K^T
   constexpr int ND = D / 8;                        // n-tiles of P V
-  constexpr int CH = D / 8;                        // 16-byte chunks per row
 
   extern __shared__ unsigned char fill_smem_raw[];
   unsigned char* smem =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(fill_smem_raw) + 1023) & ~(uintptr_t)1023);
-  unsigned char* q_s = smem;                               // [64][D] swizzled
-  unsigned char* kv_s = smem + TILE_BYTES;                 // stage s: K at 2s, V at 2s+1
+  unsigned char* kv_s = smem;                              // stage s: K at 2s, V at 2s+1
   __shared__ __align__(8) uint64_t bars[2];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -149,24 +147,21 @@ __global__ void __launch_bounds__(FILL_THREADS) tova_fill_attn_kernel(const Fill
   };
   if (tid == 0) issue(0);
 
-  // Q tile -> shared memory (swizzled like the K/V tiles); rows past the run repeat its last token.
-  {
-    const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q);
-    for (int i = tid; i < FILL_Q_ROWS * CH; i += FILL_THREADS) {
-      const int r = i / CH, ch = i % CH;
-      const int t = min(t0 + r, p.F - 1);
-      const uint4 w = *reinterpret_cast<const uint4*>(qg + (((size_t)t * p.B + b) * p.H + h) * D + ch * 8);
-      *reinterpret_cast<uint4*>(q_s + fill_swz(r, ch)) = w;
-    }
-  }
-  __syncthreads();
-
-  // A fragments of this warp's 16 query rows, kept in registers for the whole kernel.
+  // A fragments of this warp's 16 query rows straight from global memory (every 32-byte sector is used in
+  // full), kept in registers for the whole kernel; rows past the run repeat its last token.
   uint32_t qa[KS][4];
   {
-    const int r = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+    const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q);
+    const int ra = min(t0 + warp * 16 + (lane >> 2), p.F - 1), rb = min(t0 + warp * 16 + (lane >> 2) + 8, p.F - 1);
+    const uint32_t* qra = reinterpret_cast<const uint32_t*>(qg + (((size_t)ra * p.B + b) * p.H + h) * D) + (lane & 3);
+    const uint32_t* qrb = reinterpret_cast<const uint32_t*>(qg + (((size_t)rb * p.B + b) * p.H + h) * D) + (lane & 3);
 #pragma unroll
-    for (int ks = 0; ks < KS; ++ks) ldmatrix_x4(qa[ks], smem_addr(q_s) + fill_swz(r, 2 * ks + (lane >> 4)));
+    for (int ks = 0; ks < KS; ++ks) {
+      qa[ks][0] = __ldg(qra + ks * 8);
+      qa[ks][1] = __ldg(qrb + ks * 8);
+      qa[ks][2] = __ldg(qra + ks * 8 + 4);
+      qa[ks][3] = __ldg(qrb + ks * 8 + 4);
+    }
   }
 
   float o[ND][4];
