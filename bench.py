@@ -55,6 +55,7 @@ def parse_args():
                     help="time tova_prefill of a T-token prompt into an empty state instead of decode steps "
                          "(-1: as many tokens as the state holds); a step is one whole prompt")
     ap.add_argument("--no-bulk-prefill", action="store_true", help="with --prefill: every prompt token takes the decode kernels")
+    ap.add_argument("--warp-mma-prefill", action="store_true", help="with --prefill: bulk fill through the warp-level MMA kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
@@ -437,8 +438,8 @@ def run_prefill(args):
     caches = []
     for _ in range(steps + warm):
         c = tova.TovaCache(B, H, Hkv, D, cap, dtype=w.dtype, device=dev)
-        if args.no_bulk_prefill:
-            c.tova_cache_set_bulk_prefill(False)
+        if args.no_bulk_prefill or args.warp_mma_prefill:
+            c.tova_cache_set_bulk_prefill(0 if args.no_bulk_prefill else 2)
         caches.append(c)
     torch.cuda.synchronize()
     for c in caches[:warm]:
@@ -474,7 +475,8 @@ def run_prefill(args):
                                       "parallelism": "single GPU"}),
         "roofline": ({"bound": "tensor", "achieved": flops / (ms * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
                       "frac": flops / (ms * 1e-3) / 1e12 / peak, "traffic": None, "peak_kind": kind,
-                      "note": "causal-attention flops of the bulk run / whole prefill time; warp-level MMA kernel"}
+                      "note": "causal-attention flops of the bulk run / whole prefill time; "
+                              + ("warp-level MMA kernel" if args.warp_mma_prefill or D != 128 else "tcgen05 kernel")}
                      if bulk and T == F else None),
         "cpu_baseline": None, "e2e": None, "gpu_launches": launches * steps, "clocks": clocks,
     }

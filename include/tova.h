@@ -109,7 +109,8 @@ int tova_decode_step(tova_cache* c, const void* q, const void* k, const void* v,
  * the cache is within its size), so for them Eq. 6-7 are ordinary causal
  * attention.  On bf16 states a run of at least 4 such tokens is therefore
  * processed in bulk - one copy of the rows, one tensor-core causal-attention
- * kernel (skipped when out is NULL), one small commit kernel - instead of
+ * kernel (skipped when out is NULL; tcgen05 with accumulators in tensor memory
+ * where head_dim is 128), one small commit kernel - instead of
  * token by token; its outputs equal the per-token ones up to floating-point
  * summation order (within the library's output tolerance), everything else
  * bit for bit.  The tokens that remain once the state is full are processed
@@ -194,9 +195,12 @@ int tova_cache_set_policy(tova_cache* c, int32_t policy, int32_t keep_first);
 int tova_cache_set_fused_merge(tova_cache* c, int32_t on);
 
 /* Bulk processing of the prompt tokens that fill free rows (see tova_prefill;
- * on by default, used on bf16 states).  on = 0: every prompt token takes the
- * decode kernels.  Returns TOVA_ERR_NULL for a null handle. */
-int tova_cache_set_bulk_prefill(tova_cache* c, int32_t on);
+ * used on bf16 states).  mode 1 (default): the causal attention of the run
+ * goes through the tcgen05 / tensor-memory kernel where head_dim is 128, else
+ * through the warp-level MMA kernel; mode 2: always the warp-level MMA kernel;
+ * mode 0: every prompt token takes the decode kernels.  Returns TOVA_ERR_NULL
+ * for a null handle, TOVA_ERR_BAD_SHAPE for any other mode. */
+int tova_cache_set_bulk_prefill(tova_cache* c, int32_t mode);
 
 /* Rows each sequence holds now, min(tokens fed, capacity) = g(t) of Section
  * 3.3, tracked on the host (sequences advance in lock step). */

@@ -174,8 +174,10 @@ class TovaCache:
     def tova_cache_set_fused_merge(self, on: bool) -> None:
         _check(lib().tova_cache_set_fused_merge(self._h, 1 if on else 0), "tova_cache_set_fused_merge")
 
-    def tova_cache_set_bulk_prefill(self, on: bool) -> None:
-        _check(lib().tova_cache_set_bulk_prefill(self._h, 1 if on else 0), "tova_cache_set_bulk_prefill")
+    def tova_cache_set_bulk_prefill(self, mode) -> None:
+        """0 / False: prompt tokens one at a time; 1 / True: bulk fill (tcgen05 kernel where head_dim is 128);
+        2: bulk fill with the warp-level MMA kernel."""
+        _check(lib().tova_cache_set_bulk_prefill(self._h, int(mode)), "tova_cache_set_bulk_prefill")
 
     def tova_cache_set_deferred_eviction(self, on: bool) -> None:
         _check(lib().tova_cache_set_deferred_eviction(self._h, 1 if on else 0),

@@ -15,6 +15,7 @@
 #include "tova_kernels.cuh"
 #include "tova_split_mma.cuh"
 #include "tova_fill.cuh"
+#include "tova_fill_tc.cuh"
 
 namespace {
 
@@ -85,7 +86,8 @@ struct tova_cache {
   CUtensorMap map_k, map_v;  // tiled views of K and V for the tensor-core split kernel
   bool use_mma;
   CUtensorMap fill_map_k, fill_map_v;  // the same matrices in boxes of 64 rows, for the bulk fill of a prompt
-  bool fill_maps, bulk_fill;
+  bool fill_maps;
+  int bulk_fill;   // 0: prompts token by token; 1: bulk fill, tcgen05 kernel where head_dim is 128; 2: bulk fill, warp-level MMA kernel
   int policy, keep_first;  // which row is dropped once the state is over capacity (tova_cache_set_policy)
   bool fuse_merge;      // the split warps of a head group form one CTA and merge the outputs themselves
   // deferred eviction: victim choice and insert run on a side stream, overlapping later work
@@ -552,15 +554,27 @@ cudaError_t launch_fill_d(tova_cache* c, const tova::FillParams& p, cudaStream_t
   if (e != cudaSuccess) return e;
   c->launches += 1;
   if (p.out) {
-    constexpr size_t smem = 4 * (size_t)tova::FILL_K_ROWS * D * 2 + 1024;
-    static bool configured[64] = {};
-    if (c->device >= 0 && c->device < 64 && !configured[c->device]) {
-      e = cudaFuncSetAttribute(tova::tova_fill_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return e;
-      configured[c->device] = true;
+    if (D == 128 && c->bulk_fill == 1) {
+      constexpr size_t smem_tc = 96 * 1024 + 1024;
+      static bool configured_tc[64] = {};
+      if (c->device >= 0 && c->device < 64 && !configured_tc[c->device]) {
+        e = cudaFuncSetAttribute(tova::tova_fill_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_tc);
+        if (e != cudaSuccess) return e;
+        configured_tc[c->device] = true;
+      }
+      dim3 grid((p.F + tova::FILLTC_Q_ROWS - 1) / tova::FILLTC_Q_ROWS, p.H, p.B);
+      tova::tova_fill_attn_tc_kernel<<<grid, tova::FILLTC_THREADS, smem_tc, st>>>(p, c->fill_map_k, c->fill_map_v);
+    } else {
+      constexpr size_t smem = 4 * (size_t)tova::FILL_K_ROWS * D * 2 + 1024;
+      static bool configured[64] = {};
+      if (c->device >= 0 && c->device < 64 && !configured[c->device]) {
+        e = cudaFuncSetAttribute(tova::tova_fill_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured[c->device] = true;
+      }
+      dim3 grid((p.F + tova::FILL_Q_ROWS - 1) / tova::FILL_Q_ROWS, p.H, p.B);
+      tova::tova_fill_attn_kernel<D><<<grid, tova::FILL_THREADS, smem, st>>>(p, c->fill_map_k, c->fill_map_v);
     }
-    dim3 grid((p.F + tova::FILL_Q_ROWS - 1) / tova::FILL_Q_ROWS, p.H, p.B);
-    tova::tova_fill_attn_kernel<D><<<grid, tova::FILL_THREADS, smem, st>>>(p, c->fill_map_k, c->fill_map_v);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     c->launches += 1;
   }
@@ -696,7 +710,7 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   }
   // Bulk fill of a prompt (bf16 states): tiled views in boxes of 64 rows.  Where they cannot be had
   // (a state of fewer rows than one box, 2^31 rows or more) prompts go token by token.
-  c->bulk_fill = true;
+  c->bulk_fill = 1;
   c->fill_maps = false;
   {
     const long long rows = (long long)cfg->batch * cfg->n_kv_heads * cfg->capacity;
@@ -751,7 +765,8 @@ int tova_cache_set_policy(tova_cache* c, int32_t policy, int32_t keep_first) {
 
 int tova_cache_set_bulk_prefill(tova_cache* c, int32_t on) {
   if (!c) return TOVA_ERR_NULL;
-  c->bulk_fill = on != 0;
+  if (on < 0 || on > 2) return TOVA_ERR_BAD_SHAPE;
+  c->bulk_fill = on;
   return TOVA_OK;
 }
 

@@ -1,0 +1,303 @@
+// Causal attention of a prompt run on the 5th-generation tensor cores (sm_100a): the same
+// operation as tova_fill_attn_kernel (tova_fill.cuh; Eq. 6-7 while the state has free rows),
+// with both contractions issued as tcgen05.mma from shared-memory descriptors and their
+// accumulators in tensor memory (TMEM).
+//
+// One CTA of 128 threads per (128 query tokens, query head, sequence); thread i owns query
+// row i = TMEM lane i.  Per tile of 64 state rows:
+//   TMA (tiled, 128-byte swizzle)  K tile, V tile -> shared memory
+//   tcgen05.mma  S[128 x 64]  = Q[128 x D] . K^T          (A, B K-major; fp32 in TMEM)
+//   tcgen05.ld   S row -> registers; scale, causal mask, online soft-max in the base-2 domain;
+//                weights as hi + lo bf16 terms -> shared memory (K-major, 128-byte swizzle);
+//                if a row's running max moved, O is rescaled in TMEM (tcgen05.ld / tcgen05.st)
+//   tcgen05.mma  O[128 x D] += P_hi . V + P_lo . V         (B = V tile as stored, MN-major)
+// The steps of one CTA run one after the other (completion through tcgen05.commit on an
+// mbarrier); two CTAs share an SM (97 KiB of shared memory, 256 of the 512 TMEM columns
+// each), so one CTA's soft-max overlaps the other's contractions.  Every wait is bounded;
+// a wait that runs out sets the status word, and the CTA still frees its TMEM.
+#pragma once
+
+#include "tova_fill.cuh"
+
+namespace tova {
+
+constexpr int FILLTC_Q_ROWS = 128;
+constexpr int FILLTC_THREADS = 128;
+constexpr int FILLTC_TMEM_COLS = 256;   // S: 64 columns, O: 128 columns; allocations are powers of two
+
+// Shared-memory matrix descriptor: start address, leading / stride byte offsets (units of 16 bytes),
+// descriptor version 1 (sm_100), 128-byte swizzle.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3ffffu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, A K-major, B K-major or MN-major.
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int M, int N, bool b_mn_major) {
+  uint32_t d = 0;
+  d |= 1u << 4;                        // D format: f32
+  d |= 1u << 7;                        // A format: bf16
+  d |= 1u << 10;                       // B format: bf16
+  d |= (b_mn_major ? 1u : 0u) << 16;   // B major
+  d |= (uint32_t)(N >> 3) << 17;
+  d |= (uint32_t)(M >> 4) << 24;
+  return d;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// The mbarrier receives one arrival once every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(bar))
+               : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])),
+        "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])),
+        "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+        "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])),
+        "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])),
+        "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])),
+        "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// grid = (ceil(F/128), H, B), block = 128.  Dynamic shared memory: Q (32 KiB) + K, V tiles (16 KiB each) +
+// P_hi, P_lo (16 KiB each) + 1 KiB alignment slack.  head_dim 128 only.
+__global__ void __launch_bounds__(FILLTC_THREADS, 2)
+    tova_fill_attn_tc_kernel(const FillParams p, const __grid_constant__ CUtensorMap map_k,
+                             const __grid_constant__ CUtensorMap map_v) {
+  constexpr int D = 128;
+  constexpr int KT = FILL_K_ROWS;                 // 64 state rows per tile
+  constexpr int Q_BYTES = FILLTC_Q_ROWS * D * 2;  // two boxes of [128 rows][128 bytes]
+  constexpr int T_BYTES = KT * D * 2;             // two boxes of [64 rows][128 bytes]
+  constexpr int P_BYTES = FILLTC_Q_ROWS * KT * 2; // one box of [128 rows][128 bytes]
+
+  extern __shared__ unsigned char filltc_smem_raw[];
+  unsigned char* smem =
+      reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(filltc_smem_raw) + 1023) & ~(uintptr_t)1023);
+  unsigned char* q_s = smem;
+  unsigned char* k_s = q_s + Q_BYTES;
+  unsigned char* v_s = k_s + T_BYTES;
+  unsigned char* ph_s = v_s + T_BYTES;
+  unsigned char* pl_s = ph_s + P_BYTES;
+  __shared__ __align__(8) uint64_t bar_kv, bar_mma;
+  __shared__ uint32_t tmem_base_s;
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tile_q = gridDim.x - 1 - blockIdx.x;          // longest rows first
+  const int t0 = tile_q * FILLTC_Q_ROWS;
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int kvh = h / p.G;
+  const int head_row0 = (b * p.Hkv + kvh) * p.cap;
+  const int t_last = min(t0 + FILLTC_Q_ROWS, p.F) - 1;
+  const int n_keys = p.n0 + t_last + 1;
+  const int n_tiles = (n_keys + KT - 1) / KT;
+
+  if (tid == 0) {
+    mbar_init(&bar_kv, 1);
+    mbar_init(&bar_mma, 1);
+    mbar_fence_init();
+  }
+  if (warp == 0) {   // one warp allocates the CTA's tensor memory and gives up the right to allocate more
+    __syncwarp();
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&tmem_base_s)),
+                 "r"(FILLTC_TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // Q tile -> shared memory, K-major with the 128-byte swizzle; rows past the run repeat its last token.
+  {
+    const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q);
+    for (int i = tid; i < FILLTC_Q_ROWS * (D / 8); i += FILLTC_THREADS) {
+      const int r = i / (D / 8), ch = i % (D / 8);
+      const int t = min(t0 + r, p.F - 1);
+      const uint4 w = *reinterpret_cast<const uint4*>(qg + (((size_t)t * p.B + b) * p.H + h) * D + ch * 8);
+      *reinterpret_cast<uint4*>(q_s + (ch >> 3) * (FILLTC_Q_ROWS * 128) + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = w;
+    }
+  }
+  fence_proxy_async_smem();   // the tensor cores read Q through the asynchronous proxy
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base_s;
+  const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 TMEM lanes
+  const uint32_t tm_s = 0, tm_o = 64;                                // column offsets of S and O
+
+  const uint32_t idesc_s = umma_idesc_bf16(FILLTC_Q_ROWS, KT, false);
+  const uint32_t idesc_o = umma_idesc_bf16(FILLTC_Q_ROWS, D, true);
+  const uint32_t q_a = smem_addr(q_s), k_a = smem_addr(k_s), v_a = smem_addr(v_s), ph_a = smem_addr(ph_s),
+                 pl_a = smem_addr(pl_s);
+
+  const int my_t = min(t0 + tid, p.F - 1);
+  const int vis = p.n0 + my_t;            // last state row this thread's query sees
+  float m_run = -INFINITY, l_run = 0.f;
+  uint32_t ph_kv = 0, ph_mma = 0;         // phases of the two barriers
+  bool ok = true;
+
+  for (int i = 0; i < n_tiles && ok; ++i) {
+    const int j0 = i * KT;
+    if (tid == 0) {
+      mbar_expect_tx(&bar_kv, 2u * T_BYTES);
+      const int y = head_row0 + j0;
+      tma_load_2d_keep(k_s, &map_k, 0, y, &bar_kv);
+      tma_load_2d_keep(k_s + KT * 128, &map_k, 64, y, &bar_kv);
+      tma_load_2d_keep(v_s, &map_v, 0, y, &bar_kv);
+      tma_load_2d_keep(v_s + KT * 128, &map_v, 64, y, &bar_kv);
+      ok = mbar_wait_bounded(&bar_kv, ph_kv);
+      if (ok) {
+        // S = Q K^T: 8 steps of 16 along D; a step moves 32 bytes inside the 128-byte row, 4 steps per box
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint64_t a = umma_desc_sw128(q_a + (ks >> 2) * (FILLTC_Q_ROWS * 128) + (ks & 3) * 32, 16, 1024);
+          const uint64_t bd = umma_desc_sw128(k_a + (ks >> 2) * (KT * 128) + (ks & 3) * 32, 16, 1024);
+          umma_bf16(tmem + tm_s, a, bd, idesc_s, ks > 0 ? 1u : 0u);
+        }
+        umma_commit(&bar_mma);
+      }
+    }
+    ph_kv ^= 1u;
+    ok = __syncthreads_and(ok ? 1 : 0) != 0;
+    if (!ok) break;
+    ok = mbar_wait_bounded(&bar_mma, ph_mma);
+    ph_mma ^= 1u;
+    tc_fence_after();
+
+    // ---- soft-max of this thread's row -------------------------------------------------
+    __syncwarp();
+    float s[KT];
+    {
+      float part[32];
+      tmem_ld32(lane_base + tm_s, part);
+#pragma unroll
+      for (int c = 0; c < 32; ++c) s[c] = part[c];
+      tmem_ld32(lane_base + tm_s + 32, part);
+#pragma unroll
+      for (int c = 0; c < 32; ++c) s[32 + c] = part[c];
+    }
+    float mx = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < KT; ++c) {
+      s[c] = (j0 + c <= vis) ? s[c] * p.scale2 : -INFINITY;
+      mx = fmaxf(mx, s[c]);
+    }
+    const float m_new = fmaxf(m_run, mx);       // finite from tile 0 on: row 0 of the state is visible to every query
+    const float corr = exp2_diff(m_run, m_new);
+    m_run = m_new;
+    float lsum = 0.f;
+#pragma unroll
+    for (int c8 = 0; c8 < KT / 8; ++c8) {
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float e0 = exp2f(s[c8 * 8 + 2 * e] - m_new), e1 = exp2f(s[c8 * 8 + 2 * e + 1] - m_new);
+        lsum += e0 + e1;
+        split_hi_lo(e0, e1, hi[e], lo[e]);
+      }
+      const uint32_t off = (uint32_t)tid * 128u + (uint32_t)((c8 ^ (tid & 7)) << 4);
+      *reinterpret_cast<uint4*>(ph_s + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      *reinterpret_cast<uint4*>(pl_s + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    }
+    l_run = l_run * corr + lsum;
+    // O of the tiles so far was accumulated against the old max
+    if (i > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
+#pragma unroll
+      for (int c0 = 0; c0 < D; c0 += 32) {
+        float o[32];
+        tmem_ld32(lane_base + tm_o + c0, o);
+#pragma unroll
+        for (int c = 0; c < 32; ++c) o[c] *= corr;
+        tmem_st32(lane_base + tm_o + c0, o);
+      }
+      tmem_st_wait();
+    }
+    fence_proxy_async_smem();   // P was written through the generic proxy, the tensor cores read it asynchronously
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- O += P V: 4 steps of 16 state rows; V as stored is MN-major (D contiguous) --------
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int kk = 0; kk < KT / 16; ++kk) {
+        const uint64_t bd = umma_desc_sw128(v_a + kk * 2048, KT * 128, 1024);
+        const uint64_t ah = umma_desc_sw128(ph_a + kk * 32, 16, 1024);
+        const uint64_t al = umma_desc_sw128(pl_a + kk * 32, 16, 1024);
+        umma_bf16(tmem + tm_o, ah, bd, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
+        umma_bf16(tmem + tm_o, al, bd, idesc_o, 1u);
+      }
+      umma_commit(&bar_mma);
+    }
+    ok = mbar_wait_bounded(&bar_mma, ph_mma);   // K, V, P may be overwritten and O read after this
+    ph_mma ^= 1u;
+    tc_fence_after();
+    ok = __syncthreads_and(ok ? 1 : 0) != 0;
+  }
+
+  if (ok) {
+    const float rl = 1.f / l_run;
+    const int t = t0 + tid;
+#pragma unroll
+    for (int c0 = 0; c0 < D; c0 += 32) {
+      float o[32];
+      tmem_ld32(lane_base + tm_o + c0, o);
+      if (t < p.F) {
+        float4* dst = reinterpret_cast<float4*>(p.out + (((size_t)t * p.B + b) * p.H + h) * D + c0);
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          dst[c] = make_float4(o[4 * c] * rl, o[4 * c + 1] * rl, o[4 * c + 2] * rl, o[4 * c + 3] * rl);
+      }
+    }
+  } else if (tid == 0) {
+    atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(FILLTC_TMEM_COLS) : "memory");
+  }
+}
+
+}  // namespace tova

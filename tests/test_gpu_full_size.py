@@ -116,8 +116,9 @@ def test_full_shapes_as_the_benchmark_launches_them(name, cap):
         assert torch.equal(a["positions"], b["positions"]) and torch.equal(a["len"], b["len"])
 
 
+@pytest.mark.parametrize("mode", [1, 2])   # 1: tcgen05 kernel; 2: warp-level MMA kernel
 @pytest.mark.parametrize("name,cap", [("llama2_7b_layer", 512), ("mistral_7b_gqa", 1024), ("yi_6b_long", 4096)])
-def test_bulk_prefill_full_shapes_on_sampled_tokens(name, cap):
+def test_bulk_prefill_full_shapes_on_sampled_tokens(name, cap, mode):
     """A prompt that fills the whole state in one tova_prefill call (one bulk run: rows copied, one causal-attention
     launch, one commit).  The state must be the prompt in order; the outputs of sampled (token, sequence) pairs are
     recomputed by the checker, whose state is written with the tokens before the sampled one."""
@@ -127,6 +128,7 @@ def test_bulk_prefill_full_shapes_on_sampled_tokens(name, cap):
     T = cap
     q, k, v = W.tokens(w, 0, T)
     cache = make_cache(w)
+    cache.tova_cache_set_bulk_prefill(mode)
     out, ev = gpu_block(cache, w, q, k, v, 0)
     assert cache.tova_cache_launches() == 1 + 3
     assert np.all(ev == -1)

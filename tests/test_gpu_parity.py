@@ -133,13 +133,15 @@ def test_prefill_equals_decode_steps_bitwise():
     (4, 4, 64, 96, 96, 40),        # D = 64; the run fills the state exactly
     (16, 1, 128, 257, 3, 254),     # below the bulk threshold first (per-token), then a run from 3 held rows
 ])
-def test_bulk_prefill_against_decode_steps(H, Hkv, D, cap, T0, T1):
+@pytest.mark.parametrize("mode", [1, 2])   # 1: tcgen05 kernel where D = 128; 2: warp-level MMA kernel
+def test_bulk_prefill_against_decode_steps(H, Hkv, D, cap, T0, T1, mode):
     """The bulk route for tokens that fill free rows: state, dropped positions and all later outputs bit-identical
     to decode steps; outputs of the bulk tokens within the output tolerance (other summation order)."""
     w = LLAMA.scaled(batch=3, n_q_heads=H, n_kv_heads=Hkv, head_dim=D, capacity=cap)
     T = T0 + T1
     q, k, v = W.tokens(w, 0, T)
     a, b = make_cache(w), make_cache(w)
+    a.tova_cache_set_bulk_prefill(mode)
     o0, e0 = gpu_block(a, w, q[:T0], k[:T0], v[:T0], 0, use_prefill=True)
     o1, e1 = gpu_block(a, w, q[T0:], k[T0:], v[T0:], T0, use_prefill=True)
     oa, ea = np.concatenate([o0, o1]), np.concatenate([e0, e1])
