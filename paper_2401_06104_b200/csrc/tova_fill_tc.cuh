@@ -67,6 +67,13 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// 2^x, hardware approximation (relative error about 2^-22; -inf gives 0; results below 2^-126 flush to 0).
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // 32 consecutive fp32 columns of this thread's TMEM lane.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   uint32_t r[32];
@@ -122,7 +129,7 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   unsigned char* v_s = k_s + T_BYTES;
   unsigned char* ph_s = v_s + T_BYTES;
   unsigned char* pl_s = ph_s + P_BYTES;
-  __shared__ __align__(8) uint64_t bar_kv, bar_mma;
+  __shared__ __align__(8) uint64_t bar_k, bar_v, bar_mma;
   __shared__ uint32_t tmem_base_s;
 
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -136,7 +143,8 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   const int n_tiles = (n_keys + KT - 1) / KT;
 
   if (tid == 0) {
-    mbar_init(&bar_kv, 1);
+    mbar_init(&bar_k, 1);
+    mbar_init(&bar_v, 1);
     mbar_init(&bar_mma, 1);
     mbar_fence_init();
   }
@@ -176,16 +184,30 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   uint32_t ph_kv = 0, ph_mma = 0;         // phases of the two barriers
   bool ok = true;
 
+  // K and V tiles have one buffer each and a barrier each: the next K tile is requested as soon as S = Q K^T
+  // of the current one has completed, the next V tile as soon as O += P V has, so the copies run under the
+  // soft-max and the other contraction.
+  auto load_k = [&](int i) {
+    mbar_expect_tx(&bar_k, (uint32_t)T_BYTES);
+    const int y = head_row0 + i * KT;
+    tma_load_2d_keep(k_s, &map_k, 0, y, &bar_k);
+    tma_load_2d_keep(k_s + KT * 128, &map_k, 64, y, &bar_k);
+  };
+  auto load_v = [&](int i) {
+    mbar_expect_tx(&bar_v, (uint32_t)T_BYTES);
+    const int y = head_row0 + i * KT;
+    tma_load_2d_keep(v_s, &map_v, 0, y, &bar_v);
+    tma_load_2d_keep(v_s + KT * 128, &map_v, 64, y, &bar_v);
+  };
+  if (tid == 0) {
+    load_k(0);
+    load_v(0);
+  }
+
   for (int i = 0; i < n_tiles && ok; ++i) {
     const int j0 = i * KT;
     if (tid == 0) {
-      mbar_expect_tx(&bar_kv, 2u * T_BYTES);
-      const int y = head_row0 + j0;
-      tma_load_2d_keep(k_s, &map_k, 0, y, &bar_kv);
-      tma_load_2d_keep(k_s + KT * 128, &map_k, 64, y, &bar_kv);
-      tma_load_2d_keep(v_s, &map_v, 0, y, &bar_kv);
-      tma_load_2d_keep(v_s + KT * 128, &map_v, 64, y, &bar_kv);
-      ok = mbar_wait_bounded(&bar_kv, ph_kv);
+      ok = mbar_wait_bounded(&bar_k, ph_kv);
       if (ok) {
         // S = Q K^T: 8 steps of 16 along D; a step moves 32 bytes inside the 128-byte row, 4 steps per box
         tc_fence_after();
@@ -198,12 +220,11 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
         umma_commit(&bar_mma);
       }
     }
-    ph_kv ^= 1u;
-    ok = __syncthreads_and(ok ? 1 : 0) != 0;
-    if (!ok) break;
-    ok = mbar_wait_bounded(&bar_mma, ph_mma);
+    // (a K wait that ran out shows up as a missing commit: the wait below then runs out for every thread)
+    ok = mbar_wait_bounded(&bar_mma, ph_mma) && ok;
     ph_mma ^= 1u;
     tc_fence_after();
+    if (tid == 0 && ok && i + 1 < n_tiles) load_k(i + 1);   // the K buffer is free: S has been computed
 
     // ---- soft-max of this thread's row -------------------------------------------------
     __syncwarp();
@@ -218,10 +239,18 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
       for (int c = 0; c < 32; ++c) s[32 + c] = part[c];
     }
     float mx = -INFINITY;
+    if (j0 + KT - 1 > p.n0 + t0) {   // some query of this CTA cannot see the whole tile (CTA-uniform)
 #pragma unroll
-    for (int c = 0; c < KT; ++c) {
-      s[c] = (j0 + c <= vis) ? s[c] * p.scale2 : -INFINITY;
-      mx = fmaxf(mx, s[c]);
+      for (int c = 0; c < KT; ++c) {
+        s[c] = (j0 + c <= vis) ? s[c] * p.scale2 : -INFINITY;
+        mx = fmaxf(mx, s[c]);
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < KT; ++c) {
+        s[c] *= p.scale2;
+        mx = fmaxf(mx, s[c]);
+      }
     }
     const float m_new = fmaxf(m_run, mx);       // finite from tile 0 on: row 0 of the state is visible to every query
     const float corr = exp2_diff(m_run, m_new);
@@ -232,7 +261,7 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
       uint32_t hi[4], lo[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const float e0 = exp2f(s[c8 * 8 + 2 * e] - m_new), e1 = exp2f(s[c8 * 8 + 2 * e + 1] - m_new);
+        const float e0 = ex2_approx(s[c8 * 8 + 2 * e] - m_new), e1 = ex2_approx(s[c8 * 8 + 2 * e + 1] - m_new);
         lsum += e0 + e1;
         split_hi_lo(e0, e1, hi[e], lo[e]);
       }
@@ -258,7 +287,7 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
     __syncthreads();
 
     // ---- O += P V: 4 steps of 16 state rows; V as stored is MN-major (D contiguous) --------
-    if (tid == 0) {
+    if (tid == 0 && mbar_wait_bounded(&bar_v, ph_kv)) {   // (a wait that ran out shows up as a missing commit below)
       tc_fence_after();
 #pragma unroll
       for (int kk = 0; kk < KT / 16; ++kk) {
@@ -270,9 +299,11 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
       }
       umma_commit(&bar_mma);
     }
-    ok = mbar_wait_bounded(&bar_mma, ph_mma);   // K, V, P may be overwritten and O read after this
+    ok = mbar_wait_bounded(&bar_mma, ph_mma);   // V and P may be overwritten and O read after this
     ph_mma ^= 1u;
+    ph_kv ^= 1u;
     tc_fence_after();
+    if (tid == 0 && ok && i + 1 < n_tiles) load_v(i + 1);
     ok = __syncthreads_and(ok ? 1 : 0) != 0;
   }
 
