@@ -23,7 +23,7 @@ namespace tova {
 
 constexpr int FILLTC_Q_ROWS = 128;
 constexpr int FILLTC_THREADS = 128;
-constexpr int FILLTC_TMEM_COLS = 256;   // S: 64 columns, O: 128 columns; allocations are powers of two
+constexpr int FILLTC_TMEM_COLS = 256;   // S of even and odd tiles: 64 columns each, O: 128 columns
 
 // Shared-memory matrix descriptor: start address, leading / stride byte offsets (units of 16 bytes),
 // descriptor version 1 (sm_100), 128-byte swizzle.
@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
   const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 TMEM lanes
-  const uint32_t tm_s = 0, tm_o = 64;                                // column offsets of S and O
+  const uint32_t tm_o = 128;                                         // S of tile i at column 64 (i & 1), O at 128
 
   const uint32_t idesc_s = umma_idesc_bf16(FILLTC_Q_ROWS, KT, false);
   const uint32_t idesc_o = umma_idesc_bf16(FILLTC_Q_ROWS, D, true);
@@ -181,7 +181,7 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   const int my_t = min(t0 + tid, p.F - 1);
   const int vis = p.n0 + my_t;            // last state row this thread's query sees
   float m_run = -INFINITY, l_run = 0.f;
-  uint32_t ph_kv = 0, ph_mma = 0;         // phases of the two barriers
+  uint32_t ph_mma = 0;                    // phase of the tensor-core completion barrier (K, V tile i: parity i & 1)
   bool ok = true;
 
   // K and V tiles have one buffer each and a barrier each: the next K tile is requested as soon as S = Q K^T
@@ -204,27 +204,34 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
     load_v(0);
   }
 
+  // S = Q K^T of tile i into S buffer i & 1: 8 steps of 16 along D; a step moves 32 bytes inside the 128-byte
+  // row, 4 steps per box.  Issued by one thread once the K tile has landed.
+  auto issue_qk = [&](int i) {
+    tc_fence_after();
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+      const uint64_t a = umma_desc_sw128(q_a + (ks >> 2) * (FILLTC_Q_ROWS * 128) + (ks & 3) * 32, 16, 1024);
+      const uint64_t bd = umma_desc_sw128(k_a + (ks >> 2) * (KT * 128) + (ks & 3) * 32, 16, 1024);
+      umma_bf16(tmem + (uint32_t)(64 * (i & 1)), a, bd, idesc_s, ks > 0 ? 1u : 0u);
+    }
+  };
+  // Tile 0's S by itself; from then on S of tile i+1 is issued together with O += P V of tile i (one commit,
+  // one wait per tile), so a tile's logits are ready when its soft-max starts.
+  if (tid == 0) {
+    if (mbar_wait_bounded(&bar_k, 0u)) {
+      issue_qk(0);
+      umma_commit(&bar_mma);
+    }
+  }
+  ok = mbar_wait_bounded(&bar_mma, ph_mma);   // (a K wait that ran out shows up as a missing commit)
+  ph_mma ^= 1u;
+  tc_fence_after();
+  if (tid == 0 && ok && n_tiles > 1) load_k(1);   // the K buffer is free: S of tile 0 has been computed
+  ok = __syncthreads_and(ok ? 1 : 0) != 0;
+
   for (int i = 0; i < n_tiles && ok; ++i) {
     const int j0 = i * KT;
-    if (tid == 0) {
-      ok = mbar_wait_bounded(&bar_k, ph_kv);
-      if (ok) {
-        // S = Q K^T: 8 steps of 16 along D; a step moves 32 bytes inside the 128-byte row, 4 steps per box
-        tc_fence_after();
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          const uint64_t a = umma_desc_sw128(q_a + (ks >> 2) * (FILLTC_Q_ROWS * 128) + (ks & 3) * 32, 16, 1024);
-          const uint64_t bd = umma_desc_sw128(k_a + (ks >> 2) * (KT * 128) + (ks & 3) * 32, 16, 1024);
-          umma_bf16(tmem + tm_s, a, bd, idesc_s, ks > 0 ? 1u : 0u);
-        }
-        umma_commit(&bar_mma);
-      }
-    }
-    // (a K wait that ran out shows up as a missing commit: the wait below then runs out for every thread)
-    ok = mbar_wait_bounded(&bar_mma, ph_mma) && ok;
-    ph_mma ^= 1u;
-    tc_fence_after();
-    if (tid == 0 && ok && i + 1 < n_tiles) load_k(i + 1);   // the K buffer is free: S has been computed
+    const uint32_t tm_s = (uint32_t)(64 * (i & 1));
 
     // ---- soft-max of this thread's row -------------------------------------------------
     __syncwarp();
@@ -287,7 +294,10 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
     __syncthreads();
 
     // ---- O += P V: 4 steps of 16 state rows; V as stored is MN-major (D contiguous) --------
-    if (tid == 0 && mbar_wait_bounded(&bar_v, ph_kv)) {   // (a wait that ran out shows up as a missing commit below)
+    // (a K or V wait that ran out shows up as a missing commit below)
+    if (tid == 0 && (i + 1 >= n_tiles || mbar_wait_bounded(&bar_k, (uint32_t)((i + 1) & 1))) &&
+        mbar_wait_bounded(&bar_v, (uint32_t)(i & 1))) {
+      if (i + 1 < n_tiles) issue_qk(i + 1);
       tc_fence_after();
 #pragma unroll
       for (int kk = 0; kk < KT / 16; ++kk) {
@@ -299,11 +309,13 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
       }
       umma_commit(&bar_mma);
     }
-    ok = mbar_wait_bounded(&bar_mma, ph_mma);   // V and P may be overwritten and O read after this
+    ok = mbar_wait_bounded(&bar_mma, ph_mma);   // K, V and P may be overwritten and O and the next S read after this
     ph_mma ^= 1u;
-    ph_kv ^= 1u;
     tc_fence_after();
-    if (tid == 0 && ok && i + 1 < n_tiles) load_v(i + 1);
+    if (tid == 0 && ok) {
+      if (i + 2 < n_tiles) load_k(i + 2);
+      if (i + 1 < n_tiles) load_v(i + 1);
+    }
     ok = __syncthreads_and(ok ? 1 : 0) != 0;
   }
 
