@@ -22,7 +22,7 @@
 namespace tova {
 
 constexpr int FILLTC_Q_ROWS = 128;
-constexpr int FILLTC_THREADS = 128;
+constexpr int FILLTC_THREADS = 256;   // two threads per query row: each takes half of a tile's 64 logits, half of O's columns
 constexpr int FILLTC_TMEM_COLS = 256;   // S of even and odd tiles: 64 columns each, O: 128 columns
 
 // Shared-memory matrix descriptor: start address, leading / stride byte offsets (units of 16 bytes),
@@ -131,6 +131,7 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   unsigned char* pl_s = ph_s + P_BYTES;
   __shared__ __align__(8) uint64_t bar_k, bar_v, bar_mma;
   __shared__ uint32_t tmem_base_s;
+  __shared__ float half_max[2][FILLTC_Q_ROWS];   // the two halves of a row exchange their tile maxima (and, at the end, sums)
 
   const int tid = threadIdx.x, warp = tid >> 5;
   const int tile_q = gridDim.x - 1 - blockIdx.x;          // longest rows first
@@ -170,7 +171,10 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
-  const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 TMEM lanes
+  // A warp reaches the 32 TMEM lanes of its quarter (warp mod 4); warps 0-3 take the first half of a row's
+  // columns, warps 4-7 the second half.
+  const int row = (warp & 3) * 32 + (tid & 31), half = warp >> 2;
+  const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
   const uint32_t tm_o = 128;                                         // S of tile i at column 64 (i & 1), O at 128
 
   const uint32_t idesc_s = umma_idesc_bf16(FILLTC_Q_ROWS, KT, false);
@@ -178,7 +182,7 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   const uint32_t q_a = smem_addr(q_s), k_a = smem_addr(k_s), v_a = smem_addr(v_s), ph_a = smem_addr(ph_s),
                  pl_a = smem_addr(pl_s);
 
-  const int my_t = min(t0 + tid, p.F - 1);
+  const int my_t = min(t0 + row, p.F - 1);
   const int vis = p.n0 + my_t;            // last state row this thread's query sees
   float m_run = -INFINITY, l_run = 0.f;
   uint32_t ph_mma = 0;                    // phase of the tensor-core completion barrier (K, V tile i: parity i & 1)
@@ -235,36 +239,33 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
 
     // ---- soft-max of this thread's row -------------------------------------------------
     __syncwarp();
-    float s[KT];
-    {
-      float part[32];
-      tmem_ld32(lane_base + tm_s, part);
-#pragma unroll
-      for (int c = 0; c < 32; ++c) s[c] = part[c];
-      tmem_ld32(lane_base + tm_s + 32, part);
-#pragma unroll
-      for (int c = 0; c < 32; ++c) s[32 + c] = part[c];
-    }
+    constexpr int KH = KT / 2;   // logits per thread
+    float s[KH];
+    tmem_ld32(lane_base + tm_s + (uint32_t)(KH * half), s);
+    const int jh = j0 + KH * half;
     float mx = -INFINITY;
     if (j0 + KT - 1 > p.n0 + t0) {   // some query of this CTA cannot see the whole tile (CTA-uniform)
 #pragma unroll
-      for (int c = 0; c < KT; ++c) {
-        s[c] = (j0 + c <= vis) ? s[c] * p.scale2 : -INFINITY;
+      for (int c = 0; c < KH; ++c) {
+        s[c] = (jh + c <= vis) ? s[c] * p.scale2 : -INFINITY;
         mx = fmaxf(mx, s[c]);
       }
     } else {
 #pragma unroll
-      for (int c = 0; c < KT; ++c) {
+      for (int c = 0; c < KH; ++c) {
         s[c] *= p.scale2;
         mx = fmaxf(mx, s[c]);
       }
     }
+    half_max[half][row] = mx;
+    __syncthreads();
+    mx = fmaxf(mx, half_max[half ^ 1][row]);
     const float m_new = fmaxf(m_run, mx);       // finite from tile 0 on: row 0 of the state is visible to every query
     const float corr = exp2_diff(m_run, m_new);
     m_run = m_new;
     float lsum = 0.f;
 #pragma unroll
-    for (int c8 = 0; c8 < KT / 8; ++c8) {
+    for (int c8 = 0; c8 < KH / 8; ++c8) {
       uint32_t hi[4], lo[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
@@ -272,7 +273,7 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
         lsum += e0 + e1;
         split_hi_lo(e0, e1, hi[e], lo[e]);
       }
-      const uint32_t off = (uint32_t)tid * 128u + (uint32_t)((c8 ^ (tid & 7)) << 4);
+      const uint32_t off = (uint32_t)row * 128u + (uint32_t)(((c8 + 4 * half) ^ (row & 7)) << 4);
       *reinterpret_cast<uint4*>(ph_s + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
       *reinterpret_cast<uint4*>(pl_s + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     }
@@ -280,7 +281,7 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
     // O of the tiles so far was accumulated against the old max
     if (i > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
 #pragma unroll
-      for (int c0 = 0; c0 < D; c0 += 32) {
+      for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
         float o[32];
         tmem_ld32(lane_base + tm_o + c0, o);
 #pragma unroll
@@ -320,10 +321,12 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   }
 
   if (ok) {
-    const float rl = 1.f / l_run;
-    const int t = t0 + tid;
+    half_max[half][row] = l_run;     // (the last use of the array was followed by two CTA barriers)
+    __syncthreads();
+    const float rl = 1.f / (half_max[0][row] + half_max[1][row]);
+    const int t = t0 + row;
 #pragma unroll
-    for (int c0 = 0; c0 < D; c0 += 32) {
+    for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
       float o[32];
       tmem_ld32(lane_base + tm_o + c0, o);
       if (t < p.F) {
