@@ -3,18 +3,22 @@
 // with both contractions issued as tcgen05.mma from shared-memory descriptors and their
 // accumulators in tensor memory (TMEM).
 //
-// One CTA of 128 threads per (128 query tokens, query head, sequence); thread i owns query
-// row i = TMEM lane i.  Per tile of 64 state rows:
-//   TMA (tiled, 128-byte swizzle)  K tile, V tile -> shared memory
-//   tcgen05.mma  S[128 x 64]  = Q[128 x D] . K^T          (A, B K-major; fp32 in TMEM)
-//   tcgen05.ld   S row -> registers; scale, causal mask, online soft-max in the base-2 domain;
+// One CTA of 256 threads per (128 query tokens, query head, sequence); query row i = TMEM
+// lane i, shared by two threads (warps w and w + 4), each taking half of a tile's logits and
+// half of O's columns.  Per tile of 64 state rows:
+//   TMA (tiled, 128-byte swizzle)  K tile, V tile -> shared memory (one buffer each; the next
+//                tile is requested as soon as the contraction that read the buffer is complete)
+//   tcgen05.mma  S[128 x 64]  = Q[128 x D] . K^T          (A, B K-major; fp32 in TMEM, two S
+//                buffers: S of tile i+1 is issued together with O += P V of tile i)
+//   tcgen05.ld   half a row of S -> registers; scale, causal mask, online soft-max in the base-2
+//                domain (row maxima of the two halves exchanged through shared memory);
 //                weights as hi + lo bf16 terms -> shared memory (K-major, 128-byte swizzle);
 //                if a row's running max moved, O is rescaled in TMEM (tcgen05.ld / tcgen05.st)
 //   tcgen05.mma  O[128 x D] += P_hi . V + P_lo . V         (B = V tile as stored, MN-major)
-// The steps of one CTA run one after the other (completion through tcgen05.commit on an
-// mbarrier); two CTAs share an SM (97 KiB of shared memory, 256 of the 512 TMEM columns
-// each), so one CTA's soft-max overlaps the other's contractions.  Every wait is bounded;
-// a wait that runs out sets the status word, and the CTA still frees its TMEM.
+// Completion through tcgen05.commit on an mbarrier, one commit and one wait per tile; two
+// CTAs share an SM (98 KiB of shared memory, 256 of the 512 TMEM columns each), so one CTA's
+// soft-max overlaps the other's contractions.  Every wait is bounded; a wait that runs out
+// sets the status word, and the CTA still frees its TMEM.
 #pragma once
 
 #include "tova_fill.cuh"
@@ -110,7 +114,7 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// grid = (ceil(F/128), H, B), block = 128.  Dynamic shared memory: Q (32 KiB) + K, V tiles (16 KiB each) +
+// grid = (ceil(F/128), H, B), block = 256.  Dynamic shared memory: Q (32 KiB) + K, V tiles (16 KiB each) +
 // P_hi, P_lo (16 KiB each) + 1 KiB alignment slack.  head_dim 128 only.
 __global__ void __launch_bounds__(FILLTC_THREADS, 2)
     tova_fill_attn_tc_kernel(const FillParams p, const __grid_constant__ CUtensorMap map_k,
