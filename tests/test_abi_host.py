@@ -72,6 +72,7 @@ def test_null_handles_are_rejected():
     assert L.tova_cache_read(None, None, None, None, None, None, None) == -1
     assert L.tova_cache_destroy(None) == -1
     assert L.tova_cache_len(None) == -1
+    assert L.tova_cache_set_bulk_prefill(None, 1) == -1
     assert tova.strerror(0) == "ok" and "aligned" in tova.strerror(-4)
 
 

@@ -158,6 +158,15 @@ def test_bulk_prefill_against_decode_steps(H, Hkv, D, cap, T0, T1, mode):
     assert a.tova_cache_launches() < b.tova_cache_launches()
 
 
+def test_bulk_prefill_mode_argument():
+    c = make_cache(LLAMA.scaled(batch=1, n_q_heads=2, n_kv_heads=2, capacity=70))
+    for mode in (0, 1, 2, True, False):
+        c.tova_cache_set_bulk_prefill(mode)
+    for bad in (3, -1):
+        with pytest.raises(tova.TovaError):
+            c.tova_cache_set_bulk_prefill(bad)
+
+
 def test_bulk_prefill_against_the_checker_with_automatic_positions():
     """Bulk runs of several query tiles held against the checker token by token; positions continue from
     the device counter (TOVA_POS_AUTO) across a bulk run and the per-token steps after it."""
