@@ -29,15 +29,22 @@ METRIC = "tova_decode_tokens_per_s_per_layer"
 UNIT = "tokens/s"
 RING = 128                      # distinct pre-generated tokens per workload
 WORKING_SET = 1 << 30           # rotate layer caches until this many bytes are touched per round
+# The largest single-GPU configuration: 32 layers of the LLaMA-2-7B shape, batch 64, state of 1024 rows
+# (32 layer caches of 1 GiB; a step is one layer-step).
+DEFAULT_WORKLOAD = "llama2_7b_full"
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=16384)
-    ap.add_argument("--warmup", type=int, default=2048)
+    ap.add_argument("--steps", type=int, default=64, help="K: steps per timed unit (one CUDA graph of K steps)")
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--repeats", type=int, default=0,
+                    help="how often the K timed steps are repeated (0 = until the timed region lasts 50 ms)")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="time the headline workload only, not the other graded configurations after it")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="llama2_7b_layer")
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--capacity", type=int, default=0)
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--layers", type=int, default=0, help="independent layer caches to rotate over (0 = auto)")
@@ -163,6 +170,11 @@ def time_oracle(w, ring, seconds: float, max_seqs: int = 0):
     return S * n_steps / dt, used, f"{n_steps} steady-state steps of {S} of {w.batch} sequences on a full state (k={w.capacity})"
 
 
+def storage_name(w):
+    """Type of q, k, v and the cached rows; sums and soft-max run in fp32."""
+    return "bf16" if w.elem_bytes == 2 else "f32"
+
+
 def workload_config(w, extra):
     cfg = {"workload": w.name, "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
            "head_dim": w.head_dim, "capacity": w.capacity,
@@ -185,7 +197,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.batch / val,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-            "data": "synthetic", "config": workload_config(w, {"sample": sample}),
+            "data": "synthetic", "config": workload_config(w, {"l2": "not applicable: host cores", "parallelism": "replicas only" if args.gpus > 1 else "single GPU"}),
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -233,28 +245,28 @@ def max_over_ranks(x: float, device) -> float:
     return float(t.item())
 
 
-def run_ours(args):
+MIN_TIMED_MS = 50.0             # the K timed steps are repeated until the timed region lasts at least this long
+
+# The other roofline-graded configurations (state of 1024 rows and more), timed after the headline in the same
+# run: (workload, capacity, layer caches).
+SWEEP = [("mistral_7b_gqa", 1024, 0), ("mistral_7b_gqa", 4096, 0), ("yi_6b_long", 4096, 0),
+         ("llama2_7b_full", 8192, 2)]
+
+
+def measure(w, args, dev, world, layers=0, want_e2e=False):
+    """Steady-state decode steps of workload `w` on the current device: fills `layers` caches past their capacity,
+    captures args.steps steps as one CUDA graph and replays it until the timed region lasts MIN_TIMED_MS.
+    Returns a dict of measurements (host numbers; times are the max over ranks)."""
     import torch
     import torch.distributed as dist
 
     import paper_2401_06104_b200 as tova
     from paper_2401_06104_b200 import workloads as W
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py: no CUDA device; the decode path has no CPU fallback")
-    torch.cuda.set_device(local)
-    dev = f"cuda:{local}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(dev))
-
-    w = pick_workload(args)
     B, H, Hkv, D, cap = w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity
     step_bytes = w.step_bytes()
     # at least two layers: consecutive steps then belong to different caches, as in a model
-    L = args.layers or min(64, max(2, -(-WORKING_SET // step_bytes)))
+    L = layers or args.layers or min(64, max(2, w.n_layers, -(-WORKING_SET // step_bytes)))
     deferred = (not args.no_deferred and L >= 2) or args.deferred
     ring = W.tokens(w, 0, RING)                                   # seeded, host
     dq, dk, dv = (tova.to_device(a, w.dtype, dev) for a in ring)
@@ -276,8 +288,8 @@ def run_ours(args):
     # steady state: fill every layer past its capacity (positions from the device counter)
     for l, c in enumerate(caches):
         fed, r = 0, (17 * l) % RING
-        while fed < cap + 64:
-            T = min(RING - r, cap + 64 - fed)
+        while fed < cap + 16:
+            T = min(RING - r, cap + 16 - fed)
             c.tova_prefill(dq[r:], dk[r:], dv[r:], T, -1, None, None)
             fed += T
             r = (r + T) % RING
@@ -304,49 +316,59 @@ def run_ours(args):
             step(counter[0])
             counter[0] += 1
 
+    # Warm-up, part 1: host-launched steps, at least one per cache (sets function attributes before capture).
     l0 = sum(c.tova_cache_launches() for c in caches)
-    n_direct = min(64, max(args.warmup, 3))
-    run_direct(n_direct)                                          # sets function attributes before capture
-    launches_per_step = (sum(c.tova_cache_launches() for c in caches) - l0) // n_direct
+    n_direct = max(args.warmup, 3, L)
+    run_direct(n_direct)
+    launches_per_step = (sum(c.tova_cache_launches() for c in caches) - l0) / n_direct
     join_all()
     torch.cuda.synchronize()
 
-    graph, G = None, 0
+    # The K timed steps as ONE graph of C-ABI calls, whatever K is.
+    K = args.steps
+    graph = None
     launch_mode = "stream"
-    if not args.no_graph and args.steps >= 2 * L:
-        G = min(args.steps, 512)
-        G = max(L, G // L * L)
+    if not args.no_graph:
         try:
             graph = torch.cuda.CUDAGraph()
             base = counter[0]
             with torch.cuda.graph(graph):
-                for j in range(G):
+                for j in range(K):
                     step(base + j)
                 join_all()                                        # side streams rejoin before the capture ends
             launch_mode = "cuda_graph"
         except Exception as e:  # pragma: no cover
             print(f"bench.py: graph capture failed ({e}); launching from the host", file=sys.stderr)
-            graph, G = None, 0
+            graph = None
             torch.cuda.synchronize()
 
-    def run(n):
+    def run_k():
         if graph is not None:
-            for _ in range(n // G):
-                graph.replay()
-            n = n % G
-        run_direct(n)
-        join_all()
+            graph.replay()
+        else:
+            run_direct(K)
+            join_all()
 
-    launches_before = sum(c.tova_cache_launches() for c in caches)
-    run(max(args.warmup, 3))
-    sampler = ClockSampler(local)
+    # Warm-up, part 2: the timed unit itself, and an estimate of how often to repeat it.
+    for _ in range(2):
+        run_k()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    run_k()
+    e1.record()
+    torch.cuda.synchronize()
+    est = max(max_over_ranks(e0.elapsed_time(e1), dev), 1e-3)
+    repeats = args.repeats or max(1, int(-(-MIN_TIMED_MS // est)) + 1)
+
+    sampler = ClockSampler(torch.cuda.current_device())
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    run(args.steps)
+    for _ in range(repeats):
+        run_k()
     e1.record()
     torch.cuda.synchronize()
     clocks = sampler.stop()
@@ -356,19 +378,22 @@ def run_ours(args):
     for c in caches:
         assert c.tova_cache_read()["status"] == 0, "a kernel reported a failed check"
 
-    ms_per_step = ms / args.steps
-    value = world * B * args.steps / (ms * 1e-3)
-    gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
-    peak, peak_kind = load_peaks()
+    timed_steps = repeats * K
+    ms_per_step = ms / timed_steps
+    res = {
+        "ms": ms, "ms_per_step": ms_per_step, "timed_steps": timed_steps, "repeats": repeats,
+        "value": world * B * timed_steps / (ms * 1e-3), "gbs": step_bytes / (ms_per_step * 1e-3) / 1e9,
+        "launch": launch_mode, "layers": L, "deferred": deferred, "step_bytes": step_bytes,
+        "launches": int(round(launches_per_step * timed_steps)), "clocks": clocks, "ring": ring, "e2e": None,
+    }
 
     # end to end: host buffers in, host buffers out, through tova_decode_step_host
-    e2e = None
-    if not args.no_e2e:
+    if want_e2e:
         hq, hk, hv = (torch.from_numpy(a).to(dq.dtype).pin_memory() for a in ring)
         hout = torch.empty(B, H, D, dtype=torch.float32).pin_memory()
         hev = torch.empty(B, dtype=torch.int32).pin_memory()
-        n_e = min(args.steps, 2048)
-        for i in range(8):
+        n_e = max(K, min(2048, int(4 * MIN_TIMED_MS / ms_per_step) + 1))
+        for i in range(max(8, L)):
             caches[i % L].tova_decode_step_host(hq[i % RING], hk[i % RING], hv[i % RING], -1, hout, hev)
         if world > 1:
             dist.barrier()
@@ -379,37 +404,85 @@ def run_ours(args):
             caches[i % L].tova_decode_step_host(hq[r], hk[r], hv[r], -1, hout, hev)
         torch.cuda.synchronize()
         dt = max_over_ranks(time.perf_counter() - t0, dev)
-        e2e = {"value": world * B * n_e / dt, "unit": UNIT, "steps": n_e,
-               "h2d_bytes_per_step": int(hq[0].nbytes + hk[0].nbytes + hv[0].nbytes),
-               "d2h_bytes_per_step": int(hout.nbytes + hev.nbytes)}
+        res["e2e"] = {"value": world * B * n_e / dt, "unit": UNIT, "steps": n_e,
+                      "h2d_bytes_per_step": int(hq[0].nbytes + hk[0].nbytes + hv[0].nbytes),
+                      "d2h_bytes_per_step": int(hout.nbytes + hev.nbytes)}
+    for c in caches:
+        c.close()
+    del caches, outs, evs, graph
+    torch.cuda.empty_cache()
+    return res
+
+
+def roofline_of(w, res, peak, peak_kind):
+    return {"bound": "hbm", "achieved": res["gbs"], "peak": peak, "unit": "GB/s", "frac": res["gbs"] / peak,
+            "traffic": recorded_traffic(w, res["step_bytes"]), "peak_kind": peak_kind,
+            "frac_of_nominal_8TBs": res["gbs"] / 8000.0,
+            "note": "algorithmic bytes (K/V read + one slot written) / whole-step time (split + combine kernels)"}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2401_06104_b200 import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the decode path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    w = pick_workload(args)
+    peak, peak_kind = load_peaks()
+    res = measure(w, args, dev, world, want_e2e=not args.no_e2e)
+    L, step_bytes = res["layers"], res["step_bytes"]
+
+    # the other graded configurations, one GPU only (with several ranks all of them would be held meanwhile)
+    sweep = []
+    if world == 1 and not args.no_sweep and args.workload == DEFAULT_WORKLOAD and not args.capacity and not args.batch:
+        for name, capacity, layers in SWEEP:
+            ws = W.WORKLOADS[name].scaled(capacity=capacity)
+            r = measure(ws, args, dev, world, layers=layers)
+            sweep.append({"workload": name, "capacity": capacity, "batch": ws.batch, "bytes_per_step": r["step_bytes"],
+                          "layers_rotated": r["layers"], "ms_per_step": r["ms_per_step"], "value": r["value"],
+                          "achieved_gbs": r["gbs"], "frac": r["gbs"] / peak, "launch": r["launch"],
+                          "timed_steps": r["timed_steps"], "timed_ms": r["ms"], "clocks": r["clocks"]})
 
     if rank != 0:
         return 0
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        val, cores, sample = time_oracle(w, ring, args.cpu_seconds)
+        val, cores, sample = time_oracle(w, res["ring"], args.cpu_seconds)
         cpu = {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
 
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": storage_name(w), "data": "synthetic",
+        "timed_steps": res["timed_steps"], "repeats": res["repeats"], "timed_ms": res["ms"],
         "config": workload_config(w, {
-            "layers_rotated": L, "working_set_bytes": L * step_bytes, "l2": "inputs larger than L2" if L * step_bytes > 2 * 126e6 else "working set near or below L2 size",
-            "launch": launch_mode, "graph_steps": G, "bytes_per_step": step_bytes,
-            "policy": args.policy + (f"+{args.keep_first}" if args.keep_first else ""),
-            "eviction": "deferred to the cache's side stream, overlaps the next layer's step" if deferred
-                        else "on the caller's stream",
+            "l2": "inputs larger than L2" if min(L, args.steps) * step_bytes > 2 * 126e6
+                  else "working set near or below L2 size",
             "parallelism": "replicas only" if world > 1 else "single GPU"}),
-        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                     "traffic": recorded_traffic(w, step_bytes), "peak_kind": peak_kind,
-                     "frac_of_nominal_8TBs": gbs / 8000.0,
-                     "note": "algorithmic bytes (K/V read + one slot written) / whole-step time (split + combine kernels)"},
+        "run": {
+            "layers_rotated": L, "working_set_bytes": min(L, args.steps) * step_bytes,
+            "launch": res["launch"], "graph_steps": args.steps if res["launch"] == "cuda_graph" else 0,
+            "bytes_per_step": step_bytes, "accumulate": "fp32",
+            "policy": args.policy + (f"+{args.keep_first}" if args.keep_first else ""),
+            "eviction": "deferred to the cache's side stream, overlaps the next layer's step" if res["deferred"]
+                        else "on the caller's stream"},
+        "roofline": roofline_of(w, res, peak, peak_kind),
         "cpu_baseline": cpu,
-        "e2e": e2e,
-        "gpu_launches": launches_per_step * args.steps,
-        "clocks": clocks,
+        "e2e": res["e2e"],
+        "gpu_launches": res["launches"],
+        "clocks": res["clocks"],
+        "sweep": sweep,
     }
     print(json.dumps(line))
     if world > 1:
@@ -467,7 +540,7 @@ def run_prefill(args):
     line = {
         "metric": "tova_prefill_tokens_per_s_per_layer", "value": B * T / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
         "steps": steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": storage_name(w), "data": "synthetic",
         "config": workload_config(w, {"prompt_tokens": T, "tokens_into_free_rows": F,
                                       "route": "bulk fill + per-token steps" if bulk else "per-token steps",
                                       "l2": "a fresh cache per step; inputs larger than L2" if q.numel() * 2 > 126e6

@@ -238,6 +238,11 @@ const char* tova_strerror(int status);
  *                                min(tokens fed so far, capacity): the caller
  *                                tracks it
  *   q, k, v, pos, out, evicted_pos   as for tova_decode_step (pos >= 0)
+ *   status [1] int32 or NULL     device word that receives 0, or the code of a
+ *                                device-side check this call failed (a copy that
+ *                                did not land, an arg-min out of range); cleared
+ *                                by the call.  With NULL such failures go
+ *                                unreported: there is no handle to read them from
  *
  * Scratch need: about 4*B*H*(capacity+5) bytes of logits plus
  * B*H*(D*4+8)*ceil(capacity/chunk) bytes of partials (chunk = 32..256 rows,
@@ -247,16 +252,20 @@ const char* tova_strerror(int status);
  *
  * The call allocates nothing, on the device or through any library.  Its first
  * use on a device looks up the array's device address (cudaGetSymbolAddress)
- * and the SM count; make that first call outside any stream capture.  All calls
- * on a device share the one array, which keeps whatever the previous call left:
- * the call clears its status words itself (a memset on `cuda_stream`),
- * but two calls whose kernels overlap on the GPU - different streams, or
- * different host threads without ordering - race on it.  Issue them on one
- * stream or order them with events. */
+ * and the SM count, and the first use of each kind of shape (dtype, head_dim,
+ * query-group size, state short or long) sets launch attributes of the kernels
+ * it picks and may look up a driver entry point: make the first call on a
+ * device, and the first call of every shape, outside any stream capture.
+ * That one-time set-up is guarded, so first calls may come from several host
+ * threads.  All calls on a device share the one array, which keeps whatever the
+ * previous call left: the call clears its status words itself (a memset on
+ * `cuda_stream`), but two calls whose kernels overlap on the GPU - different
+ * streams, or different host threads without ordering - race on it.  Issue them
+ * on one stream or order them with events. */
 #define TOVA_STATIC_SCRATCH_BYTES (8u << 20)
 int tova_decode_step_static(const tova_config* cfg, void* K, void* V, int32_t* positions,
                             int32_t n_live, const void* q, const void* k, const void* v, int32_t pos,
-                            float* out, int32_t* evicted_pos, void* cuda_stream);
+                            float* out, int32_t* evicted_pos, int32_t* status, void* cuda_stream);
 
 #ifdef __cplusplus
 }

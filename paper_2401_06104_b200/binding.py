@@ -79,7 +79,7 @@ def lib() -> ctypes.CDLL:
         L.tova_cache_destroy.argtypes = [vp]
         L.tova_decode_step_static.restype = ctypes.c_int
         L.tova_decode_step_static.argtypes = [ctypes.POINTER(tova_config), vp, vp, vp, i32, vp, vp, vp,
-                                              i32, vp, vp, vp]
+                                              i32, vp, vp, vp, vp]
         L.tova_strerror.restype = ctypes.c_char_p
         L.tova_strerror.argtypes = [ctypes.c_int]
         _lib = L
@@ -205,14 +205,15 @@ class TovaCache:
 
 
 def tova_decode_step_static(cfg: tova_config, K, V, positions, n_live: int, q, k, v, pos: int, out,
-                            evicted_pos=None, stream=None) -> None:
+                            evicted_pos=None, status=None, stream=None) -> None:
     """One decode step on caller-held state tensors, using the scratch array
     built into the library instead of a workspace: for callers that may not
     allocate device memory (see include/tova.h).  K, V [B,Hkv,cap,D] and
-    positions [B,cap] are updated in place; the caller tracks n_live."""
+    positions [B,cap] are updated in place; the caller tracks n_live.  status: an
+    int32 device tensor of one element that receives 0 or a device-side check's code."""
     _check(lib().tova_decode_step_static(ctypes.byref(cfg), _p(K), _p(V), _p(positions), int(n_live),
                                          _p(q), _p(k), _p(v), int(pos), _p(out), _p(evicted_pos),
-                                         _stream(stream)), "tova_decode_step_static")
+                                         _p(status), _stream(stream)), "tova_decode_step_static")
 
 
 def to_device(x, dtype: int, device="cuda:0") -> torch.Tensor:

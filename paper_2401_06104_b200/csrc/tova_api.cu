@@ -5,10 +5,12 @@
 // there is no CPU fallback.
 #include "../../include/tova.h"
 
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <type_traits>
 
@@ -163,7 +165,7 @@ cudaError_t launch_split_f(int dev, const StepParams& p, dim3 grid, cudaStream_t
   split_launch_shape(p, grid, block);
   const size_t smem = warp_smem * block.y + cluster_partial_bytes(p, GU, D);
   auto kern = tova::tova_split_kernel<T, D, GU, GB, FUSED>;
-  static bool attr_set[64] = {};  // per instantiation and device: the attribute is per function
+  static std::atomic<bool> attr_set[64];  // per instantiation and device: the attribute is per function
   if (!attr_set[dev & 63]) {
     cudaError_t e = cudaFuncSetAttribute(
         kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -222,7 +224,7 @@ cudaError_t launch_combine_ct(int dev, const StepParams& p, cudaStream_t st, boo
   const size_t logit_bytes = p.stage_logits ? (size_t)p.H * p.cand_per_cta * sizeof(float) : 0;
   const size_t smem = combine_smem_bytes(p.H, p.n_chunks + 1, CT, row_bytes, logit_bytes);
   auto kern = tova::tova_combine_kernel<T, D, CT, MODE>;
-  static bool attr_set[64] = {};
+  static std::atomic<bool> attr_set[64];
   if (!attr_set[dev & 63]) {
     cudaError_t e =
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)COMBINE_SMEM_LIMIT);
@@ -279,7 +281,7 @@ cudaError_t launch_split_mma_t(int dev, const StepParams& p, const CUtensorMap& 
   split_launch_shape(p, grid, block);
   const size_t smem = warp_smem * block.y + 1024 + cluster_partial_bytes(p, tova::MMA_UNIT_HEADS, D);
   auto kern = tova::tova_split_mma_kernel<D, TWO, FUSED>;
-  static bool attr_set[64] = {};
+  static std::atomic<bool> attr_set[64];
   if (!attr_set[dev & 63]) {
     cudaError_t e = cudaFuncSetAttribute(
         kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -381,7 +383,7 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, boo
   pa.v_stage = c->base + c->lay.df_v;
   // Outputs-only launch: half-size CTAs once the batch would otherwise fill the
   // register files and keep the next split kernel from becoming resident early.
-  if ((long long)p.B * p.nx > 148) set_combine_threads(pa, tova::COMBINE_THREADS_SMALL);
+  if ((long long)p.B * p.nx > c->sm_count) set_combine_threads(pa, tova::COMBINE_THREADS_SMALL);
   pa.stage_logits = 0;
   e = launch_combine<T, D>(c->device, pa, st);
   if (e != cudaSuccess) return e;
@@ -467,7 +469,7 @@ void set_combine_threads(StepParams& p, int ct) {
 }
 
 // Launch geometry of one step for n live rows.
-void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows) {
+void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows, int sm_count) {
   p.B = cfg.batch; p.H = cfg.n_q_heads; p.Hkv = cfg.n_kv_heads; p.G = cfg.n_q_heads / cfg.n_kv_heads;
   p.cap = cfg.capacity;
   p.n = n;
@@ -478,10 +480,9 @@ void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows)
   // Combine CTAs per sequence (one cluster): 512-thread CTAs (two per SM)
   // while they all fit on the GPU at once, else 256-thread CTAs (four per SM).
   // Per thread: about one output quad and at most 8 logits per pass.
-  const int sm_guess = 148;
   const int cl_max = tova::COMBINE_CLUSTER_MAX;
   const long long ctas = (long long)cfg.batch * cl_max;
-  const int ct = ctas <= 2 * sm_guess ? tova::COMBINE_THREADS_LARGE : tova::COMBINE_THREADS_SMALL;
+  const int ct = ctas <= 2LL * sm_count ? tova::COMBINE_THREADS_LARGE : tova::COMBINE_THREADS_SMALL;
   const int lg = 8;
   const long long items = (long long)cfg.n_q_heads * cfg.head_dim;
   int nx = (int)((items + ct - 1) / ct);
@@ -514,7 +515,7 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
   p.last_slot = reinterpret_cast<int32_t*>(base + c->lay.last_slot);
   p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.evicted = evicted_pos; p.pos_t = pos;
   p.ld = c->lay.ld; p.pc = c->lay.pc;
-  fill_geometry(p, cfg, n, c->chunk_rows);
+  fill_geometry(p, cfg, n, c->chunk_rows, c->sm_count);
   p.scale2 = c->scale2;
   cudaError_t e;
   const bool defer = c->deferred && allow_defer;
@@ -556,7 +557,7 @@ cudaError_t launch_fill_d(tova_cache* c, const tova::FillParams& p, cudaStream_t
   if (p.out) {
     if (D == 128 && c->bulk_fill == 1) {
       constexpr size_t smem_tc = 96 * 1024 + 1024;
-      static bool configured_tc[64] = {};
+      static std::atomic<bool> configured_tc[64];
       if (c->device >= 0 && c->device < 64 && !configured_tc[c->device]) {
         e = cudaFuncSetAttribute(tova::tova_fill_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_tc);
         if (e != cudaSuccess) return e;
@@ -566,7 +567,7 @@ cudaError_t launch_fill_d(tova_cache* c, const tova::FillParams& p, cudaStream_t
       tova::tova_fill_attn_tc_kernel<<<grid, tova::FILLTC_THREADS, smem_tc, st>>>(p, c->fill_map_k, c->fill_map_v);
     } else {
       constexpr size_t smem = 4 * (size_t)tova::FILL_K_ROWS * D * 2 + 1024;
-      static bool configured[64] = {};
+      static std::atomic<bool> configured[64];
       if (c->device >= 0 && c->device < 64 && !configured[c->device]) {
         e = cudaFuncSetAttribute(tova::tova_fill_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -631,7 +632,8 @@ int encode_state_map(CUtensorMap* map, void* base, const tova_config& cfg, int b
   typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-  static encode_fn fn = nullptr;
+  static std::atomic<encode_fn> fn_cache{nullptr};
+  encode_fn fn = fn_cache.load(std::memory_order_acquire);
   if (!fn) {
     void* sym = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -639,6 +641,7 @@ int encode_state_map(CUtensorMap* map, void* base, const tova_config& cfg, int b
         qres != cudaDriverEntryPointSuccess || !sym)
       return TOVA_ERR_CUDA;
     fn = reinterpret_cast<encode_fn>(sym);
+    fn_cache.store(fn, std::memory_order_release);
   }
   const cuuint64_t rows = (cuuint64_t)cfg.batch * cfg.n_kv_heads * cfg.capacity;
   const cuuint64_t dims[2] = {(cuuint64_t)cfg.head_dim, rows};
@@ -980,11 +983,12 @@ constexpr size_t STATIC_SCRATCH_BYTES = (size_t)TOVA_STATIC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
 
 struct StaticDevice {
-  bool ready;
-  unsigned char* scratch;  // device address of g_static_scratch on this device
-  int sm_count;
+  std::atomic<bool> ready{false};
+  unsigned char* scratch = nullptr;  // device address of g_static_scratch on this device
+  int sm_count = 0;
 };
-StaticDevice g_static_dev[64] = {};
+StaticDevice g_static_dev[64];
+std::mutex g_static_setup;   // first calls from several host threads: one of them does the look-up
 
 struct StaticLayout {
   size_t logits, part_ml, part_acc, control, total;
@@ -1010,7 +1014,8 @@ StaticLayout make_static_layout(const tova_config& c, int chunk_rows) {
 
 extern "C" int tova_decode_step_static(const tova_config* cfg, void* K, void* V, int32_t* positions,
                                        int32_t n_live, const void* q, const void* k, const void* v,
-                                       int32_t pos, float* out, int32_t* evicted_pos, void* cuda_stream) {
+                                       int32_t pos, float* out, int32_t* evicted_pos, int32_t* status,
+                                       void* cuda_stream) {
   int why;
   if (!config_ok(cfg, &why)) return why;
   if (!K || !V || !positions || !q || !k || !v || !out) return TOVA_ERR_NULL;
@@ -1024,14 +1029,17 @@ extern "C" int tova_decode_step_static(const tova_config* cfg, void* K, void* V,
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return TOVA_ERR_CUDA;
   StaticDevice& sd = g_static_dev[dev];
-  if (!sd.ready) {
-    void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return TOVA_ERR_CUDA;
-    int sms = 0;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return TOVA_ERR_CUDA;
-    sd.scratch = static_cast<unsigned char*>(ptr);
-    sd.sm_count = sms;
-    sd.ready = true;
+  if (!sd.ready.load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> guard(g_static_setup);
+    if (!sd.ready.load(std::memory_order_relaxed)) {
+      void* ptr = nullptr;
+      if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return TOVA_ERR_CUDA;
+      int sms = 0;
+      if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return TOVA_ERR_CUDA;
+      sd.scratch = static_cast<unsigned char*>(ptr);
+      sd.sm_count = sms;
+      sd.ready.store(true, std::memory_order_release);
+    }
   }
 
   const int chunk_rows = pick_chunk_rows(*cfg, sd.sm_count);
@@ -1042,27 +1050,30 @@ extern "C" int tova_decode_step_static(const tova_config* cfg, void* K, void* V,
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   unsigned char* base = sd.scratch;
   const size_t B = cfg->batch;
-  // the status word must start at zero; the array keeps the previous call's contents
+  // The status word must start at zero; the array keeps the previous call's contents.  A caller that
+  // wants to see a failed device-side check passes its own word, which is cleared the same way.
   if (cudaMemsetAsync(base + lay.control, 0, B * 4 + 8, st) != cudaSuccess) return TOVA_ERR_CUDA;
+  if (status && cudaMemsetAsync(status, 0, 4, st) != cudaSuccess) return TOVA_ERR_CUDA;
 
   StepParams p{};
   p.K = K;
   p.V = V;
   p.pos = positions;
   p.len = reinterpret_cast<int32_t*>(base + lay.control);
-  p.status = reinterpret_cast<int32_t*>(base + lay.control + B * 4);
-  p.cur_pos = p.status + 1;
+  p.cur_pos = reinterpret_cast<int32_t*>(base + lay.control + B * 4) + 1;
+  p.status = status ? status : p.cur_pos - 1;
   p.logits = reinterpret_cast<float*>(base + lay.logits);
   p.part_ml = reinterpret_cast<float2*>(base + lay.part_ml);
   p.part_acc = reinterpret_cast<float*>(base + lay.part_acc);
   p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.evicted = evicted_pos; p.pos_t = pos;
   p.ld = lay.ld; p.pc = lay.pc;
-  fill_geometry(p, *cfg, n_live, chunk_rows);
+  fill_geometry(p, *cfg, n_live, chunk_rows, sd.sm_count);
   const float scale = cfg->sm_scale == 0.f ? 1.f / std::sqrt((float)cfg->head_dim) : cfg->sm_scale;
   p.scale2 = scale * 1.4426950408889634f;
 
   tova_cache shim{};  // launch_step reads the device, the tensor maps and counts launches
   shim.device = dev;
+  shim.sm_count = sd.sm_count;
   shim.use_mma = wants_mma(*cfg);
   if (shim.use_mma) {
     if ((long long)cfg->batch * cfg->n_kv_heads * cfg->capacity >= (1LL << 31)) return TOVA_ERR_BAD_SHAPE;

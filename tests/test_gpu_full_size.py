@@ -40,6 +40,96 @@ def test_full_layer_shapes(name, cap, extra, seqs, direct_fill):
           f"self {rep.self_evictions}")
 
 
+def test_32_layer_configuration_at_full_batch():
+    """Batch 64, 32 MHA heads, state of 1024 rows: 2048 eight-warp thread blocks of 128-row chunks per streaming
+    launch (the launch the benchmark's headline times).  The checker follows three of the 64 sequences."""
+    w = W.WORKLOADS["llama2_7b_full"]
+    extra = 64
+    rep = run_lockstep(w, w.capacity + extra, seqs=[0, 29, 63], block=128, check_state_every=1000, direct_fill=True)
+    assert rep.evictions == 3 * extra
+    assert rep.resyncs <= rep.evictions // 2
+    check_all_sequences(rep, w, w.capacity + extra)
+    print(f"llama2_7b_full k=1024 B=64: max_err {rep.max_err:.2e} resyncs {rep.resyncs}/{rep.evictions} "
+          f"max_rel_gap {rep.max_rel_gap:.2e} self {rep.self_evictions}")
+
+
+def test_unbounded_arm_state_of_8192_rows_at_full_batch():
+    """The 8192-token context held whole at batch 64: 64 chunks per head, more than a cluster merges, so every
+    streaming warp is its own thread block and the partials go through global memory (131072 blocks per launch).
+    The state fills without any deletion; the last steps run on the full state and drop rows.  Tokens repeat with
+    period 512 (see run_lockstep), so the lowest average is shared by 16 rows and the lowest slot must win."""
+    w = W.WORKLOADS["llama2_7b_full"].scaled(capacity=8192)
+    extra = 6
+    rep = run_lockstep(w, w.capacity + extra, seqs=[1, 62], block=128, check_state_every=1000, direct_fill=True,
+                       period=512)
+    assert rep.evictions == 2 * extra
+    check_all_sequences(rep, w, w.capacity + extra)
+    print(f"llama2_7b_full k=8192 B=64: max_err {rep.max_err:.2e} resyncs {rep.resyncs}/{rep.evictions} "
+          f"max_rel_gap {rep.max_rel_gap:.2e}")
+
+
+def test_long_stream_of_70000_tokens():
+    """The whole long-stream configuration on the GPU: 4096 prompt tokens and 65,904 decode tokens through a state
+    of 4096 rows, all four sequences.  The checker cannot follow 70,000 tokens (minutes per thousand at this
+    size), so it joins at checkpoints: there its state is written from the GENERATOR's tokens at the positions the
+    GPU's slot table holds (after checking that the GPU's cached rows are bit for bit those tokens), and the next 32
+    tokens are compared token by token - dropped positions exact, outputs within tolerance.  Over the whole stream
+    an integer replay of the dropped-position log must reproduce the final slot table, and no kernel may have
+    reported a failed check."""
+    import torch
+    import paper_2401_06104_b200 as tova
+    from oracle.tova_oracle import OracleCache
+    w = W.WORKLOADS["yi_6b_long"]
+    total = w.prompt + w.decode
+    assert total == 70000 and w.capacity == 4096
+    cache = make_cache(w)
+    checkpoints = [4096, 4128, 9001, 20000, 33333, 47111, 61000, total - 32]
+    span = 32
+    logs = []
+    pos = 0
+    worst, resyncs, evictions = 0.0, 0, 0
+    for cp in checkpoints:
+        while pos < cp:                                   # plain GPU run up to the checkpoint
+            T = min(1024, cp - pos)
+            q, k, v = W.tokens(w, pos, T)
+            dq, dk, dv = (tova.to_device(a, w.dtype) for a in (q, k, v))
+            ev = torch.empty(T, w.batch, dtype=torch.int32, device="cuda:0")
+            cache.tova_prefill(dq, dk, dv, T, pos, None, ev)
+            torch.cuda.synchronize()
+            logs.append(ev.cpu().numpy())
+            pos += T
+        st = cache.tova_cache_read(want_kv=True)
+        assert st["status"] == 0 and np.all(st["len"].numpy() == w.capacity)
+        held = st["positions"].numpy()
+        orc = OracleCache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, precision="f32")
+        for p_held in np.unique(held):
+            _, k1, v1 = W.token(w, int(p_held))
+            for b, s in zip(*np.nonzero(held == p_held)):
+                orc.K[b, :, s] = k1[b]
+                orc.V[b, :, s] = v1[b]
+        assert np.array_equal(st["K"].numpy(), orc.K) and np.array_equal(st["V"].numpy(), orc.V), cp
+        orc.pos[:] = held
+        orc.len[:] = w.capacity
+        rep = run_lockstep(w, span, cache=cache, oracle=orc, first_pos=pos, block=span)
+        logs.extend(rep.evicted_log)
+        pos += span
+        worst = max(worst, rep.max_err)
+        resyncs += rep.resyncs
+        evictions += rep.evictions
+    assert pos == total
+    log = np.concatenate(logs, axis=0)
+    assert log.shape == (total, w.batch)
+    held = replay_slot_table(log, w.capacity)
+    st = cache.tova_cache_read()
+    assert st["status"] == 0
+    for b in range(w.batch):
+        live = st["positions"].numpy()[b].tolist()
+        assert len(set(live)) == w.capacity and set(live) == held[b]
+        assert 0 in held[b]                               # the sink (position 0) is still held, as in Section 7.3
+    assert evictions == w.batch * span * len(checkpoints)
+    print(f"yi_6b_long 70000 tokens: max_err {worst:.2e} resyncs {resyncs}/{evictions}")
+
+
 @pytest.mark.parametrize("name,cap", [("llama2_7b_layer", 512), ("mistral_7b_gqa", 1024), ("yi_6b_long", 4096)])
 def test_full_shapes_as_the_benchmark_launches_them(name, cap):
     """Deferred eviction, two layer caches taking turns, steps replayed from a CUDA

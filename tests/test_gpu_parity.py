@@ -10,7 +10,7 @@ import torch
 import paper_2401_06104_b200 as tova
 from paper_2401_06104_b200 import workloads as W
 from oracle.tova_oracle import OracleCache
-from parity import gpu_block, make_cache, out_tol, replay_slot_table, run_lockstep
+from parity import gpu_block, hand_tol, make_cache, out_tol, replay_slot_table, run_lockstep
 from test_oracle_pins import parse_golden
 
 pytestmark = pytest.mark.gpu
@@ -38,7 +38,7 @@ def test_hand_worked_example_on_gpu():
         assert int(ev.item()) == e, t
         assert st["positions"][0].tolist() == rows_after, t
         o = out.cpu().numpy()
-        assert abs(o[0, 0, 0] - float(o0)) < 1e-4 and abs(o[0, 1, 0] - float(o1)) < 1e-4
+        assert abs(o[0, 0, 0] - float(o0)) <= hand_tol(float(o0)) and abs(o[0, 1, 0] - float(o1)) <= hand_tol(float(o1))
         assert np.all(o[0, :, 1:] == 0)
         assert st["status"] == 0 and c.tova_cache_len() == min(t + 1, 3)
 
@@ -343,7 +343,7 @@ def test_policy_hand_worked_traces_on_gpu():
             assert int(ev.item()) == e, (policy, keep, t)
             assert st["positions"][0].tolist() == rows_after, (policy, keep, t)
             o = out.cpu().numpy()
-            assert abs(o[0, 0, 0] - float(o0)) < 1e-4 and abs(o[0, 1, 0] - float(o1)) < 1e-4
+            assert abs(o[0, 0, 0] - float(o0)) <= hand_tol(float(o0)) and abs(o[0, 1, 0] - float(o1)) <= hand_tol(float(o1))
 
 
 def test_policy_argument_errors():

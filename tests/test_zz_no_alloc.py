@@ -42,13 +42,16 @@ def run_both(w, n_tokens):
     o_st = torch.empty_like(o_ref)
     e_ref = torch.empty(w.batch, dtype=torch.int32, device=dev)
     e_st = torch.empty_like(e_ref)
+    status = torch.full((1,), 77, dtype=torch.int32, device=dev)
     tol = 2e-3 if w.dtype == W.DTYPE_BF16 else 1e-5
     n_live = 0
     for t in range(n_tokens):
         ref.tova_decode_step(dq[t], dk[t], dv[t], t, o_ref, e_ref)
-        tova.tova_decode_step_static(cfg, K, V, P, n_live, dq[t], dk[t], dv[t], t, o_st, e_st)
+        tova.tova_decode_step_static(cfg, K, V, P, n_live, dq[t], dk[t], dv[t], t, o_st, e_st,
+                                     status if t % 2 == 0 else None)
         n_live = min(n_live + 1, w.capacity)
         torch.cuda.synchronize()
+        assert int(status.item()) == 0, t
         assert float((o_ref - o_st).abs().max()) <= tol, t
         assert torch.equal(e_ref, e_st), t
     st = ref.tova_cache_read(want_kv=True)
@@ -69,9 +72,19 @@ def test_static_step_again_with_another_shape_on_the_same_array():
     run_both(w, 33 + 40)
 
 
+def test_static_step_on_the_tensor_core_kernel_with_caller_held_state():
+    """Query groups of 4 and more (bf16) take the tensor-core streaming kernel, which reads the state through
+    tiled tensor maps: the call encodes them over the caller's K and V every time.  Capacity 70 is not a multiple
+    of the 16-row tile, and the run crosses from filling to evicting."""
+    w = W.WORKLOADS["mistral_7b_gqa"].scaled(batch=3, n_q_heads=8, n_kv_heads=2, capacity=70)
+    run_both(w, 70 + 50)
+    w = W.WORKLOADS["yi_6b_long"].scaled(batch=1, n_q_heads=16, n_kv_heads=1, capacity=300)   # 16 heads: two N tiles
+    run_both(w, 300 + 30)
+
+
 def test_static_step_refuses_shapes_beyond_its_array():
     cfg = tova.tova_config(64, 32, 32, 128, 4096, tova.TOVA_DTYPE_BF16, 0.0, 1)
     one = ctypes.c_void_p(256)
-    rc = tova.lib().tova_decode_step_static(ctypes.byref(cfg), one, one, one, 0, one, one, one, 0, one, None, None)
+    rc = tova.lib().tova_decode_step_static(ctypes.byref(cfg), one, one, one, 0, one, one, one, 0, one, None, None, None)
     assert rc == -9
     assert "8 MiB" in tova.strerror(rc)
