@@ -35,8 +35,24 @@
  *     part;
  *   - "+i" (Window+i, TOVA+i): rows holding the first i positions (0..i-1) are
  *     never deleted; the policy picks among the others.
- * The layer output does not depend on the policy (it is computed before the
- * deletion).
+ *   - TOVA-head (Section 4: the policy "computes the attention scores of each
+ *     head separately, and can thus retain different tokens at different
+ *     heads"; appendix ablation row TOVA-head): every head keeps its own rows
+ *     and drops the row with ITS lowest weight;
+ *   - H2O, layer-wise and head-wise (Section 4.1): a window of the most recent
+ *     tokens is always kept; among the older rows the one whose attention
+ *     weight, summed over all the steps it has been in the state, is lowest
+ *     goes.  The number of non-window rows is half the multi-state size unless
+ *     the caller says otherwise.
+ * Readings for these (the paper gives one paragraph each): a "head" that owns
+ * rows is a KV head, and its score for a row is the mean weight of the query
+ * heads that read it (for multi-head attention: the head's own weight); a
+ * row's accumulated score starts with the weight it received as the new token
+ * and grows by its weight at every later step, before the victim of that step
+ * is chosen; window membership is "fewer than `recent` positions behind the new
+ * token"; ties go to the lowest row index.
+ * The layer output of the current step does not depend on the policy (it is
+ * computed before the deletion).
  *
  * Precision: every operation is carried out in REAL (float for the parity
  * checker, double for the reference the float build is itself checked with).
@@ -50,6 +66,11 @@
  * retained positions (the first i and the most recent k-i), hand-worked
  * traces of the 3-row example, "+0" equal to the plain policy, and the
  * invariant that a protected position is never reported as dropped.
+ * TOVA-head and H2O: per-head and accumulated-score restatements over the full
+ * token history in double (order-preserving lists), hand-worked traces of the
+ * 3-row example in exact arithmetic, "one head = the layer policy", H2O with
+ * a window as large as the state = Window, accumulated scores = column sums
+ * of the textbook causal soft-max matrix while nothing is dropped.
  */
 #include <math.h>
 #include <stdlib.h>
@@ -64,6 +85,45 @@
 #endif
 
 static REAL real_exp(REAL x) { return sizeof(REAL) == 4 ? (REAL)expf((float)x) : (REAL)exp((double)x); }
+
+/*
+ * Attention of the new query over the appended state, for one sequence:
+ * weights (Eq. 4) into work[h][0..n] (row n = the new token) and the layer
+ * output over all n+1 rows (Eq. 7) into out.  work is [H][cap+1].
+ */
+static void attend(int H, int Hkv, int D, int cap, REAL scale, int n,
+                   const REAL *K, const REAL *V, const REAL *q, const REAL *k_new, const REAL *v_new,
+                   REAL *out, REAL *work)
+{
+    const int m = n + 1;
+    const int G = H / Hkv;
+    const int ld = cap + 1;
+    for (int h = 0; h < H; ++h) {
+        const int kv = h / G;
+        REAL *p = work + (size_t)h * ld;
+        for (int j = 0; j < m; ++j) {
+            const REAL *krow = (j < n) ? K + ((size_t)kv * cap + j) * D : k_new + (size_t)kv * D;
+            REAL s = 0;
+            for (int d = 0; d < D; ++d) s += q[(size_t)h * D + d] * krow[d];
+            p[j] = scale * s;
+        }
+        REAL mx = p[0];
+        for (int j = 1; j < m; ++j) if (p[j] > mx) mx = p[j];
+        REAL l = 0;
+        for (int j = 0; j < m; ++j) { p[j] = real_exp(p[j] - mx); l += p[j]; }
+        for (int j = 0; j < m; ++j) p[j] = p[j] / l;
+        /* Layer output before any row is dropped (Eq. 7). */
+        for (int d = 0; d < D; ++d) {
+            REAL o = 0;
+            for (int j = 0; j < m; ++j) {
+                const REAL *vrow = (j < n) ? V + ((size_t)kv * cap + j) * D : v_new + (size_t)kv * D;
+                o += p[j] * vrow[d];
+            }
+            out[(size_t)h * D + d] = o;
+        }
+    }
+
+}
 
 /*
  * One token for one sequence.
@@ -97,34 +157,9 @@ static void step_one(int H, int Hkv, int D, int cap, REAL scale, int policy, int
 {
     const int n = *len;          /* rows before the append */
     const int m = n + 1;         /* rows after the append (Eq. 6) */
-    const int G = H / Hkv;
     const int ld = cap + 1;
 
-    /* Attention weights of the new query over the appended state (Eq. 4). */
-    for (int h = 0; h < H; ++h) {
-        const int kv = h / G;
-        REAL *p = work + (size_t)h * ld;
-        for (int j = 0; j < m; ++j) {
-            const REAL *krow = (j < n) ? K + ((size_t)kv * cap + j) * D : k_new + (size_t)kv * D;
-            REAL s = 0;
-            for (int d = 0; d < D; ++d) s += q[(size_t)h * D + d] * krow[d];
-            p[j] = scale * s;
-        }
-        REAL mx = p[0];
-        for (int j = 1; j < m; ++j) if (p[j] > mx) mx = p[j];
-        REAL l = 0;
-        for (int j = 0; j < m; ++j) { p[j] = real_exp(p[j] - mx); l += p[j]; }
-        for (int j = 0; j < m; ++j) p[j] = p[j] / l;
-        /* Layer output before any row is dropped (Eq. 7). */
-        for (int d = 0; d < D; ++d) {
-            REAL o = 0;
-            for (int j = 0; j < m; ++j) {
-                const REAL *vrow = (j < n) ? V + ((size_t)kv * cap + j) * D : v_new + (size_t)kv * D;
-                o += p[j] * vrow[d];
-            }
-            out[(size_t)h * D + d] = o;
-        }
-    }
+    attend(H, Hkv, D, cap, scale, n, K, V, q, k_new, v_new, out, work);
 
     *gap = 0;
     if (m <= cap) {              /* Algorithm 1: num_kv <= cache_max_size -> keep all */
@@ -236,6 +271,146 @@ int tova_oracle_step(int B, int H, int Hkv, int D, int cap, REAL scale,
 {
     return tova_oracle_step_policy(B, H, Hkv, D, cap, scale, POLICY_TOVA, 0, len, pos, K, V, q, k_new, v_new,
                                    pos_t, forced, out, evicted_pos, victim, argmin, gap, mean_out, nthreads);
+}
+
+/* ------------------------------------------------------------------------
+ * Policies in which rows are owned per unit: a unit is the whole layer (one
+ * unit, U = 1) or one KV head (U = Hkv).  TOVA-head, H2O-layer, H2O-head.
+ * ------------------------------------------------------------------------ */
+#define POLICY_TOVA_HEAD 2
+#define POLICY_H2O_LAYER 3
+#define POLICY_H2O_HEAD 4
+
+/*
+ * One token for one sequence under a unit policy.
+ *   len      in/out  live rows n, the same for every unit
+ *   pos      in/out  [U][cap]  position held by each row of each unit, -1 if unused
+ *   acc      in/out  [U][cap]  H2O: accumulated score of each row (unused otherwise)
+ *   K, V     in/out  [Hkv][cap][D]  (row j of KV head kv belongs to unit kv, or to the one unit)
+ *   recent   H2O: candidates fewer than `recent` positions behind the new token are never dropped
+ *   forced   [U] or NULL: candidate to drop instead of the unit's arg-min (-1: none)
+ *   evicted_pos, victim, argmin, gap   [U], as in step_one; gap is measured in the
+ *            quantity the policy minimises (weight, or accumulated score)
+ *   score_out [U][cap+1] or NULL: that quantity for every candidate
+ *   work     scratch [H+1][cap+1]
+ */
+static void step_units(int H, int Hkv, int D, int cap, REAL scale, int policy, int recent,
+                       int *len, int *pos, REAL *acc, REAL *K, REAL *V,
+                       const REAL *q, const REAL *k_new, const REAL *v_new,
+                       int pos_t, const int *forced,
+                       REAL *out, int *evicted_pos, int *victim, int *argmin, REAL *gap,
+                       REAL *score_out, REAL *work)
+{
+    const int n = *len;
+    const int m = n + 1;
+    const int G = H / Hkv;
+    const int ld = cap + 1;
+    const int U = (policy == POLICY_H2O_LAYER) ? 1 : Hkv;
+    const int h2o = (policy == POLICY_H2O_LAYER || policy == POLICY_H2O_HEAD);
+
+    attend(H, Hkv, D, cap, scale, n, K, V, q, k_new, v_new, out, work);
+
+    REAL *key = work + (size_t)H * ld;          /* what the unit minimises, per candidate */
+    for (int u = 0; u < U; ++u) {
+        const int h0 = (U == 1) ? 0 : u * G;    /* query heads that read this unit's rows */
+        const int nh = (U == 1) ? H : G;
+        const int kv0 = (U == 1) ? 0 : u, kv1 = (U == 1) ? Hkv : u + 1;
+        int *upos = pos + (size_t)u * cap;
+        REAL *uacc = acc + (size_t)u * cap;
+        /* the unit's weight on every candidate: mean over its query heads */
+        for (int j = 0; j < m; ++j) {
+            REAL a = 0;
+            for (int h = h0; h < h0 + nh; ++h) a += work[(size_t)h * ld + j];
+            key[j] = a / (REAL)nh;
+        }
+        if (h2o) {                              /* scores accumulate over the steps (Section 4.1) */
+            for (int j = 0; j < n; ++j) { uacc[j] += key[j]; key[j] = uacc[j]; }
+            /* key[n]: the new token's score so far is its weight at this step */
+        }
+        if (score_out) {
+            for (int j = 0; j < ld; ++j) score_out[(size_t)u * ld + j] = (j < m) ? key[j] : 0;
+        }
+        gap[u] = 0;
+        if (m <= cap) {                         /* g(t) = min(t, k): keep all */
+            for (int kv = kv0; kv < kv1; ++kv) {
+                memcpy(K + ((size_t)kv * cap + n) * D, k_new + (size_t)kv * D, sizeof(REAL) * D);
+                memcpy(V + ((size_t)kv * cap + n) * D, v_new + (size_t)kv * D, sizeof(REAL) * D);
+            }
+            upos[n] = pos_t;
+            if (h2o) uacc[n] = key[n];
+            evicted_pos[u] = -1; victim[u] = -1; argmin[u] = -1;
+            continue;
+        }
+        int jmin = -1;
+        for (int j = 0; j < m; ++j) {
+            const int pj = (j < n) ? upos[j] : pos_t;
+            if (h2o && pos_t - pj < recent) continue;   /* inside the recent window */
+            if (jmin < 0 || key[j] < key[jmin]) jmin = j;
+        }
+        if (jmin < 0) jmin = n;
+        int drop = jmin;
+        argmin[u] = jmin;
+        if (forced && forced[u] >= 0 && forced[u] < m) {
+            drop = forced[u];
+            const int pd = (drop < n) ? upos[drop] : pos_t;
+            if (h2o && pos_t - pd < recent && drop != jmin) gap[u] = (REAL)1e30;
+            else gap[u] = key[drop] - key[jmin];
+        }
+        victim[u] = drop;
+        if (drop < cap) {
+            evicted_pos[u] = upos[drop];
+            for (int kv = kv0; kv < kv1; ++kv) {
+                memcpy(K + ((size_t)kv * cap + drop) * D, k_new + (size_t)kv * D, sizeof(REAL) * D);
+                memcpy(V + ((size_t)kv * cap + drop) * D, v_new + (size_t)kv * D, sizeof(REAL) * D);
+            }
+            upos[drop] = pos_t;
+            if (h2o) uacc[drop] = key[n];
+        } else {
+            evicted_pos[u] = pos_t;
+        }
+    }
+    if (m <= cap) *len = m;
+}
+
+/*
+ * Batch wrapper of step_units.  U = 1 for POLICY_H2O_LAYER, Hkv otherwise.
+ * Layouts: len [B], pos [B][U][cap], acc [B][U][cap], K,V [B][Hkv][cap][D],
+ * forced/evicted_pos/victim/argmin/gap [B][U] (forced may be NULL),
+ * score_out [B][U][cap+1] or NULL.  Returns 0, or -1 on a bad argument.
+ */
+int tova_oracle_step_units(int B, int H, int Hkv, int D, int cap, REAL scale, int policy, int recent,
+                           int *len, int *pos, REAL *acc, REAL *K, REAL *V,
+                           const REAL *q, const REAL *k_new, const REAL *v_new,
+                           int pos_t, const int *forced,
+                           REAL *out, int *evicted_pos, int *victim, int *argmin, REAL *gap,
+                           REAL *score_out, int nthreads)
+{
+    if (B < 1 || H < 1 || Hkv < 1 || D < 1 || cap < 1 || H % Hkv != 0) return -1;
+    if (policy != POLICY_TOVA_HEAD && policy != POLICY_H2O_LAYER && policy != POLICY_H2O_HEAD) return -1;
+    const int h2o = policy != POLICY_TOVA_HEAD;
+    if (h2o && (recent < 1 || recent > cap)) return -1;
+    const size_t ld = (size_t)cap + 1;
+    const size_t U = (policy == POLICY_H2O_LAYER) ? 1 : (size_t)Hkv;
+    if (nthreads < 1) nthreads = 1;
+    int bad = 0;
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(nthreads) schedule(static)
+#endif
+    for (int b = 0; b < B; ++b) {
+        REAL *work = (REAL *)malloc(sizeof(REAL) * (size_t)(H + 1) * ld);
+        if (!work) { bad = 1; continue; }
+        if (len[b] < 0 || len[b] > cap) { bad = 1; free(work); continue; }
+        step_units(H, Hkv, D, cap, scale, policy, recent,
+                   len + b, pos + (size_t)b * U * cap, acc + (size_t)b * U * cap,
+                   K + (size_t)b * Hkv * cap * D, V + (size_t)b * Hkv * cap * D,
+                   q + (size_t)b * H * D, k_new + (size_t)b * Hkv * D, v_new + (size_t)b * Hkv * D,
+                   pos_t, forced ? forced + (size_t)b * U : NULL,
+                   out + (size_t)b * H * D, evicted_pos + (size_t)b * U, victim + (size_t)b * U,
+                   argmin + (size_t)b * U, gap + (size_t)b * U,
+                   score_out ? score_out + (size_t)b * U * ld : NULL, work);
+        free(work);
+    }
+    return bad ? -1 : 0;
 }
 
 int tova_oracle_real_bytes(void) { return (int)sizeof(REAL); }

@@ -39,6 +39,7 @@ def _lib(precision: str):
         lib = ctypes.CDLL(os.path.join(_HERE, f"libtova_oracle_{tag}.so"))
         lib.tova_oracle_step.restype = ctypes.c_int
         lib.tova_oracle_step_policy.restype = ctypes.c_int
+        lib.tova_oracle_step_units.restype = ctypes.c_int
         lib.tova_oracle_real_bytes.restype = ctypes.c_int
         lib.tova_oracle_max_threads.restype = ctypes.c_int
         _LIBS[precision] = lib
@@ -108,3 +109,58 @@ class OracleCache:
         if rc != 0:
             raise RuntimeError("tova_oracle_step rejected its arguments")
         return out, ev, victim, argmin, gap, mean
+
+
+UNIT_POLICIES = {"tova_head": 2, "h2o_layer": 3, "h2o_head": 4}
+
+
+class OracleUnitsCache:
+    """Bounded multi-state under the policies that own rows per unit: TOVA-head
+    (Section 4, appendix ablation), H2O layer-wise and head-wise (Section 4.1).
+    A unit is the layer (h2o_layer: U = 1) or one KV head (U = n_kv_heads)."""
+
+    def __init__(self, batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int, capacity: int,
+                 policy: str, recent: int = 0, sm_scale: float = 0.0, precision: str = "f32",
+                 threads: Optional[int] = None):
+        if n_q_heads % n_kv_heads:
+            raise ValueError("n_q_heads must be a multiple of n_kv_heads")
+        self.B, self.H, self.Hkv, self.D, self.cap = batch, n_q_heads, n_kv_heads, head_dim, capacity
+        self.scale = float(sm_scale) if sm_scale else 1.0 / float(np.sqrt(head_dim))
+        self.real = np.float32 if precision == "f32" else np.float64
+        self.creal = ctypes.c_float if precision == "f32" else ctypes.c_double
+        self.lib = _lib(precision)
+        self.threads = threads or host_threads()
+        self.policy = UNIT_POLICIES[policy]
+        self.U = 1 if policy == "h2o_layer" else n_kv_heads
+        # H2O: the non-window rows are half the multi-state size unless told otherwise (Section 4.1)
+        self.recent = int(recent) if recent else capacity - capacity // 2
+        self.len = np.zeros(batch, np.int32)
+        self.pos = np.full((batch, self.U, capacity), -1, np.int32)
+        self.acc = np.zeros((batch, self.U, capacity), self.real)
+        self.K = np.zeros((batch, n_kv_heads, capacity, head_dim), self.real)
+        self.V = np.zeros_like(self.K)
+
+    def step(self, q, k_new, v_new, pos_t: int, forced=None, want_score: bool = False):
+        """Returns (out [B,H,D], evicted_pos [B,U], victim [B,U], argmin [B,U], gap [B,U],
+        score [B,U,cap+1] or None)."""
+        B, H, Hkv, D, cap, U = self.B, self.H, self.Hkv, self.D, self.cap, self.U
+        q = np.ascontiguousarray(q, self.real).reshape(B, H, D)
+        k_new = np.ascontiguousarray(k_new, self.real).reshape(B, Hkv, D)
+        v_new = np.ascontiguousarray(v_new, self.real).reshape(B, Hkv, D)
+        out = np.empty((B, H, D), self.real)
+        ev = np.empty((B, U), np.int32)
+        victim = np.empty((B, U), np.int32)
+        argmin = np.empty((B, U), np.int32)
+        gap = np.zeros((B, U), self.real)
+        score = np.zeros((B, U, cap + 1), self.real) if want_score else None
+        f = None if forced is None else np.ascontiguousarray(forced, np.int32).reshape(B, U)
+        rc = self.lib.tova_oracle_step_units(
+            ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D),
+            ctypes.c_int(cap), self.creal(self.scale), ctypes.c_int(self.policy), ctypes.c_int(self.recent),
+            _ptr(self.len), _ptr(self.pos), _ptr(self.acc), _ptr(self.K), _ptr(self.V),
+            _ptr(q), _ptr(k_new), _ptr(v_new), ctypes.c_int(int(pos_t)), _ptr(f),
+            _ptr(out), _ptr(ev), _ptr(victim), _ptr(argmin), _ptr(gap), _ptr(score),
+            ctypes.c_int(self.threads))
+        if rc != 0:
+            raise RuntimeError("tova_oracle_step_units rejected its arguments")
+        return out, ev, victim, argmin, gap, score
