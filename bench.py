@@ -50,9 +50,10 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="independent layer caches to rotate over (0 = auto)")
     ap.add_argument("--chunk-rows", type=int, default=0)
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of CUDA graphs")
-    ap.add_argument("--policy", choices=["tova", "window"], default="tova",
+    ap.add_argument("--policy", choices=["tova", "window", "tova_head", "h2o_layer", "h2o_head"], default="tova",
                     help="which row is dropped once the state is over capacity")
-    ap.add_argument("--keep-first", type=int, default=0, help="the +i of Window+i / TOVA+i")
+    ap.add_argument("--keep-first", type=int, default=0,
+                    help="the +i of Window+i / TOVA+i; under H2O the size of the recent window (0 = half the state)")
     ap.add_argument("--no-fused-merge", action="store_true",
                     help="merge the chunk partials through global memory even where a cluster could")
     ap.add_argument("--deferred", action="store_true", help="force deferred eviction on")
@@ -208,12 +209,16 @@ def run_reference(args):
 # ----------------------------------------------------------------------------
 # the CUDA path
 # ----------------------------------------------------------------------------
+# Sources of the streaming (split) kernels, the ones the recorded DRAM counters describe.
+SPLIT_KERNEL_SOURCES = ("tova_device.cuh", "tova_kernels.cuh", "tova_split_mma.cuh")
+
+
 def kernel_digest() -> str:
-    """Hash of the kernel sources: DRAM counters in profiles/ apply to one digest only."""
+    """Hash of the streaming kernels' sources: DRAM counters in profiles/ apply to one digest only."""
     import hashlib
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_2401_06104_b200", "csrc")
-    for f in sorted(os.listdir(d)):
+    for f in SPLIT_KERNEL_SOURCES:
         with open(os.path.join(d, f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -279,11 +284,12 @@ def measure(w, args, dev, world, layers=0, want_e2e=False):
         if args.no_fused_merge:
             c.tova_cache_set_fused_merge(False)
         if args.policy != "tova" or args.keep_first:
-            c.tova_cache_set_policy(tova.TOVA_POLICY_WINDOW if args.policy == "window" else tova.TOVA_POLICY_TOVA,
-                                    args.keep_first)
+            c.tova_cache_set_policy({"tova": tova.TOVA_POLICY_TOVA, "window": tova.TOVA_POLICY_WINDOW,
+                                     "tova_head": tova.TOVA_POLICY_TOVA_HEAD, "h2o_layer": tova.TOVA_POLICY_H2O_LAYER,
+                                     "h2o_head": tova.TOVA_POLICY_H2O_HEAD}[args.policy], args.keep_first)
         caches.append(c)
     outs = torch.empty(L, B, H, D, dtype=torch.float32, device=dev)
-    evs = torch.empty(L, B, dtype=torch.int32, device=dev)
+    evs = torch.empty(L, B, caches[0].tova_cache_units(), dtype=torch.int32, device=dev)
 
     # steady state: fill every layer past its capacity (positions from the device counter)
     for l, c in enumerate(caches):
@@ -391,7 +397,7 @@ def measure(w, args, dev, world, layers=0, want_e2e=False):
     if want_e2e:
         hq, hk, hv = (torch.from_numpy(a).to(dq.dtype).pin_memory() for a in ring)
         hout = torch.empty(B, H, D, dtype=torch.float32).pin_memory()
-        hev = torch.empty(B, dtype=torch.int32).pin_memory()
+        hev = torch.empty(B, evs.shape[2], dtype=torch.int32).pin_memory()
         n_e = max(K, min(2048, int(4 * MIN_TIMED_MS / ms_per_step) + 1))
         for i in range(max(8, L)):
             caches[i % L].tova_decode_step_host(hq[i % RING], hk[i % RING], hv[i % RING], -1, hout, hev)

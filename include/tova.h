@@ -166,23 +166,49 @@ int tova_cache_join(tova_cache* c, void* cuda_stream);
  * not depend on it beyond floating-point summation order. */
 int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows);
 
-/* Other compression policies of the paper, on the same kernels (only the
- * choice of the row to drop changes; the attention output never depends on
- * it):
- *   policy TOVA_POLICY_TOVA (default)  the row with the lowest head-averaged
- *          attention weight goes (Section 4, Algorithm 1);
- *   policy TOVA_POLICY_WINDOW          first in, first out: the row holding the
- *          earliest position goes (Section 4.1, "Window");
- *   keep_first = i >= 0                rows holding positions 0..i-1 are never
- *          dropped: Window+i (Section 4.1) and TOVA+i (appendix ablation).
- * Allowed only while the state is empty (before the first token) and with
- * keep_first < capacity, else TOVA_ERR_BAD_SHAPE; an unknown policy gives
- * TOVA_ERR_UNSUPPORTED.  Positions passed to the step calls must be >= 0 and
- * distinct for these policies to mean what the paper describes; ties go to the
- * lowest slot as everywhere.  Not available through tova_decode_step_static. */
+/* Other compression policies of the paper, on the same streaming kernels (only
+ * the choice of the row to drop changes; the attention output of a step never
+ * depends on it):
+ *   TOVA_POLICY_TOVA (default)   the row with the lowest head-averaged attention
+ *          weight goes (Section 4, Algorithm 1);
+ *   TOVA_POLICY_WINDOW           first in, first out: the row holding the earliest
+ *          position goes (Section 4.1, "Window");
+ *     for these two, arg = i >= 0: rows holding positions 0..i-1 are never dropped:
+ *          Window+i (Section 4.1) and TOVA+i (appendix ablation); i < capacity;
+ *   TOVA_POLICY_TOVA_HEAD        every head drops the row with ITS lowest weight, so
+ *          heads come to hold different tokens (Section 4; appendix ablation,
+ *          "TOVA-head"); arg must be 0;
+ *   TOVA_POLICY_H2O_LAYER, TOVA_POLICY_H2O_HEAD   a window of the most recent tokens
+ *          always stays; among the older rows the one whose attention weight, summed
+ *          over all the steps it has spent in the state, is lowest goes (Section 4.1,
+ *          "H2O"), with weights averaged over the layer's heads or per head;
+ *          arg = size of the recent window, 1..capacity, or 0 for capacity minus
+ *          half the capacity (the paper's setting: half the state for non-window rows).
+ * Under grouped-query attention the "head" that owns rows is a KV head, scored by
+ * the mean weight of the query heads that read it.  For the head-wise policies
+ * evicted_pos of the step calls is [B,Hkv] ([T,B,Hkv] for tova_prefill) and
+ * tova_cache_read returns positions as [B,Hkv,capacity]: one slot table per KV head.
+ * Allowed only while the state is empty (before the first token), else
+ * TOVA_ERR_BAD_SHAPE; an unknown policy gives TOVA_ERR_UNSUPPORTED.  Positions
+ * passed to the step calls must be >= 0, distinct and increasing for Window, "+i"
+ * and H2O to mean what the paper describes; ties go to the lowest slot as
+ * everywhere.  Head-wise and H2O policies process prompts token by token and
+ * ignore deferred eviction.  Not available through tova_decode_step_static. */
 #define TOVA_POLICY_TOVA 0
 #define TOVA_POLICY_WINDOW 1
-int tova_cache_set_policy(tova_cache* c, int32_t policy, int32_t keep_first);
+#define TOVA_POLICY_TOVA_HEAD 2
+#define TOVA_POLICY_H2O_LAYER 3
+#define TOVA_POLICY_H2O_HEAD 4
+int tova_cache_set_policy(tova_cache* c, int32_t policy, int32_t arg);
+
+/* H2O policies: copy out the accumulated attention weight of every slot
+ * (Section 4.1), scores [B,U,capacity] fp32 on the DEVICE, U = 1 (layer-wise) or
+ * Hkv (head-wise); entries of unused slots are 0.  TOVA_ERR_UNSUPPORTED under
+ * any other policy. */
+int tova_cache_read_scores(const tova_cache* c, float* scores, void* cuda_stream);
+
+/* Slot tables this cache keeps per sequence: Hkv under a head-wise policy, else 1. */
+int32_t tova_cache_units(const tova_cache* c);
 
 /* Tuning: where the per-chunk partial results of a head are merged into the
  * attention output (Eq. 7 evaluated chunk by chunk).  on (default): when the

@@ -18,6 +18,9 @@ TOVA_DTYPE_FP32 = 0
 TOVA_DTYPE_BF16 = 1
 TOVA_POLICY_TOVA = 0
 TOVA_POLICY_WINDOW = 1
+TOVA_POLICY_TOVA_HEAD = 2
+TOVA_POLICY_H2O_LAYER = 3
+TOVA_POLICY_H2O_HEAD = 4
 TOVA_POS_AUTO = -1       # "the previous token's position + 1"
 
 
@@ -63,6 +66,10 @@ def lib() -> ctypes.CDLL:
         L.tova_cache_set_chunk_rows.argtypes = [vp, i32]
         L.tova_cache_set_policy.restype = ctypes.c_int
         L.tova_cache_set_policy.argtypes = [vp, i32, i32]
+        L.tova_cache_read_scores.restype = ctypes.c_int
+        L.tova_cache_read_scores.argtypes = [vp, vp, vp]
+        L.tova_cache_units.restype = i32
+        L.tova_cache_units.argtypes = [vp]
         L.tova_cache_set_fused_merge.restype = ctypes.c_int
         L.tova_cache_set_fused_merge.argtypes = [vp, i32]
         L.tova_cache_set_bulk_prefill.restype = ctypes.c_int
@@ -151,7 +158,9 @@ class TovaCache:
         """Returns dict(len [B], positions [B,cap], status int, K, V or None) on the host."""
         c = self.cfg
         ln = torch.empty(c.batch, dtype=torch.int32, device=self.device)
-        ps = torch.empty(c.batch, c.capacity, dtype=torch.int32, device=self.device)
+        units = self.tova_cache_units()
+        ps = (torch.empty(c.batch, c.capacity, dtype=torch.int32, device=self.device) if units == 1 else
+              torch.empty(c.batch, units, c.capacity, dtype=torch.int32, device=self.device))
         stt = torch.empty(1, dtype=torch.int32, device=self.device)
         K = V = None
         if want_kv:
@@ -167,9 +176,21 @@ class TovaCache:
     def tova_cache_set_chunk_rows(self, rows: int) -> None:
         _check(lib().tova_cache_set_chunk_rows(self._h, int(rows)), "tova_cache_set_chunk_rows")
 
-    def tova_cache_set_policy(self, policy: int, keep_first: int = 0) -> None:
-        """policy: TOVA_POLICY_TOVA (0) or TOVA_POLICY_WINDOW (1); keep_first = i of the "+i" variants."""
-        _check(lib().tova_cache_set_policy(self._h, int(policy), int(keep_first)), "tova_cache_set_policy")
+    def tova_cache_set_policy(self, policy: int, arg: int = 0) -> None:
+        """policy: one of TOVA_POLICY_*; arg = i of the "+i" variants, or the recent window of H2O."""
+        _check(lib().tova_cache_set_policy(self._h, int(policy), int(arg)), "tova_cache_set_policy")
+
+    def tova_cache_units(self) -> int:
+        return int(lib().tova_cache_units(self._h))
+
+    def tova_cache_read_scores(self, stream=None):
+        """H2O: accumulated attention weight of every slot, [B,U,cap] on the host."""
+        c = self.cfg
+        sc = torch.empty(c.batch, self.tova_cache_units() if self.tova_cache_units() > 1 else 1, c.capacity,
+                         dtype=torch.float32, device=self.device)
+        _check(lib().tova_cache_read_scores(self._h, _p(sc), _stream(stream)), "tova_cache_read_scores")
+        torch.cuda.synchronize(self.device)
+        return sc.cpu()
 
     def tova_cache_set_fused_merge(self, on: bool) -> None:
         _check(lib().tova_cache_set_fused_merge(self._h, 1 if on else 0), "tova_cache_set_fused_merge")

@@ -18,6 +18,7 @@
 #include "tova_split_mma.cuh"
 #include "tova_fill.cuh"
 #include "tova_fill_tc.cuh"
+#include "tova_units.cuh"
 
 namespace {
 
@@ -29,6 +30,7 @@ struct Layout {
   size_t K, V, pos, len, last_slot, logits, part_ml, part_acc, head_ml, status, cur_pos;
   size_t st_q, st_k, st_v, st_out, st_ev;  // staging for host-buffer calls
   size_t df_k, df_v;                       // the new token's rows kept for a deferred eviction
+  size_t upos, uacc;                       // per-KV-head slot tables and accumulated scores (head-wise policies, H2O)
   size_t total;
   int ld, pc;
 };
@@ -74,9 +76,11 @@ Layout make_layout(const tova_config& c) {
   L.st_k = take(B * Hkv * D * E);
   L.st_v = take(B * Hkv * D * E);
   L.st_out = take(B * H * D * 4);
-  L.st_ev = take(B * 4);
+  L.st_ev = take(B * Hkv * 4);
   L.df_k = take(B * Hkv * D * E);
   L.df_v = take(B * Hkv * D * E);
+  L.upos = take(B * Hkv * cap * 4);
+  L.uacc = take(B * Hkv * cap * 4);
   L.total = off;
   return L;
 }
@@ -91,6 +95,8 @@ struct tova_cache {
   bool fill_maps;
   int bulk_fill;   // 0: prompts token by token; 1: bulk fill, tcgen05 kernel where head_dim is 128; 2: bulk fill, warp-level MMA kernel
   int policy, keep_first;  // which row is dropped once the state is over capacity (tova_cache_set_policy)
+  int units;               // 0: the layer policies of the combine kernel; else units that own rows (1 or Hkv)
+  int recent;              // H2O: size of the window of most recent tokens that always stay
   bool fuse_merge;      // the split warps of a head group form one CTA and merge the outputs themselves
   // deferred eviction: victim choice and insert run on a side stream, overlapping later work
   bool deferred, pending;
@@ -331,6 +337,31 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, boo
     e = launch_split_g<T, D>(c->device, p.G, p, grid, st);
   }
   if (e != cudaSuccess) return e;
+  if (c->units > 0) {
+    // Policies whose rows are owned per unit (a KV head, or the layer with accumulated scores): outputs as for
+    // the layer policy, then one thread block per (unit, sequence) scores, picks and inserts.
+    int n_launch = 2;
+    if (!p.fuse_out) {
+      StepParams pa = p;
+      pa.mode = tova::COMBINE_OUTPUTS;
+      pa.k_stage = c->base + c->lay.df_k;
+      pa.v_stage = c->base + c->lay.df_v;
+      pa.stage_logits = 0;
+      if ((e = launch_combine<T, D>(c->device, pa, st)) != cudaSuccess) return e;
+      n_launch = 3;
+    }
+    tova::UnitParams up{};
+    up.units = c->units;
+    up.table = reinterpret_cast<int32_t*>(c->base + (c->units == 1 ? c->lay.pos : c->lay.upos));
+    up.acc = reinterpret_cast<float*>(c->base + c->lay.uacc);
+    up.recent = c->recent;
+    up.h2o = (c->policy == tova::POLICY_H2O_LAYER || c->policy == tova::POLICY_H2O_HEAD) ? 1 : 0;
+    const int nh = c->units == 1 ? p.H : p.G;
+    tova::tova_unit_policy_kernel<T, D><<<dim3(c->units, p.B), tova::UNIT_THREADS, sizeof(float) * nh, st>>>(p, up);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    c->launches += n_launch;
+    return cudaSuccess;
+  }
   if (p.fuse_out) {
     // The split kernel has written the outputs; what is left is the victim and
     // the insert, on the caller's stream or (deferred) on the side stream.
@@ -518,10 +549,13 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
   fill_geometry(p, cfg, n, c->chunk_rows, c->sm_count);
   p.scale2 = c->scale2;
   cudaError_t e;
-  const bool defer = c->deferred && allow_defer;
+  const bool defer = c->deferred && allow_defer && c->units == 0;
   p.head_ml = reinterpret_cast<float2*>(base + c->lay.head_ml);
-  p.policy = c->policy;
+  p.policy = c->units > 0 ? tova::POLICY_TOVA : c->policy;
   p.keep_first = c->keep_first;
+  // Head-wise policies write a different row in every KV head: no single "last written row" to fetch again,
+  // so the streaming kernel requests its first tiles only after the dependency wait.
+  if (c->units > 0) p.last_slot = nullptr;
   p.fuse_out = (c->fuse_merge && fused_merge_fits(cfg, c->chunk_rows, c->sm_count)) ? 1 : 0;
   p.merge_ctas = p.fuse_out ? (p.n_chunks + tova::SPLIT_MERGE_MAX_WARPS - 1) / tova::SPLIT_MERGE_MAX_WARPS : 1;
   if (p.merge_ctas < 1) p.merge_ctas = 1;
@@ -698,6 +732,8 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   c->fuse_merge = true;
   c->policy = tova::POLICY_TOVA;
   c->keep_first = 0;
+  c->units = 0;
+  c->recent = 0;
   c->deferred = false;
   c->pending = false;
   c->side = nullptr;
@@ -731,6 +767,13 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
     delete c;
     return TOVA_ERR_CUDA;
   }
+  // per-unit slot tables start at -1 (all bytes 0xff), accumulated scores at zero
+  const size_t unit_bytes = (size_t)cfg->batch * cfg->n_kv_heads * cfg->capacity * 4;
+  if (cudaMemsetAsync(c->base + lay.upos, 0xff, unit_bytes, st) != cudaSuccess ||
+      cudaMemsetAsync(c->base + lay.uacc, 0, unit_bytes, st) != cudaSuccess) {
+    delete c;
+    return TOVA_ERR_CUDA;
+  }
   const size_t n = (size_t)cfg->batch * cfg->capacity;
   const int threads = 256;
   const unsigned blocks = (unsigned)((n + threads - 1) / threads);
@@ -755,14 +798,32 @@ int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows) {
   return TOVA_OK;
 }
 
-int tova_cache_set_policy(tova_cache* c, int32_t policy, int32_t keep_first) {
+int tova_cache_set_policy(tova_cache* c, int32_t policy, int32_t arg) {
   if (!c) return TOVA_ERR_NULL;
-  if (policy != TOVA_POLICY_TOVA && policy != TOVA_POLICY_WINDOW) return TOVA_ERR_UNSUPPORTED;
-  // a droppable row must always exist, and Window compares ages that stay below the capacity only if the
-  // state has been under this policy from the start
-  if (keep_first < 0 || keep_first >= c->cfg.capacity || c->len != 0) return TOVA_ERR_BAD_SHAPE;
-  c->policy = policy == TOVA_POLICY_WINDOW ? tova::POLICY_WINDOW : tova::POLICY_TOVA;
-  c->keep_first = keep_first;
+  if (policy < TOVA_POLICY_TOVA || policy > TOVA_POLICY_H2O_HEAD) return TOVA_ERR_UNSUPPORTED;
+  if (c->len != 0 || c->pending) return TOVA_ERR_BAD_SHAPE;   // the policy is fixed while the state is empty
+  if (policy == TOVA_POLICY_TOVA || policy == TOVA_POLICY_WINDOW) {
+    // a droppable row must always exist, and Window compares ages that stay below the capacity only if the
+    // state has been under this policy from the start
+    if (arg < 0 || arg >= c->cfg.capacity) return TOVA_ERR_BAD_SHAPE;
+    c->policy = policy == TOVA_POLICY_WINDOW ? tova::POLICY_WINDOW : tova::POLICY_TOVA;
+    c->keep_first = arg;
+    c->units = 0;
+    return TOVA_OK;
+  }
+  if (policy == TOVA_POLICY_TOVA_HEAD) {
+    if (arg != 0) return TOVA_ERR_BAD_SHAPE;
+    c->policy = tova::POLICY_TOVA_HEAD;
+    c->units = c->cfg.n_kv_heads;
+    c->keep_first = 0;
+    return TOVA_OK;
+  }
+  // H2O: arg = size of the recent window; 0 = the other half of the multi-state (Section 4.1)
+  if (arg < 0 || arg > c->cfg.capacity) return TOVA_ERR_BAD_SHAPE;
+  c->recent = arg ? arg : c->cfg.capacity - c->cfg.capacity / 2;
+  c->policy = policy == TOVA_POLICY_H2O_LAYER ? tova::POLICY_H2O_LAYER : tova::POLICY_H2O_HEAD;
+  c->units = policy == TOVA_POLICY_H2O_LAYER ? 1 : c->cfg.n_kv_heads;
+  c->keep_first = 0;
   return TOVA_OK;
 }
 
@@ -803,7 +864,8 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
   {
     const int room = c->cfg.capacity - c->len;
     const int F = n_tokens < room ? n_tokens : room;
-    if (c->bulk_fill && c->fill_maps && F >= BULK_FILL_MIN_TOKENS) {
+    // (the per-unit policies keep their own slot tables and scores: token by token)
+    if (c->bulk_fill && c->fill_maps && F >= BULK_FILL_MIN_TOKENS && c->units == 0) {
       rc = launch_fill(c, q, k, v, F, first_pos, out, evicted_pos, static_cast<cudaStream_t>(cuda_stream));
       if (rc != TOVA_OK) return rc;
       done = F;
@@ -815,7 +877,8 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
                    static_cast<const unsigned char*>(v) + t * kv_stride,
                    first_pos < 0 ? first_pos : first_pos + t,
                    out ? out + (size_t)t * B * H * D : scratch_out,
-                   evicted_pos ? evicted_pos + (size_t)t * B : nullptr, static_cast<cudaStream_t>(cuda_stream),
+                   evicted_pos ? evicted_pos + (size_t)t * B * (c->units > 0 ? c->units : 1) : nullptr,
+                   static_cast<cudaStream_t>(cuda_stream),
                    /*allow_defer=*/false);  // consecutive tokens of one cache cannot overlap anyway
     if (rc != TOVA_OK) return rc;
   }
@@ -887,7 +950,7 @@ int tova_decode_step_host(tova_cache* c, const void* q_host, const void* k_host,
   if (cudaMemcpyAsync(out_host, base + c->lay.st_out, ob, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return TOVA_ERR_CUDA;
   if (evicted_pos_host &&
-      cudaMemcpyAsync(evicted_pos_host, base + c->lay.st_ev, B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+      cudaMemcpyAsync(evicted_pos_host, base + c->lay.st_ev, B * (c->units > 0 ? c->units : 1) * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return TOVA_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return TOVA_ERR_CUDA;
   return TOVA_OK;
@@ -927,13 +990,26 @@ int tova_cache_read(const tova_cache* c_in, int32_t* len, int32_t* positions, vo
   const unsigned char* base = c->base;
   bool ok = true;
   if (len) ok &= cudaMemcpyAsync(len, base + c->lay.len, B * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
-  if (positions)
-    ok &= cudaMemcpyAsync(positions, base + c->lay.pos, B * cap * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (positions) {
+    const bool per_head = c->units > 1;     // head-wise policies: one slot table per KV head
+    ok &= cudaMemcpyAsync(positions, base + (per_head ? c->lay.upos : c->lay.pos), B * (per_head ? Hkv : 1) * cap * 4,
+                          cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  }
   if (k_out) ok &= cudaMemcpyAsync(k_out, base + c->lay.K, kvb, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
   if (v_out) ok &= cudaMemcpyAsync(v_out, base + c->lay.V, kvb, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
   if (status) ok &= cudaMemcpyAsync(status, base + c->lay.status, 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
   return ok ? TOVA_OK : TOVA_ERR_CUDA;
 }
+
+int tova_cache_read_scores(const tova_cache* c, float* scores, void* cuda_stream) {
+  if (!c || !scores) return TOVA_ERR_NULL;
+  if (c->policy != tova::POLICY_H2O_LAYER && c->policy != tova::POLICY_H2O_HEAD) return TOVA_ERR_UNSUPPORTED;
+  const size_t bytes = (size_t)c->cfg.batch * c->units * c->cfg.capacity * 4;
+  return cudaMemcpyAsync(scores, c->base + c->lay.uacc, bytes, cudaMemcpyDeviceToDevice,
+                         static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? TOVA_OK : TOVA_ERR_CUDA;
+}
+
+int32_t tova_cache_units(const tova_cache* c) { return c ? (c->units > 0 ? c->units : 1) : -1; }
 
 int32_t tova_cache_len(const tova_cache* c) { return c ? c->len : -1; }
 int64_t tova_cache_launches(const tova_cache* c) { return c ? c->launches : -1; }

@@ -54,7 +54,9 @@ class ParityReport:
     evicted_log: List[np.ndarray] = field(default_factory=list)
 
 
-POLICIES = {"tova": tova.TOVA_POLICY_TOVA, "window": tova.TOVA_POLICY_WINDOW}
+POLICIES = {"tova": tova.TOVA_POLICY_TOVA, "window": tova.TOVA_POLICY_WINDOW,
+            "tova_head": tova.TOVA_POLICY_TOVA_HEAD, "h2o_layer": tova.TOVA_POLICY_H2O_LAYER,
+            "h2o_head": tova.TOVA_POLICY_H2O_HEAD}
 
 
 def make_cache(w: W.Workload, sm_scale: float = 0.0, evict: bool = True, chunk_rows: int = 0,
@@ -186,6 +188,71 @@ def _periodic_token(w, pos, layer):
             _token_memo.clear()
         _token_memo[key] = W.token(w, pos, layer)
     return _token_memo[key]
+
+
+def run_lockstep_units(w: W.Workload, n_tokens: int, policy: str, recent: int = 0, *, block: int = 64,
+                       use_prefill: bool = True, chunk_rows: int = 0, fused_merge: bool = True,
+                       score_tol: float = 1e-5) -> ParityReport:
+    """run_lockstep for the policies whose rows are owned per unit (TOVA-head, H2O): dropped positions and slot
+    tables per unit bit-exact under the same victim rule (gap measured in the quantity the policy minimises),
+    outputs within tolerance, and for H2O the accumulated scores of all slots within score_tol at the end."""
+    from oracle.tova_oracle import OracleUnitsCache
+    cache = make_cache(w, chunk_rows=chunk_rows, fused_merge=fused_merge, policy=policy, keep_first=recent)
+    orc = OracleUnitsCache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, policy, recent=recent,
+                           precision="f32")
+    U = orc.U
+    assert cache.tova_cache_units() == U
+    tol = out_tol(w)
+    rep = ParityReport()
+    done = 0
+    while done < n_tokens:
+        T = min(block, n_tokens - done)
+        q, k, v = W.tokens(w, done, T)
+        dq, dk, dv = (tova.to_device(a, w.dtype) for a in (q, k, v))
+        out = torch.empty(T, w.batch, w.n_q_heads, w.head_dim, dtype=torch.float32, device="cuda:0")
+        ev = torch.full((T, w.batch, U), -12345, dtype=torch.int32, device="cuda:0")
+        if use_prefill:
+            cache.tova_prefill(dq, dk, dv, T, done, out, ev)
+        else:
+            for t in range(T):
+                cache.tova_decode_step(dq[t], dk[t], dv[t], done + t, out[t], ev[t])
+        torch.cuda.synchronize()
+        g_out, g_ev = out.cpu().numpy(), ev.cpu().numpy()
+        for t in range(T):
+            pos_t = done + t
+            full = orc.len[0] == w.capacity
+            forced = np.full((w.batch, U), -1, np.int32)
+            if full:
+                for b in range(w.batch):
+                    for u in range(U):
+                        e = int(g_ev[t, b, u])
+                        if e == pos_t:
+                            forced[b, u] = w.capacity
+                        else:
+                            hit = np.nonzero(orc.pos[b, u] == e)[0]
+                            assert hit.size == 1, f"token {pos_t} seq {b} unit {u}: GPU dropped {e}, not held by the checker"
+                            forced[b, u] = int(hit[0])
+            o_out, o_ev, victim, argmin, gap, _ = orc.step(q[t], k[t], v[t], pos_t, forced=forced)
+            assert np.all(gap < GAP_TOL), f"token {pos_t}: GPU victim lies {gap.max():.3e} above the minimum"
+            assert np.array_equal(o_ev, g_ev[t]), f"token {pos_t}: dropped {g_ev[t].tolist()} vs {o_ev.tolist()}"
+            err = float(np.abs(g_out[t] - o_out).max())
+            assert err <= tol, f"token {pos_t}: output error {err:.3e} > {tol}"
+            rep.max_err = max(rep.max_err, err)
+            if full:
+                rep.evictions += w.batch * U
+                rep.resyncs += int(np.sum(victim != argmin))
+                rep.self_evictions += int(np.sum(victim == w.capacity))
+        done += T
+        rep.steps = done
+        st = cache.tova_cache_read()
+        assert st["status"] == 0
+        assert np.array_equal(st["len"].numpy(), orc.len)
+        assert np.array_equal(st["positions"].numpy().reshape(w.batch, U, w.capacity), orc.pos), f"slot tables differ after {done} tokens"
+    if policy.startswith("h2o"):
+        sc = cache.tova_cache_read_scores().numpy()
+        assert np.abs(sc - orc.acc).max() <= score_tol, float(np.abs(sc - orc.acc).max())
+    rep.cache, rep.oracle = cache, orc
+    return rep
 
 
 def replay_slot_table(evicted: np.ndarray, capacity: int, first_pos: int = 0) -> np.ndarray:

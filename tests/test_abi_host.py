@@ -73,6 +73,9 @@ def test_null_handles_are_rejected():
     assert L.tova_cache_destroy(None) == -1
     assert L.tova_cache_len(None) == -1
     assert L.tova_cache_set_bulk_prefill(None, 1) == -1
+    assert L.tova_cache_set_policy(None, 2, 0) == -1
+    assert L.tova_cache_read_scores(None, None, None) == -1
+    assert L.tova_cache_units(None) == -1
     assert tova.strerror(0) == "ok" and "aligned" in tova.strerror(-4)
 
 

@@ -10,7 +10,7 @@ import torch
 import paper_2401_06104_b200 as tova
 from paper_2401_06104_b200 import workloads as W
 from oracle.tova_oracle import OracleCache
-from parity import gpu_block, hand_tol, make_cache, out_tol, replay_slot_table, run_lockstep
+from parity import gpu_block, hand_tol, make_cache, out_tol, replay_slot_table, run_lockstep, run_lockstep_units
 from test_oracle_pins import parse_golden
 
 pytestmark = pytest.mark.gpu
@@ -346,6 +346,58 @@ def test_policy_hand_worked_traces_on_gpu():
             assert abs(o[0, 0, 0] - float(o0)) <= hand_tol(float(o0)) and abs(o[0, 1, 0] - float(o1)) <= hand_tol(float(o1))
 
 
+@pytest.mark.parametrize("policy,recent", [("tova_head", 0), ("h2o_layer", 0), ("h2o_head", 0), ("h2o_head", 7),
+                                           ("h2o_layer", 150)])
+@pytest.mark.parametrize("shape", ["mha", "gqa4", "gqa16"])
+def test_unit_policies_against_the_checker(policy, recent, shape):
+    """TOVA-head, H2O layer-wise and head-wise: per-unit dropped positions and slot tables bit-exact, outputs within
+    tolerance, accumulated scores within 1e-5; outputs merged inside the streaming kernel (capacity 150: one thread
+    block per head group) and through global memory (32-row chunks, merge off)."""
+    w = {"mha": LLAMA.scaled(batch=2, n_q_heads=6, n_kv_heads=6, capacity=150),
+         "gqa4": MISTRAL.scaled(batch=2, n_q_heads=8, n_kv_heads=2, capacity=150),
+         "gqa16": YI.scaled(batch=1, n_q_heads=32, n_kv_heads=2, capacity=150, heavy_period=40)}[shape]
+    U = 1 if policy == "h2o_layer" else w.n_kv_heads
+    rep = run_lockstep_units(w, 150 + 170, policy, recent, block=80)
+    assert rep.evictions == w.batch * U * 170
+    held = rep.cache.tova_cache_read()["positions"].numpy().reshape(w.batch, U, -1)
+    if policy.startswith("h2o"):
+        window = recent or 75
+        for b in range(w.batch):
+            for u in range(U):
+                assert set(range(320 - window, 320)) <= set(held[b, u].tolist())
+                if window == 150:        # a window as large as the state: first in, first out
+                    assert sorted(held[b, u].tolist()) == list(range(170, 320))
+    if policy == "tova_head" and U > 1:
+        assert any(set(held[b, 0].tolist()) != set(held[b, 1].tolist()) for b in range(w.batch))
+    rep = run_lockstep_units(w, 150 + 50, policy, recent, block=50, fused_merge=False, chunk_rows=32)
+    assert rep.evictions == w.batch * U * 50
+
+
+def test_unit_policy_hand_worked_traces_on_gpu():
+    from test_oracle_unit_policies import parse_unit_golden
+    toks, _ = parse_golden()
+    D = 64
+    for policy, recent, steps in parse_unit_golden():
+        c = tova.TovaCache(1, 2, 2, D, 3, dtype=tova.TOVA_DTYPE_FP32, sm_scale=1.0)
+        c.tova_cache_set_policy({"tova_head": 2, "h2o_layer": 3, "h2o_head": 4}[policy], recent)
+        U = c.tova_cache_units()
+        out = torch.empty(1, 2, D, device="cuda:0")
+        ev = torch.empty(1, U, dtype=torch.int32, device="cuda:0")
+        for (t, e, rows_after, o0, o1) in steps:
+            q = np.zeros((1, 2, D), np.float32); q[..., 0] = 1.0
+            k = np.zeros((1, 2, D), np.float32); v = np.zeros((1, 2, D), np.float32)
+            a0, v0, a1, v1 = toks[t]
+            k[0, 0, 0], k[0, 1, 0] = np.log(a0), np.log(a1)
+            v[0, 0, 0], v[0, 1, 0] = v0, v1
+            c.tova_decode_step(*(tova.to_device(a, 0) for a in (q, k, v)), t, out, ev)
+            st = c.tova_cache_read()
+            assert ev.cpu().numpy()[0].tolist() == e, (policy, recent, t)
+            assert st["positions"].numpy().reshape(U, 3).tolist() == rows_after, (policy, recent, t)
+            o = out.cpu().numpy()
+            assert abs(o[0, 0, 0] - float(o0)) <= hand_tol(float(o0)) and abs(o[0, 1, 0] - float(o1)) <= hand_tol(float(o1))
+            assert st["status"] == 0
+
+
 def test_policy_argument_errors():
     w = LLAMA.scaled(batch=1, n_q_heads=2, n_kv_heads=2, capacity=8)
     c = make_cache(w)
@@ -355,7 +407,19 @@ def test_policy_argument_errors():
     for bad in (-1, 8):
         with pytest.raises(tova.TovaError):
             c.tova_cache_set_policy(tova.TOVA_POLICY_WINDOW, bad)
+    with pytest.raises(tova.TovaError):
+        c.tova_cache_set_policy(tova.TOVA_POLICY_TOVA_HEAD, 1)       # the per-head policy takes no argument
+    with pytest.raises(tova.TovaError):
+        c.tova_cache_set_policy(tova.TOVA_POLICY_H2O_HEAD, 9)        # a window larger than the state
+    with pytest.raises(tova.TovaError) as e:
+        c.tova_cache_read_scores()                                   # scores exist under H2O only
+    assert e.value.code == -3
+    c.tova_cache_set_policy(tova.TOVA_POLICY_H2O_LAYER, 0)
+    assert c.tova_cache_units() == 1
+    c.tova_cache_set_policy(tova.TOVA_POLICY_TOVA_HEAD, 0)
+    assert c.tova_cache_units() == 2
     c.tova_cache_set_policy(tova.TOVA_POLICY_WINDOW, 7)
+    assert c.tova_cache_units() == 1
     q = torch.zeros(1, 2, 128, dtype=torch.bfloat16, device="cuda:0")
     c.tova_decode_step(q, q, q, 0, torch.zeros(1, 2, 128, device="cuda:0"))
     with pytest.raises(tova.TovaError):            # the state is no longer empty
