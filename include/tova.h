@@ -114,10 +114,42 @@ int tova_decode_step(tova_cache* c, const void* q, const void* k, const void* v,
  * token by token; its outputs equal the per-token ones up to floating-point
  * summation order (within the library's output tolerance), everything else
  * bit for bit.  The tokens that remain once the state is full are processed
- * one at a time.  tova_cache_set_bulk_prefill(c, 0) forces the per-token
- * route for all of them (then outputs are bit-identical to decode steps). */
+ * one at a time, or - where tova_cache_set_prefill_workspace has given the
+ * cache a workspace - in chunks of up to 64 tokens (see there).
+ * tova_cache_set_bulk_prefill(c, 0) forces the per-token route for all of
+ * them (then outputs are bit-identical to decode steps). */
 int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int32_t n_tokens,
                  int32_t first_pos, float* out, int32_t* evicted_pos, void* cuda_stream);
+
+/* Prompt tokens that meet a FULL state, many per launch.  Each of them drops a
+ * row (Algorithm 1) and thereby changes what the next one attends to; the
+ * paper's language-modelling runs handle whole chunks of tokens at once by
+ * masking the attention according to the layer's attention weights (appendix
+ * "Experimental Details").  With a workspace, tova_prefill does the same,
+ * exactly: per chunk of up to 64 tokens one dense pass computes the logits of
+ * all its queries against the state as the chunk found it and against the
+ * chunk's own tokens, one thread block per sequence replays the chunk's
+ * deletions in order from those logits alone (the same candidates, head-averaged
+ * weights and arg-min as token-by-token steps), a second dense pass forms the
+ * outputs with every query's weights masked to the rows alive at its step, and
+ * the surviving tokens are written to the slots they took.  Five launches per
+ * 64 tokens instead of 128.  Results equal token-by-token processing up to
+ * floating-point summation order (the library's output tolerance; a victim may
+ * differ only between candidates whose averages differ by rounding).
+ *   tova_prefill_workspace_bytes   device bytes needed (about
+ *        B*H*64*(capacity+64)*4 for the logits); 0 for an invalid or fp32
+ *        configuration.
+ *   tova_cache_set_prefill_workspace   dev_mem: 256-byte aligned device memory of
+ *        at least that size, owned by the caller, to outlive the handle (or
+ *        until replaced; NULL switches the chunked route off).  It may be
+ *        shared by caches of one shape whose calls are ordered on one stream.
+ *        TOVA_ERR_UNSUPPORTED for fp32 states and for capacities beyond what the
+ *        deletion kernel's shared memory holds (about 25,000 rows).
+ * Used for the TOVA policy (with or without protected first positions) on bf16
+ * states, for runs of at least 8 tokens; everything else takes the per-token
+ * route as before. */
+size_t tova_prefill_workspace_bytes(const tova_config* cfg);
+int tova_cache_set_prefill_workspace(tova_cache* c, void* dev_mem, size_t dev_bytes);
 
 /* tova_decode_step with HOST buffers; returns after `cuda_stream` has been
  * synchronised, when out (and evicted_pos if not NULL) hold the results.

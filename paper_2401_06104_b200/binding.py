@@ -66,6 +66,10 @@ def lib() -> ctypes.CDLL:
         L.tova_cache_set_chunk_rows.argtypes = [vp, i32]
         L.tova_cache_set_policy.restype = ctypes.c_int
         L.tova_cache_set_policy.argtypes = [vp, i32, i32]
+        L.tova_prefill_workspace_bytes.restype = ctypes.c_size_t
+        L.tova_prefill_workspace_bytes.argtypes = [ctypes.POINTER(tova_config)]
+        L.tova_cache_set_prefill_workspace.restype = ctypes.c_int
+        L.tova_cache_set_prefill_workspace.argtypes = [vp, vp, ctypes.c_size_t]
         L.tova_cache_read_scores.restype = ctypes.c_int
         L.tova_cache_read_scores.argtypes = [vp, vp, vp]
         L.tova_cache_units.restype = i32
@@ -172,6 +176,25 @@ class TovaCache:
         torch.cuda.synchronize(self.device)
         return {"len": ln.cpu(), "positions": ps.cpu(), "status": int(stt.item()),
                 "K": None if K is None else K.float().cpu(), "V": None if V is None else V.float().cpu()}
+
+    def tova_cache_set_prefill_workspace(self, mem: Optional[torch.Tensor] = None, allocate: bool = True):
+        """Gives the cache the scratch of the chunked prompt route: `mem`, a uint8 device tensor the caller
+        keeps alive (it may serve several caches of one shape), or a fresh one when allocate is set.
+        mem=None with allocate=False switches the route off.  Returns the tensor in use."""
+        if mem is None and not allocate:
+            _check(lib().tova_cache_set_prefill_workspace(self._h, None, 0), "tova_cache_set_prefill_workspace")
+            self._prefill_ws = None
+            return None
+        need = int(lib().tova_prefill_workspace_bytes(ctypes.byref(self.cfg)))
+        if need == 0:
+            raise TovaError(-3, "tova_prefill_workspace_bytes rejected the configuration")
+        if mem is None:
+            mem = torch.empty(need + 256, dtype=torch.uint8, device=self.device)
+        off = (-mem.data_ptr()) % 256
+        _check(lib().tova_cache_set_prefill_workspace(self._h, ctypes.c_void_p(mem.data_ptr() + off),
+                                                      mem.numel() - off), "tova_cache_set_prefill_workspace")
+        self._prefill_ws = mem
+        return mem
 
     def tova_cache_set_chunk_rows(self, rows: int) -> None:
         _check(lib().tova_cache_set_chunk_rows(self._h, int(rows)), "tova_cache_set_chunk_rows")

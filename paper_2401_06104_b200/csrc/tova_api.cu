@@ -19,6 +19,7 @@
 #include "tova_fill.cuh"
 #include "tova_fill_tc.cuh"
 #include "tova_units.cuh"
+#include "tova_chunk.cuh"
 
 namespace {
 
@@ -85,6 +86,31 @@ Layout make_layout(const tova_config& c) {
   return L;
 }
 
+// Caller-provided scratch of the chunked prompt path (tova_cache_set_prefill_workspace).
+struct ChunkLayout {
+  size_t Kst, Vst, lg, rt, ml, death, slot_token, first, total;
+  int ldc;
+};
+
+ChunkLayout make_chunk_layout(const tova_config& c) {
+  ChunkLayout L{};
+  const size_t B = c.batch, H = c.n_q_heads, Hkv = c.n_kv_heads, D = c.head_dim, cap = c.capacity;
+  const size_t CT = tova::CHUNK_TOKENS;
+  L.ldc = (int)((cap + CT + 3) / 4 * 4);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L.Kst = take(B * Hkv * CT * D * 2);
+  L.Vst = take(B * Hkv * CT * D * 2);
+  L.lg = take(B * H * CT * L.ldc * 4);
+  L.rt = take(B * H * CT * 8);
+  L.ml = take(B * H * CT * 8);
+  L.death = take(B * L.ldc * 4);
+  L.slot_token = take(B * cap * 4);
+  L.first = take(4);
+  L.total = off;
+  return L;
+}
+
 }  // namespace
 
 struct tova_cache {
@@ -104,6 +130,10 @@ struct tova_cache {
   cudaEvent_t ev_fork, ev_join;
   Layout lay;
   unsigned char* base;
+  // chunked prompt path: caller-provided workspace and tiled views of its staging tiles
+  unsigned char* chunk_ws;
+  ChunkLayout chunk_lay;
+  CUtensorMap chunk_map_k, chunk_map_v;
   int32_t len;          // rows per sequence (host mirror; sequences move in lock step)
   int64_t launches;
   int chunk_rows;       // rows of the state per split warp
@@ -650,6 +680,89 @@ int launch_fill(tova_cache* c, const void* q, const void* k, const void* v, int 
   return TOVA_OK;
 }
 
+// Fewest prompt tokens worth a chunk's five launches.
+constexpr int CHUNK_MIN_TOKENS = 8;
+constexpr size_t CHUNK_RESOLVE_SMEM_LIMIT = 200 * 1024;
+
+inline size_t chunk_resolve_smem(const tova_config& cfg) {
+  return sizeof(int32_t) * 2 * (size_t)cfg.capacity + sizeof(float) * (size_t)cfg.n_q_heads;
+}
+
+template <int D>
+cudaError_t launch_chunk_d(tova_cache* c, const tova::ChunkParams& p, cudaStream_t st) {
+  const unsigned cap_blocks = (unsigned)c->sm_count * 16u;
+  auto blocks_for = [&](size_t items) {
+    unsigned b = (unsigned)((items + 255) / 256);
+    return b < 1 ? 1u : (b > cap_blocks ? cap_blocks : b);
+  };
+  cudaError_t e;
+  tova::tova_chunk_stage_kernel<D><<<blocks_for((size_t)p.B * p.Hkv * tova::CHUNK_TOKENS * (D * 2 / 16)), 256, 0, st>>>(p);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  constexpr size_t smem = 4 * (size_t)tova::FILL_K_ROWS * D * 2 + 1024;
+  static std::atomic<bool> configured[64];
+  if (c->device >= 0 && c->device < 64 && !configured[c->device]) {
+    if ((e = cudaFuncSetAttribute(tova::tova_chunk_attn_kernel<D, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(tova::tova_chunk_attn_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(tova::tova_chunk_resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)CHUNK_RESOLVE_SMEM_LIMIT)) != cudaSuccess) return e;
+    configured[c->device] = true;
+  }
+  const dim3 grid(p.H, p.B);
+  tova::tova_chunk_attn_kernel<D, 0><<<grid, tova::FILL_THREADS, smem, st>>>(p, c->fill_map_k, c->fill_map_v, c->chunk_map_k,
+                                                                         c->chunk_map_v);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  tova::tova_chunk_resolve_kernel<<<p.B, tova::CHUNK_RESOLVE_THREADS, chunk_resolve_smem(c->cfg), st>>>(p);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  c->launches += 3;
+  if (p.out) {
+    tova::tova_chunk_attn_kernel<D, 1><<<grid, tova::FILL_THREADS, smem, st>>>(p, c->fill_map_k, c->fill_map_v, c->chunk_map_k,
+                                                                           c->chunk_map_v);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    c->launches += 1;
+  }
+  tova::tova_chunk_scatter_kernel<D><<<blocks_for((size_t)p.B * p.cap * p.Hkv * (D * 2 / 16)), 256, 0, st>>>(p);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  c->launches += 1;
+  return cudaSuccess;
+}
+
+// C prompt tokens (CHUNK_MIN_TOKENS..64) onto a full bf16 state under the TOVA policy, through the caller's workspace.
+int launch_chunk(tova_cache* c, const void* q, const void* k, const void* v, int C, int32_t first_pos, float* out,
+                 int32_t* evicted_pos, cudaStream_t st) {
+  if (c->pending) {
+    if (cudaStreamWaitEvent(st, c->ev_join, 0) != cudaSuccess) return TOVA_ERR_CUDA;
+    c->pending = false;
+  }
+  tova::ChunkParams p{};
+  unsigned char* base = c->base;
+  unsigned char* ws = c->chunk_ws;
+  const ChunkLayout& L = c->chunk_lay;
+  p.K = base + c->lay.K;
+  p.V = base + c->lay.V;
+  p.pos = reinterpret_cast<int32_t*>(base + c->lay.pos);
+  p.cur_pos = reinterpret_cast<int32_t*>(base + c->lay.cur_pos);
+  p.last_slot = reinterpret_cast<int32_t*>(base + c->lay.last_slot);
+  p.status = reinterpret_cast<int32_t*>(base + c->lay.status);
+  p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.evicted = evicted_pos;
+  p.Kst = ws + L.Kst;
+  p.Vst = ws + L.Vst;
+  p.lg = reinterpret_cast<float*>(ws + L.lg);
+  p.rt = reinterpret_cast<float2*>(ws + L.rt);
+  p.ml = reinterpret_cast<float2*>(ws + L.ml);
+  p.death = reinterpret_cast<int32_t*>(ws + L.death);
+  p.slot_token = reinterpret_cast<int32_t*>(ws + L.slot_token);
+  p.first = reinterpret_cast<int32_t*>(ws + L.first);
+  p.B = c->cfg.batch; p.H = c->cfg.n_q_heads; p.Hkv = c->cfg.n_kv_heads; p.G = p.H / p.Hkv;
+  p.cap = c->cfg.capacity;
+  p.ldc = L.ldc;
+  p.C = C;
+  p.first_pos = first_pos;
+  p.keep_first = c->keep_first;
+  p.scale2 = c->scale2;
+  const cudaError_t e = c->cfg.head_dim == 128 ? launch_chunk_d<128>(c, p, st) : launch_chunk_d<64>(c, p, st);
+  return e == cudaSuccess ? TOVA_OK : TOVA_ERR_CUDA;
+}
+
 int check_step_args(const tova_cache* c, const void* q, const void* k, const void* v, const void* out) {
   if (!c || !q || !k || !v || !out) return TOVA_ERR_NULL;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return TOVA_ERR_ALIGN;
@@ -662,7 +775,8 @@ int check_step_args(const tova_cache* c, const void* q, const void* k, const voi
 // kernel: boxes of 16 rows x 64 columns (128 bytes) with the 128-byte swizzle.
 // The driver's encoder is looked up through the runtime, so the library has no
 // link-time dependency on the driver.
-int encode_state_map(CUtensorMap* map, void* base, const tova_config& cfg, int box_rows = tova::TILE_ROWS) {
+int encode_state_map(CUtensorMap* map, void* base, const tova_config& cfg, int box_rows = tova::TILE_ROWS,
+                     long long rows_per_head = 0) {
   typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -677,7 +791,7 @@ int encode_state_map(CUtensorMap* map, void* base, const tova_config& cfg, int b
     fn = reinterpret_cast<encode_fn>(sym);
     fn_cache.store(fn, std::memory_order_release);
   }
-  const cuuint64_t rows = (cuuint64_t)cfg.batch * cfg.n_kv_heads * cfg.capacity;
+  const cuuint64_t rows = (cuuint64_t)cfg.batch * cfg.n_kv_heads * (rows_per_head ? rows_per_head : cfg.capacity);
   const cuuint64_t dims[2] = {(cuuint64_t)cfg.head_dim, rows};
   const cuuint64_t strides[1] = {(cuuint64_t)cfg.head_dim * 2};
   const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
@@ -734,6 +848,7 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   c->keep_first = 0;
   c->units = 0;
   c->recent = 0;
+  c->chunk_ws = nullptr;
   c->deferred = false;
   c->pending = false;
   c->side = nullptr;
@@ -871,7 +986,21 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
       done = F;
     }
   }
-  for (int32_t t = done; t < n_tokens; ++t) {
+  // Tokens that meet a full state: chunks of up to 64 through the caller's workspace, where one was given
+  // (TOVA policy, with or without protected first positions; bf16 states).
+  const bool chunked = c->chunk_ws && c->bulk_fill && c->cfg.evict && c->units == 0 && c->policy == tova::POLICY_TOVA;
+  for (int32_t t = done; t < n_tokens;) {
+    if (chunked && c->len == c->cfg.capacity && n_tokens - t >= CHUNK_MIN_TOKENS) {
+      const int C = n_tokens - t < tova::CHUNK_TOKENS ? n_tokens - t : tova::CHUNK_TOKENS;
+      rc = launch_chunk(c, static_cast<const unsigned char*>(q) + t * q_stride,
+                        static_cast<const unsigned char*>(k) + t * kv_stride,
+                        static_cast<const unsigned char*>(v) + t * kv_stride, C,
+                        first_pos < 0 ? first_pos : first_pos + t, out ? out + (size_t)t * B * H * D : nullptr,
+                        evicted_pos ? evicted_pos + (size_t)t * B : nullptr, static_cast<cudaStream_t>(cuda_stream));
+      if (rc != TOVA_OK) return rc;
+      t += C;
+      continue;
+    }
     rc = step_impl(c, static_cast<const unsigned char*>(q) + t * q_stride,
                    static_cast<const unsigned char*>(k) + t * kv_stride,
                    static_cast<const unsigned char*>(v) + t * kv_stride,
@@ -881,7 +1010,31 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
                    static_cast<cudaStream_t>(cuda_stream),
                    /*allow_defer=*/false);  // consecutive tokens of one cache cannot overlap anyway
     if (rc != TOVA_OK) return rc;
+    ++t;
   }
+  return TOVA_OK;
+}
+
+size_t tova_prefill_workspace_bytes(const tova_config* cfg) {
+  int why;
+  if (!config_ok(cfg, &why) || cfg->dtype != TOVA_DTYPE_BF16) return 0;
+  return make_chunk_layout(*cfg).total;
+}
+
+int tova_cache_set_prefill_workspace(tova_cache* c, void* dev_mem, size_t dev_bytes) {
+  if (!c) return TOVA_ERR_NULL;
+  if (!dev_mem) { c->chunk_ws = nullptr; return TOVA_OK; }      // back to token-by-token
+  if (c->cfg.dtype != TOVA_DTYPE_BF16 || !c->fill_maps || chunk_resolve_smem(c->cfg) > CHUNK_RESOLVE_SMEM_LIMIT)
+    return TOVA_ERR_UNSUPPORTED;
+  if (reinterpret_cast<uintptr_t>(dev_mem) % ALIGN != 0) return TOVA_ERR_ALIGN;
+  const ChunkLayout L = make_chunk_layout(c->cfg);
+  if (dev_bytes < L.total) return TOVA_ERR_WORKSPACE;
+  unsigned char* ws = static_cast<unsigned char*>(dev_mem);
+  if (encode_state_map(&c->chunk_map_k, ws + L.Kst, c->cfg, tova::FILL_K_ROWS, tova::CHUNK_TOKENS) != TOVA_OK ||
+      encode_state_map(&c->chunk_map_v, ws + L.Vst, c->cfg, tova::FILL_K_ROWS, tova::CHUNK_TOKENS) != TOVA_OK)
+    return TOVA_ERR_CUDA;
+  c->chunk_lay = L;
+  c->chunk_ws = ws;
   return TOVA_OK;
 }
 

@@ -1,0 +1,446 @@
+// Prompt tokens beyond the capacity, many per launch (sm_100a).
+//
+// Once the state is full every prompt token drops a row (Algorithm 1), and the
+// row it drops changes what the next token attends to: taken literally that is
+// one dependent decode step per token.  The paper's language-modelling runs
+// avoid this by editing the attention mask of a whole chunk of tokens according
+// to the attention weights of the layer (appendix "Experimental Details"); the
+// same idea, made exact, drives this file.  For a chunk of up to 64 tokens that
+// meets a full state:
+//
+//   stage     the chunk's keys and values are copied next to the state
+//             (tova_chunk_stage_kernel) so that tiled copies can reach them;
+//   logits    ONE dense pass computes the scaled logits of all the chunk's
+//             queries against every row they could possibly attend to - the k
+//             rows of the state as the chunk found it, and the chunk's own
+//             earlier tokens - plus each query's row maximum R and the sum T of
+//             exp2(logit - R) over all those columns (tova_chunk_attn_kernel,
+//             MODE 0; warp-level bf16 MMAs, as in the bulk fill);
+//   resolve   one thread block per sequence replays the chunk's deletions in
+//             order from those logits alone (tova_chunk_resolve_kernel): for
+//             token i it removes the rows dropped by tokens < i from the
+//             normaliser (L = T - their terms), scores the k+1 live candidates
+//             by the head-averaged soft-max weight (Eq. 4, Algorithm 1), takes
+//             the arg-min - lowest slot on ties, the token itself being slot k -
+//             records the dropped position and lets the token take the slot.
+//             No key or value is touched: per token the work is H*(k+1) exp2;
+//   outputs   a second dense pass forms Eq. 7 for every query with the weights
+//             masked to the rows alive at ITS step and normalised by ITS L
+//             (tova_chunk_attn_kernel, MODE 1);
+//   scatter   the surviving tokens' rows go to the slots they won
+//             (tova_chunk_scatter_kernel).
+//
+// The result is what token-by-token steps give: the same candidates, weights
+// and arg-min per token, up to floating-point summation order (near-ties closer
+// than rounding can fall either way, as between any two implementations).
+#pragma once
+
+#include <cuda.h>
+
+#include "tova_fill.cuh"
+
+namespace tova {
+
+constexpr int CHUNK_TOKENS = 64;        // tokens per chunk = query rows of one attention CTA = rows of one staging tile
+constexpr int CHUNK_RESOLVE_THREADS = 1024;
+
+struct ChunkParams {
+  // state
+  unsigned char* K;        // [B,Hkv,cap,D]
+  unsigned char* V;
+  int32_t* pos;            // [B,cap]
+  int32_t* cur_pos;        // [1]
+  int32_t* last_slot;      // [B]
+  int32_t* status;         // [1]
+  // the chunk's tokens
+  const void* q;           // [C,B,H,D]
+  const void* k_new;       // [C,B,Hkv,D]
+  const void* v_new;
+  float* out;              // [C,B,H,D] or null
+  int32_t* evicted;        // [C,B] or null
+  // workspace
+  unsigned char* Kst;      // [B,Hkv,64,D] the chunk's keys
+  unsigned char* Vst;
+  float* lg;               // [B,H,64,ldc] base-2 logits: columns 0..cap-1 = state rows, cap+j = chunk token j
+  float2* rt;              // [B,H,64] (row maximum R, sum T of exp2(logit - R) over all columns a query can see)
+  float2* ml;              // [B,H,64] (R, sum L over the candidates alive at the query's step)
+  int32_t* death;          // [B,ldc] step at which a column's token is dropped (it is still attended at that step)
+  int32_t* slot_token;     // [B,cap] chunk token that ends up in a slot, -1: the slot keeps its row
+  int32_t* first;          // [1] position of the chunk's first token
+  int B, H, Hkv, G, cap, ldc;
+  int C;                   // tokens in this chunk (1..64)
+  int first_pos;           // position of the chunk's first token, or < 0: current position + 1
+  int keep_first;          // rows holding positions 0..keep_first-1 are never dropped
+  float scale2;
+};
+
+constexpr int32_t CHUNK_ALIVE = 0x7fffffff;
+
+// The chunk's keys/values into the staging tiles (rows past the chunk are zeroed: they are read with weight zero),
+// every column's death step reset, the first position fixed for the later kernels.
+template <int D>
+__global__ void tova_chunk_stage_kernel(const ChunkParams p) {
+  constexpr int CH = D * 2 / 16;
+  const size_t total = (size_t)p.B * p.Hkv * CHUNK_TOKENS * CH;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int ch = (int)(i % CH);
+    const size_t row = i / CH;                         // (b, kvh, t)
+    const int t = (int)(row % CHUNK_TOKENS);
+    const size_t bk = row / CHUNK_TOKENS;              // b * Hkv + kvh
+    uint4 kq = make_uint4(0u, 0u, 0u, 0u), vq = kq;
+    if (t < p.C) {
+      const size_t src = ((size_t)t * p.B * p.Hkv + bk) * CH + ch;
+      kq = static_cast<const uint4*>(p.k_new)[src];
+      vq = static_cast<const uint4*>(p.v_new)[src];
+    }
+    reinterpret_cast<uint4*>(p.Kst)[i] = kq;
+    reinterpret_cast<uint4*>(p.Vst)[i] = vq;
+  }
+  const size_t nd = (size_t)p.B * p.ldc;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nd; i += (size_t)gridDim.x * blockDim.x)
+    p.death[i] = CHUNK_ALIVE;
+  if (blockIdx.x == 0 && threadIdx.x == 0) *p.first = (p.first_pos < 0) ? *p.cur_pos + 1 : p.first_pos;
+}
+
+// MODE 0: logits of the chunk's queries against the state and the chunk, row maxima and row sums.
+// MODE 1: attention outputs with the weights masked per query step and normalised by the resolved sums.
+// grid = (H, B), block = 128: warp w owns queries 16w..16w+15 of the chunk.  Tiles of 64 rows: the state's
+// (through map_k / map_v), then the chunk's own (map_ks / map_vs).  Dynamic shared memory as the bulk fill's.
+template <int D, int MODE>
+__global__ void __launch_bounds__(FILL_THREADS, 3) tova_chunk_attn_kernel(const ChunkParams p,
+                                                                       const __grid_constant__ CUtensorMap map_k,
+                                                                       const __grid_constant__ CUtensorMap map_v,
+                                                                       const __grid_constant__ CUtensorMap map_ks,
+                                                                       const __grid_constant__ CUtensorMap map_vs) {
+  constexpr int TILE_BYTES = FILL_K_ROWS * D * 2;
+  constexpr int BOXES = D / 64;
+  constexpr int KS = D / 16;
+  constexpr int ND = D / 8;
+
+  extern __shared__ unsigned char chunk_smem_raw[];
+  unsigned char* smem =
+      reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(chunk_smem_raw) + 1023) & ~(uintptr_t)1023);
+  unsigned char* kv_s = smem;                              // stage s: K at 2s, V at 2s+1
+  __shared__ __align__(8) uint64_t bars[2];
+  __shared__ int32_t dth[2][FILL_K_ROWS];                  // MODE 1: death step of the tile's columns
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int h = blockIdx.x, b = blockIdx.y;
+  const int kvh = h / p.G;
+  const int head_row0 = (b * p.Hkv + kvh) * p.cap;         // first row of this head in the [B*Hkv*cap, D] view
+  const int stage_row0 = (b * p.Hkv + kvh) * CHUNK_TOKENS; // ... in the [B*Hkv*64, D] view of the staging tiles
+  const int n_state = (p.cap + FILL_K_ROWS - 1) / FILL_K_ROWS;
+  const int n_tiles = n_state + 1;
+
+  if (tid == 0) {
+    mbar_init(&bars[0], 1);
+    mbar_init(&bars[1], 1);
+    mbar_fence_init();
+  }
+  __syncthreads();
+
+  auto issue = [&](int i) {
+    uint64_t* bar = &bars[i & 1];
+    unsigned char* kd = kv_s + (size_t)(2 * (i & 1)) * TILE_BYTES;
+    unsigned char* vd = kd + TILE_BYTES;
+    mbar_expect_tx(bar, (MODE == 1 ? 2u : 1u) * TILE_BYTES);
+    const bool st = i < n_state;
+    const int y = st ? head_row0 + i * FILL_K_ROWS : stage_row0;
+#pragma unroll
+    for (int bx = 0; bx < BOXES; ++bx) {
+      tma_load_2d_keep(kd + bx * (FILL_K_ROWS * 128), st ? &map_k : &map_ks, bx * 64, y, bar);
+      if (MODE == 1) tma_load_2d_keep(vd + bx * (FILL_K_ROWS * 128), st ? &map_v : &map_vs, bx * 64, y, bar);
+    }
+  };
+  if (tid == 0) issue(0);
+
+  // A fragments of this warp's 16 query rows, straight from global memory; rows past the chunk repeat its last token.
+  const int row_lo = warp * 16 + (lane >> 2);
+  const int qa_i = min(row_lo, p.C - 1), qb_i = min(row_lo + 8, p.C - 1);
+  uint32_t qa[KS][4];
+  {
+    const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q);
+    const uint32_t* qra = reinterpret_cast<const uint32_t*>(qg + (((size_t)qa_i * p.B + b) * p.H + h) * D) + (lane & 3);
+    const uint32_t* qrb = reinterpret_cast<const uint32_t*>(qg + (((size_t)qb_i * p.B + b) * p.H + h) * D) + (lane & 3);
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      qa[ks][0] = __ldg(qra + ks * 8);
+      qa[ks][1] = __ldg(qrb + ks * 8);
+      qa[ks][2] = __ldg(qra + ks * 8 + 4);
+      qa[ks][3] = __ldg(qrb + ks * 8 + 4);
+    }
+  }
+  const size_t bh = (size_t)b * p.H + h;
+  float* lg0 = p.lg + (bh * CHUNK_TOKENS + qa_i) * p.ldc;   // this lane's two logit rows
+  float* lg1 = p.lg + (bh * CHUNK_TOKENS + qb_i) * p.ldc;
+  const bool real0 = row_lo < p.C, real1 = row_lo + 8 < p.C;
+
+  float o[ND][4];
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+  float R0 = 0.f, R1 = 0.f, iL0 = 0.f, iL1 = 0.f;
+  if (MODE == 1) {
+#pragma unroll
+    for (int nd = 0; nd < ND; ++nd) o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f;
+    const float2 a = p.ml[bh * CHUNK_TOKENS + qa_i], c = p.ml[bh * CHUNK_TOKENS + qb_i];
+    R0 = a.x; iL0 = 1.f / a.y;
+    R1 = c.x; iL1 = 1.f / c.y;
+  }
+  const int32_t* death = p.death + (size_t)b * p.ldc;
+  bool ok = true;
+
+  for (int i = 0; i < n_tiles; ++i) {
+    if (tid == 0 && i + 1 < n_tiles) issue(i + 1);
+    const bool st = i < n_state;
+    const int c0 = st ? i * FILL_K_ROWS : p.cap;            // column of the tile's first row
+    if (MODE == 1 && tid < FILL_K_ROWS) {
+      const int c = c0 + tid;
+      dth[i & 1][tid] = (c < p.ldc) ? death[c] : -1;
+    }
+    ok = warp_wait(&bars[i & 1], (uint32_t)((i >> 1) & 1)) && ok;
+    if (MODE == 1) __syncthreads();
+    const uint32_t kt = smem_addr(kv_s + (size_t)(2 * (i & 1)) * TILE_BYTES);
+    const uint32_t vt = kt + TILE_BYTES;
+
+    float s[8][4];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+      const int kr = nt * 8 + (lane & 7);
+#pragma unroll
+      for (int ks = 0; ks < KS; ks += 2) {
+        uint32_t kb[4];
+        ldmatrix_x4(kb, kt + fill_swz(kr, 2 * ks + (lane >> 3)));
+        mma_bf16(s[nt], qa[ks], kb[0], kb[1]);
+        mma_bf16(s[nt], qa[ks + 1], kb[2], kb[3]);
+      }
+    }
+
+    // Which columns a query may see: every row of the state (tile rows past the capacity belong to the next head),
+    // and the chunk's tokens up to itself.
+    const int lim = st ? p.cap - c0 : 0;                    // state tile: rows < lim are this head's
+    if (MODE == 0) {
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt) {
+        const int r = nt * 8 + 2 * (lane & 3);
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const bool v0 = st ? (r + e < lim) : (r + e <= qa_i);
+          const bool v1 = st ? (r + e < lim) : (r + e <= qb_i);
+          const float a = v0 ? s[nt][e] * p.scale2 : -INFINITY, c = v1 ? s[nt][2 + e] * p.scale2 : -INFINITY;
+          s[nt][e] = a;
+          s[nt][2 + e] = c;
+          mx0 = fmaxf(mx0, a);
+          mx1 = fmaxf(mx1, c);
+        }
+        // keep the logits: two neighbouring columns per store (columns a query cannot see are never read back)
+        // (the chunk's columns start at `capacity`, which may be odd: then one column per store)
+        const int c = c0 + r;
+        const bool k0 = !st || r < lim, k1 = !st || r + 1 < lim;
+        if (k0 && k1 && !(c & 1)) {
+          if (real0) *reinterpret_cast<float2*>(lg0 + c) = make_float2(s[nt][0], s[nt][1]);
+          if (real1) *reinterpret_cast<float2*>(lg1 + c) = make_float2(s[nt][2], s[nt][3]);
+        } else {
+          if (k0 && real0) lg0[c] = s[nt][0];
+          if (k0 && real1) lg1[c] = s[nt][2];
+          if (k1 && real0) lg0[c + 1] = s[nt][1];
+          if (k1 && real1) lg1[c + 1] = s[nt][3];
+        }
+      }
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);   // finite from tile 0 on: the state is full
+      l_run[0] *= exp2_diff(m_run[0], mn0);
+      l_run[1] *= exp2_diff(m_run[1], mn1);
+      m_run[0] = mn0;
+      m_run[1] = mn1;
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt) {
+        l_run[0] += exp2f(s[nt][0] - mn0) + exp2f(s[nt][1] - mn0);
+        l_run[1] += exp2f(s[nt][2] - mn1) + exp2f(s[nt][3] - mn1);
+      }
+    } else {
+      // weights of the rows alive at the query's step: born no later (chunk tokens), dropped no earlier
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        uint32_t ph[4], pl[4];
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const int nt = 2 * kk + half;
+          const int r = nt * 8 + 2 * (lane & 3);
+          float e4[4];
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int dd = dth[i & 1][r + e];
+            const bool v0 = (st ? (r + e < lim) : (r + e <= qa_i)) && dd >= qa_i;
+            const bool v1 = (st ? (r + e < lim) : (r + e <= qb_i)) && dd >= qb_i;
+            e4[e] = v0 ? exp2f(s[nt][e] * p.scale2 - R0) : 0.f;
+            e4[2 + e] = v1 ? exp2f(s[nt][2 + e] * p.scale2 - R1) : 0.f;
+          }
+          split_hi_lo(e4[0], e4[1], ph[2 * half], pl[2 * half]);
+          split_hi_lo(e4[2], e4[3], ph[2 * half + 1], pl[2 * half + 1]);
+        }
+        const int vr = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+        for (int nd = 0; nd < ND; nd += 2) {
+          uint32_t vb[4];
+          ldmatrix_x4_trans(vb, vt + fill_swz(vr, nd + (lane >> 4)));
+          mma_bf16(o[nd], ph, vb[0], vb[1]);
+          mma_bf16(o[nd], pl, vb[0], vb[1]);
+          mma_bf16(o[nd + 1], ph, vb[2], vb[3]);
+          mma_bf16(o[nd + 1], pl, vb[2], vb[3]);
+        }
+      }
+    }
+    fence_proxy_async_smem();
+    __syncthreads();
+  }
+
+  if (!ok) {
+    if (tid == 0) atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
+    return;
+  }
+
+  if (MODE == 0) {
+    float l0 = l_run[0], l1 = l_run[1];
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    if ((lane & 3) == 0) {
+      if (real0) p.rt[bh * CHUNK_TOKENS + row_lo] = make_float2(m_run[0], l0);
+      if (real1) p.rt[bh * CHUNK_TOKENS + row_lo + 8] = make_float2(m_run[1], l1);
+    }
+  } else {
+#pragma unroll
+    for (int nd = 0; nd < ND; ++nd) {
+      const int d = nd * 8 + 2 * (lane & 3);
+      if (real0)
+        *reinterpret_cast<float2*>(p.out + (((size_t)row_lo * p.B + b) * p.H + h) * D + d) =
+            make_float2(o[nd][0] * iL0, o[nd][1] * iL0);
+      if (real1)
+        *reinterpret_cast<float2*>(p.out + (((size_t)(row_lo + 8) * p.B + b) * p.H + h) * D + d) =
+            make_float2(o[nd][2] * iL1, o[nd][3] * iL1);
+    }
+  }
+}
+
+// The chunk's deletions, in order, from the logits alone.  grid = (B), block = CHUNK_RESOLVE_THREADS.
+// Dynamic shared memory: occupant column and position of every slot (2 x cap ints), per-head constants (H floats).
+__global__ void __launch_bounds__(CHUNK_RESOLVE_THREADS) tova_chunk_resolve_kernel(const ChunkParams p) {
+  constexpr int NT = CHUNK_RESOLVE_THREADS, NW = NT / 32;
+  extern __shared__ __align__(16) int32_t rsm[];
+  int32_t* occ = rsm;                    // [cap] column whose token sits in the slot
+  int32_t* posv = occ + p.cap;           // [cap] position that token holds
+  float* hc = reinterpret_cast<float*>(posv + p.cap);   // [H] -R - log2(L * H) of the current query
+  __shared__ int32_t dead[CHUNK_TOKENS]; // columns dropped so far in this chunk
+  __shared__ float red_v[NW];
+  __shared__ int red_i[NW];
+  __shared__ int s_ndead;
+
+  const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int first = *p.first;
+  for (int s = tid; s < p.cap; s += NT) {
+    occ[s] = s;
+    posv[s] = p.pos[(size_t)b * p.cap + s];
+  }
+  if (tid == 0) s_ndead = 0;
+  __syncthreads();
+
+  const float* lgb = p.lg + (size_t)b * p.H * CHUNK_TOKENS * p.ldc;
+  const size_t hstride = (size_t)CHUNK_TOKENS * p.ldc;  // between heads
+  for (int i = 0; i < p.C; ++i) {
+    const int pos_i = first + i;
+    const float* row = lgb + (size_t)i * p.ldc;          // head 0's logits of query i
+    const int ndead = s_ndead;
+    // ---- each head's normaliser over the rows alive now: the sum over all columns minus the dropped ones ----
+    for (int h = warp; h < p.H; h += NW) {
+      const float2 rt = p.rt[((size_t)b * p.H + h) * CHUNK_TOKENS + i];
+      float gone = 0.f;
+      for (int d = lane; d < ndead; d += 32) gone += exp2f(row[h * hstride + dead[d]] - rt.x);
+      gone = warp_sum(gone);
+      if (lane == 0) {
+        const float L = rt.y - gone;
+        hc[h] = -rt.x - __log2f(L * (float)p.H);
+        p.ml[((size_t)b * p.H + h) * CHUNK_TOKENS + i] = make_float2(rt.x, L);
+      }
+    }
+    __syncthreads();
+    // ---- head-averaged weight of the k+1 candidates (Algorithm 1), lowest first -------------------------
+    float val = INFINITY;
+    int idx = 0x7fffffff;
+    for (int s = tid; s <= p.cap; s += NT) {
+      const int c = (s < p.cap) ? occ[s] : p.cap + i;
+      const int pj = (s < p.cap) ? posv[s] : pos_i;
+      const float* col = row + c;
+      float a = 0.f;
+#pragma unroll 8
+      for (int h = 0; h < p.H; ++h) a += exp2f(col[h * hstride] + hc[h]);
+      if (pj < p.keep_first) a = INFINITY;               // one of the first i token states: never dropped
+      if (a < val) { val = a; idx = s; }                 // s ascends: strict < keeps the lowest slot
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, val, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+      if (ov < val || (ov == val && oi < idx)) { val = ov; idx = oi; }
+    }
+    if (lane == 0) { red_v[warp] = val; red_i[warp] = idx; }
+    __syncthreads();
+    if (tid == 0) {
+      for (int w = 1; w < NW; ++w)
+        if (red_v[w] < val || (red_v[w] == val && red_i[w] < idx)) { val = red_v[w]; idx = red_i[w]; }
+      if (idx < 0 || idx > p.cap) { atomicExch(p.status, DEV_ERR_BAD_VICTIM); idx = p.cap; }
+      int gone_col, gone_pos;
+      if (idx < p.cap) {                                 // the token takes the dropped row's slot (Eq. 9, in place)
+        gone_col = occ[idx];
+        gone_pos = posv[idx];
+        occ[idx] = p.cap + i;
+        posv[idx] = pos_i;
+      } else {                                           // the token itself had the lowest weight
+        gone_col = p.cap + i;
+        gone_pos = pos_i;
+      }
+      p.death[(size_t)b * p.ldc + gone_col] = i;
+      dead[ndead] = gone_col;
+      s_ndead = ndead + 1;
+      if (p.evicted) p.evicted[(size_t)i * p.B + b] = gone_pos;
+    }
+    __syncthreads();
+  }
+  for (int s = tid; s < p.cap; s += NT) {
+    p.pos[(size_t)b * p.cap + s] = posv[s];
+    p.slot_token[(size_t)b * p.cap + s] = (occ[s] >= p.cap) ? occ[s] - p.cap : -1;
+  }
+}
+
+// Rows of the chunk's surviving tokens into the slots they took; bookkeeping for the kernels that follow
+// (a plain launch: a later streaming kernel, which requests rows before its own dependency wait, starts only
+// once these copies are complete; no single "last written row" exists, so that hint is cleared).
+template <int D>
+__global__ void tova_chunk_scatter_kernel(const ChunkParams p) {
+  constexpr int CH = D * 2 / 16;
+  const size_t total = (size_t)p.B * p.cap * p.Hkv * CH;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int ch = (int)(i % CH);
+    const size_t r = i / CH;                           // (b, s, kvh)
+    const int kvh = (int)(r % p.Hkv);
+    const size_t bs = r / p.Hkv;                       // b * cap + s
+    const int t = p.slot_token[bs];
+    if (t < 0) continue;
+    const int b = (int)(bs / p.cap), s = (int)(bs % p.cap);
+    const size_t src = (((size_t)b * p.Hkv + kvh) * CHUNK_TOKENS + t) * CH + ch;
+    const size_t dst = (((size_t)b * p.Hkv + kvh) * p.cap + s) * CH + ch;
+    reinterpret_cast<uint4*>(p.K)[dst] = reinterpret_cast<const uint4*>(p.Kst)[src];
+    reinterpret_cast<uint4*>(p.V)[dst] = reinterpret_cast<const uint4*>(p.Vst)[src];
+  }
+  if (blockIdx.x == 0) {
+    for (int b = threadIdx.x; b < p.B; b += blockDim.x) p.last_slot[b] = -1;
+    if (threadIdx.x == 0) *p.cur_pos = *p.first + p.C - 1;
+  }
+}
+
+}  // namespace tova

@@ -60,7 +60,7 @@ POLICIES = {"tova": tova.TOVA_POLICY_TOVA, "window": tova.TOVA_POLICY_WINDOW,
 
 
 def make_cache(w: W.Workload, sm_scale: float = 0.0, evict: bool = True, chunk_rows: int = 0,
-               fused_merge: bool = True, policy: str = "tova", keep_first: int = 0):
+               fused_merge: bool = True, policy: str = "tova", keep_first: int = 0, prefill_ws: bool = False):
     c = tova.TovaCache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, dtype=w.dtype,
                        sm_scale=sm_scale, evict=evict)
     if chunk_rows:
@@ -69,6 +69,8 @@ def make_cache(w: W.Workload, sm_scale: float = 0.0, evict: bool = True, chunk_r
         c.tova_cache_set_fused_merge(False)
     if policy != "tova" or keep_first:
         c.tova_cache_set_policy(POLICIES[policy], keep_first)
+    if prefill_ws:                       # prompt tokens that meet a full state go in chunks of up to 64
+        c.tova_cache_set_prefill_workspace()
     return c
 
 
@@ -92,7 +94,7 @@ def run_lockstep(w: W.Workload, n_tokens: int, *, seqs: Optional[Sequence[int]] 
                  sm_scale: float = 0.0, layer: int = 0, cache=None, oracle=None,
                  first_pos: int = 0, check_state_every: int = 4, direct_fill: bool = False,
                  fused_merge: bool = True, policy: str = "tova", keep_first: int = 0,
-                 period: int = 0) -> ParityReport:
+                 period: int = 0, prefill_ws: bool = False) -> ParityReport:
     """Feed n_tokens tokens to both sides and compare at every token.
 
     direct_fill: while the state is filling nothing is dropped (Section 3.3), so
@@ -108,7 +110,7 @@ def run_lockstep(w: W.Workload, n_tokens: int, *, seqs: Optional[Sequence[int]] 
     seqs = list(range(w.batch)) if seqs is None else list(seqs)
     own = cache is None
     cache = cache or make_cache(w, sm_scale=sm_scale, chunk_rows=chunk_rows, fused_merge=fused_merge,
-                                policy=policy, keep_first=keep_first)
+                                policy=policy, keep_first=keep_first, prefill_ws=prefill_ws)
     orc = oracle or OracleCache(len(seqs), w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity,
                                 sm_scale=sm_scale, precision="f32", policy=policy, keep_first=keep_first)
     tol = out_tol(w)
@@ -192,10 +194,11 @@ def _periodic_token(w, pos, layer):
 
 def run_lockstep_units(w: W.Workload, n_tokens: int, policy: str, recent: int = 0, *, block: int = 64,
                        use_prefill: bool = True, chunk_rows: int = 0, fused_merge: bool = True,
-                       score_tol: float = 1e-5) -> ParityReport:
+                       score_rtol: float = 1e-5) -> ParityReport:
     """run_lockstep for the policies whose rows are owned per unit (TOVA-head, H2O): dropped positions and slot
     tables per unit bit-exact under the same victim rule (gap measured in the quantity the policy minimises),
-    outputs within tolerance, and for H2O the accumulated scores of all slots within score_tol at the end."""
+    outputs within tolerance, and for H2O the accumulated scores of all slots at the end within score_rtol of their
+    size (a sink row's score grows by about half a unit per step: hundreds of fp32 additions on either side)."""
     from oracle.tova_oracle import OracleUnitsCache
     cache = make_cache(w, chunk_rows=chunk_rows, fused_merge=fused_merge, policy=policy, keep_first=recent)
     orc = OracleUnitsCache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, policy, recent=recent,
@@ -250,7 +253,7 @@ def run_lockstep_units(w: W.Workload, n_tokens: int, policy: str, recent: int = 
         assert np.array_equal(st["positions"].numpy().reshape(w.batch, U, w.capacity), orc.pos), f"slot tables differ after {done} tokens"
     if policy.startswith("h2o"):
         sc = cache.tova_cache_read_scores().numpy()
-        assert np.abs(sc - orc.acc).max() <= score_tol, float(np.abs(sc - orc.acc).max())
+        assert np.all(np.abs(sc - orc.acc) <= score_rtol * np.maximum(1.0, np.abs(orc.acc))), float(np.abs(sc - orc.acc).max())
     rep.cache, rep.oracle = cache, orc
     return rep
 

@@ -42,6 +42,15 @@ def test_cache_bytes_counts_state_and_scratch():
     assert 64 * 2**20 < big < 80 * 2**20          # 64 MiB of K/V plus scratch
 
 
+def test_prefill_workspace_size_is_dominated_by_the_logits():
+    c = cfg(batch=4, n_q_heads=8, n_kv_heads=2, capacity=1000)
+    n = tova.lib().tova_prefill_workspace_bytes(ctypes.byref(c))
+    logits = 4 * 8 * 64 * (1000 + 64) * 4
+    assert logits < n < logits + 2 * 2**20
+    assert tova.lib().tova_prefill_workspace_bytes(ctypes.byref(cfg(dtype=tova.TOVA_DTYPE_FP32))) == 0
+    assert tova.lib().tova_prefill_workspace_bytes(ctypes.byref(cfg(capacity=0))) == 0
+
+
 @pytest.mark.parametrize("bad", [dict(batch=0), dict(n_q_heads=6), dict(capacity=0), dict(n_kv_heads=0),
                                  dict(head_dim=96), dict(dtype=7), dict(sm_scale=-1.0)])
 def test_invalid_configurations_are_rejected(bad):
@@ -76,6 +85,7 @@ def test_null_handles_are_rejected():
     assert L.tova_cache_set_policy(None, 2, 0) == -1
     assert L.tova_cache_read_scores(None, None, None) == -1
     assert L.tova_cache_units(None) == -1
+    assert L.tova_cache_set_prefill_workspace(None, None, 0) == -1
     assert tova.strerror(0) == "ok" and "aligned" in tova.strerror(-4)
 
 

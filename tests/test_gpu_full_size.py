@@ -40,6 +40,20 @@ def test_full_layer_shapes(name, cap, extra, seqs, direct_fill):
           f"self {rep.self_evictions}")
 
 
+@pytest.mark.parametrize("name,cap,seqs", [("mistral_7b_gqa", 1024, [5, 31]), ("llama2_7b_layer", 512, [0, 7]),
+                                           ("yi_6b_long", 4096, [2])])
+def test_chunked_prompt_at_full_layer_shapes(name, cap, seqs):
+    """512-token tova_prefill calls onto a full state (eight chunks of 64 each), full batch, the checker on
+    sampled sequences, the slot tables of all sequences replayed from the log."""
+    w = W.WORKLOADS[name].scaled(capacity=cap)
+    n = cap + (512 if cap <= 1024 else 128)
+    rep = run_lockstep(w, n, seqs=seqs, block=512 if cap <= 1024 else 128, check_state_every=1000, direct_fill=True,
+                       prefill_ws=True)
+    assert rep.evictions == len(seqs) * (n - cap)
+    check_all_sequences(rep, w, n)
+    print(f"{name} k={cap} chunked prompt: max_err {rep.max_err:.2e} resyncs {rep.resyncs}/{rep.evictions}")
+
+
 def test_32_layer_configuration_at_full_batch():
     """Batch 64, 32 MHA heads, state of 1024 rows: 2048 eight-warp thread blocks of 128-row chunks per streaming
     launch (the launch the benchmark's headline times).  The checker follows three of the 64 sequences."""

@@ -158,6 +158,79 @@ def test_bulk_prefill_against_decode_steps(H, Hkv, D, cap, T0, T1, mode):
     assert a.tova_cache_launches() < b.tova_cache_launches()
 
 
+# ---------------------------------------------------------------------------
+# prompt tokens that meet a full state, in chunks (appendix "Experimental Details": whole chunks at once,
+# the attention masked according to the layer's attention weights)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("H,Hkv,D,cap,B,block,keep", [
+    (8, 8, 128, 203, 2, 64, 0),      # MHA, odd capacity (the chunk's logit columns start at an odd index), whole chunks
+    (8, 2, 128, 256, 3, 50, 0),      # GQA, ragged chunks of 50
+    (16, 1, 128, 130, 2, 200, 0),    # 200-token calls: three chunks of 64, then 8 tokens as a short chunk
+    (4, 4, 64, 96, 2, 71, 0),        # D = 64; 64 + 7: the 7 left over go token by token
+    (8, 2, 128, 300, 2, 64, 4),      # the first four positions protected (TOVA+4)
+    (32, 4, 128, 1100, 1, 64, 0),    # 18 state tiles, the last one ragged
+])
+def test_chunked_prompt_against_the_checker(H, Hkv, D, cap, B, block, keep):
+    """Every token of every chunk held against the checker: dropped positions and slot tables exact, outputs
+    within tolerance.  The state fills through the bulk route first, then the chunks begin."""
+    w = MISTRAL.scaled(batch=B, n_q_heads=H, n_kv_heads=Hkv, head_dim=D, capacity=cap)
+    n = cap + 3 * block + 30
+    rep = run_lockstep(w, n, block=block, prefill_ws=True, keep_first=keep, check_state_every=1,
+                       direct_fill=cap > 1000)
+    assert rep.evictions == B * (n - cap)
+    calls = -(-n // block)
+    assert rep.cache.tova_cache_launches() < 1 + 3 * calls + 5 * (n - cap) // 8     # far fewer than 2 per token
+    st = rep.cache.tova_cache_read(want_kv=True)
+    q, k, v = W.tokens(w, 0, n)
+    pos = st["positions"].numpy()
+    for b in range(B):                    # the cached rows are the tokens the slot table names
+        for s in range(0, cap, 7):
+            assert np.array_equal(st["K"][b, :, s].numpy(), k[pos[b, s], b])
+            assert np.array_equal(st["V"][b, :, s].numpy(), v[pos[b, s], b])
+
+
+def test_chunked_prompt_equals_token_by_token_processing():
+    """Same prompt through the chunked route and through decode steps: the same dropped positions, the same
+    state, outputs within the output tolerance; later decode steps bit-identical.  Also: no outputs wanted,
+    positions from the device counter, and the route switched off again."""
+    w = LLAMA.scaled(batch=2, n_q_heads=8, n_kv_heads=4, capacity=150)
+    T = 150 + 64 * 3 + 20
+    q, k, v = W.tokens(w, 0, T + 10)
+    a, b, c = make_cache(w, prefill_ws=True), make_cache(w), make_cache(w, prefill_ws=True)
+    oa, ea = gpu_block(a, w, q[:T], k[:T], v[:T], 0, use_prefill=True)
+    ob, eb = gpu_block(b, w, q[:T], k[:T], v[:T], 0, use_prefill=False)
+    assert np.array_equal(ea, eb)
+    assert np.abs(oa - ob).max() <= out_tol(w)
+    assert a.tova_cache_launches() < b.tova_cache_launches() // 4
+    dq, dk, dv = (tova.to_device(x, w.dtype) for x in (q, k, v))
+    ev = torch.empty(T, w.batch, dtype=torch.int32, device="cuda:0")
+    c.tova_prefill(dq[:9], dk[:9], dv[:9], 9, 0, None, ev[:9])
+    c.tova_prefill(dq[9:T], dk[9:T], dv[9:T], T - 9, tova.TOVA_POS_AUTO, None, ev[9:])
+    torch.cuda.synchronize()
+    assert np.array_equal(ev.cpu().numpy(), ea)
+    a.tova_cache_set_prefill_workspace(None, allocate=False)
+    o1, e1 = gpu_block(a, w, q[T:], k[T:], v[T:], T, use_prefill=True)
+    o2, e2 = gpu_block(b, w, q[T:], k[T:], v[T:], T, use_prefill=False)
+    o3, e3 = gpu_block(c, w, q[T:], k[T:], v[T:], T, use_prefill=False)
+    assert np.array_equal(o1, o2) and np.array_equal(e1, e2) and np.array_equal(o1, o3) and np.array_equal(e1, e3)
+    sa, sb, sc = (x.tova_cache_read(want_kv=True) for x in (a, b, c))
+    for key in ("len", "positions", "K", "V"):
+        assert torch.equal(sa[key], sb[key]) and torch.equal(sa[key], sc[key]), key
+    assert sa["status"] == 0 and sc["status"] == 0
+
+
+def test_prefill_workspace_argument_errors():
+    w = LLAMA.scaled(batch=1, n_q_heads=2, n_kv_heads=2, capacity=70)
+    c = make_cache(w)
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda:0")
+    with pytest.raises(tova.TovaError) as e:
+        c.tova_cache_set_prefill_workspace(small)
+    assert e.value.code == -5
+    f = make_cache(W.WORKLOADS["tiny"])
+    with pytest.raises(tova.TovaError):
+        f.tova_cache_set_prefill_workspace()                   # fp32 states keep the per-token route
+
+
 def test_bulk_prefill_mode_argument():
     c = make_cache(LLAMA.scaled(batch=1, n_q_heads=2, n_kv_heads=2, capacity=70))
     for mode in (0, 1, 2, True, False):
@@ -351,7 +424,7 @@ def test_policy_hand_worked_traces_on_gpu():
 @pytest.mark.parametrize("shape", ["mha", "gqa4", "gqa16"])
 def test_unit_policies_against_the_checker(policy, recent, shape):
     """TOVA-head, H2O layer-wise and head-wise: per-unit dropped positions and slot tables bit-exact, outputs within
-    tolerance, accumulated scores within 1e-5; outputs merged inside the streaming kernel (capacity 150: one thread
+    tolerance, accumulated scores within 1e-5 of their size; outputs merged inside the streaming kernel (capacity 150: one thread
     block per head group) and through global memory (32-row chunks, merge off)."""
     w = {"mha": LLAMA.scaled(batch=2, n_q_heads=6, n_kv_heads=6, capacity=150),
          "gqa4": MISTRAL.scaled(batch=2, n_q_heads=8, n_kv_heads=2, capacity=150),
