@@ -64,6 +64,8 @@ def parse_args():
                          "(-1: as many tokens as the state holds); a step is one whole prompt")
     ap.add_argument("--no-bulk-prefill", action="store_true", help="with --prefill: every prompt token takes the decode kernels")
     ap.add_argument("--warp-mma-prefill", action="store_true", help="with --prefill: bulk fill through the warp-level MMA kernel")
+    ap.add_argument("--no-chunked-prefill", action="store_true",
+                    help="with --prefill: prompt tokens that meet a full state go one at a time instead of in chunks of 64")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
@@ -515,10 +517,14 @@ def run_prefill(args):
     out = torch.empty(T, B, H, D, dtype=torch.float32, device=dev)
     ev = torch.empty(T, B, dtype=torch.int32, device=dev)
     caches = []
+    chunked = not (args.no_chunked_prefill or args.no_bulk_prefill) and w.dtype == W.DTYPE_BF16 and T > cap
+    ws = None
     for _ in range(steps + warm):
         c = tova.TovaCache(B, H, Hkv, D, cap, dtype=w.dtype, device=dev)
         if args.no_bulk_prefill or args.warp_mma_prefill:
             c.tova_cache_set_bulk_prefill(0 if args.no_bulk_prefill else 2)
+        if chunked:
+            ws = c.tova_cache_set_prefill_workspace(ws)          # one workspace serves all: calls share a stream
         caches.append(c)
     torch.cuda.synchronize()
     for c in caches[:warm]:
@@ -548,7 +554,8 @@ def run_prefill(args):
         "steps": steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": storage_name(w), "data": "synthetic",
         "config": workload_config(w, {"prompt_tokens": T, "tokens_into_free_rows": F,
-                                      "route": "bulk fill + per-token steps" if bulk else "per-token steps",
+                                      "route": ("bulk fill + chunks of 64" if chunked else "bulk fill + per-token steps") if bulk
+                                               else "per-token steps",
                                       "l2": "a fresh cache per step; inputs larger than L2" if q.numel() * 2 > 126e6
                                             else "a fresh cache per step",
                                       "parallelism": "single GPU"}),

@@ -151,6 +151,15 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
 size_t tova_prefill_workspace_bytes(const tova_config* cfg);
 int tova_cache_set_prefill_workspace(tova_cache* c, void* dev_mem, size_t dev_bytes);
 
+/* Tuning of the chunked prompt route: thread blocks per sequence in the kernel
+ * that replays a chunk's deletions.  0 (default): as many as keep all
+ * sequences resident at once, up to 8, as one thread-block cluster with the
+ * logits staged in shared memory; 1, 2, 4, 8: that many; -1: one block per
+ * sequence reading the logits from global memory (also taken where not even
+ * one token's logits fit the shared memory).  Results do not depend on it
+ * beyond floating-point summation order.  Other values: TOVA_ERR_BAD_SHAPE. */
+int tova_cache_set_chunk_cluster(tova_cache* c, int32_t ctas);
+
 /* tova_decode_step with HOST buffers; returns after `cuda_stream` has been
  * synchronised, when out (and evicted_pos if not NULL) hold the results.
  * Page-locked buffers (pinned or registered, 16-byte aligned; all of them):

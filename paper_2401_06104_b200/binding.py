@@ -70,6 +70,8 @@ def lib() -> ctypes.CDLL:
         L.tova_prefill_workspace_bytes.argtypes = [ctypes.POINTER(tova_config)]
         L.tova_cache_set_prefill_workspace.restype = ctypes.c_int
         L.tova_cache_set_prefill_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+        L.tova_cache_set_chunk_cluster.restype = ctypes.c_int
+        L.tova_cache_set_chunk_cluster.argtypes = [vp, i32]
         L.tova_cache_read_scores.restype = ctypes.c_int
         L.tova_cache_read_scores.argtypes = [vp, vp, vp]
         L.tova_cache_units.restype = i32
@@ -195,6 +197,9 @@ class TovaCache:
                                                       mem.numel() - off), "tova_cache_set_prefill_workspace")
         self._prefill_ws = mem
         return mem
+
+    def tova_cache_set_chunk_cluster(self, ctas: int) -> None:
+        _check(lib().tova_cache_set_chunk_cluster(self._h, int(ctas)), "tova_cache_set_chunk_cluster")
 
     def tova_cache_set_chunk_rows(self, rows: int) -> None:
         _check(lib().tova_cache_set_chunk_rows(self._h, int(rows)), "tova_cache_set_chunk_rows")

@@ -96,7 +96,7 @@ ChunkLayout make_chunk_layout(const tova_config& c) {
   ChunkLayout L{};
   const size_t B = c.batch, H = c.n_q_heads, Hkv = c.n_kv_heads, D = c.head_dim, cap = c.capacity;
   const size_t CT = tova::CHUNK_TOKENS;
-  L.ldc = (int)((cap + CT + 3) / 4 * 4);
+  L.ldc = (int)((cap + 3) / 4 * 4 + CT);      // state columns, then (16-byte aligned) the chunk's own
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   L.Kst = take(B * Hkv * CT * D * 2);
@@ -132,6 +132,7 @@ struct tova_cache {
   unsigned char* base;
   // chunked prompt path: caller-provided workspace and tiled views of its staging tiles
   unsigned char* chunk_ws;
+  int chunk_cluster;       // 0: automatic; 1, 2, 4, 8: CTAs per sequence of the deletion kernel; -1: the one-CTA kernel
   ChunkLayout chunk_lay;
   CUtensorMap chunk_map_k, chunk_map_v;
   int32_t len;          // rows per sequence (host mirror; sequences move in lock step)
@@ -683,6 +684,7 @@ int launch_fill(tova_cache* c, const void* q, const void* k, const void* v, int 
 // Fewest prompt tokens worth a chunk's five launches.
 constexpr int CHUNK_MIN_TOKENS = 8;
 constexpr size_t CHUNK_RESOLVE_SMEM_LIMIT = 200 * 1024;
+constexpr size_t CHUNK_CLUSTER_SMEM_LIMIT = 216 * 1024;
 
 inline size_t chunk_resolve_smem(const tova_config& cfg) {
   return sizeof(int32_t) * 2 * (size_t)cfg.capacity + sizeof(float) * (size_t)cfg.n_q_heads;
@@ -711,8 +713,44 @@ cudaError_t launch_chunk_d(tova_cache* c, const tova::ChunkParams& p, cudaStream
   tova::tova_chunk_attn_kernel<D, 0><<<grid, tova::FILL_THREADS, smem, st>>>(p, c->fill_map_k, c->fill_map_v, c->chunk_map_k,
                                                                          c->chunk_map_v);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  tova::tova_chunk_resolve_kernel<<<p.B, tova::CHUNK_RESOLVE_THREADS, chunk_resolve_smem(c->cfg), st>>>(p);
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  // The deletions: a cluster of CTAs per sequence with the logits staged in shared memory ahead of time, as
+  // many CTAs as keep all sequences resident at once; one CTA per sequence reading global memory where
+  // even one staged token does not fit.
+  {
+    int nc = tova::CHUNK_CLUSTER_MAX;
+    while (nc > 1 && (long long)p.B * nc > c->sm_count) nc >>= 1;
+    if (c->chunk_cluster > 0) nc = c->chunk_cluster;
+    const int S = ((p.cap + nc - 1) / nc + 3) / 4 * 4;
+    int nstage = tova::CHUNK_STAGES_MAX;
+    while (nstage > 0 && tova::chunk_cluster_smem(p.H, S, nstage) > CHUNK_CLUSTER_SMEM_LIMIT) --nstage;
+    if (nstage > 0 && c->chunk_cluster >= 0) {
+      static std::atomic<bool> cl_configured[64];
+      if (c->device >= 0 && c->device < 64 && !cl_configured[c->device]) {
+        if ((e = cudaFuncSetAttribute(tova::tova_chunk_resolve_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)CHUNK_CLUSTER_SMEM_LIMIT)) != cudaSuccess) return e;
+        cl_configured[c->device] = true;
+      }
+      cudaLaunchConfig_t cfg{};
+      cfg.gridDim = dim3(nc, p.B);
+      int nt = 256;                            // about one thread per candidate of a CTA
+      while (nt < tova::CHUNK_CLUSTER_THREADS_MAX && nt < S + 1) nt *= 2;
+      cfg.blockDim = dim3(nt);
+      cfg.dynamicSmemBytes = tova::chunk_cluster_smem(p.H, S, nstage);
+      cfg.stream = st;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = nc;
+      at[0].val.clusterDim.y = 1;
+      at[0].val.clusterDim.z = 1;
+      cfg.attrs = at;
+      cfg.numAttrs = 1;
+      e = cudaLaunchKernelEx(&cfg, tova::tova_chunk_resolve_cluster_kernel, p, S, nstage);
+    } else {
+      tova::tova_chunk_resolve_kernel<<<p.B, tova::CHUNK_RESOLVE_THREADS, chunk_resolve_smem(c->cfg), st>>>(p);
+      e = cudaGetLastError();
+    }
+    if (e != cudaSuccess) return e;
+  }
   c->launches += 3;
   if (p.out) {
     tova::tova_chunk_attn_kernel<D, 1><<<grid, tova::FILL_THREADS, smem, st>>>(p, c->fill_map_k, c->fill_map_v, c->chunk_map_k,
@@ -755,6 +793,7 @@ int launch_chunk(tova_cache* c, const void* q, const void* k, const void* v, int
   p.B = c->cfg.batch; p.H = c->cfg.n_q_heads; p.Hkv = c->cfg.n_kv_heads; p.G = p.H / p.Hkv;
   p.cap = c->cfg.capacity;
   p.ldc = L.ldc;
+  p.capA = L.ldc - tova::CHUNK_TOKENS;
   p.C = C;
   p.first_pos = first_pos;
   p.keep_first = c->keep_first;
@@ -849,6 +888,7 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   c->units = 0;
   c->recent = 0;
   c->chunk_ws = nullptr;
+  c->chunk_cluster = 0;
   c->deferred = false;
   c->pending = false;
   c->side = nullptr;
@@ -946,6 +986,13 @@ int tova_cache_set_bulk_prefill(tova_cache* c, int32_t on) {
   if (!c) return TOVA_ERR_NULL;
   if (on < 0 || on > 2) return TOVA_ERR_BAD_SHAPE;
   c->bulk_fill = on;
+  return TOVA_OK;
+}
+
+int tova_cache_set_chunk_cluster(tova_cache* c, int32_t ctas) {
+  if (!c) return TOVA_ERR_NULL;
+  if (ctas != -1 && ctas != 0 && ctas != 1 && ctas != 2 && ctas != 4 && ctas != 8) return TOVA_ERR_BAD_SHAPE;
+  c->chunk_cluster = ctas;
   return TOVA_OK;
 }
 

@@ -35,6 +35,7 @@
 // than rounding can fall either way, as between any two implementations).
 #pragma once
 
+#include <cooperative_groups.h>
 #include <cuda.h>
 
 #include "tova_fill.cuh"
@@ -61,13 +62,14 @@ struct ChunkParams {
   // workspace
   unsigned char* Kst;      // [B,Hkv,64,D] the chunk's keys
   unsigned char* Vst;
-  float* lg;               // [B,H,64,ldc] base-2 logits: columns 0..cap-1 = state rows, cap+j = chunk token j
+  float* lg;               // [B,64,H,ldc] base-2 logits of query i, head h: columns 0..cap-1 = state rows,
+                           // capA+j = chunk token j (capA = cap rounded up to 4: 16-byte aligned blocks)
   float2* rt;              // [B,H,64] (row maximum R, sum T of exp2(logit - R) over all columns a query can see)
   float2* ml;              // [B,H,64] (R, sum L over the candidates alive at the query's step)
   int32_t* death;          // [B,ldc] step at which a column's token is dropped (it is still attended at that step)
   int32_t* slot_token;     // [B,cap] chunk token that ends up in a slot, -1: the slot keeps its row
   int32_t* first;          // [1] position of the chunk's first token
-  int B, H, Hkv, G, cap, ldc;
+  int B, H, Hkv, G, cap, capA, ldc;
   int C;                   // tokens in this chunk (1..64)
   int first_pos;           // position of the chunk's first token, or < 0: current position + 1
   int keep_first;          // rows holding positions 0..keep_first-1 are never dropped
@@ -171,8 +173,8 @@ __global__ void __launch_bounds__(FILL_THREADS, 3) tova_chunk_attn_kernel(const 
     }
   }
   const size_t bh = (size_t)b * p.H + h;
-  float* lg0 = p.lg + (bh * CHUNK_TOKENS + qa_i) * p.ldc;   // this lane's two logit rows
-  float* lg1 = p.lg + (bh * CHUNK_TOKENS + qb_i) * p.ldc;
+  float* lg0 = p.lg + (((size_t)b * CHUNK_TOKENS + qa_i) * p.H + h) * p.ldc;   // this lane's two logit rows
+  float* lg1 = p.lg + (((size_t)b * CHUNK_TOKENS + qb_i) * p.H + h) * p.ldc;
   const bool real0 = row_lo < p.C, real1 = row_lo + 8 < p.C;
 
   float o[ND][4];
@@ -191,7 +193,7 @@ __global__ void __launch_bounds__(FILL_THREADS, 3) tova_chunk_attn_kernel(const 
   for (int i = 0; i < n_tiles; ++i) {
     if (tid == 0 && i + 1 < n_tiles) issue(i + 1);
     const bool st = i < n_state;
-    const int c0 = st ? i * FILL_K_ROWS : p.cap;            // column of the tile's first row
+    const int c0 = st ? i * FILL_K_ROWS : p.capA;           // column of the tile's first row
     if (MODE == 1 && tid < FILL_K_ROWS) {
       const int c = c0 + tid;
       dth[i & 1][tid] = (c < p.ldc) ? death[c] : -1;
@@ -235,10 +237,9 @@ __global__ void __launch_bounds__(FILL_THREADS, 3) tova_chunk_attn_kernel(const 
           mx1 = fmaxf(mx1, c);
         }
         // keep the logits: two neighbouring columns per store (columns a query cannot see are never read back)
-        // (the chunk's columns start at `capacity`, which may be odd: then one column per store)
-        const int c = c0 + r;
+        const int c = c0 + r;                       // even: 8-byte aligned pairs
         const bool k0 = !st || r < lim, k1 = !st || r + 1 < lim;
-        if (k0 && k1 && !(c & 1)) {
+        if (k0 && k1) {
           if (real0) *reinterpret_cast<float2*>(lg0 + c) = make_float2(s[nt][0], s[nt][1]);
           if (real1) *reinterpret_cast<float2*>(lg1 + c) = make_float2(s[nt][2], s[nt][3]);
         } else {
@@ -350,11 +351,11 @@ __global__ void __launch_bounds__(CHUNK_RESOLVE_THREADS) tova_chunk_resolve_kern
   if (tid == 0) s_ndead = 0;
   __syncthreads();
 
-  const float* lgb = p.lg + (size_t)b * p.H * CHUNK_TOKENS * p.ldc;
-  const size_t hstride = (size_t)CHUNK_TOKENS * p.ldc;  // between heads
+  const float* lgb = p.lg + (size_t)b * CHUNK_TOKENS * p.H * p.ldc;
+  const size_t hstride = (size_t)p.ldc;                 // between heads
   for (int i = 0; i < p.C; ++i) {
     const int pos_i = first + i;
-    const float* row = lgb + (size_t)i * p.ldc;          // head 0's logits of query i
+    const float* row = lgb + (size_t)i * p.H * p.ldc;    // head 0's logits of query i
     const int ndead = s_ndead;
     // ---- each head's normaliser over the rows alive now: the sum over all columns minus the dropped ones ----
     for (int h = warp; h < p.H; h += NW) {
@@ -373,7 +374,7 @@ __global__ void __launch_bounds__(CHUNK_RESOLVE_THREADS) tova_chunk_resolve_kern
     float val = INFINITY;
     int idx = 0x7fffffff;
     for (int s = tid; s <= p.cap; s += NT) {
-      const int c = (s < p.cap) ? occ[s] : p.cap + i;
+      const int c = (s < p.cap) ? occ[s] : p.capA + i;
       const int pj = (s < p.cap) ? posv[s] : pos_i;
       const float* col = row + c;
       float a = 0.f;
@@ -398,10 +399,10 @@ __global__ void __launch_bounds__(CHUNK_RESOLVE_THREADS) tova_chunk_resolve_kern
       if (idx < p.cap) {                                 // the token takes the dropped row's slot (Eq. 9, in place)
         gone_col = occ[idx];
         gone_pos = posv[idx];
-        occ[idx] = p.cap + i;
+        occ[idx] = p.capA + i;
         posv[idx] = pos_i;
       } else {                                           // the token itself had the lowest weight
-        gone_col = p.cap + i;
+        gone_col = p.capA + i;
         gone_pos = pos_i;
       }
       p.death[(size_t)b * p.ldc + gone_col] = i;
@@ -413,7 +414,209 @@ __global__ void __launch_bounds__(CHUNK_RESOLVE_THREADS) tova_chunk_resolve_kern
   }
   for (int s = tid; s < p.cap; s += NT) {
     p.pos[(size_t)b * p.cap + s] = posv[s];
-    p.slot_token[(size_t)b * p.cap + s] = (occ[s] >= p.cap) ? occ[s] - p.cap : -1;
+    p.slot_token[(size_t)b * p.cap + s] = (occ[s] >= p.capA) ? occ[s] - p.capA : -1;
+  }
+}
+
+// The same replay with the candidates of a sequence spread over a thread-block cluster and the logits staged in
+// shared memory ahead of time.  grid = (NC, B), cluster (NC,1,1), block = 256.  CTA r owns slots [r*S, r*S+S)
+// (S a multiple of 4); CTA 0 also owns the new token (candidate `capacity`).  Per token every CTA needs, of each
+// head's logit row, its own S state columns and the 64 chunk columns (a slot's occupant may by now be a chunk
+// token): 2*H bulk copies into one of `nstage` buffers, requested nstage tokens ahead - what a token reads
+// does not depend on earlier deletions, only which of the staged columns it uses does.  Per token:
+//   A. every warp takes heads, its lanes the CTA's candidates: e = exp2(logit - R) in place, the head's partial sum
+//      goes to every CTA of the cluster (distributed shared memory);           cluster barrier
+//   B. L_h = the partial sums in rank order; every thread scores a candidate: sum_h e[h] / (L_h * H); block arg-min;
+//      the CTA's best (value, slot) goes to every CTA;                          cluster barrier
+//   C. every CTA takes the same arg-min over the NC entries (lowest slot on ties); the owner of the slot
+//      replaces its occupant; the buffer is handed back to the copy engine for token i + nstage.
+// All waits on copies are bounded; a wait that runs out sets the status word and the kernel carries on through
+// its barriers (peers must not be left waiting).
+constexpr int CHUNK_CLUSTER_THREADS_MAX = 1024;   // block size: about one thread per candidate of the CTA, 256..1024
+constexpr int CHUNK_CLUSTER_MAX = 8;
+constexpr int CHUNK_STAGES_MAX = 4;
+
+__host__ __device__ inline size_t chunk_cluster_smem(int H, int S, int nstage) {
+  return sizeof(float) * ((size_t)nstage * H * (S + CHUNK_TOKENS) + (size_t)CHUNK_TOKENS * H +
+                          2 * (size_t)CHUNK_CLUSTER_MAX * H + H) + sizeof(int32_t) * 2 * (size_t)S + 64;
+}
+
+__global__ void __launch_bounds__(CHUNK_CLUSTER_THREADS_MAX) tova_chunk_resolve_cluster_kernel(const ChunkParams p,
+                                                                                           const int S, const int nstage) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cl = cg::this_cluster();
+  constexpr int NWM = CHUNK_CLUSTER_THREADS_MAX / 32, NCM = CHUNK_CLUSTER_MAX;
+  const int NT = (int)blockDim.x, NW = NT / 32;
+  const int NC = (int)cl.num_blocks(), r = (int)cl.block_rank();
+  const int b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int H = p.H, SW = S + CHUNK_TOKENS;
+
+  extern __shared__ __align__(16) float csm2[];
+  float* stage = csm2;                                        // [nstage][H][SW]
+  float* Rs = stage + (size_t)nstage * H * SW;               // [64][H] row maxima of the chunk's queries
+  float* part = Rs + (size_t)CHUNK_TOKENS * H;               // [2][NCM][H] partial sums of every CTA, double-buffered
+  float* invLH = part + 2 * (size_t)NCM * H;                 // [H] 1 / (L_h * H)
+  int32_t* occl = reinterpret_cast<int32_t*>(invLH + H);     // [S] staged column holding the slot's occupant
+  int32_t* posv = occl + S;                                  // [S] position it holds
+  __shared__ __align__(8) uint64_t full[CHUNK_STAGES_MAX];
+  __shared__ float2 best[2][NCM];                            // (value, slot) of every CTA, double-buffered
+  __shared__ float red_v[NWM];
+  __shared__ int red_i[NWM];
+
+  const int s_begin = r * S;
+  const int n_loc = max(0, min(S, p.cap - s_begin));          // slots this CTA really owns
+  const int n_cand = n_loc + (r == 0 ? 1 : 0);                // plus the new token
+  const int first = *p.first;
+  const float* lgb = p.lg + (size_t)b * CHUNK_TOKENS * H * p.ldc;
+
+  if (tid == 0) {
+    for (int s = 0; s < nstage; ++s) mbar_init(&full[s], 1);
+    mbar_fence_init();
+  }
+  for (int t = tid; t < S; t += NT) {
+    occl[t] = t;
+    posv[t] = (t < n_loc) ? p.pos[(size_t)b * p.cap + s_begin + t] : 0;
+  }
+  for (int t = tid; t < CHUNK_TOKENS * H; t += NT) {
+    const int i = t / H, h = t % H;
+    Rs[t] = (i < p.C) ? p.rt[((size_t)b * H + h) * CHUNK_TOKENS + i].x : 0.f;
+  }
+  __syncthreads();
+  // logits of token i into buffer i % nstage (warp 0): per head the CTA's state columns and the chunk's columns
+  auto request = [&](int i) {
+    uint64_t* bar = &full[i % nstage];
+    float* dst = stage + (size_t)(i % nstage) * H * SW;
+    if (lane == 0) mbar_expect_tx(bar, (uint32_t)H * (uint32_t)SW * 4u);
+    __syncwarp();
+    const float* src = lgb + (size_t)i * H * p.ldc;
+    for (int h = lane; h < H; h += 32) {
+      bulk_g2s(dst + (size_t)h * SW, src + (size_t)h * p.ldc + s_begin, (uint32_t)S * 4u, bar);
+      bulk_g2s(dst + (size_t)h * SW + S, src + (size_t)h * p.ldc + p.capA, (uint32_t)CHUNK_TOKENS * 4u, bar);
+    }
+  };
+  if (warp == 0)
+    for (int i = 0; i < min(nstage, p.C); ++i) request(i);
+  cl.sync();                                                  // every CTA of the cluster runs: its shared memory may be written
+
+  bool ok = true;
+  for (int i = 0; i < p.C; ++i) {
+    const int pos_i = first + i;
+    const int par = i & 1;
+    float* st = stage + (size_t)(i % nstage) * H * SW;
+    ok = warp_wait(&full[i % nstage], (uint32_t)((i / nstage) & 1)) && ok;
+    // ---- A: un-normalised weights in place, per-head partial sums to every CTA ---------------------
+    for (int h = warp; h < H; h += NW) {
+      const float R = Rs[i * H + h];
+      float* row = st + (size_t)h * SW;
+      float sum = 0.f;
+      int t = lane;
+      for (; t + 96 < n_cand; t += 128) {                 // four independent candidates in flight per lane
+        int c[4];
+        float e[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) c[u] = (t + 32 * u < n_loc) ? occl[t + 32 * u] : S + i;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) e[u] = exp2f(row[c[u]] - R);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { row[c[u]] = e[u]; sum += e[u]; }
+      }
+      for (; t < n_cand; t += 32) {
+        const int c = (t < n_loc) ? occl[t] : S + i;
+        const float e = exp2f(row[c] - R);
+        row[c] = e;
+        sum += e;
+      }
+      sum = warp_sum(sum);
+      if (lane < NC) *cl.map_shared_rank(&part[((size_t)par * NCM + r) * H + h], lane) = sum;
+    }
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    for (int h = tid; h < H; h += NT) {
+      float L = 0.f;
+      for (int rr = 0; rr < NC; ++rr) L += part[((size_t)par * NCM + rr) * H + h];
+      invLH[h] = 1.f / (L * (float)H);
+      if (r == 0) p.ml[((size_t)b * H + h) * CHUNK_TOKENS + i] = make_float2(Rs[i * H + h], L);
+    }
+    __syncthreads();
+    // ---- B: head-averaged weight of this CTA's candidates, lowest (value, slot) ----------------------
+    float val = INFINITY;
+    int idx = 0x7fffffff;
+    for (int t = tid; t < n_cand; t += NT) {
+      const int c = (t < n_loc) ? occl[t] : S + i;
+      const int pj = (t < n_loc) ? posv[t] : pos_i;
+      const float* col = st + c;
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;       // fixed order: heads h = 0,4,8,.. / 1,5,.. / 2,6,.. / 3,7,..
+      int h = 0;
+      for (; h + 3 < H; h += 4) {
+        a0 = fmaf(col[(size_t)h * SW], invLH[h], a0);
+        a1 = fmaf(col[(size_t)(h + 1) * SW], invLH[h + 1], a1);
+        a2 = fmaf(col[(size_t)(h + 2) * SW], invLH[h + 2], a2);
+        a3 = fmaf(col[(size_t)(h + 3) * SW], invLH[h + 3], a3);
+      }
+      for (; h < H; ++h) a0 = fmaf(col[(size_t)h * SW], invLH[h], a0);
+      float a = (a0 + a1) + (a2 + a3);
+      if (pj < p.keep_first) a = INFINITY;
+      const int g = (t < n_loc) ? s_begin + t : p.cap;
+      if (a < val) { val = a; idx = g; }               // t ascends and with it the slot: strict < keeps the lowest
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, val, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+      if (ov < val || (ov == val && oi < idx)) { val = ov; idx = oi; }
+    }
+    if (lane == 0) { red_v[warp] = val; red_i[warp] = idx; }
+    __syncthreads();
+    if (warp == 0) {
+      val = (lane < NW) ? red_v[lane] : INFINITY;
+      idx = (lane < NW) ? red_i[lane] : 0x7fffffff;
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, val, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+        if (ov < val || (ov == val && oi < idx)) { val = ov; idx = oi; }
+      }
+      if (lane < NC) *cl.map_shared_rank(&best[par][r], lane) = make_float2(val, __int_as_float(idx));
+    }
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    // ---- C: the same arg-min in every CTA; the slot's owner lets the token in ---------------------------------
+    float bv = INFINITY;
+    int bi = 0x7fffffff;
+    for (int rr = 0; rr < NC; ++rr) {
+      const float2 e = best[par][rr];
+      const int ei = __float_as_int(e.y);
+      if (e.x < bv || (e.x == bv && ei < bi)) { bv = e.x; bi = ei; }
+    }
+    if (bi < 0 || bi > p.cap) {                          // cannot happen with finite logits: report, drop the token
+      if (tid == 0 && r == 0) atomicExch(p.status, DEV_ERR_BAD_VICTIM);
+      bi = p.cap;
+    }
+    if (tid == 0) {
+      if (bi < p.cap) {
+        const int l = bi - s_begin;
+        if (l >= 0 && l < n_loc) {                      // Eq. 9 in place: the token takes the dropped row's slot
+          const int old = occl[l];
+          p.death[(size_t)b * p.ldc + (old < S ? s_begin + old : p.capA + (old - S))] = i;
+          if (p.evicted) p.evicted[(size_t)i * p.B + b] = posv[l];
+          occl[l] = S + i;
+          posv[l] = pos_i;
+        }
+      } else if (r == 0) {                               // the token itself had the lowest weight
+        p.death[(size_t)b * p.ldc + p.capA + i] = i;
+        if (p.evicted) p.evicted[(size_t)i * p.B + b] = pos_i;
+      }
+    }
+    __syncthreads();                                     // the buffer has been read by everybody; occl is up to date
+    if (warp == 0 && i + nstage < p.C) {
+      fence_proxy_async_smem();
+      request(i + nstage);
+    }
+  }
+  if (!ok && tid == 0) atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
+  for (int t = tid; t < n_loc; t += NT) {
+    p.pos[(size_t)b * p.cap + s_begin + t] = posv[t];
+    p.slot_token[(size_t)b * p.cap + s_begin + t] = (occl[t] >= S) ? occl[t] - S : -1;
   }
 }
 

@@ -86,6 +86,7 @@ def test_null_handles_are_rejected():
     assert L.tova_cache_read_scores(None, None, None) == -1
     assert L.tova_cache_units(None) == -1
     assert L.tova_cache_set_prefill_workspace(None, None, 0) == -1
+    assert L.tova_cache_set_chunk_cluster(None, 0) == -1
     assert tova.strerror(0) == "ok" and "aligned" in tova.strerror(-4)
 
 

@@ -189,6 +189,18 @@ def test_chunked_prompt_against_the_checker(H, Hkv, D, cap, B, block, keep):
             assert np.array_equal(st["V"][b, :, s].numpy(), v[pos[b, s], b])
 
 
+@pytest.mark.parametrize("ctas", [-1, 1, 2, 4, 8])
+def test_chunked_prompt_every_cluster_size(ctas):
+    """The deletion kernel as one thread block reading global memory (-1) and as clusters of 1 to 8 blocks
+    with staged logits; capacity 333 leaves the last block of a cluster a ragged share (8 x 44 > 333)."""
+    w = MISTRAL.scaled(batch=2, n_q_heads=8, n_kv_heads=2, capacity=333)
+    rep = run_lockstep(w, 333 + 64 + 40, block=64, prefill_ws=True, chunk_cluster=ctas, check_state_every=1)
+    assert rep.evictions == 2 * 104
+    w = LLAMA.scaled(batch=1, n_q_heads=4, n_kv_heads=4, capacity=20)      # fewer slots than blocks can share out
+    rep = run_lockstep(w, 20 + 64 * 2, block=64, prefill_ws=True, chunk_cluster=ctas, check_state_every=1)
+    assert rep.evictions == 128
+
+
 def test_chunked_prompt_equals_token_by_token_processing():
     """Same prompt through the chunked route and through decode steps: the same dropped positions, the same
     state, outputs within the output tolerance; later decode steps bit-identical.  Also: no outputs wanted,
@@ -229,6 +241,9 @@ def test_prefill_workspace_argument_errors():
     f = make_cache(W.WORKLOADS["tiny"])
     with pytest.raises(tova.TovaError):
         f.tova_cache_set_prefill_workspace()                   # fp32 states keep the per-token route
+    for bad in (3, 16, -2):
+        with pytest.raises(tova.TovaError):
+            c.tova_cache_set_chunk_cluster(bad)
 
 
 def test_bulk_prefill_mode_argument():
