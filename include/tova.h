@@ -251,6 +251,49 @@ int tova_cache_read_scores(const tova_cache* c, float* scores, void* cuda_stream
 /* Slot tables this cache keeps per sequence: Hkv under a head-wise policy, else 1. */
 int32_t tova_cache_units(const tova_cache* c);
 
+/* One layer sharded by KV head over several GPUs (one process per GPU).
+ * Algorithm 1 averages the last query's weights over the heads of the layer - a
+ * sum over heads - so ranks that each hold some of the KV heads (with the
+ * query heads that read them) only have to exchange, once a row is due to go,
+ * their partial head sums: one fp32 vector of capacity+1 entries per sequence.
+ * Everything else of the step (Eq. 4, Eq. 6, Eq. 7, the insert of Eq. 9) is
+ * local to a rank's heads.  A sharded cache is created like any other, with
+ * cfg.n_q_heads / cfg.n_kv_heads = the heads THIS rank holds, and then:
+ *
+ *   tova_cache_set_shard(c, rank, world, n_q_heads_total, peer_tables, peer_flags)
+ *       while the state is empty; world <= 8; TOVA policy (with or without
+ *       protected first positions).  Two ways to exchange:
+ *       peer stores - peer_tables[r] / peer_flags[r] (HOST arrays of `world`
+ *         DEVICE pointers) address rank r's score table of
+ *         tova_shard_table_bytes(cfg, world) bytes and its `world` int32 flags
+ *         (zeroed by the caller once), mapped into this process (CUDA IPC or
+ *         symmetric memory; for a single-process emulation plain device
+ *         memory).  The scores kernel stores this rank's partial sums into
+ *         every rank's table with ordinary stores and raises its flag there;
+ *         the commit kernel waits - bounded: a rank that never reports leaves
+ *         status code 3 and the state untouched - and adds the parts in rank
+ *         order, so every rank computes the same bits and the same victim;
+ *       caller reduces - peer_flags = NULL: only peer_tables[rank] is used,
+ *         [B, ld] floats with ld = capacity+1 rounded up to 4; between the two
+ *         calls below the caller sums that vector over the ranks in place
+ *         (e.g. an NCCL all-reduce on the same stream).
+ *   tova_decode_step_scores(c, q, k, v, pos, out, stream)
+ *       this rank's heads: q [B,H_local,D], k and v [B,Hkv_local,D]; attention
+ *       output for them; the rank's partial head sums published.
+ *   tova_decode_step_commit(c, k, v, evicted_pos, stream)
+ *       the victim from the summed vector (arg-min, lowest slot on ties, the new
+ *       token being slot `capacity`) and the insert into this rank's KV heads.
+ *       evicted_pos [B] or NULL: the same on every rank.
+ * The two calls alternate; tova_decode_step, tova_prefill and
+ * tova_decode_step_host are refused (TOVA_ERR_BAD_SHAPE) on a sharded cache.
+ * No TMA multicast and no library kernel reads or writes peer memory. */
+size_t tova_shard_table_bytes(const tova_config* cfg, int32_t world);
+int tova_cache_set_shard(tova_cache* c, int32_t rank, int32_t world, int32_t n_q_heads_total,
+                         void* const* peer_tables, void* const* peer_flags);
+int tova_decode_step_scores(tova_cache* c, const void* q, const void* k, const void* v, int32_t pos, float* out,
+                            void* cuda_stream);
+int tova_decode_step_commit(tova_cache* c, const void* k, const void* v, int32_t* evicted_pos, void* cuda_stream);
+
 /* Tuning: where the per-chunk partial results of a head are merged into the
  * attention output (Eq. 7 evaluated chunk by chunk).  on (default): when the
  * state splits into at most 8 chunks, the streaming warps of a head group run

@@ -70,6 +70,14 @@ def lib() -> ctypes.CDLL:
         L.tova_prefill_workspace_bytes.argtypes = [ctypes.POINTER(tova_config)]
         L.tova_cache_set_prefill_workspace.restype = ctypes.c_int
         L.tova_cache_set_prefill_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+        L.tova_shard_table_bytes.restype = ctypes.c_size_t
+        L.tova_shard_table_bytes.argtypes = [ctypes.POINTER(tova_config), i32]
+        L.tova_cache_set_shard.restype = ctypes.c_int
+        L.tova_cache_set_shard.argtypes = [vp, i32, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(vp)]
+        L.tova_decode_step_scores.restype = ctypes.c_int
+        L.tova_decode_step_scores.argtypes = [vp, vp, vp, vp, i32, vp, vp]
+        L.tova_decode_step_commit.restype = ctypes.c_int
+        L.tova_decode_step_commit.argtypes = [vp, vp, vp, vp, vp]
         L.tova_cache_set_chunk_cluster.restype = ctypes.c_int
         L.tova_cache_set_chunk_cluster.argtypes = [vp, i32]
         L.tova_cache_read_scores.restype = ctypes.c_int
@@ -197,6 +205,31 @@ class TovaCache:
                                                       mem.numel() - off), "tova_cache_set_prefill_workspace")
         self._prefill_ws = mem
         return mem
+
+    def tova_shard_table_bytes(self, world: int) -> int:
+        return int(lib().tova_shard_table_bytes(ctypes.byref(self.cfg), int(world)))
+
+    def tova_cache_set_shard(self, rank: int, world: int, n_q_heads_total: int, peer_tables, peer_flags=None) -> None:
+        """peer_tables / peer_flags: lists of `world` device tensors (or data pointers) as mapped into this process;
+        peer_flags None = the caller sums peer_tables[rank] over the ranks between scores and commit."""
+        def ptrs(xs):
+            arr = (ctypes.c_void_p * world)()
+            for i, x in enumerate(xs):
+                arr[i] = None if x is None else (x.data_ptr() if hasattr(x, "data_ptr") else int(x))
+            return arr
+        tabs = ptrs(peer_tables)
+        flags = None if peer_flags is None else ptrs(peer_flags)
+        self._shard_keep = (peer_tables, peer_flags)
+        _check(lib().tova_cache_set_shard(self._h, int(rank), int(world), int(n_q_heads_total), tabs, flags),
+               "tova_cache_set_shard")
+
+    def tova_decode_step_scores(self, q, k, v, pos: int, out, stream=None) -> None:
+        _check(lib().tova_decode_step_scores(self._h, _p(q), _p(k), _p(v), int(pos), _p(out), _stream(stream)),
+               "tova_decode_step_scores")
+
+    def tova_decode_step_commit(self, k, v, evicted_pos=None, stream=None) -> None:
+        _check(lib().tova_decode_step_commit(self._h, _p(k), _p(v), _p(evicted_pos), _stream(stream)),
+               "tova_decode_step_commit")
 
     def tova_cache_set_chunk_cluster(self, ctas: int) -> None:
         _check(lib().tova_cache_set_chunk_cluster(self._h, int(ctas)), "tova_cache_set_chunk_cluster")

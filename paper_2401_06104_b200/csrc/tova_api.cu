@@ -20,6 +20,7 @@
 #include "tova_fill_tc.cuh"
 #include "tova_units.cuh"
 #include "tova_chunk.cuh"
+#include "tova_shard.cuh"
 
 namespace {
 
@@ -32,6 +33,7 @@ struct Layout {
   size_t st_q, st_k, st_v, st_out, st_ev;  // staging for host-buffer calls
   size_t df_k, df_v;                       // the new token's rows kept for a deferred eviction
   size_t upos, uacc;                       // per-KV-head slot tables and accumulated scores (head-wise policies, H2O)
+  size_t shard_words;                      // epoch and ticket of the sharded step
   size_t total;
   int ld, pc;
 };
@@ -82,6 +84,7 @@ Layout make_layout(const tova_config& c) {
   L.df_v = take(B * Hkv * D * E);
   L.upos = take(B * Hkv * cap * 4);
   L.uacc = take(B * Hkv * cap * 4);
+  L.shard_words = take(8);
   L.total = off;
   return L;
 }
@@ -131,6 +134,9 @@ struct tova_cache {
   Layout lay;
   unsigned char* base;
   // chunked prompt path: caller-provided workspace and tiled views of its staging tiles
+  // state sharded by KV head over several ranks (tova_cache_set_shard)
+  bool shard_on, shard_scored;
+  tova::ShardParams shard;
   unsigned char* chunk_ws;
   int chunk_cluster;       // 0: automatic; 1, 2, 4, 8: CTAs per sequence of the deletion kernel; -1: the one-CTA kernel
   ChunkLayout chunk_lay;
@@ -368,6 +374,27 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, boo
     e = launch_split_g<T, D>(c->device, p.G, p, grid, st);
   }
   if (e != cudaSuccess) return e;
+  if (c->shard_on) {
+    // This rank's heads of a sharded layer: outputs as on one GPU, then (once a row is due to go) the rank's partial
+    // head sums into every rank's table.  Victim and insert follow in tova_decode_step_commit.
+    int n_launch = 1;
+    if (!p.fuse_out) {
+      StepParams pa = p;
+      pa.mode = tova::COMBINE_OUTPUTS;
+      pa.k_stage = c->base + c->lay.df_k;
+      pa.v_stage = c->base + c->lay.df_v;
+      pa.stage_logits = 0;
+      if ((e = launch_combine<T, D>(c->device, pa, st)) != cudaSuccess) return e;
+      ++n_launch;
+    }
+    if (p.do_evict) {
+      tova::tova_shard_scores_kernel<<<dim3(p.nx, p.B), tova::SHARD_THREADS, sizeof(float) * p.H, st>>>(p, c->shard);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      ++n_launch;
+    }
+    c->launches += n_launch;
+    return cudaSuccess;
+  }
   if (c->units > 0) {
     // Policies whose rows are owned per unit (a KV head, or the layer with accumulated scores): outputs as for
     // the layer policy, then one thread block per (unit, sequence) scores, picks and inserts.
@@ -558,12 +585,11 @@ void fill_geometry(StepParams& p, const tova_config& cfg, int n, int chunk_rows,
   set_combine_threads(p, ct);
 }
 
-int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_t pos, float* out,
-              int32_t* evicted_pos, cudaStream_t st, bool allow_defer = true) {
+// Pointers and launch geometry of one step of cache c for its current length.
+void step_params(tova_cache* c, const void* q, const void* k, const void* v, int32_t pos, float* out,
+                 int32_t* evicted_pos, bool defer, StepParams& p) {
   const tova_config& cfg = c->cfg;
   const int n = c->len;
-  if (n >= cfg.capacity && !cfg.evict) return TOVA_ERR_FULL;
-  StepParams p{};
   unsigned char* base = c->base;
   p.K = base + c->lay.K;
   p.V = base + c->lay.V;
@@ -579,8 +605,6 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
   p.ld = c->lay.ld; p.pc = c->lay.pc;
   fill_geometry(p, cfg, n, c->chunk_rows, c->sm_count);
   p.scale2 = c->scale2;
-  cudaError_t e;
-  const bool defer = c->deferred && allow_defer && c->units == 0;
   p.head_ml = reinterpret_cast<float2*>(base + c->lay.head_ml);
   p.policy = c->units > 0 ? tova::POLICY_TOVA : c->policy;
   p.keep_first = c->keep_first;
@@ -594,6 +618,17 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
     p.k_stage = base + c->lay.df_k;
     p.v_stage = base + c->lay.df_v;
   }
+}
+
+int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_t pos, float* out,
+              int32_t* evicted_pos, cudaStream_t st, bool allow_defer = true) {
+  const tova_config& cfg = c->cfg;
+  if (c->len >= cfg.capacity && !cfg.evict) return TOVA_ERR_FULL;
+  if (c->shard_on) return TOVA_ERR_BAD_SHAPE;   // a sharded layer steps through its two-phase calls
+  const bool defer = c->deferred && allow_defer && c->units == 0;
+  StepParams p{};
+  step_params(c, q, k, v, pos, out, evicted_pos, defer, p);
+  cudaError_t e;
   if (cfg.dtype == TOVA_DTYPE_BF16) {
     e = cfg.head_dim == 128 ? launch_step<__nv_bfloat16, 128>(c, p, st, defer)
                             : launch_step<__nv_bfloat16, 64>(c, p, st, defer);
@@ -888,6 +923,8 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   c->units = 0;
   c->recent = 0;
   c->chunk_ws = nullptr;
+  c->shard_on = false;
+  c->shard_scored = false;
   c->chunk_cluster = 0;
   c->deferred = false;
   c->pending = false;
@@ -922,6 +959,7 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
     delete c;
     return TOVA_ERR_CUDA;
   }
+  if (cudaMemsetAsync(c->base + lay.shard_words, 0, 8, st) != cudaSuccess) { delete c; return TOVA_ERR_CUDA; }
   // per-unit slot tables start at -1 (all bytes 0xff), accumulated scores at zero
   const size_t unit_bytes = (size_t)cfg->batch * cfg->n_kv_heads * cfg->capacity * 4;
   if (cudaMemsetAsync(c->base + lay.upos, 0xff, unit_bytes, st) != cudaSuccess ||
@@ -986,6 +1024,80 @@ int tova_cache_set_bulk_prefill(tova_cache* c, int32_t on) {
   if (!c) return TOVA_ERR_NULL;
   if (on < 0 || on > 2) return TOVA_ERR_BAD_SHAPE;
   c->bulk_fill = on;
+  return TOVA_OK;
+}
+
+size_t tova_shard_table_bytes(const tova_config* cfg, int32_t world) {
+  int why;
+  if (!config_ok(cfg, &why) || world < 1 || world > tova::SHARD_MAX_WORLD) return 0;
+  return 2 * (size_t)world * cfg->batch * make_layout(*cfg).ld * sizeof(float);   // two halves, used alternately
+}
+
+int tova_cache_set_shard(tova_cache* c, int32_t rank, int32_t world, int32_t n_q_heads_total, void* const* peer_tables,
+                         void* const* peer_flags) {
+  if (!c) return TOVA_ERR_NULL;
+  if (world < 1 || world > tova::SHARD_MAX_WORLD || rank < 0 || rank >= world || n_q_heads_total < c->cfg.n_q_heads)
+    return TOVA_ERR_BAD_SHAPE;
+  if (c->len != 0 || c->pending || !c->cfg.evict) return TOVA_ERR_BAD_SHAPE;
+  if (c->units != 0 || c->policy != tova::POLICY_TOVA) return TOVA_ERR_UNSUPPORTED;   // the layer-wise TOVA policy (with "+i")
+  if (!peer_tables || !peer_tables[rank]) return TOVA_ERR_NULL;
+  tova::ShardParams sp{};
+  sp.rank = rank;
+  sp.world = world;
+  sp.h_total = n_q_heads_total;
+  sp.tables = peer_flags ? world : 1;        // without flags the caller adds the ranks' vectors itself (a library all-reduce)
+  for (int r = 0; r < world; ++r) {
+    if (sp.tables > 1 && (!peer_tables[r] || !peer_flags[r])) return TOVA_ERR_NULL;
+    sp.parts[r] = static_cast<float*>(peer_tables[sp.tables > 1 ? r : rank]);
+    sp.flags[r] = sp.tables > 1 ? static_cast<int32_t*>(peer_flags[r]) : nullptr;
+    if (!aligned16(sp.parts[r])) return TOVA_ERR_ALIGN;
+  }
+  sp.epoch = reinterpret_cast<int32_t*>(c->base + c->lay.shard_words);
+  sp.ticket = sp.epoch + 1;
+  c->shard = sp;
+  c->shard_on = true;
+  c->shard_scored = false;
+  c->deferred = false;
+  return TOVA_OK;
+}
+
+int tova_decode_step_scores(tova_cache* c, const void* q, const void* k, const void* v, int32_t pos, float* out,
+                            void* cuda_stream) {
+  int rc = check_step_args(c, q, k, v, out);
+  if (rc != TOVA_OK) return rc;
+  if (!c->shard_on || c->shard_scored) return TOVA_ERR_BAD_SHAPE;   // not sharded, or a commit is outstanding
+  StepParams p{};
+  step_params(c, q, k, v, pos, out, nullptr, false, p);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e;
+  if (c->cfg.dtype == TOVA_DTYPE_BF16) {
+    e = c->cfg.head_dim == 128 ? launch_step<__nv_bfloat16, 128>(c, p, st, false) : launch_step<__nv_bfloat16, 64>(c, p, st, false);
+  } else {
+    e = c->cfg.head_dim == 128 ? launch_step<float, 128>(c, p, st, false) : launch_step<float, 64>(c, p, st, false);
+  }
+  if (e != cudaSuccess) return TOVA_ERR_CUDA;
+  c->shard_scored = true;
+  return TOVA_OK;
+}
+
+int tova_decode_step_commit(tova_cache* c, const void* k, const void* v, int32_t* evicted_pos, void* cuda_stream) {
+  if (!c || !k || !v) return TOVA_ERR_NULL;
+  if (!aligned16(k) || !aligned16(v)) return TOVA_ERR_ALIGN;
+  if (!c->shard_on || !c->shard_scored) return TOVA_ERR_BAD_SHAPE;
+  StepParams p{};
+  step_params(c, nullptr, k, v, 0, nullptr, evicted_pos, false, p);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (c->cfg.dtype == TOVA_DTYPE_BF16) {
+    if (c->cfg.head_dim == 128) tova::tova_shard_commit_kernel<__nv_bfloat16, 128><<<p.B, tova::SHARD_THREADS, 0, st>>>(p, c->shard);
+    else tova::tova_shard_commit_kernel<__nv_bfloat16, 64><<<p.B, tova::SHARD_THREADS, 0, st>>>(p, c->shard);
+  } else {
+    if (c->cfg.head_dim == 128) tova::tova_shard_commit_kernel<float, 128><<<p.B, tova::SHARD_THREADS, 0, st>>>(p, c->shard);
+    else tova::tova_shard_commit_kernel<float, 64><<<p.B, tova::SHARD_THREADS, 0, st>>>(p, c->shard);
+  }
+  if (cudaGetLastError() != cudaSuccess) return TOVA_ERR_CUDA;
+  c->launches += 1;
+  c->shard_scored = false;
+  if (c->len < c->cfg.capacity) c->len += 1;
   return TOVA_OK;
 }
 

@@ -87,6 +87,11 @@ def test_null_handles_are_rejected():
     assert L.tova_cache_units(None) == -1
     assert L.tova_cache_set_prefill_workspace(None, None, 0) == -1
     assert L.tova_cache_set_chunk_cluster(None, 0) == -1
+    assert L.tova_cache_set_shard(None, 0, 1, 8, None, None) == -1
+    assert L.tova_decode_step_scores(None, None, None, None, 0, None, None) == -1
+    assert L.tova_decode_step_commit(None, None, None, None, None) == -1
+    c = cfg()
+    assert L.tova_shard_table_bytes(ctypes.byref(c), 2) == 2 * 2 * 2 * 104 * 4 and L.tova_shard_table_bytes(ctypes.byref(c), 9) == 0
     assert tova.strerror(0) == "ok" and "aligned" in tova.strerror(-4)
 
 
