@@ -66,6 +66,10 @@
  * retained positions (the first i and the most recent k-i), hand-worked
  * traces of the 3-row example, "+0" equal to the plain policy, and the
  * invariant that a protected position is never reported as dropped.
+ * Position compression: the gap function's printed examples, "no gap above 10
+ * = ordinary rotary attention" against a library routine, invariance under a
+ * shift of all positions, and a restatement over the full token history with
+ * complex exponentials in double.
  * TOVA-head and H2O: per-head and accumulated-score restatements over the full
  * token history in double (order-preserving lists), hand-worked traces of the
  * 3-row example in exact arithmetic, "one head = the layer policy", H2O with
@@ -148,6 +152,13 @@ static void attend(int H, int Hkv, int D, int cap, REAL scale, int n,
 #define POLICY_TOVA 0
 #define POLICY_WINDOW 1
 
+static void drop_and_insert(int H, int Hkv, int D, int cap, int policy, int keep_first,
+                            int *len, int *pos, REAL *K, REAL *V,
+                            const REAL *k_new, const REAL *v_new,
+                            int pos_t, int forced,
+                            int *evicted_pos, int *victim, int *argmin, REAL *gap,
+                            REAL *mean_out, REAL *work);
+
 static void step_one(int H, int Hkv, int D, int cap, REAL scale, int policy, int keep_first,
                      int *len, int *pos, REAL *K, REAL *V,
                      const REAL *q, const REAL *k_new, const REAL *v_new,
@@ -155,11 +166,27 @@ static void step_one(int H, int Hkv, int D, int cap, REAL scale, int policy, int
                      REAL *out, int *evicted_pos, int *victim, int *argmin, REAL *gap,
                      REAL *mean_out, REAL *work)
 {
+    attend(H, Hkv, D, cap, scale, *len, K, V, q, k_new, v_new, out, work);
+    drop_and_insert(H, Hkv, D, cap, policy, keep_first, len, pos, K, V, k_new, v_new, pos_t, forced,
+                    evicted_pos, victim, argmin, gap, mean_out, work);
+}
+
+/*
+ * The second half of a step: given the weights of the new query over the
+ * appended state (work[h][0..n], from attend), keep all rows while the state
+ * has room, else pick the row to delete and let the new token take its place.
+ * Arguments as for step_one.
+ */
+static void drop_and_insert(int H, int Hkv, int D, int cap, int policy, int keep_first,
+                            int *len, int *pos, REAL *K, REAL *V,
+                            const REAL *k_new, const REAL *v_new,
+                            int pos_t, int forced,
+                            int *evicted_pos, int *victim, int *argmin, REAL *gap,
+                            REAL *mean_out, REAL *work)
+{
     const int n = *len;          /* rows before the append */
     const int m = n + 1;         /* rows after the append (Eq. 6) */
     const int ld = cap + 1;
-
-    attend(H, Hkv, D, cap, scale, n, K, V, q, k_new, v_new, out, work);
 
     *gap = 0;
     if (m <= cap) {              /* Algorithm 1: num_kv <= cache_max_size -> keep all */
@@ -409,6 +436,133 @@ int tova_oracle_step_units(int B, int H, int Hkv, int D, int cap, REAL scale, in
                    argmin + (size_t)b * U, gap + (size_t)b * U,
                    score_out ? score_out + (size_t)b * U * ld : NULL, work);
         free(work);
+    }
+    return bad ? -1 : 0;
+}
+
+/* ------------------------------------------------------------------------
+ * Position compression for streams longer than the training context
+ * (Section "Extrapolation with TOVA"): the keys are cached WITHOUT rotary
+ * embedding; at every step the retained tokens and the new token, taken in
+ * position order, get new positions in which the gap g between neighbours is
+ * ln(ln(g)), or g itself while g <= 10; the rotary embedding is then applied
+ * with those positions to the cached keys and to the query, and the step
+ * proceeds as usual (the un-rotated key of the new token is what is cached).
+ * Readings: the new positions accumulate along the chain (p'_{m+1} = p'_m +
+ * f(p_{m+1} - p_m)); the earliest retained token sits at 0 - attention depends
+ * on differences only, so the origin is immaterial; rotary embedding in the
+ * rotate-half form (component d pairs with d + D/2, angle p' * base^(-2d/D)),
+ * as in the model families the paper runs; the chain of new positions and the
+ * angles are worked out in double, whatever REAL is.
+ * ------------------------------------------------------------------------ */
+double tova_oracle_compress_gap(int g)
+{
+    return (g <= 10) ? (double)g : log(log((double)g));
+}
+
+/* x[0..D) rotated by position p (rotate-half pairs), into y. */
+static void rope_rotate(const REAL *x, REAL *y, int D, double p, double base)
+{
+    const int half = D / 2;
+    for (int d = 0; d < half; ++d) {
+        const double ang = p * pow(base, -2.0 * (double)d / (double)D);
+        const REAL c = (REAL)cos(ang), s = (REAL)sin(ang);
+        const REAL a = x[d], b = x[d + half];
+        y[d] = a * c - b * s;
+        y[d + half] = b * c + a * s;
+    }
+}
+
+/*
+ * One token for one sequence with position compression.  As step_one, plus:
+ *   rope_base      base of the rotary embedding (10000 in the LLaMA family)
+ *   cpos_out       [cap+1] or NULL: the new position of every candidate
+ *                  (slot order, the new token last)
+ *   rot            scratch [Hkv][cap+1][D] + [H][D] REAL
+ */
+static void step_one_poscomp(int H, int Hkv, int D, int cap, REAL scale, int policy, int keep_first, double rope_base,
+                             int *len, int *pos, REAL *K, REAL *V,
+                             const REAL *q, const REAL *k_new, const REAL *v_new,
+                             int pos_t, int forced,
+                             REAL *out, int *evicted_pos, int *victim, int *argmin, REAL *gap,
+                             REAL *mean_out, double *cpos_out, REAL *work, REAL *rot)
+{
+    const int n = *len, m = n + 1;
+    /* candidates in position order: insertion sort of (position, candidate index) */
+    int *order = (int *)malloc(sizeof(int) * (size_t)m);
+    double *cp = (double *)malloc(sizeof(double) * (size_t)m);
+    for (int j = 0; j < m; ++j) {
+        const int pj = (j < n) ? pos[j] : pos_t;
+        int i = j;
+        while (i > 0) {
+            const int o = order[i - 1];
+            const int po = (o < n) ? pos[o] : pos_t;
+            if (po <= pj) break;
+            order[i] = o;
+            --i;
+        }
+        order[i] = j;
+    }
+    /* the chain of compressed positions */
+    double acc = 0.0;
+    for (int r = 0; r < m; ++r) {
+        const int j = order[r];
+        if (r > 0) {
+            const int jp = order[r - 1];
+            const int g = ((j < n) ? pos[j] : pos_t) - ((jp < n) ? pos[jp] : pos_t);
+            acc += tova_oracle_compress_gap(g);
+        }
+        cp[j] = acc;
+    }
+    if (cpos_out) for (int j = 0; j <= cap; ++j) cpos_out[j] = (j < m) ? cp[j] : 0.0;
+    /* rotated copies: keys of the state as [Hkv][cap][D] (stride cap, as attend expects), the new key, the query */
+    REAL *Krot = rot;
+    REAL *knew_rot = rot + (size_t)Hkv * cap * D;
+    REAL *q_rot = knew_rot + (size_t)Hkv * D;
+    for (int kv = 0; kv < Hkv; ++kv) {
+        for (int j = 0; j < n; ++j)
+            rope_rotate(K + ((size_t)kv * cap + j) * D, Krot + ((size_t)kv * cap + j) * D, D, cp[j], rope_base);
+        rope_rotate(k_new + (size_t)kv * D, knew_rot + (size_t)kv * D, D, cp[n], rope_base);
+    }
+    for (int h = 0; h < H; ++h) rope_rotate(q + (size_t)h * D, q_rot + (size_t)h * D, D, cp[n], rope_base);
+    attend(H, Hkv, D, cap, scale, n, Krot, V, q_rot, knew_rot, v_new, out, work);
+    drop_and_insert(H, Hkv, D, cap, policy, keep_first, len, pos, K, V, k_new, v_new, pos_t, forced,
+                    evicted_pos, victim, argmin, gap, mean_out, work);
+    free(order);
+    free(cp);
+}
+
+/* Batch wrapper; layouts as tova_oracle_step_policy, cpos_out [B][cap+1] doubles or NULL. */
+int tova_oracle_step_poscomp(int B, int H, int Hkv, int D, int cap, REAL scale, int policy, int keep_first,
+                             double rope_base,
+                             int *len, int *pos, REAL *K, REAL *V,
+                             const REAL *q, const REAL *k_new, const REAL *v_new,
+                             int pos_t, const int *forced,
+                             REAL *out, int *evicted_pos, int *victim, int *argmin, REAL *gap,
+                             REAL *mean_out, double *cpos_out, int nthreads)
+{
+    if (B < 1 || H < 1 || Hkv < 1 || D < 2 || D % 2 || cap < 1 || H % Hkv != 0 || !(rope_base > 1.0)) return -1;
+    if ((policy != POLICY_TOVA && policy != POLICY_WINDOW) || keep_first < 0) return -1;
+    const size_t ld = (size_t)cap + 1;
+    if (nthreads < 1) nthreads = 1;
+    int bad = 0;
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(nthreads) schedule(static)
+#endif
+    for (int b = 0; b < B; ++b) {
+        REAL *work = (REAL *)malloc(sizeof(REAL) * (size_t)(H + 1) * ld);
+        REAL *rot = (REAL *)malloc(sizeof(REAL) * ((size_t)Hkv * ld + (size_t)H) * D);
+        if (!work || !rot || len[b] < 0 || len[b] > cap) { bad = 1; free(work); free(rot); continue; }
+        step_one_poscomp(H, Hkv, D, cap, scale, policy, keep_first, rope_base,
+                         len + b, pos + (size_t)b * cap,
+                         K + (size_t)b * Hkv * cap * D, V + (size_t)b * Hkv * cap * D,
+                         q + (size_t)b * H * D, k_new + (size_t)b * Hkv * D, v_new + (size_t)b * Hkv * D,
+                         pos_t, forced ? forced[b] : -1,
+                         out + (size_t)b * H * D, evicted_pos + b, victim + b, argmin + b, gap + b,
+                         mean_out ? mean_out + (size_t)b * ld : NULL, cpos_out ? cpos_out + (size_t)b * ld : NULL,
+                         work, rot);
+        free(work);
+        free(rot);
     }
     return bad ? -1 : 0;
 }

@@ -40,10 +40,18 @@ def _lib(precision: str):
         lib.tova_oracle_step.restype = ctypes.c_int
         lib.tova_oracle_step_policy.restype = ctypes.c_int
         lib.tova_oracle_step_units.restype = ctypes.c_int
+        lib.tova_oracle_step_poscomp.restype = ctypes.c_int
+        lib.tova_oracle_compress_gap.restype = ctypes.c_double
+        lib.tova_oracle_compress_gap.argtypes = [ctypes.c_int]
         lib.tova_oracle_real_bytes.restype = ctypes.c_int
         lib.tova_oracle_max_threads.restype = ctypes.c_int
         _LIBS[precision] = lib
     return _LIBS[precision]
+
+
+def compress_gap(g: int) -> float:
+    """The checker's gap function of the position compression (double build)."""
+    return float(_lib("f64").tova_oracle_compress_gap(int(g)))
 
 
 def host_threads() -> int:
@@ -63,7 +71,10 @@ class OracleCache:
 
     def __init__(self, batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
                  capacity: int, sm_scale: float = 0.0, precision: str = "f32",
-                 threads: Optional[int] = None, policy: str = "tova", keep_first: int = 0):
+                 threads: Optional[int] = None, policy: str = "tova", keep_first: int = 0,
+                 rope_base: float = 0.0):
+        """rope_base > 0: position compression (Section "Extrapolation with TOVA"): keys are cached without
+        rotary embedding, which is applied at every step with the compressed positions."""
         if n_q_heads % n_kv_heads:
             raise ValueError("n_q_heads must be a multiple of n_kv_heads")
         self.B, self.H, self.Hkv, self.D, self.cap = batch, n_q_heads, n_kv_heads, head_dim, capacity
@@ -76,6 +87,8 @@ class OracleCache:
         self.threads = threads or host_threads()
         self.policy = {"tova": 0, "window": 1}[policy]   # Section 4 / Section 4.1
         self.keep_first = int(keep_first)                  # "+i": positions 0..i-1 are never dropped
+        self.rope_base = float(rope_base)
+        self.last_cpos = None                              # compressed positions of the last step's candidates
         self.len = np.zeros(batch, np.int32)
         self.pos = np.full((batch, capacity), -1, np.int32)
         self.K = np.zeros((batch, n_kv_heads, capacity, head_dim), self.real)
@@ -99,6 +112,20 @@ class OracleCache:
         gap = np.zeros(B, self.real)
         mean = np.zeros((B, cap + 1), self.real) if want_mean else None
         f = None if forced is None else np.ascontiguousarray(forced, np.int32)
+        if self.rope_base > 0.0:
+            cpos = np.zeros((B, cap + 1), np.float64)
+            rc = self.lib.tova_oracle_step_poscomp(
+                ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D),
+                ctypes.c_int(cap), self.creal(self.scale), ctypes.c_int(self.policy), ctypes.c_int(self.keep_first),
+                ctypes.c_double(self.rope_base),
+                _ptr(self.len), _ptr(self.pos), _ptr(self.K), _ptr(self.V),
+                _ptr(q), _ptr(k_new), _ptr(v_new), ctypes.c_int(int(pos_t)), _ptr(f),
+                _ptr(out), _ptr(ev), _ptr(victim), _ptr(argmin), _ptr(gap), _ptr(mean), _ptr(cpos),
+                ctypes.c_int(self.threads))
+            if rc != 0:
+                raise RuntimeError("tova_oracle_step_poscomp rejected its arguments")
+            self.last_cpos = cpos
+            return out, ev, victim, argmin, gap, mean
         rc = self.lib.tova_oracle_step_policy(
             ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D),
             ctypes.c_int(cap), self.creal(self.scale), ctypes.c_int(self.policy), ctypes.c_int(self.keep_first),
