@@ -251,6 +251,35 @@ int tova_cache_read_scores(const tova_cache* c, float* scores, void* cuda_stream
 /* Slot tables this cache keeps per sequence: Hkv under a head-wise policy, else 1. */
 int32_t tova_cache_units(const tova_cache* c);
 
+/* Position compression for streams longer than the model's training context
+ * (Section "Extrapolation with TOVA").  The positional encoding of the cached
+ * tokens is adapted so that no distance unseen in training occurs: between
+ * neighbouring retained tokens (in position order, the new token last) a gap g
+ * becomes ln(ln(g)), and stays g while g <= 10; the new positions accumulate
+ * along that chain, the earliest retained token at 0 (attention depends on
+ * differences only).  In this mode the LIBRARY applies the rotary embedding:
+ * callers pass q and k WITHOUT it, keys are cached as given, and at every step
+ * the query and every cached key are rotated at their current compressed
+ * position (rotate-half pairs d, d + D/2, angle p' * rope_base^(-2d/D), the
+ * convention of the model families the paper runs; rope_base 10000 there).
+ * Everything after the logits is the ordinary step, under the TOVA or Window
+ * policy with or without protected first positions.
+ *   tova_position_workspace_bytes  device bytes needed: a (cos, sin) table of
+ *        B*(capacity+1)*D/2 pairs, the rotated query, the positions.
+ *   tova_cache_set_position_compression  dev_mem: 256-byte aligned device
+ *        memory of that size, owned by the caller, to outlive the handle (NULL:
+ *        off); only while the state is empty; capacity up to about 8000 rows
+ *        (TOVA_ERR_UNSUPPORTED beyond, and together with head-wise policies or
+ *        sharding).  The step then takes three launches and a slower streaming
+ *        kernel (a table read and a rotation per cached row); prompts go token
+ *        by token; deferred eviction is ignored.
+ *   tova_cache_read_compressed_positions  cpos [B,capacity+1] doubles on the
+ *        DEVICE: the positions the LAST step used, by slot, the new token's at
+ *        index min(tokens before it, capacity). */
+size_t tova_position_workspace_bytes(const tova_config* cfg);
+int tova_cache_set_position_compression(tova_cache* c, void* dev_mem, size_t dev_bytes, float rope_base);
+int tova_cache_read_compressed_positions(const tova_cache* c, double* cpos, void* cuda_stream);
+
 /* One layer sharded by KV head over several GPUs (one process per GPU).
  * Algorithm 1 averages the last query's weights over the heads of the layer - a
  * sum over heads - so ranks that each hold some of the KV heads (with the

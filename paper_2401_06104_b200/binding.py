@@ -70,6 +70,12 @@ def lib() -> ctypes.CDLL:
         L.tova_prefill_workspace_bytes.argtypes = [ctypes.POINTER(tova_config)]
         L.tova_cache_set_prefill_workspace.restype = ctypes.c_int
         L.tova_cache_set_prefill_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+        L.tova_position_workspace_bytes.restype = ctypes.c_size_t
+        L.tova_position_workspace_bytes.argtypes = [ctypes.POINTER(tova_config)]
+        L.tova_cache_set_position_compression.restype = ctypes.c_int
+        L.tova_cache_set_position_compression.argtypes = [vp, vp, ctypes.c_size_t, ctypes.c_float]
+        L.tova_cache_read_compressed_positions.restype = ctypes.c_int
+        L.tova_cache_read_compressed_positions.argtypes = [vp, vp, vp]
         L.tova_shard_table_bytes.restype = ctypes.c_size_t
         L.tova_shard_table_bytes.argtypes = [ctypes.POINTER(tova_config), i32]
         L.tova_cache_set_shard.restype = ctypes.c_int
@@ -205,6 +211,28 @@ class TovaCache:
                                                       mem.numel() - off), "tova_cache_set_prefill_workspace")
         self._prefill_ws = mem
         return mem
+
+    def tova_cache_set_position_compression(self, rope_base: float = 10000.0, on: bool = True) -> None:
+        """Switches the position compression on (allocating its workspace) or off; callers then pass q and k
+        without rotary embedding."""
+        if not on:
+            _check(lib().tova_cache_set_position_compression(self._h, None, 0, 0.0), "tova_cache_set_position_compression")
+            self._poscomp_ws = None
+            return
+        need = int(lib().tova_position_workspace_bytes(ctypes.byref(self.cfg)))
+        mem = torch.empty(need + 256, dtype=torch.uint8, device=self.device)
+        off = (-mem.data_ptr()) % 256
+        _check(lib().tova_cache_set_position_compression(self._h, ctypes.c_void_p(mem.data_ptr() + off), need,
+                                                         float(rope_base)), "tova_cache_set_position_compression")
+        self._poscomp_ws = mem
+
+    def tova_cache_read_compressed_positions(self, stream=None):
+        c = self.cfg
+        cp = torch.empty(c.batch, c.capacity + 1, dtype=torch.float64, device=self.device)
+        _check(lib().tova_cache_read_compressed_positions(self._h, _p(cp), _stream(stream)),
+               "tova_cache_read_compressed_positions")
+        torch.cuda.synchronize(self.device)
+        return cp.cpu()
 
     def tova_shard_table_bytes(self, world: int) -> int:
         return int(lib().tova_shard_table_bytes(ctypes.byref(self.cfg), int(world)))

@@ -21,6 +21,7 @@
 #include "tova_units.cuh"
 #include "tova_chunk.cuh"
 #include "tova_shard.cuh"
+#include "tova_poscomp.cuh"
 
 namespace {
 
@@ -134,6 +135,9 @@ struct tova_cache {
   Layout lay;
   unsigned char* base;
   // chunked prompt path: caller-provided workspace and tiled views of its staging tiles
+  // position compression: caller-provided workspace (table of cosines and sines, rotated query, positions)
+  unsigned char* poscomp_ws;
+  tova::PosCompParams poscomp;
   // state sharded by KV head over several ranks (tova_cache_set_shard)
   bool shard_on, shard_scored;
   tova::ShardParams shard;
@@ -357,6 +361,7 @@ cudaError_t launch_split_mma(int dev, const StepParams& p, const CUtensorMap& mk
 }
 
 void set_combine_threads(StepParams& p, int ct);
+constexpr size_t POSCOMP_SMEM_LIMIT = 200 * 1024;
 
 template <typename T, int D>
 cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, bool defer) {
@@ -366,6 +371,23 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, boo
     e = cudaStreamWaitEvent(st, c->ev_join, 0);
     if (e != cudaSuccess) return e;
     c->pending = false;
+  }
+  if (c->poscomp_ws) {
+    // Position compression: new positions and their cosines/sines per sequence, the rotating streaming kernel,
+    // then the ordinary combine kernel (merge, outputs, victim, insert of the un-rotated key).
+    static std::atomic<bool> pc_configured[64];
+    if (c->device >= 0 && c->device < 64 && !pc_configured[c->device]) {
+      if ((e = cudaFuncSetAttribute(tova::tova_poscomp_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)POSCOMP_SMEM_LIMIT)) != cudaSuccess) return e;
+      pc_configured[c->device] = true;
+    }
+    tova::tova_poscomp_kernel<T, D><<<p.B, tova::POSCOMP_THREADS, tova::poscomp_smem_bytes(p.cap, D), st>>>(p, c->poscomp);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    tova::tova_split_rope_kernel<T, D><<<grid, 32, 0, st>>>(p, c->poscomp);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = launch_combine<T, D>(c->device, p, st)) != cudaSuccess) return e;
+    c->launches += 3;
+    return cudaSuccess;
   }
   if constexpr (std::is_same<T, __nv_bfloat16>::value) {
     e = c->use_mma ? launch_split_mma<D>(c->device, p, c->map_k, c->map_v, grid, st)
@@ -614,6 +636,11 @@ void step_params(tova_cache* c, const void* q, const void* k, const void* v, int
   p.fuse_out = (c->fuse_merge && fused_merge_fits(cfg, c->chunk_rows, c->sm_count)) ? 1 : 0;
   p.merge_ctas = p.fuse_out ? (p.n_chunks + tova::SPLIT_MERGE_MAX_WARPS - 1) / tova::SPLIT_MERGE_MAX_WARPS : 1;
   if (p.merge_ctas < 1) p.merge_ctas = 1;
+  if (c->poscomp_ws) {         // the rotating streaming kernel: partials through global memory, 4 heads per warp
+    p.fuse_out = 0;
+    p.merge_ctas = 1;
+    p.hgroups = (p.G + tova::ROPE_UNIT_HEADS - 1) / tova::ROPE_UNIT_HEADS;
+  }
   if (p.fuse_out && defer) {   // the split kernel keeps copies of the new token's rows for the later insert
     p.k_stage = base + c->lay.df_k;
     p.v_stage = base + c->lay.df_v;
@@ -625,7 +652,7 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
   const tova_config& cfg = c->cfg;
   if (c->len >= cfg.capacity && !cfg.evict) return TOVA_ERR_FULL;
   if (c->shard_on) return TOVA_ERR_BAD_SHAPE;   // a sharded layer steps through its two-phase calls
-  const bool defer = c->deferred && allow_defer && c->units == 0;
+  const bool defer = c->deferred && allow_defer && c->units == 0 && !c->poscomp_ws;
   StepParams p{};
   step_params(c, q, k, v, pos, out, evicted_pos, defer, p);
   cudaError_t e;
@@ -923,6 +950,7 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   c->units = 0;
   c->recent = 0;
   c->chunk_ws = nullptr;
+  c->poscomp_ws = nullptr;
   c->shard_on = false;
   c->shard_scored = false;
   c->chunk_cluster = 0;
@@ -1004,6 +1032,7 @@ int tova_cache_set_policy(tova_cache* c, int32_t policy, int32_t arg) {
     c->units = 0;
     return TOVA_OK;
   }
+  if (c->poscomp_ws || c->shard_on) return TOVA_ERR_UNSUPPORTED;   // per-unit policies: not with compression or sharding
   if (policy == TOVA_POLICY_TOVA_HEAD) {
     if (arg != 0) return TOVA_ERR_BAD_SHAPE;
     c->policy = tova::POLICY_TOVA_HEAD;
@@ -1027,6 +1056,54 @@ int tova_cache_set_bulk_prefill(tova_cache* c, int32_t on) {
   return TOVA_OK;
 }
 
+namespace {
+struct PosCompLayout { size_t table, q_rot, cpos, total; };
+PosCompLayout make_poscomp_layout(const tova_config& c) {
+  PosCompLayout L{};
+  const size_t B = c.batch, H = c.n_q_heads, D = c.head_dim, cap = c.capacity;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L.table = take(B * (cap + 1) * (D / 2) * 8);
+  L.q_rot = take(B * H * D * 4);
+  L.cpos = take(B * (cap + 1) * 8);
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+size_t tova_position_workspace_bytes(const tova_config* cfg) {
+  int why;
+  if (!config_ok(cfg, &why)) return 0;
+  return make_poscomp_layout(*cfg).total;
+}
+
+int tova_cache_set_position_compression(tova_cache* c, void* dev_mem, size_t dev_bytes, float rope_base) {
+  if (!c) return TOVA_ERR_NULL;
+  if (c->len != 0 || c->pending) return TOVA_ERR_BAD_SHAPE;      // keys must be cached un-rotated from the first token
+  if (!dev_mem) { c->poscomp_ws = nullptr; return TOVA_OK; }
+  if (!(rope_base > 1.f) || !std::isfinite(rope_base)) return TOVA_ERR_BAD_SHAPE;
+  if (c->units != 0 || c->shard_on || tova::poscomp_smem_bytes(c->cfg.capacity, c->cfg.head_dim) > POSCOMP_SMEM_LIMIT)
+    return TOVA_ERR_UNSUPPORTED;
+  if (reinterpret_cast<uintptr_t>(dev_mem) % ALIGN != 0) return TOVA_ERR_ALIGN;
+  const PosCompLayout L = make_poscomp_layout(c->cfg);
+  if (dev_bytes < L.total) return TOVA_ERR_WORKSPACE;
+  unsigned char* ws = static_cast<unsigned char*>(dev_mem);
+  c->poscomp.table = reinterpret_cast<float2*>(ws + L.table);
+  c->poscomp.q_rot = reinterpret_cast<float*>(ws + L.q_rot);
+  c->poscomp.cpos = reinterpret_cast<double*>(ws + L.cpos);
+  c->poscomp.rope_base = (double)rope_base;
+  c->poscomp_ws = ws;
+  return TOVA_OK;
+}
+
+int tova_cache_read_compressed_positions(const tova_cache* c, double* cpos, void* cuda_stream) {
+  if (!c || !cpos) return TOVA_ERR_NULL;
+  if (!c->poscomp_ws) return TOVA_ERR_UNSUPPORTED;
+  const size_t bytes = (size_t)c->cfg.batch * (c->cfg.capacity + 1) * 8;
+  return cudaMemcpyAsync(cpos, c->poscomp.cpos, bytes, cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(cuda_stream)) ==
+                 cudaSuccess ? TOVA_OK : TOVA_ERR_CUDA;
+}
+
 size_t tova_shard_table_bytes(const tova_config* cfg, int32_t world) {
   int why;
   if (!config_ok(cfg, &why) || world < 1 || world > tova::SHARD_MAX_WORLD) return 0;
@@ -1039,7 +1116,7 @@ int tova_cache_set_shard(tova_cache* c, int32_t rank, int32_t world, int32_t n_q
   if (world < 1 || world > tova::SHARD_MAX_WORLD || rank < 0 || rank >= world || n_q_heads_total < c->cfg.n_q_heads)
     return TOVA_ERR_BAD_SHAPE;
   if (c->len != 0 || c->pending || !c->cfg.evict) return TOVA_ERR_BAD_SHAPE;
-  if (c->units != 0 || c->policy != tova::POLICY_TOVA) return TOVA_ERR_UNSUPPORTED;   // the layer-wise TOVA policy (with "+i")
+  if (c->units != 0 || c->policy != tova::POLICY_TOVA || c->poscomp_ws) return TOVA_ERR_UNSUPPORTED;   // layer-wise TOVA (with "+i")
   if (!peer_tables || !peer_tables[rank]) return TOVA_ERR_NULL;
   tova::ShardParams sp{};
   sp.rank = rank;
@@ -1139,7 +1216,7 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
     const int room = c->cfg.capacity - c->len;
     const int F = n_tokens < room ? n_tokens : room;
     // (the per-unit policies keep their own slot tables and scores: token by token)
-    if (c->bulk_fill && c->fill_maps && F >= BULK_FILL_MIN_TOKENS && c->units == 0) {
+    if (c->bulk_fill && c->fill_maps && F >= BULK_FILL_MIN_TOKENS && c->units == 0 && !c->poscomp_ws) {
       rc = launch_fill(c, q, k, v, F, first_pos, out, evicted_pos, static_cast<cudaStream_t>(cuda_stream));
       if (rc != TOVA_OK) return rc;
       done = F;
@@ -1147,7 +1224,8 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
   }
   // Tokens that meet a full state: chunks of up to 64 through the caller's workspace, where one was given
   // (TOVA policy, with or without protected first positions; bf16 states).
-  const bool chunked = c->chunk_ws && c->bulk_fill && c->cfg.evict && c->units == 0 && c->policy == tova::POLICY_TOVA;
+  const bool chunked = c->chunk_ws && c->bulk_fill && c->cfg.evict && c->units == 0 && c->policy == tova::POLICY_TOVA &&
+                       !c->poscomp_ws;
   for (int32_t t = done; t < n_tokens;) {
     if (chunked && c->len == c->cfg.capacity && n_tokens - t >= CHUNK_MIN_TOKENS) {
       const int C = n_tokens - t < tova::CHUNK_TOKENS ? n_tokens - t : tova::CHUNK_TOKENS;

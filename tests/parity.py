@@ -61,7 +61,7 @@ POLICIES = {"tova": tova.TOVA_POLICY_TOVA, "window": tova.TOVA_POLICY_WINDOW,
 
 def make_cache(w: W.Workload, sm_scale: float = 0.0, evict: bool = True, chunk_rows: int = 0,
                fused_merge: bool = True, policy: str = "tova", keep_first: int = 0, prefill_ws: bool = False,
-               chunk_cluster: int = 0):
+               chunk_cluster: int = 0, rope_base: float = 0.0):
     c = tova.TovaCache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, dtype=w.dtype,
                        sm_scale=sm_scale, evict=evict)
     if chunk_rows:
@@ -70,6 +70,8 @@ def make_cache(w: W.Workload, sm_scale: float = 0.0, evict: bool = True, chunk_r
         c.tova_cache_set_fused_merge(False)
     if policy != "tova" or keep_first:
         c.tova_cache_set_policy(POLICIES[policy], keep_first)
+    if rope_base:                        # position compression: q and k come without rotary embedding
+        c.tova_cache_set_position_compression(rope_base)
     if prefill_ws:                       # prompt tokens that meet a full state go in chunks of up to 64
         c.tova_cache_set_prefill_workspace()
         if chunk_cluster:
@@ -97,7 +99,8 @@ def run_lockstep(w: W.Workload, n_tokens: int, *, seqs: Optional[Sequence[int]] 
                  sm_scale: float = 0.0, layer: int = 0, cache=None, oracle=None,
                  first_pos: int = 0, check_state_every: int = 4, direct_fill: bool = False,
                  fused_merge: bool = True, policy: str = "tova", keep_first: int = 0,
-                 period: int = 0, prefill_ws: bool = False, chunk_cluster: int = 0) -> ParityReport:
+                 period: int = 0, prefill_ws: bool = False, chunk_cluster: int = 0,
+                 rope_base: float = 0.0) -> ParityReport:
     """Feed n_tokens tokens to both sides and compare at every token.
 
     direct_fill: while the state is filling nothing is dropped (Section 3.3), so
@@ -114,9 +117,10 @@ def run_lockstep(w: W.Workload, n_tokens: int, *, seqs: Optional[Sequence[int]] 
     own = cache is None
     cache = cache or make_cache(w, sm_scale=sm_scale, chunk_rows=chunk_rows, fused_merge=fused_merge,
                                 policy=policy, keep_first=keep_first, prefill_ws=prefill_ws,
-                                chunk_cluster=chunk_cluster)
+                                chunk_cluster=chunk_cluster, rope_base=rope_base)
     orc = oracle or OracleCache(len(seqs), w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity,
-                                sm_scale=sm_scale, precision="f32", policy=policy, keep_first=keep_first)
+                                sm_scale=sm_scale, precision="f32", policy=policy, keep_first=keep_first,
+                                rope_base=rope_base)
     tol = out_tol(w)
     rep = ParityReport()
     done = 0

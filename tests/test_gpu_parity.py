@@ -486,6 +486,53 @@ def test_unit_policy_hand_worked_traces_on_gpu():
             assert st["status"] == 0
 
 
+# ---------------------------------------------------------------------------
+# position compression (Section "Extrapolation with TOVA")
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("H,Hkv,D,dtype,cap,B,policy,keep", [
+    (8, 8, 128, W.DTYPE_BF16, 64, 2, "tova", 0),      # MHA
+    (8, 2, 128, W.DTYPE_BF16, 100, 2, "tova", 2),     # GQA 4, two protected positions
+    (16, 1, 64, W.DTYPE_BF16, 70, 1, "tova", 0),      # GQA 16 (four head groups per KV head), D = 64
+    (4, 4, 64, W.DTYPE_FP32, 48, 2, "tova", 0),       # fp32
+    (4, 2, 128, W.DTYPE_FP32, 40, 1, "window", 4),    # Window+4 on compressed positions
+])
+def test_position_compression_against_the_checker(H, Hkv, D, dtype, cap, B, policy, keep):
+    """q and k come without rotary embedding; 500 tokens through a small state leave retained tokens hundreds of
+    positions apart, so the ln ln rule is at work in almost every step.  Dropped positions and slot tables exact,
+    outputs within tolerance, and the compressed positions of the last step equal to the checker's."""
+    w = MISTRAL.scaled(batch=B, n_q_heads=H, n_kv_heads=Hkv, head_dim=D, dtype=dtype, capacity=cap)
+    assert not w.rope
+    rep = run_lockstep(w, 500, block=50, rope_base=10000.0, policy=policy, keep_first=keep)
+    assert rep.evictions == B * (500 - cap)
+    cp = rep.cache.tova_cache_read_compressed_positions().numpy()
+    assert np.abs(cp - rep.oracle.last_cpos).max() < 1e-9
+    pos = rep.cache.tova_cache_read()["positions"].numpy()
+    assert max(np.diff(np.sort(pos[0]))) > 10                      # gaps above 10 were there to compress
+    assert rep.cache.tova_cache_launches() == 1 + 3 * 500
+
+
+def test_position_compression_argument_errors():
+    w = MISTRAL.scaled(batch=1, n_q_heads=2, n_kv_heads=2, capacity=8)
+    c = make_cache(w)
+    with pytest.raises(tova.TovaError) as e:
+        c.tova_cache_read_compressed_positions()
+    assert e.value.code == -3
+    q = torch.zeros(1, 2, 128, dtype=torch.bfloat16, device="cuda:0")
+    c.tova_decode_step(q, q, q, 0, torch.zeros(1, 2, 128, device="cuda:0"))
+    with pytest.raises(tova.TovaError):            # keys already cached: too late to switch
+        c.tova_cache_set_position_compression(10000.0)
+    big = make_cache(MISTRAL.scaled(batch=1, n_q_heads=2, n_kv_heads=2, capacity=20000))
+    with pytest.raises(tova.TovaError) as e:
+        big.tova_cache_set_position_compression(10000.0)
+    assert e.value.code == -3
+    d = make_cache(w)
+    d.tova_cache_set_position_compression(10000.0)
+    with pytest.raises(tova.TovaError):
+        d.tova_cache_set_policy(tova.TOVA_POLICY_TOVA_HEAD, 0)
+    d.tova_cache_set_position_compression(on=False)
+    d.tova_cache_set_policy(tova.TOVA_POLICY_TOVA_HEAD, 0)
+
+
 def test_policy_argument_errors():
     w = LLAMA.scaled(batch=1, n_q_heads=2, n_kv_heads=2, capacity=8)
     c = make_cache(w)
