@@ -54,6 +54,9 @@ def parse_args():
                     help="which row is dropped once the state is over capacity")
     ap.add_argument("--keep-first", type=int, default=0,
                     help="the +i of Window+i / TOVA+i; under H2O the size of the recent window (0 = half the state)")
+    ap.add_argument("--position-compression", type=float, default=0.0, metavar="BASE",
+                    help="time the position-compression mode (rotary embedding applied by the library with the "
+                         "compressed positions); BASE = rotary base, e.g. 10000")
     ap.add_argument("--no-fused-merge", action="store_true",
                     help="merge the chunk partials through global memory even where a cluster could")
     ap.add_argument("--deferred", action="store_true", help="force deferred eviction on")
@@ -285,6 +288,8 @@ def measure(w, args, dev, world, layers=0, want_e2e=False):
             c.tova_cache_set_chunk_rows(args.chunk_rows)
         if args.no_fused_merge:
             c.tova_cache_set_fused_merge(False)
+        if args.position_compression:
+            c.tova_cache_set_position_compression(args.position_compression)
         if args.policy != "tova" or args.keep_first:
             c.tova_cache_set_policy({"tova": tova.TOVA_POLICY_TOVA, "window": tova.TOVA_POLICY_WINDOW,
                                      "tova_head": tova.TOVA_POLICY_TOVA_HEAD, "h2o_layer": tova.TOVA_POLICY_H2O_LAYER,
