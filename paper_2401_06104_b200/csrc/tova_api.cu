@@ -198,9 +198,13 @@ inline int split_launch_attrs(const StepParams& p, cudaLaunchAttribute* at) {
   at[1].val.clusterDim.z = 1;
   return 2;
 }
-// Shared memory behind the rings for a CTA's merged partial (cluster merge only).
+// Shared memory behind the rings for a CTA's inbox of the cluster merge: one partial from every CTA of the
+// cluster for each of the heads this CTA owns (heads dealt out over the CTAs, rounded up).
+inline size_t cluster_inbox_bytes(int heads, int D) {
+  return sizeof(float) * (size_t)(heads + tova::COMBINE_CLUSTER_MAX) * (D + tova::PART_STRIDE_EXTRA);
+}
 inline size_t cluster_partial_bytes(const StepParams& p, int heads, int D) {
-  return (p.fuse_out && p.merge_ctas > 1) ? sizeof(float) * heads * (D + tova::PART_STRIDE_EXTRA) : 0;
+  return (p.fuse_out && p.merge_ctas > 1) ? cluster_inbox_bytes(heads, D) : 0;
 }
 
 template <typename T, int D, int GU, int GB, bool FUSED>
@@ -216,7 +220,7 @@ cudaError_t launch_split_f(int dev, const StepParams& p, dim3 grid, cudaStream_t
   if (!attr_set[dev & 63]) {
     cudaError_t e = cudaFuncSetAttribute(
         kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-        (int)(warp_smem * tova::SPLIT_MERGE_MAX_WARPS + sizeof(float) * GU * (D + tova::PART_STRIDE_EXTRA)));
+        (int)(warp_smem * tova::SPLIT_MERGE_MAX_WARPS + cluster_inbox_bytes(GU, D)));
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     if (e != cudaSuccess) return e;
@@ -332,8 +336,7 @@ cudaError_t launch_split_mma_t(int dev, const StepParams& p, const CUtensorMap& 
   if (!attr_set[dev & 63]) {
     cudaError_t e = cudaFuncSetAttribute(
         kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-        (int)(warp_smem * tova::SPLIT_MERGE_MAX_WARPS + 1024 +
-              sizeof(float) * tova::MMA_UNIT_HEADS * (D + tova::PART_STRIDE_EXTRA)));
+        (int)(warp_smem * tova::SPLIT_MERGE_MAX_WARPS + 1024 + cluster_inbox_bytes(tova::MMA_UNIT_HEADS, D)));
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     if (e != cudaSuccess) return e;
@@ -524,6 +527,8 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, boo
 // the warps; 32-row chunks lose more in the combine kernel (twice the
 // partials) than they gain.  Larger chunks only where the combine kernel's
 // shared memory would not hold all partials of a sequence.
+bool fused_merge_fits(const tova_config& cfg, int chunk_rows, int sm_count);
+
 int pick_chunk_rows(const tova_config& cfg, int sm_count) {
   const size_t smem = split_smem_bytes(cfg) + 1024 /* per-CTA reserve */ + 64;
   long long per_sm = (long long)(227 * 1024) / (long long)smem;
@@ -546,6 +551,16 @@ int pick_chunk_rows(const tova_config& cfg, int sm_count) {
   if (wants_mma(cfg) && 2 * pairs >= 3LL * sm_count) {
     const int cr8 = (int)(((cfg.capacity + 7) / 8 + 31) / 32 * 32);
     if (cr8 > cr) cr = cr8;
+  }
+  // More than 8 x 8 chunks cannot merge inside the streaming kernel.  Where chunks long enough to get back under
+  // that limit keep the launch within what clusters merge well (fused_merge_fits), take them: at 4 sequences x 4 KV
+  // heads x 8192 rows the step is 18.0 us with 128-row chunks in clusters against 35.5 us with 64-row chunks and
+  // partials through global memory (16384 rows: 32.1 against 47.7 us).
+  {
+    const int limit = tova::SPLIT_MERGE_MAX_WARPS * tova::COMBINE_CLUSTER_MAX;
+    int cr2 = cr;
+    while (cr2 < 8192 && (cfg.capacity + cr2 - 1) / cr2 > limit) cr2 *= 2;
+    if (cr2 != cr && (cfg.capacity + cr2 - 1) / cr2 <= limit && fused_merge_fits(cfg, cr2, sm_count)) cr = cr2;
   }
   while (cr <= 8192 && combine_smem_bound(cfg.n_q_heads, (int)((cfg.capacity + cr - 1) / cr) + 1) > COMBINE_BASE_LIMIT)
     cr *= 2;

@@ -176,12 +176,16 @@ __device__ __noinline__ void block_merge_outputs(float* out, float2* head_ml, co
 
 // The same across a thread-block cluster, for states of up to 8 x 8 chunks: the
 // CTAs that share a head group (cluster dimension x, CTA r streams chunks 8r ..
-// 8r+7) first merge their own warps' partials into one partial per head
-// (`cpart`, shared memory of their own), meet at a cluster barrier, and then
-// split the output quads among all threads of the cluster, each reading the
-// CTAs' partials through distributed shared memory.  CTA 0's warp 0 holds the
-// new token's logits.  Nobody leaves before the second cluster barrier: a peer
-// may still be reading its shared memory.
+// 8r+7) each merge their own warps' partials into one partial per head and
+// SEND it to the CTA that owns that head (heads are dealt out over the CTAs of
+// the cluster) - stores into the owner's shared memory (`cpart`, its inbox:
+// [heads per CTA][CTAs][D+4] floats; CTA 0 adds the new token's logit) - then
+// meet at ONE cluster barrier, after which every CTA merges what it received
+// for its heads from its own shared memory and writes their outputs.  Nobody
+// reads a peer's memory, so a CTA may leave as soon as it is done.  The inbox
+// may only be written once its CTA runs: every thread arrives at the cluster
+// barrier at kernel entry (split kernels) and waits for that phase here, just
+// before the first remote store.
 template <typename T, int D>
 __device__ __noinline__ void cluster_merge_outputs(float* out, float2* head_ml, const T* v_new_row, const float* part0,
                                                    int warp_stride, float* snew0, float* cpart, size_t bh0,
@@ -193,12 +197,17 @@ __device__ __noinline__ void cluster_merge_outputs(float* out, float2* head_ml, 
   const int nw = (int)blockDim.y, nthreads = nw * 32;
   const int tid = (int)(threadIdx.y * 32 + threadIdx.x);
   const int ncta = (int)cl.num_blocks(), rank = (int)cl.block_rank();
+  const int hpc = (g_cnt + ncta - 1) / ncta;   // heads per owning CTA
   const int items = g_cnt * (D / 4);           // output quads of the group
   // the new token's value for this thread's first quad of the second stage: on its way before the barriers
-  const int it0 = rank * nthreads + tid;
+  const int my_items = min(hpc, max(g_cnt - rank * hpc, 0)) * (D / 4);
   float4 vq = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (it0 < items) vq = load_quad<T>(v_new_row + (it0 % (D / 4)) * 4);
+  if (tid < my_items) vq = load_quad<T>(v_new_row + (tid % (D / 4)) * 4);
   __syncthreads();                             // every warp's partial is in shared memory
+  cluster_wait_acquire();                      // every CTA of the cluster has started: its inbox may be written
+  float* inbox[COMBINE_CLUSTER_MAX];
+#pragma unroll
+  for (int r = 0; r < COMBINE_CLUSTER_MAX; ++r) inbox[r] = cl.map_shared_rank(cpart, r < ncta ? r : 0);
   for (int it = tid; it < items; it += nthreads) {
     const int g = it / (D / 4), d4 = it % (D / 4);
     float mr[NW], lr[NW];
@@ -222,28 +231,34 @@ __device__ __noinline__ void cluster_merge_outputs(float* out, float2* head_ml, 
         L = fmaf(lr[r], w, L);
       }
     }
-    *reinterpret_cast<float4*>(cpart + g * PS + d4 * 4) = o;
+    const int owner = g / hpc, slot = g % hpc;
+    float* dst = nullptr;
+#pragma unroll
+    for (int r = 0; r < COMBINE_CLUSTER_MAX; ++r)
+      if (r == owner) dst = inbox[r];
+    dst += (size_t)(slot * ncta + rank) * PS;
+    *reinterpret_cast<float4*>(dst + d4 * 4) = o;
     if (d4 == 0) {
-      cpart[g * PS + D] = M;
-      cpart[g * PS + D + 1] = L;
+      dst[D] = M;
+      dst[D + 1] = L;
+      if (rank == 0) dst[D + 2] = snew0[g];    // the new token's logit travels with CTA 0's partial
     }
   }
-  cl.sync();                                   // every CTA's partial is in its shared memory
-  const float* rp[COMBINE_CLUSTER_MAX];
-#pragma unroll
-  for (int r = 0; r < COMBINE_CLUSTER_MAX; ++r) rp[r] = cl.map_shared_rank(cpart, r < ncta ? r : 0);
-  const float* rs = cl.map_shared_rank(snew0, 0);
-  for (int it = it0; it < items; it += ncta * nthreads) {
-    const int g = it / (D / 4), d4 = it % (D / 4);
-    if (it != it0) vq = load_quad<T>(v_new_row + d4 * 4);
-    const float s_new = rs[g];
+  cluster_arrive_release();                    // orders the stores above before the barrier completes
+  cluster_wait_acquire();
+  for (int it = tid; it < my_items; it += nthreads) {
+    const int slot = it / (D / 4), d4 = it % (D / 4);
+    const int g = rank * hpc + slot;
+    if (it != tid) vq = load_quad<T>(v_new_row + d4 * 4);
+    const float* src = cpart + (size_t)slot * ncta * PS;
+    const float s_new = src[D + 2];
     float mr[COMBINE_CLUSTER_MAX], lr[COMBINE_CLUSTER_MAX];
     float M = s_new;
 #pragma unroll
     for (int r = 0; r < COMBINE_CLUSTER_MAX; ++r) {
       if (r < ncta) {
-        mr[r] = rp[r][g * PS + D];
-        lr[r] = rp[r][g * PS + D + 1];
+        mr[r] = src[r * PS + D];
+        lr[r] = src[r * PS + D + 1];
         M = fmaxf(M, mr[r]);
       }
     }
@@ -253,7 +268,7 @@ __device__ __noinline__ void cluster_merge_outputs(float* out, float2* head_ml, 
     for (int r = 0; r < COMBINE_CLUSTER_MAX; ++r) {
       if (r < ncta) {
         const float w = exp2_diff(mr[r], M);
-        const float4 a = *reinterpret_cast<const float4*>(rp[r] + g * PS + d4 * 4);
+        const float4 a = *reinterpret_cast<const float4*>(src + r * PS + d4 * 4);
         o.x = fmaf(a.x, w, o.x); o.y = fmaf(a.y, w, o.y); o.z = fmaf(a.z, w, o.z); o.w = fmaf(a.w, w, o.w);
         L = fmaf(lr[r], w, L);
       }
@@ -266,7 +281,6 @@ __device__ __noinline__ void cluster_merge_outputs(float* out, float2* head_ml, 
     reinterpret_cast<float4*>(out + (bh0 + g) * D)[d4] = o;
     if (d4 == 0) head_ml[bh0 + g] = make_float2(M, L);
   }
-  cl.sync();
 }
 
 // One CTA per head group, or a cluster of them (merge_ctas > 1).
@@ -318,8 +332,11 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32) tova_
   uint64_t* bars = bars_all[wib];
   const float* part0 = reinterpret_cast<const float*>(smem_all);    // warp 0's partial
   __shared__ float snew_s[MAX_UNIT_HEADS];                          // the new token's logit per head (chunk 0's warp)
-  // merge_ctas > 1: this CTA's merged partial, behind the rings
+  // merge_ctas > 1: this CTA's inbox for the cluster merge, behind the rings
   float* cpart = reinterpret_cast<float*>(smem_all + (size_t)(FUSED ? blockDim.y : 1) * WARP_SMEM);
+
+  // Merge across a cluster: peers will store into this CTA's shared memory; report in (see cluster_merge_outputs).
+  if (FUSED && p.merge_ctas > 1) cluster_arrive_release();
 
   const int lane = threadIdx.x;
   const int lig = lane % LPR;   // lane in row group

@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(32) tova_split_rope_kernel(const StepParams p,
     const float2* tr = tab + (size_t)j * HALF + d0;
 #pragma unroll
     for (int e = 0; e < EPL; ++e) {
-      const float2 cs = tr[e];
+      const float2 cs = __ldg(tr + e);
       // lower half: a*c - b*s with a = own, b = partner; upper half: b*c + a*s with b = own, a = partner
       kf[e] = upper ? fmaf(oth[e], cs.y, own[e] * cs.x) : fmaf(-oth[e], cs.y, own[e] * cs.x);
     }
@@ -190,6 +190,7 @@ __global__ void __launch_bounds__(32) tova_split_rope_kernel(const StepParams p,
   }
   const unsigned char* k_src = static_cast<const unsigned char*>(p.K) + (((size_t)b * p.Hkv + kvh) * p.cap + row_begin) * RB;
   const unsigned char* v_src = static_cast<const unsigned char*>(p.V) + (((size_t)b * p.Hkv + kvh) * p.cap + row_begin) * RB;
+#pragma unroll 4
   for (int r0 = 0; r0 < rows; r0 += RPW) {          // uniform trip count: the shuffles need the whole warp
     const int r = r0 + sub;
     const bool live = r < rows;

@@ -103,13 +103,16 @@ __global__ void __launch_bounds__(FUSED ? 32 * SPLIT_MERGE_MAX_WARPS : 32, FUSED
   uint64_t* bars = bars_all[wib];
   const float* part0 = reinterpret_cast<const float*>(ring0);      // warp 0's partial
   __shared__ float snew_s[MMA_UNIT_HEADS];                         // the new token's logit per head (chunk 0's warp)
-  // merge_ctas > 1: this CTA's merged partial, behind the rings
+  // merge_ctas > 1: this CTA's inbox for the cluster merge, behind the rings
   float* cpart = reinterpret_cast<float*>(ring0 + (size_t)(FUSED ? blockDim.y : 1) * WARP_SMEM);
   // fuse_out: once all tiles are consumed the ring holds this warp's partial
   // [MMA_UNIT_HEADS][D+4] and (rank 0) the new token's logits
   float* part = reinterpret_cast<float*>(ring);
   static_assert((MMA_UNIT_HEADS * (D + PART_STRIDE_EXTRA) + MMA_UNIT_HEADS) * sizeof(float) <= (size_t)NB * TILE_BYTES,
                 "partial fits the ring");
+
+  // Merge across a cluster: peers will store into this CTA's shared memory; report in (see cluster_merge_outputs).
+  if (FUSED && p.merge_ctas > 1) cluster_arrive_release();
 
   const int lane = threadIdx.x;
   const int qrow = lane >> 2, qcol = (lane & 3) * 2;   // fragment coordinates of this lane

@@ -84,6 +84,7 @@ __global__ void __launch_bounds__(UNIT_THREADS) tova_unit_policy_kernel(const St
   int idx = 0x7fffffff, cpos = pos_t;
   for (int j = tid; j <= p.n; j += UNIT_THREADS) {
     float w = 0.f;
+#pragma unroll 8
     for (int h = 0; h < nh; ++h) w += exp2f(lg[(size_t)h * p.ld + j] + hc[h]);
     float key = w;
     const int pj = (j < p.n) ? table[j] : pos_t;
