@@ -67,6 +67,8 @@ def parse_args():
                          "(-1: as many tokens as the state holds); a step is one whole prompt")
     ap.add_argument("--no-bulk-prefill", action="store_true", help="with --prefill: every prompt token takes the decode kernels")
     ap.add_argument("--warp-mma-prefill", action="store_true", help="with --prefill: bulk fill through the warp-level MMA kernel")
+    ap.add_argument("--chunk-cluster", type=int, default=0,
+                    help="with --prefill: thread blocks per sequence in the kernel that replays a chunk's deletions (0 = auto)")
     ap.add_argument("--no-chunked-prefill", action="store_true",
                     help="with --prefill: prompt tokens that meet a full state go one at a time instead of in chunks of 64")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -530,6 +532,8 @@ def run_prefill(args):
             c.tova_cache_set_bulk_prefill(0 if args.no_bulk_prefill else 2)
         if chunked:
             ws = c.tova_cache_set_prefill_workspace(ws)          # one workspace serves all: calls share a stream
+            if args.chunk_cluster:
+                c.tova_cache_set_chunk_cluster(args.chunk_cluster)
         caches.append(c)
     torch.cuda.synchronize()
     for c in caches[:warm]:
