@@ -35,6 +35,7 @@ def test_full_layer_shapes(name, cap, extra, seqs, direct_fill):
     n = cap + extra
     rep = run_lockstep(w, n, seqs=seqs, block=128, check_state_every=1000, direct_fill=direct_fill)
     assert rep.evictions == len(seqs) * extra
+    assert rep.resyncs <= max(1, rep.evictions // 20)      # the two sides may differ on near-ties only: rare
     check_all_sequences(rep, w, n)
     print(f"{name} k={cap}: max_err {rep.max_err:.2e} resyncs {rep.resyncs}/{rep.evictions} "
           f"self {rep.self_evictions}")
@@ -50,6 +51,7 @@ def test_chunked_prompt_at_full_layer_shapes(name, cap, seqs):
     rep = run_lockstep(w, n, seqs=seqs, block=512 if cap <= 1024 else 128, check_state_every=1000, direct_fill=True,
                        prefill_ws=True)
     assert rep.evictions == len(seqs) * (n - cap)
+    assert rep.resyncs <= max(1, rep.evictions // 20)
     check_all_sequences(rep, w, n)
     print(f"{name} k={cap} chunked prompt: max_err {rep.max_err:.2e} resyncs {rep.resyncs}/{rep.evictions}")
 
@@ -61,7 +63,7 @@ def test_32_layer_configuration_at_full_batch():
     extra = 64
     rep = run_lockstep(w, w.capacity + extra, seqs=[0, 29, 63], block=128, check_state_every=1000, direct_fill=True)
     assert rep.evictions == 3 * extra
-    assert rep.resyncs <= rep.evictions // 2
+    assert rep.resyncs <= max(1, rep.evictions // 20)
     check_all_sequences(rep, w, w.capacity + extra)
     print(f"llama2_7b_full k=1024 B=64: max_err {rep.max_err:.2e} resyncs {rep.resyncs}/{rep.evictions} "
           f"max_rel_gap {rep.max_rel_gap:.2e} self {rep.self_evictions}")
@@ -140,7 +142,7 @@ def test_long_stream_of_70000_tokens():
         live = st["positions"].numpy()[b].tolist()
         assert len(set(live)) == w.capacity and set(live) == held[b]
         assert 0 in held[b]                               # the sink (position 0) is still held, as in Section 7.3
-    assert evictions == w.batch * span * len(checkpoints)
+    assert evictions == w.batch * span * len(checkpoints) and resyncs <= evictions // 20
     print(f"yi_6b_long 70000 tokens: max_err {worst:.2e} resyncs {resyncs}/{evictions}")
 
 
