@@ -200,8 +200,8 @@ def run_reference(args):
     w = pick_workload(args)
     ring = W.tokens(w, 0, RING)
     # every "step" is a bounded sample; the whole run stays within minutes
-    budget = min(60.0, max(4.0, 0.004 * (args.steps + args.warmup)))
-    val, cores, sample = time_oracle(w, ring, budget)
+    seconds = min(60.0, max(4.0, 0.004 * (args.steps + args.warmup)))
+    val, cores, sample = time_oracle(w, ring, seconds)
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.batch / val,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",

@@ -1038,6 +1038,7 @@ int tova_cache_set_policy(tova_cache* c, int32_t policy, int32_t arg) {
   if (!c) return TOVA_ERR_NULL;
   if (policy < TOVA_POLICY_TOVA || policy > TOVA_POLICY_H2O_HEAD) return TOVA_ERR_UNSUPPORTED;
   if (c->len != 0 || c->pending) return TOVA_ERR_BAD_SHAPE;   // the policy is fixed while the state is empty
+  if (c->shard_on && policy != TOVA_POLICY_TOVA) return TOVA_ERR_UNSUPPORTED;   // the sharded step sums TOVA's weights
   if (policy == TOVA_POLICY_TOVA || policy == TOVA_POLICY_WINDOW) {
     // a droppable row must always exist, and Window compares ages that stay below the capacity only if the
     // state has been under this policy from the start
@@ -1216,7 +1217,7 @@ int tova_decode_step(tova_cache* c, const void* q, const void* k, const void* v,
 int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int32_t n_tokens,
                  int32_t first_pos, float* out, int32_t* evicted_pos, void* cuda_stream) {
   if (!c) return TOVA_ERR_NULL;
-  if (n_tokens < 0) return TOVA_ERR_BAD_SHAPE;
+  if (n_tokens < 0 || c->shard_on) return TOVA_ERR_BAD_SHAPE;   // a sharded layer steps through its two-phase calls
   if (n_tokens == 0) return TOVA_OK;
   float* scratch_out = reinterpret_cast<float*>(c->base + c->lay.st_out);
   int rc = check_step_args(c, q, k, v, out ? (const void*)out : (const void*)scratch_out);

@@ -116,6 +116,10 @@ def test_sharded_step_call_order_and_refusals():
     with pytest.raises(tova.TovaError):
         c.tova_decode_step(q, k, k, 0, out)                     # the one-call step is refused on a sharded cache
     with pytest.raises(tova.TovaError):
+        c.tova_prefill(q[None], k[None], k[None], 1, 0, out[None])   # nor prompts
+    with pytest.raises(tova.TovaError):
+        c.tova_cache_set_policy(tova.TOVA_POLICY_WINDOW, 0)     # the exchange sums TOVA's weights
+    with pytest.raises(tova.TovaError):
         c.tova_decode_step_commit(k, k)                         # nothing scored yet
     c.tova_decode_step_scores(q, k, k, 0, out)
     with pytest.raises(tova.TovaError):
