@@ -56,6 +56,75 @@ def test_chunked_prompt_at_full_layer_shapes(name, cap, seqs):
     print(f"{name} k={cap} chunked prompt: max_err {rep.max_err:.2e} resyncs {rep.resyncs}/{rep.evictions}")
 
 
+def test_position_compression_at_the_layer_shape():
+    """B=8, 32 MHA heads, state of 512 rows, q and k without rotary embedding: the rotating streaming kernel at
+    the shape the paper's extrapolation experiment uses (multi-state 512), the checker on two sequences."""
+    w = W.WORKLOADS["llama2_7b_layer"].scaled(rope=False)
+    n = w.capacity + 96
+    rep = run_lockstep(w, n, seqs=[0, 6], block=128, check_state_every=1000, direct_fill=True, rope_base=10000.0)
+    assert rep.evictions == 2 * 96 and rep.resyncs <= 9
+    check_all_sequences(rep, w, n)
+    print(f"position compression k=512 B=8: max_err {rep.max_err:.2e} resyncs {rep.resyncs}/{rep.evictions}")
+
+
+def test_per_head_policy_at_the_full_gqa_shape():
+    """TOVA-head on the Mistral shape (B=32, 32 query / 8 KV heads, state of 1024 rows): while the state fills no
+    head drops anything, so the checker's per-head tables are written directly; then 40 tokens in lock step on two
+    sequences, every KV head dropping its own row."""
+    import torch
+    import paper_2401_06104_b200 as tova
+    from oracle.tova_oracle import OracleUnitsCache
+    from parity import GAP_TOL, out_tol
+    w = W.WORKLOADS["mistral_7b_gqa"].scaled(capacity=1024)
+    seqs, extra = [4, 27], 40
+    cache = make_cache(w, policy="tova_head")
+    U = w.n_kv_heads
+    orc = OracleUnitsCache(len(seqs), w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, "tova_head", precision="f32")
+    done = 0
+    while done < w.capacity + extra:
+        T = min(128, w.capacity + extra - done)
+        q, k, v = W.tokens(w, done, T)
+        dq, dk, dv = (tova.to_device(a, w.dtype) for a in (q, k, v))
+        out = torch.empty(T, w.batch, w.n_q_heads, w.head_dim, device="cuda:0")
+        ev = torch.empty(T, w.batch, U, dtype=torch.int32, device="cuda:0")
+        cache.tova_prefill(dq, dk, dv, T, done, out, ev)
+        torch.cuda.synchronize()
+        g_out, g_ev = out.cpu().numpy(), ev.cpu().numpy()
+        for t in range(T):
+            pos_t = done + t
+            if orc.len[0] < w.capacity:
+                n = int(orc.len[0])
+                assert np.all(g_ev[t] == -1)
+                orc.K[:, :, n], orc.V[:, :, n] = k[t][seqs], v[t][seqs]
+                orc.pos[:, :, n] = pos_t
+                orc.len[:] = n + 1
+                continue
+            forced = np.zeros((len(seqs), U), np.int32)
+            for i, b in enumerate(seqs):
+                for u in range(U):
+                    e = int(g_ev[t, b, u])
+                    forced[i, u] = w.capacity if e == pos_t else int(np.nonzero(orc.pos[i, u] == e)[0][0])
+            o_out, o_ev, victim, argmin, gap, _ = orc.step(q[t][seqs], k[t][seqs], v[t][seqs], pos_t, forced=forced)
+            assert np.all(gap < GAP_TOL) and np.array_equal(o_ev, g_ev[t, seqs]), pos_t
+            assert np.abs(g_out[t][seqs] - o_out).max() <= out_tol(w), pos_t
+            assert np.sum(victim != argmin) == 0
+        done += T
+    st = cache.tova_cache_read()
+    assert st["status"] == 0
+    pos = st["positions"].numpy()
+    assert np.array_equal(pos[seqs], orc.pos)
+    assert any(set(pos[seqs[0], 0].tolist()) != set(pos[seqs[0], u].tolist()) for u in range(1, U))   # heads diverged
+
+
+def test_sharded_layer_at_a_long_state():
+    """Four emulated ranks, two KV heads each, state of 1024 rows (8 chunks per head: the in-kernel merge), batch 4."""
+    from test_gpu_sharded import run_sharded
+    w = W.WORKLOADS["mistral_7b_gqa"].scaled(batch=4, capacity=1024)
+    worst, resyncs = run_sharded(w, 4, 1024 + 24, "peer")
+    assert resyncs <= 2
+    print(f"sharded mistral k=1024 B=4 world=4: max_err {worst:.2e} resyncs {resyncs}")
+
+
 def test_32_layer_configuration_at_full_batch():
     """Batch 64, 32 MHA heads, state of 1024 rows: 2048 eight-warp thread blocks of 128-row chunks per streaming
     launch (the launch the benchmark's headline times).  The checker follows three of the 64 sequences."""
