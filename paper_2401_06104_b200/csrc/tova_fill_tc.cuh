@@ -3,22 +3,23 @@
 // with both contractions issued as tcgen05.mma from shared-memory descriptors and their
 // accumulators in tensor memory (TMEM).
 //
-// One CTA of 256 threads per (128 query tokens, query head, sequence); query row i = TMEM
-// lane i, shared by two threads (warps w and w + 4), each taking half of a tile's logits and
-// half of O's columns.  Per tile of 64 state rows:
-//   TMA (tiled, 128-byte swizzle)  K tile, V tile -> shared memory (one buffer each; the next
-//                tile is requested as soon as the contraction that read the buffer is complete)
-//   tcgen05.mma  S[128 x 64]  = Q[128 x D] . K^T          (A, B K-major; fp32 in TMEM, two S
-//                buffers: S of tile i+1 is issued together with O += P V of tile i)
-//   tcgen05.ld   half a row of S -> registers; scale, causal mask, online soft-max in the base-2
-//                domain (row maxima of the two halves exchanged through shared memory);
-//                weights as hi + lo bf16 terms -> shared memory (K-major, 128-byte swizzle);
-//                if a row's running max moved, O is rescaled in TMEM (tcgen05.ld / tcgen05.st)
+// One CTA per (128 query tokens, query head, sequence): 256 soft-max threads - query row i = TMEM lane i, shared
+// by two threads (warps w and w + 4), each taking half of a tile's logits and half of O's columns - and one more
+// warp whose first lane issues every copy and every contraction.  Per tile of 64 state rows:
+//   TMA (tiled, 128-byte swizzle)  K tile, V tile -> shared memory (one buffer each; the next tile is requested
+//                as soon as the contraction that read the buffer is complete)
+//   tcgen05.mma  S[128 x 64]  = Q[128 x D] . K^T          (A, B K-major; fp32 in TMEM, two S buffers: S of tile
+//                i+1 is issued as soon as its K tile is there, ahead of O += P V of tile i)
+//   tcgen05.ld   the row of S -> registers: the maximum over the whole tile (no exchange between the two threads of
+//                a row), the weights of the thread's half; online soft-max in the base-2 domain; weights as hi + lo
+//                bf16 terms -> shared memory (K-major, 128-byte swizzle); if a row's running max moved, O is
+//                rescaled in TMEM (tcgen05.ld / tcgen05.st)
 //   tcgen05.mma  O[128 x D] += P_hi . V + P_lo . V         (B = V tile as stored, MN-major)
-// Completion through tcgen05.commit on an mbarrier, one commit and one wait per tile; two
-// CTAs share an SM (98 KiB of shared memory, 256 of the 512 TMEM columns each), so one CTA's
-// soft-max overlaps the other's contractions.  Every wait is bounded; a wait that runs out
-// sets the status word, and the CTA still frees its TMEM.
+// The roles meet through mbarriers only (tcgen05.commit for the contractions, 256 arrivals for a tile's weights):
+// the soft-max of tile i+1 runs while the tensor cores work on O += P V of tile i, and only writing the new
+// weights and touching O wait for that contraction.  Two CTAs share an SM (98 KiB of shared memory, 256 of the
+// 512 TMEM columns each).  Every wait is bounded; a wait that runs out sets the status word, the roles drain
+// through their own bounded waits, and the CTA still frees its TMEM.
 #pragma once
 
 #include "tova_fill.cuh"
@@ -26,7 +27,8 @@
 namespace tova {
 
 constexpr int FILLTC_Q_ROWS = 128;
-constexpr int FILLTC_THREADS = 256;   // two threads per query row: each takes half of a tile's 64 logits, half of O's columns
+constexpr int FILLTC_SOFTMAX_THREADS = 256;   // two threads per query row: each takes half of a tile's 64 logits, half of O's columns
+constexpr int FILLTC_THREADS = FILLTC_SOFTMAX_THREADS + 32;   // plus one warp whose first lane issues copies and contractions
 constexpr int FILLTC_TMEM_COLS = 256;   // S of even and odd tiles: 64 columns each, O: 128 columns
 
 // Shared-memory matrix descriptor: start address, leading / stride byte offsets (units of 16 bytes),
@@ -66,6 +68,25 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(bar))
                : "memory");
+}
+
+// One arrival of this thread on an mbarrier of its own CTA.
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+// Barrier `id` (1..15) among `count` threads of the CTA (a multiple of 32; whole warps take part).
+__device__ __forceinline__ void named_barrier_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+// Bounded wait of the fill kernel: every try_wait blocks for a hardware-defined slice, so the limit is far beyond
+// any legitimate copy or contraction, yet a kernel whose roles have lost each other ends within seconds.
+__device__ __forceinline__ bool fill_wait(uint64_t* bar, uint32_t parity) {
+  for (int it = 0; it < (1 << 20); ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+  }
+  return false;
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -114,7 +135,7 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// grid = (ceil(F/128), H, B), block = 256.  Dynamic shared memory: Q (32 KiB) + K, V tiles (16 KiB each) +
+// grid = (ceil(F/128), H, B), block = 288.  Dynamic shared memory: Q (32 KiB) + K, V tiles (16 KiB each) +
 // P_hi, P_lo (16 KiB each) + 1 KiB alignment slack.  head_dim 128 only.
 __global__ void __launch_bounds__(FILLTC_THREADS, 2)
     tova_fill_attn_tc_kernel(const FillParams p, const __grid_constant__ CUtensorMap map_k,
@@ -133,9 +154,11 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   unsigned char* v_s = k_s + T_BYTES;
   unsigned char* ph_s = v_s + T_BYTES;
   unsigned char* pl_s = ph_s + P_BYTES;
-  __shared__ __align__(8) uint64_t bar_k, bar_v, bar_mma;
+  // K tile, V tile landed; S = Q K^T, O += P V completed (tcgen05.commit); weights of a tile written (256 arrivals)
+  // (one S barrier per S buffer: a barrier then completes once per two tiles, and a waiter can never be two phases behind)
+  __shared__ __align__(8) uint64_t bar_k, bar_v, bar_s[2], bar_o, bar_p;
   __shared__ uint32_t tmem_base_s;
-  __shared__ float half_max[2][FILLTC_Q_ROWS];   // the two halves of a row exchange their tile maxima (and, at the end, sums)
+  __shared__ float half_sum[2][FILLTC_Q_ROWS];   // the two halves of a row add up their sums at the end
 
   const int tid = threadIdx.x, warp = tid >> 5;
   const int tile_q = gridDim.x - 1 - blockIdx.x;          // longest rows first
@@ -150,7 +173,10 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   if (tid == 0) {
     mbar_init(&bar_k, 1);
     mbar_init(&bar_v, 1);
-    mbar_init(&bar_mma, 1);
+    mbar_init(&bar_s[0], 1);
+    mbar_init(&bar_s[1], 1);
+    mbar_init(&bar_o, 1);
+    mbar_init(&bar_p, FILLTC_SOFTMAX_THREADS);
     mbar_fence_init();
   }
   if (warp == 0) {   // one warp allocates the CTA's tensor memory and gives up the right to allocate more
@@ -175,173 +201,188 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
-  // A warp reaches the 32 TMEM lanes of its quarter (warp mod 4); warps 0-3 take the first half of a row's
-  // columns, warps 4-7 the second half.
-  const int row = (warp & 3) * 32 + (tid & 31), half = warp >> 2;
-  const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
   const uint32_t tm_o = 128;                                         // S of tile i at column 64 (i & 1), O at 128
 
-  const uint32_t idesc_s = umma_idesc_bf16(FILLTC_Q_ROWS, KT, false);
-  const uint32_t idesc_o = umma_idesc_bf16(FILLTC_Q_ROWS, D, true);
-  const uint32_t q_a = smem_addr(q_s), k_a = smem_addr(k_s), v_a = smem_addr(v_s), ph_a = smem_addr(ph_s),
-                 pl_a = smem_addr(pl_s);
-
-  const int my_t = min(t0 + row, p.F - 1);
-  const int vis = p.n0 + my_t;            // last state row this thread's query sees
-  float m_run = -INFINITY, l_run = 0.f;
-  uint32_t ph_mma = 0;                    // phase of the tensor-core completion barrier (K, V tile i: parity i & 1)
-  bool ok = true;
-
-  // K and V tiles have one buffer each and a barrier each: the next K tile is requested as soon as S = Q K^T
-  // of the current one has completed, the next V tile as soon as O += P V has, so the copies run under the
-  // soft-max and the other contraction.
-  auto load_k = [&](int i) {
-    mbar_expect_tx(&bar_k, (uint32_t)T_BYTES);
-    const int y = head_row0 + i * KT;
-    tma_load_2d_keep(k_s, &map_k, 0, y, &bar_k);
-    tma_load_2d_keep(k_s + KT * 128, &map_k, 64, y, &bar_k);
-  };
-  auto load_v = [&](int i) {
-    mbar_expect_tx(&bar_v, (uint32_t)T_BYTES);
-    const int y = head_row0 + i * KT;
-    tma_load_2d_keep(v_s, &map_v, 0, y, &bar_v);
-    tma_load_2d_keep(v_s + KT * 128, &map_v, 64, y, &bar_v);
-  };
-  if (tid == 0) {
-    load_k(0);
-    load_v(0);
-  }
-
-  // S = Q K^T of tile i into S buffer i & 1: 8 steps of 16 along D; a step moves 32 bytes inside the 128-byte
-  // row, 4 steps per box.  Issued by one thread once the K tile has landed.
-  auto issue_qk = [&](int i) {
-    tc_fence_after();
+  if (warp == FILLTC_SOFTMAX_THREADS / 32) {
+    // ======================= copy + tensor-core issue: one thread =======================
+    // K and V have one buffer each.  The tensor cores execute what this thread issues in order:
+    //   S(0) | S(1) | O+=PV(0) | S(2) | O+=PV(1) | S(3) | ...
+    // S of a tile is issued as soon as its K tile has landed (the S buffer it overwrites was read two tiles ago),
+    // so the soft-max threads find their next logits waiting; O += P V of a tile once its weights are written.
+    if ((tid & 31) == 0) {
+      const uint32_t idesc_s = umma_idesc_bf16(FILLTC_Q_ROWS, KT, false);
+      const uint32_t idesc_o = umma_idesc_bf16(FILLTC_Q_ROWS, D, true);
+      const uint32_t q_a = smem_addr(q_s), k_a = smem_addr(k_s), v_a = smem_addr(v_s), ph_a = smem_addr(ph_s),
+                     pl_a = smem_addr(pl_s);
+      auto load_k = [&](int i) {
+        mbar_expect_tx(&bar_k, (uint32_t)T_BYTES);
+        const int y = head_row0 + i * KT;
+        tma_load_2d_keep(k_s, &map_k, 0, y, &bar_k);
+        tma_load_2d_keep(k_s + KT * 128, &map_k, 64, y, &bar_k);
+      };
+      auto load_v = [&](int i) {
+        mbar_expect_tx(&bar_v, (uint32_t)T_BYTES);
+        const int y = head_row0 + i * KT;
+        tma_load_2d_keep(v_s, &map_v, 0, y, &bar_v);
+        tma_load_2d_keep(v_s + KT * 128, &map_v, 64, y, &bar_v);
+      };
+      // S = Q K^T of tile i into S buffer i & 1: 8 steps of 16 along D; a step moves 32 bytes inside the 128-byte
+      // row, 4 steps per box.
+      auto issue_qk = [&](int i) {
+        tc_fence_after();
 #pragma unroll
-    for (int ks = 0; ks < D / 16; ++ks) {
-      const uint64_t a = umma_desc_sw128(q_a + (ks >> 2) * (FILLTC_Q_ROWS * 128) + (ks & 3) * 32, 16, 1024);
-      const uint64_t bd = umma_desc_sw128(k_a + (ks >> 2) * (KT * 128) + (ks & 3) * 32, 16, 1024);
-      umma_bf16(tmem + (uint32_t)(64 * (i & 1)), a, bd, idesc_s, ks > 0 ? 1u : 0u);
-    }
-  };
-  // Tile 0's S by itself; from then on S of tile i+1 is issued together with O += P V of tile i (one commit,
-  // one wait per tile), so a tile's logits are ready when its soft-max starts.
-  if (tid == 0) {
-    if (mbar_wait_bounded(&bar_k, 0u)) {
-      issue_qk(0);
-      umma_commit(&bar_mma);
-    }
-  }
-  ok = mbar_wait_bounded(&bar_mma, ph_mma);   // (a K wait that ran out shows up as a missing commit)
-  ph_mma ^= 1u;
-  tc_fence_after();
-  if (tid == 0 && ok && n_tiles > 1) load_k(1);   // the K buffer is free: S of tile 0 has been computed
-  ok = __syncthreads_and(ok ? 1 : 0) != 0;
-
-  for (int i = 0; i < n_tiles && ok; ++i) {
-    const int j0 = i * KT;
-    const uint32_t tm_s = (uint32_t)(64 * (i & 1));
-
-    // ---- soft-max of this thread's row -------------------------------------------------
-    __syncwarp();
-    constexpr int KH = KT / 2;   // logits per thread
-    float s[KH];
-    tmem_ld32(lane_base + tm_s + (uint32_t)(KH * half), s);
-    const int jh = j0 + KH * half;
-    float mx = -INFINITY;
-    if (j0 + KT - 1 > p.n0 + t0) {   // some query of this CTA cannot see the whole tile (CTA-uniform)
-#pragma unroll
-      for (int c = 0; c < KH; ++c) {
-        s[c] = (jh + c <= vis) ? s[c] * p.scale2 : -INFINITY;
-        mx = fmaxf(mx, s[c]);
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint64_t a = umma_desc_sw128(q_a + (ks >> 2) * (FILLTC_Q_ROWS * 128) + (ks & 3) * 32, 16, 1024);
+          const uint64_t bd = umma_desc_sw128(k_a + (ks >> 2) * (KT * 128) + (ks & 3) * 32, 16, 1024);
+          umma_bf16(tmem + (uint32_t)(64 * (i & 1)), a, bd, idesc_s, ks > 0 ? 1u : 0u);
+        }
+        umma_commit(&bar_s[i & 1]);
+      };
+      load_k(0);
+      load_v(0);
+      bool okp = fill_wait(&bar_k, 0u);
+      if (okp) issue_qk(0);
+      if (okp && n_tiles > 1) {
+        okp = fill_wait(&bar_s[0], 0u);              // S(0) computed: the K buffer is free
+        if (okp) load_k(1);
       }
-    } else {
+      for (int i = 0; i < n_tiles && okp; ++i) {
+        if (i + 1 < n_tiles) {                       // the next tile's logits, ahead of the soft-max that needs them
+          okp = fill_wait(&bar_k, (uint32_t)((i + 1) & 1));
+          if (!okp) break;
+          issue_qk(i + 1);
+        }
+        okp = fill_wait(&bar_p, (uint32_t)(i & 1)) && fill_wait(&bar_v, (uint32_t)(i & 1));
+        if (!okp) break;
+        tc_fence_after();
+        // O += P V: 4 steps of 16 state rows; V as stored is MN-major (D contiguous)
 #pragma unroll
-      for (int c = 0; c < KH; ++c) {
-        s[c] *= p.scale2;
-        mx = fmaxf(mx, s[c]);
+        for (int kk = 0; kk < KT / 16; ++kk) {
+          const uint64_t bd = umma_desc_sw128(v_a + kk * 2048, KT * 128, 1024);
+          const uint64_t ah = umma_desc_sw128(ph_a + kk * 32, 16, 1024);
+          const uint64_t al = umma_desc_sw128(pl_a + kk * 32, 16, 1024);
+          umma_bf16(tmem + tm_o, ah, bd, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
+          umma_bf16(tmem + tm_o, al, bd, idesc_o, 1u);
+        }
+        umma_commit(&bar_o);
+        if (i + 2 < n_tiles) {                       // S(i+1) computed: K(i+2) may overwrite K(i+1)
+          okp = fill_wait(&bar_s[(i + 1) & 1], (uint32_t)(((i + 1) >> 1) & 1));
+          if (!okp) break;
+          load_k(i + 2);
+        }
+        if (i + 1 < n_tiles) {                       // O += P V of tile i completed: V(i+1) may overwrite V(i)
+          okp = fill_wait(&bar_o, (uint32_t)(i & 1));
+          if (!okp) break;
+          load_v(i + 1);
+        }
       }
+      if (!okp) atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
     }
-    half_max[half][row] = mx;
-    __syncthreads();
-    mx = fmaxf(mx, half_max[half ^ 1][row]);
-    const float m_new = fmaxf(m_run, mx);       // finite from tile 0 on: row 0 of the state is visible to every query
-    const float corr = exp2_diff(m_run, m_new);
-    m_run = m_new;
-    float lsum = 0.f;
+  } else {
+    // ======================= soft-max: two threads per query row =======================
+    // A warp reaches the 32 TMEM lanes of its quarter (warp mod 4); warps 0-3 take the first half of a row's
+    // columns, warps 4-7 the second half.  No barrier of the whole CTA inside the loop: the threads meet the
+    // issuing thread, and each other, only through the mbarriers.
+    const int row = (warp & 3) * 32 + (tid & 31), half = warp >> 2;
+    const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const int my_t = min(t0 + row, p.F - 1);
+    const int vis = p.n0 + my_t;            // last state row this thread's query sees
+    float m_run = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    for (int i = 0; i < n_tiles; ++i) {
+      const int j0 = i * KT;
+      const uint32_t tm_s = (uint32_t)(64 * (i & 1));
+      ok = __all_sync(0xffffffffu, fill_wait(&bar_s[i & 1], (uint32_t)((i >> 1) & 1))) != 0;   // this tile's logits
+      if (!ok) break;
+      tc_fence_after();
+      // the maximum over the whole tile, the weights of this thread's half
+      constexpr int KH = KT / 2;
+      float s[KH];
+      float mx = -INFINITY;
+      {
+        float so[KH];
+        tmem_ld32(lane_base + tm_s + (uint32_t)(KH * (half ^ 1)), so);
+        const int jo = j0 + KH * (half ^ 1);
+        const bool masked = j0 + KT - 1 > p.n0 + t0;   // some query of this CTA cannot see the whole tile (CTA-uniform)
 #pragma unroll
-    for (int c8 = 0; c8 < KH / 8; ++c8) {
-      uint32_t hi[4], lo[4];
+        for (int c = 0; c < KH; ++c) mx = fmaxf(mx, (!masked || jo + c <= vis) ? so[c] : -INFINITY);
+      }
+      tmem_ld32(lane_base + tm_s + (uint32_t)(KH * half), s);
+      const int jh = j0 + KH * half;
+      if (j0 + KT - 1 > p.n0 + t0) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float e0 = ex2_approx(s[c8 * 8 + 2 * e] - m_new), e1 = ex2_approx(s[c8 * 8 + 2 * e + 1] - m_new);
+        for (int c = 0; c < KH; ++c) {
+          s[c] = (jh + c <= vis) ? s[c] : -INFINITY;
+          mx = fmaxf(mx, s[c]);
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < KH; ++c) mx = fmaxf(mx, s[c]);
+      }
+      mx *= p.scale2;                             // scale2 > 0: the maximum commutes with the scaling
+      const float m_new = fmaxf(m_run, mx);       // finite from tile 0 on: row 0 of the state is visible to every query
+      const float corr = exp2_diff(m_run, m_new);
+      m_run = m_new;
+      float lsum = 0.f;
+      uint32_t hi[KH / 2], lo[KH / 2];
+#pragma unroll
+      for (int e = 0; e < KH / 2; ++e) {
+        const float e0 = ex2_approx(fmaf(s[2 * e], p.scale2, -m_new)), e1 = ex2_approx(fmaf(s[2 * e + 1], p.scale2, -m_new));
         lsum += e0 + e1;
         split_hi_lo(e0, e1, hi[e], lo[e]);
       }
-      const uint32_t off = (uint32_t)row * 128u + (uint32_t)(((c8 + 4 * half) ^ (row & 7)) << 4);
-      *reinterpret_cast<uint4*>(ph_s + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-      *reinterpret_cast<uint4*>(pl_s + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      l_run = l_run * corr + lsum;
+      // The weights of tile i-1 are still being read, and O written, until O += P V of tile i-1 has completed.
+      if (i > 0) {
+        ok = __all_sync(0xffffffffu, fill_wait(&bar_o, (uint32_t)((i - 1) & 1))) != 0;
+        if (!ok) break;
+        tc_fence_after();
+      }
+#pragma unroll
+      for (int c8 = 0; c8 < KH / 8; ++c8) {
+        const uint32_t off = (uint32_t)row * 128u + (uint32_t)(((c8 + 4 * half) ^ (row & 7)) << 4);
+        *reinterpret_cast<uint4*>(ph_s + off) = make_uint4(hi[4 * c8], hi[4 * c8 + 1], hi[4 * c8 + 2], hi[4 * c8 + 3]);
+        *reinterpret_cast<uint4*>(pl_s + off) = make_uint4(lo[4 * c8], lo[4 * c8 + 1], lo[4 * c8 + 2], lo[4 * c8 + 3]);
+      }
+      // O of the tiles so far was accumulated against the old max
+      if (i > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
+#pragma unroll
+        for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
+          float o[32];
+          tmem_ld32(lane_base + tm_o + c0, o);
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] *= corr;
+          tmem_st32(lane_base + tm_o + c0, o);
+        }
+        tmem_st_wait();
+      }
+      fence_proxy_async_smem();   // P was written through the generic proxy, the tensor cores read it asynchronously
+      tc_fence_before();
+      mbar_arrive(&bar_p);        // this thread's part of the tile's weights (and of O) is in place
     }
-    l_run = l_run * corr + lsum;
-    // O of the tiles so far was accumulated against the old max
-    if (i > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
+    if (ok && n_tiles > 0) {
+      ok = __all_sync(0xffffffffu, fill_wait(&bar_o, (uint32_t)((n_tiles - 1) & 1))) != 0;   // the last O += P V
+      tc_fence_after();
+    }
+    half_sum[half][row] = l_run;
+    named_barrier_sync(1, FILLTC_SOFTMAX_THREADS);
+    if (ok) {
+      const float rl = 1.f / (half_sum[0][row] + half_sum[1][row]);
+      const int t = t0 + row;
 #pragma unroll
       for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
         float o[32];
         tmem_ld32(lane_base + tm_o + c0, o);
+        if (t < p.F) {
+          float4* dst = reinterpret_cast<float4*>(p.out + (((size_t)t * p.B + b) * p.H + h) * D + c0);
 #pragma unroll
-        for (int c = 0; c < 32; ++c) o[c] *= corr;
-        tmem_st32(lane_base + tm_o + c0, o);
+          for (int c = 0; c < 8; ++c)
+            dst[c] = make_float4(o[4 * c] * rl, o[4 * c + 1] * rl, o[4 * c + 2] * rl, o[4 * c + 3] * rl);
+        }
       }
-      tmem_st_wait();
+    } else if ((tid & 31) == 0) {
+      atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
     }
-    fence_proxy_async_smem();   // P was written through the generic proxy, the tensor cores read it asynchronously
-    tc_fence_before();
-    __syncthreads();
-
-    // ---- O += P V: 4 steps of 16 state rows; V as stored is MN-major (D contiguous) --------
-    // (a K or V wait that ran out shows up as a missing commit below)
-    if (tid == 0 && (i + 1 >= n_tiles || mbar_wait_bounded(&bar_k, (uint32_t)((i + 1) & 1))) &&
-        mbar_wait_bounded(&bar_v, (uint32_t)(i & 1))) {
-      if (i + 1 < n_tiles) issue_qk(i + 1);
-      tc_fence_after();
-#pragma unroll
-      for (int kk = 0; kk < KT / 16; ++kk) {
-        const uint64_t bd = umma_desc_sw128(v_a + kk * 2048, KT * 128, 1024);
-        const uint64_t ah = umma_desc_sw128(ph_a + kk * 32, 16, 1024);
-        const uint64_t al = umma_desc_sw128(pl_a + kk * 32, 16, 1024);
-        umma_bf16(tmem + tm_o, ah, bd, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
-        umma_bf16(tmem + tm_o, al, bd, idesc_o, 1u);
-      }
-      umma_commit(&bar_mma);
-    }
-    ok = mbar_wait_bounded(&bar_mma, ph_mma);   // K, V and P may be overwritten and O and the next S read after this
-    ph_mma ^= 1u;
-    tc_fence_after();
-    if (tid == 0 && ok) {
-      if (i + 2 < n_tiles) load_k(i + 2);
-      if (i + 1 < n_tiles) load_v(i + 1);
-    }
-    ok = __syncthreads_and(ok ? 1 : 0) != 0;
-  }
-
-  if (ok) {
-    half_max[half][row] = l_run;     // (the last use of the array was followed by two CTA barriers)
-    __syncthreads();
-    const float rl = 1.f / (half_max[0][row] + half_max[1][row]);
-    const int t = t0 + row;
-#pragma unroll
-    for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
-      float o[32];
-      tmem_ld32(lane_base + tm_o + c0, o);
-      if (t < p.F) {
-        float4* dst = reinterpret_cast<float4*>(p.out + (((size_t)t * p.B + b) * p.H + h) * D + c0);
-#pragma unroll
-        for (int c = 0; c < 8; ++c)
-          dst[c] = make_float4(o[4 * c] * rl, o[4 * c + 1] * rl, o[4 * c + 2] * rl, o[4 * c + 3] * rl);
-      }
-    }
-  } else if (tid == 0) {
-    atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
   }
   tc_fence_before();
   __syncthreads();
