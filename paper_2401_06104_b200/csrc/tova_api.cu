@@ -698,7 +698,7 @@ cudaError_t launch_fill_d(tova_cache* c, const tova::FillParams& p, cudaStream_t
   c->launches += 1;
   if (p.out) {
     if (D == 128 && c->bulk_fill == 1) {
-      constexpr size_t smem_tc = 96 * 1024 + 1024;
+      constexpr size_t smem_tc = 64 * 1024 + 1024;
       static std::atomic<bool> configured_tc[64];
       if (c->device >= 0 && c->device < 64 && !configured_tc[c->device]) {
         e = cudaFuncSetAttribute(tova::tova_fill_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_tc);

@@ -12,12 +12,13 @@
 //                i+1 is issued as soon as its K tile is there, ahead of O += P V of tile i)
 //   tcgen05.ld   the row of S -> registers: the maximum over the whole tile (no exchange between the two threads of
 //                a row), the weights of the thread's half; online soft-max in the base-2 domain; weights as hi + lo
-//                bf16 terms -> shared memory (K-major, 128-byte swizzle); if a row's running max moved, O is
+//                bf16 terms -> tcgen05.st back into the tile's S buffer, where they are the A operand of the
+//                second contraction (no trip through shared memory); if a row's running max moved, O is
 //                rescaled in TMEM (tcgen05.ld / tcgen05.st)
-//   tcgen05.mma  O[128 x D] += P_hi . V + P_lo . V         (B = V tile as stored, MN-major)
+//   tcgen05.mma  O[128 x D] += P_hi . V + P_lo . V         (A in tensor memory, B = V tile as stored, MN-major)
 // The roles meet through mbarriers only (tcgen05.commit for the contractions, 256 arrivals for a tile's weights):
 // the soft-max of tile i+1 runs while the tensor cores work on O += P V of tile i, and only writing the new
-// weights and touching O wait for that contraction.  Two CTAs share an SM (98 KiB of shared memory, 256 of the
+// weights and touching O wait for that contraction.  Two CTAs share an SM (65 KiB of shared memory, 256 of the
 // 512 TMEM columns each).  Every wait is bounded; a wait that runs out sets the status word, the roles drain
 // through their own bounded waits, and the CTA still frees its TMEM.
 #pragma once
@@ -61,6 +62,17 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// The same with the A operand in tensor memory: row i of A in TMEM lane i, its K elements packed two per 32-bit
+// column from a_tmem on.
+__device__ __forceinline__ void umma_bf16_a_tmem(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 
@@ -133,10 +145,19 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
         "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
       : "memory");
 }
+// 16 consecutive 32-bit columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// grid = (ceil(F/128), H, B), block = 288.  Dynamic shared memory: Q (32 KiB) + K, V tiles (16 KiB each) +
-// P_hi, P_lo (16 KiB each) + 1 KiB alignment slack.  head_dim 128 only.
+// grid = (ceil(F/128), H, B), block = 288.  Dynamic shared memory: Q (32 KiB) + K, V tiles (16 KiB each) + 1 KiB
+// alignment slack.  head_dim 128 only.
 __global__ void __launch_bounds__(FILLTC_THREADS, 2)
     tova_fill_attn_tc_kernel(const FillParams p, const __grid_constant__ CUtensorMap map_k,
                              const __grid_constant__ CUtensorMap map_v) {
@@ -144,7 +165,6 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   constexpr int KT = FILL_K_ROWS;                 // 64 state rows per tile
   constexpr int Q_BYTES = FILLTC_Q_ROWS * D * 2;  // two boxes of [128 rows][128 bytes]
   constexpr int T_BYTES = KT * D * 2;             // two boxes of [64 rows][128 bytes]
-  constexpr int P_BYTES = FILLTC_Q_ROWS * KT * 2; // one box of [128 rows][128 bytes]
 
   extern __shared__ unsigned char filltc_smem_raw[];
   unsigned char* smem =
@@ -152,8 +172,6 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   unsigned char* q_s = smem;
   unsigned char* k_s = q_s + Q_BYTES;
   unsigned char* v_s = k_s + T_BYTES;
-  unsigned char* ph_s = v_s + T_BYTES;
-  unsigned char* pl_s = ph_s + P_BYTES;
   // K tile, V tile landed; S = Q K^T, O += P V completed (tcgen05.commit); weights of a tile written (256 arrivals)
   // (one S barrier per S buffer: a barrier then completes once per two tiles, and a waiter can never be two phases behind)
   __shared__ __align__(8) uint64_t bar_k, bar_v, bar_s[2], bar_o, bar_p;
@@ -212,8 +230,7 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
     if ((tid & 31) == 0) {
       const uint32_t idesc_s = umma_idesc_bf16(FILLTC_Q_ROWS, KT, false);
       const uint32_t idesc_o = umma_idesc_bf16(FILLTC_Q_ROWS, D, true);
-      const uint32_t q_a = smem_addr(q_s), k_a = smem_addr(k_s), v_a = smem_addr(v_s), ph_a = smem_addr(ph_s),
-                     pl_a = smem_addr(pl_s);
+      const uint32_t q_a = smem_addr(q_s), k_a = smem_addr(k_s), v_a = smem_addr(v_s);
       auto load_k = [&](int i) {
         mbar_expect_tx(&bar_k, (uint32_t)T_BYTES);
         const int y = head_row0 + i * KT;
@@ -256,13 +273,13 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
         if (!okp) break;
         tc_fence_after();
         // O += P V: 4 steps of 16 state rows; V as stored is MN-major (D contiguous)
+        // (the weights sit where the tile's logits were: hi terms in the first 32 columns, lo terms in the other 32)
+        const uint32_t tm_p = tmem + (uint32_t)(64 * (i & 1));
 #pragma unroll
         for (int kk = 0; kk < KT / 16; ++kk) {
           const uint64_t bd = umma_desc_sw128(v_a + kk * 2048, KT * 128, 1024);
-          const uint64_t ah = umma_desc_sw128(ph_a + kk * 32, 16, 1024);
-          const uint64_t al = umma_desc_sw128(pl_a + kk * 32, 16, 1024);
-          umma_bf16(tmem + tm_o, ah, bd, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
-          umma_bf16(tmem + tm_o, al, bd, idesc_o, 1u);
+          umma_bf16_a_tmem(tmem + tm_o, tm_p + kk * 8, bd, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
+          umma_bf16_a_tmem(tmem + tm_o, tm_p + 32 + kk * 8, bd, idesc_o, 1u);
         }
         umma_commit(&bar_o);
         if (i + 2 < n_tiles) {                       // S(i+1) computed: K(i+2) may overwrite K(i+1)
@@ -308,6 +325,10 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
         for (int c = 0; c < KH; ++c) mx = fmaxf(mx, (!masked || jo + c <= vis) ? so[c] : -INFINITY);
       }
       tmem_ld32(lane_base + tm_s + (uint32_t)(KH * half), s);
+      // The weights will overwrite these columns: the row's other thread must have read its logits too.
+      tc_fence_before();
+      named_barrier_sync(1 + (warp & 3), 64);
+      tc_fence_after();
       const int jh = j0 + KH * half;
       if (j0 + KT - 1 > p.n0 + t0) {
 #pragma unroll
@@ -332,20 +353,17 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
         split_hi_lo(e0, e1, hi[e], lo[e]);
       }
       l_run = l_run * corr + lsum;
-      // The weights of tile i-1 are still being read, and O written, until O += P V of tile i-1 has completed.
-      if (i > 0) {
+      // The weights take the place of the tile's logits in tensor memory, as the A operand of O += P V: the
+      // row's 64 hi terms in the first 32 columns of the S buffer (two per column), the lo terms in the other 32.
+      // (The buffer of tile i-1, still being read by its contraction, is the other one.)
+      tmem_st16(lane_base + tm_s + (uint32_t)(16 * half), hi);
+      tmem_st16(lane_base + tm_s + 32u + (uint32_t)(16 * half), lo);
+      // O of the tiles so far was accumulated against the old max; it may be touched once O += P V of tile i-1
+      // has completed
+      if (i > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
         ok = __all_sync(0xffffffffu, fill_wait(&bar_o, (uint32_t)((i - 1) & 1))) != 0;
         if (!ok) break;
         tc_fence_after();
-      }
-#pragma unroll
-      for (int c8 = 0; c8 < KH / 8; ++c8) {
-        const uint32_t off = (uint32_t)row * 128u + (uint32_t)(((c8 + 4 * half) ^ (row & 7)) << 4);
-        *reinterpret_cast<uint4*>(ph_s + off) = make_uint4(hi[4 * c8], hi[4 * c8 + 1], hi[4 * c8 + 2], hi[4 * c8 + 3]);
-        *reinterpret_cast<uint4*>(pl_s + off) = make_uint4(lo[4 * c8], lo[4 * c8 + 1], lo[4 * c8 + 2], lo[4 * c8 + 3]);
-      }
-      // O of the tiles so far was accumulated against the old max
-      if (i > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
 #pragma unroll
         for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
           float o[32];
@@ -354,9 +372,8 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
           for (int c = 0; c < 32; ++c) o[c] *= corr;
           tmem_st32(lane_base + tm_o + c0, o);
         }
-        tmem_st_wait();
       }
-      fence_proxy_async_smem();   // P was written through the generic proxy, the tensor cores read it asynchronously
+      tmem_st_wait();
       tc_fence_before();
       mbar_arrive(&bar_p);        // this thread's part of the tile's weights (and of O) is in place
     }
@@ -365,7 +382,7 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
       tc_fence_after();
     }
     half_sum[half][row] = l_run;
-    named_barrier_sync(1, FILLTC_SOFTMAX_THREADS);
+    named_barrier_sync(5, FILLTC_SOFTMAX_THREADS);   // (barriers 1-4 belong to the pairs of warps that share rows)
     if (ok) {
       const float rl = 1.f / (half_sum[0][row] + half_sum[1][row]);
       const int t = t0 + row;
