@@ -10,8 +10,8 @@
 //                as soon as the contraction that read the buffer is complete)
 //   tcgen05.mma  S[128 x 64]  = Q[128 x D] . K^T          (A, B K-major; fp32 in TMEM, two S buffers: S of tile
 //                i+1 is issued as soon as its K tile is there, ahead of O += P V of tile i)
-//   tcgen05.ld   the row of S -> registers: the maximum over the whole tile (no exchange between the two threads of
-//                a row), the weights of the thread's half; online soft-max in the base-2 domain; weights as hi + lo
+//   tcgen05.ld   half a row of S -> registers (row maxima of the two halves exchanged through shared memory at the
+//                barrier the two warps of a row share); the weights of the thread's half; online soft-max in the base-2 domain; weights as hi + lo
 //                bf16 terms -> tcgen05.st back into the tile's S buffer, where they are the A operand of the
 //                second contraction (no trip through shared memory); if a row's running max moved, O is
 //                rescaled in TMEM (tcgen05.ld / tcgen05.st)
@@ -177,6 +177,7 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   __shared__ __align__(8) uint64_t bar_k, bar_v, bar_s[2], bar_o, bar_p;
   __shared__ uint32_t tmem_base_s;
   __shared__ float half_sum[2][FILLTC_Q_ROWS];   // the two halves of a row add up their sums at the end
+  __shared__ float half_max[2][2][FILLTC_Q_ROWS];   // ... and exchange their tile maxima (double-buffered by tile)
 
   const int tid = threadIdx.x, warp = tid >> 5;
   const int tile_q = gridDim.x - 1 - blockIdx.x;          // longest rows first
@@ -312,25 +313,13 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
       ok = __all_sync(0xffffffffu, fill_wait(&bar_s[i & 1], (uint32_t)((i >> 1) & 1))) != 0;   // this tile's logits
       if (!ok) break;
       tc_fence_after();
-      // the maximum over the whole tile, the weights of this thread's half
+      // this thread's half of the row's logits; the two halves exchange their maxima through shared memory
       constexpr int KH = KT / 2;
       float s[KH];
       float mx = -INFINITY;
-      {
-        float so[KH];
-        tmem_ld32(lane_base + tm_s + (uint32_t)(KH * (half ^ 1)), so);
-        const int jo = j0 + KH * (half ^ 1);
-        const bool masked = j0 + KT - 1 > p.n0 + t0;   // some query of this CTA cannot see the whole tile (CTA-uniform)
-#pragma unroll
-        for (int c = 0; c < KH; ++c) mx = fmaxf(mx, (!masked || jo + c <= vis) ? so[c] : -INFINITY);
-      }
       tmem_ld32(lane_base + tm_s + (uint32_t)(KH * half), s);
-      // The weights will overwrite these columns: the row's other thread must have read its logits too.
-      tc_fence_before();
-      named_barrier_sync(1 + (warp & 3), 64);
-      tc_fence_after();
       const int jh = j0 + KH * half;
-      if (j0 + KT - 1 > p.n0 + t0) {
+      if (j0 + KT - 1 > p.n0 + t0) {   // some query of this CTA cannot see the whole tile (CTA-uniform)
 #pragma unroll
         for (int c = 0; c < KH; ++c) {
           s[c] = (jh + c <= vis) ? s[c] : -INFINITY;
@@ -340,6 +329,12 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
 #pragma unroll
         for (int c = 0; c < KH; ++c) mx = fmaxf(mx, s[c]);
       }
+      half_max[i & 1][half][row] = mx;
+      // The weights will overwrite the logits' columns: the row's other thread must have read its logits too.
+      tc_fence_before();
+      named_barrier_sync(1 + (warp & 3), 64);
+      tc_fence_after();
+      mx = fmaxf(mx, half_max[i & 1][half ^ 1][row]);
       mx *= p.scale2;                             // scale2 > 0: the maximum commutes with the scaling
       const float m_new = fmaxf(m_run, mx);       // finite from tile 0 on: row 0 of the state is visible to every query
       const float corr = exp2_diff(m_run, m_new);
