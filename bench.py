@@ -548,6 +548,8 @@ def run_prefill(args):
     e1.record()
     torch.cuda.synchronize()
     clocks = sampler.stop()
+    for c in caches:
+        assert c.tova_cache_read()["status"] == 0, "a kernel reported a failed check"
     ms = e0.elapsed_time(e1) / steps
     launches = caches[-1].tova_cache_launches() - 1
     F = min(T, cap)

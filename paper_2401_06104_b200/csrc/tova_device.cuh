@@ -46,15 +46,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return done != 0;
 }
 
-// Bounded wait: every try_wait already blocks for a hardware-defined slice, so
-// the limit below is seconds of wall time, far beyond any legitimate copy.
-// Returns false when the limit ran out (the caller records an error and
-// carries on without touching the data).
+// Nanoseconds of the GPU's global timer.
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait: gives up two seconds after the first failed try, far beyond any legitimate copy or
+// contraction.  Returns false when the limit ran out (the caller records an error and carries on without
+// touching the data).
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-  for (int it = 0; it < (1 << 22); ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  while (!mbar_try_wait(bar, parity)) {
+    if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
   }
-  return false;
+  return true;
 }
 
 // All lanes of a warp wait for the same barrier phase; the verdict is made

@@ -92,14 +92,8 @@ __device__ __forceinline__ void named_barrier_sync(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
-// Bounded wait of the fill kernel: every try_wait blocks for a hardware-defined slice, so the limit is far beyond
-// any legitimate copy or contraction, yet a kernel whose roles have lost each other ends within seconds.
-__device__ __forceinline__ bool fill_wait(uint64_t* bar, uint32_t parity) {
-  for (int it = 0; it < (1 << 20); ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-  }
-  return false;
-}
+// Bounded wait of the fill kernel (two seconds, as everywhere).
+__device__ __forceinline__ bool fill_wait(uint64_t* bar, uint32_t parity) { return mbar_wait_bounded(bar, parity); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -178,6 +172,10 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
   __shared__ uint32_t tmem_base_s;
   __shared__ float half_sum[2][FILLTC_Q_ROWS];   // the two halves of a row add up their sums at the end
   __shared__ float half_max[2][2][FILLTC_Q_ROWS];   // ... and exchange their tile maxima (double-buffered by tile)
+
+  // A wait that ran out anywhere in this launch (or before) has left its code: the roles of that block have lost
+  // each other, and the blocks still to come give up at once instead of each waiting out its own limit.
+  if (*reinterpret_cast<volatile int32_t*>(p.status) != 0) return;
 
   const int tid = threadIdx.x, warp = tid >> 5;
   const int tile_q = gridDim.x - 1 - blockIdx.x;          // longest rows first
@@ -353,19 +351,24 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
       // (The buffer of tile i-1, still being read by its contraction, is the other one.)
       tmem_st16(lane_base + tm_s + (uint32_t)(16 * half), hi);
       tmem_st16(lane_base + tm_s + 32u + (uint32_t)(16 * half), lo);
-      // O of the tiles so far was accumulated against the old max; it may be touched once O += P V of tile i-1
-      // has completed
-      if (i > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
+      // Before this thread reports tile i, O += P V of tile i-1 must have completed: O may then be touched, and -
+      // since that contraction was only issued once EVERY thread had reported tile i-1 - no thread can report a
+      // tile while another still owes the previous one (the barrier counts arrivals, not tiles), nor can the
+      // barrier run two phases ahead of the issuing thread.
+      if (i > 0) {
         ok = __all_sync(0xffffffffu, fill_wait(&bar_o, (uint32_t)((i - 1) & 1))) != 0;
         if (!ok) break;
         tc_fence_after();
+        // O of the tiles so far was accumulated against the old max
+        if (__any_sync(0xffffffffu, corr != 1.f)) {
 #pragma unroll
-        for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
-          float o[32];
-          tmem_ld32(lane_base + tm_o + c0, o);
+          for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
+            float o[32];
+            tmem_ld32(lane_base + tm_o + c0, o);
 #pragma unroll
-          for (int c = 0; c < 32; ++c) o[c] *= corr;
-          tmem_st32(lane_base + tm_o + c0, o);
+            for (int c = 0; c < 32; ++c) o[c] *= corr;
+            tmem_st32(lane_base + tm_o + c0, o);
+          }
         }
       }
       tmem_st_wait();

@@ -50,11 +50,6 @@ __device__ __forceinline__ int32_t ld_acquire_sys(const int32_t* p) {
   asm volatile("ld.acquire.sys.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
 constexpr unsigned long long SHARD_WAIT_NS = 1000000000ull;   // how long a rank waits for its peers' parts
 
 __device__ __forceinline__ void st_release_sys(int32_t* p, int32_t v) {
