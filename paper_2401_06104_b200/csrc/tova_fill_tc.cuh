@@ -105,6 +105,26 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// Two fp32 operations in one instruction (sm_100: packed operands in a 64-bit register).
+__device__ __forceinline__ uint64_t pack_f2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t add_f2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+
 // 32 consecutive fp32 columns of this thread's TMEM lane.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   uint32_t r[32];
@@ -314,19 +334,22 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
       // this thread's half of the row's logits; the two halves exchange their maxima through shared memory
       constexpr int KH = KT / 2;
       float s[KH];
-      float mx = -INFINITY;
       tmem_ld32(lane_base + tm_s + (uint32_t)(KH * half), s);
       const int jh = j0 + KH * half;
       if (j0 + KT - 1 > p.n0 + t0) {   // some query of this CTA cannot see the whole tile (CTA-uniform)
 #pragma unroll
-        for (int c = 0; c < KH; ++c) {
-          s[c] = (jh + c <= vis) ? s[c] : -INFINITY;
-          mx = fmaxf(mx, s[c]);
-        }
-      } else {
-#pragma unroll
-        for (int c = 0; c < KH; ++c) mx = fmaxf(mx, s[c]);
+        for (int c = 0; c < KH; ++c) s[c] = (jh + c <= vis) ? s[c] : -INFINITY;
       }
+      // (four independent chains: a single running maximum would be 32 dependent instructions)
+      float mxa = fmaxf(s[0], s[1]), mxb = fmaxf(s[2], s[3]), mxc = fmaxf(s[4], s[5]), mxd = fmaxf(s[6], s[7]);
+#pragma unroll
+      for (int c = 8; c < KH; c += 8) {
+        mxa = fmaxf(mxa, fmaxf(s[c], s[c + 1]));
+        mxb = fmaxf(mxb, fmaxf(s[c + 2], s[c + 3]));
+        mxc = fmaxf(mxc, fmaxf(s[c + 4], s[c + 5]));
+        mxd = fmaxf(mxd, fmaxf(s[c + 6], s[c + 7]));
+      }
+      float mx = fmaxf(fmaxf(mxa, mxb), fmaxf(mxc, mxd));
       half_max[i & 1][half][row] = mx;
       // The weights will overwrite the logits' columns: the row's other thread must have read its logits too.
       tc_fence_before();
@@ -337,15 +360,30 @@ __global__ void __launch_bounds__(FILLTC_THREADS, 2)
       const float m_new = fmaxf(m_run, mx);       // finite from tile 0 on: row 0 of the state is visible to every query
       const float corr = exp2_diff(m_run, m_new);
       m_run = m_new;
-      float lsum = 0.f;
+      // Pairs of logits go through packed fp32 instructions: x = s * scale - m, the row sum, and the lo term
+      // e - hi(e) (as hi * -1 + e: one rounding, the same value as the subtraction).
+      const uint64_t scale_2 = pack_f2(p.scale2, p.scale2), mneg_2 = pack_f2(-m_new, -m_new);
+      const uint64_t minus1_2 = pack_f2(-1.f, -1.f);
+      uint64_t lsum2[2] = {pack_f2(0.f, 0.f), pack_f2(0.f, 0.f)};
       uint32_t hi[KH / 2], lo[KH / 2];
 #pragma unroll
       for (int e = 0; e < KH / 2; ++e) {
-        const float e0 = ex2_approx(fmaf(s[2 * e], p.scale2, -m_new)), e1 = ex2_approx(fmaf(s[2 * e + 1], p.scale2, -m_new));
-        lsum += e0 + e1;
-        split_hi_lo(e0, e1, hi[e], lo[e]);
+        float x0, x1;
+        unpack_f2(fma_f2(pack_f2(s[2 * e], s[2 * e + 1]), scale_2, mneg_2), x0, x1);
+        const float e0 = ex2_approx(x0), e1 = ex2_approx(x1);
+        const uint64_t e_2 = pack_f2(e0, e1);
+        lsum2[e & 1] = add_f2(lsum2[e & 1], e_2);
+        const __nv_bfloat162 hb = __floats2bfloat162_rn(e0, e1);
+        const uint32_t hw = *reinterpret_cast<const uint32_t*>(&hb);
+        float d0, d1;
+        unpack_f2(fma_f2(pack_f2(__uint_as_float(hw << 16), __uint_as_float(hw & 0xffff0000u)), minus1_2, e_2), d0, d1);
+        const __nv_bfloat162 lb = __floats2bfloat162_rn(d0, d1);
+        hi[e] = hw;
+        lo[e] = *reinterpret_cast<const uint32_t*>(&lb);
       }
-      l_run = l_run * corr + lsum;
+      float ls0, ls1;
+      unpack_f2(add_f2(lsum2[0], lsum2[1]), ls0, ls1);
+      l_run = l_run * corr + (ls0 + ls1);
       // The weights take the place of the tile's logits in tensor memory, as the A operand of O += P V: the
       // row's 64 hi terms in the first 32 columns of the S buffer (two per column), the lo terms in the other 32.
       // (The buffer of tile i-1, still being read by its contraction, is the other one.)
