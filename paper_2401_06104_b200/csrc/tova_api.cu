@@ -34,6 +34,7 @@ struct Layout {
   size_t st_q, st_k, st_v, st_out, st_ev;  // staging for host-buffer calls
   size_t df_k, df_v;                       // the new token's rows kept for a deferred eviction
   size_t upos, uacc;                       // per-KV-head slot tables and accumulated scores (head-wise policies, H2O)
+  size_t upart, uticket;                   // slice minima and ticket counters of the unit-policy kernel
   size_t shard_words;                      // epoch and ticket of the sharded step
   size_t total;
   int ld, pc;
@@ -85,6 +86,8 @@ Layout make_layout(const tova_config& c) {
   L.df_v = take(B * Hkv * D * E);
   L.upos = take(B * Hkv * cap * 4);
   L.uacc = take(B * Hkv * cap * 4);
+  L.upart = take(B * Hkv * tova::UNIT_MAX_SLICES * sizeof(tova::UnitPartial));
+  L.uticket = take(B * Hkv * 4);
   L.shard_words = take(8);
   L.total = off;
   return L;
@@ -439,8 +442,14 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, boo
     up.acc = reinterpret_cast<float*>(c->base + c->lay.uacc);
     up.recent = c->recent;
     up.h2o = (c->policy == tova::POLICY_H2O_LAYER || c->policy == tova::POLICY_H2O_HEAD) ? 1 : 0;
+    up.part = reinterpret_cast<tova::UnitPartial*>(c->base + c->lay.upart);
+    up.ticket = reinterpret_cast<int32_t*>(c->base + c->lay.uticket);
     const int nh = c->units == 1 ? p.H : p.G;
-    tova::tova_unit_policy_kernel<T, D><<<dim3(c->units, p.B), tova::UNIT_THREADS, sizeof(float) * nh, st>>>(p, up);
+    // Few (unit, sequence) pairs: cut each pair's candidates into slices of at least 256, up to two blocks per SM.
+    int slices = (2 * c->sm_count) / (c->units * p.B);
+    slices = std::min(slices, (p.n + 1 + 255) / 256);
+    slices = std::max(1, std::min(slices, tova::UNIT_MAX_SLICES));
+    tova::tova_unit_policy_kernel<T, D><<<dim3(c->units, p.B, slices), tova::UNIT_THREADS, sizeof(float) * nh, st>>>(p, up);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     c->launches += n_launch;
     return cudaSuccess;
@@ -1006,7 +1015,8 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   // per-unit slot tables start at -1 (all bytes 0xff), accumulated scores at zero
   const size_t unit_bytes = (size_t)cfg->batch * cfg->n_kv_heads * cfg->capacity * 4;
   if (cudaMemsetAsync(c->base + lay.upos, 0xff, unit_bytes, st) != cudaSuccess ||
-      cudaMemsetAsync(c->base + lay.uacc, 0, unit_bytes, st) != cudaSuccess) {
+      cudaMemsetAsync(c->base + lay.uacc, 0, unit_bytes, st) != cudaSuccess ||
+      cudaMemsetAsync(c->base + lay.uticket, 0, (size_t)cfg->batch * cfg->n_kv_heads * 4, st) != cudaSuccess) {
     delete c;
     return TOVA_ERR_CUDA;
   }

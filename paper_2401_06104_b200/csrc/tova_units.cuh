@@ -18,7 +18,11 @@
 // (max, sum) of the unit's heads, scores every candidate in a fixed order,
 // updates the accumulated scores (H2O), takes the arg-min - lowest slot on ties,
 // the new token counting as slot `capacity` - and puts the new token's key, value,
-// position and first score into the freed slot of the unit's KV heads.
+// position and first score into the freed slot of the unit's KV heads.  Where the
+// (unit, sequence) pairs are too few to fill the GPU (H2O layer-wise: one unit),
+// the candidates of a pair are cut into slices, one thread block each; the block
+// that finishes last (a ticket counter) merges the slices' minima in slice order
+// and does the insert, so no block ever waits for another.
 #pragma once
 
 #include "tova_kernels.cuh"
@@ -27,6 +31,13 @@ namespace tova {
 
 constexpr int POLICY_TOVA_HEAD = 2, POLICY_H2O_LAYER = 3, POLICY_H2O_HEAD = 4;
 constexpr int UNIT_THREADS = 512;
+constexpr int UNIT_MAX_SLICES = 8;
+
+struct UnitPartial {   // a slice's arg-min: value, slot, position held there; the new token's weight (its slice only)
+  float val;
+  int32_t idx, pos;
+  float wnew;
+};
 
 struct UnitParams {
   int32_t* table;     // [B,U,cap] position held by every slot of every unit
@@ -34,9 +45,11 @@ struct UnitParams {
   int32_t units;      // U: 1 (layer) or Hkv (one unit per KV head)
   int32_t recent;     // H2O: candidates fewer than `recent` positions behind the new token are never dropped
   int32_t h2o;        // scores accumulate over the steps
+  UnitPartial* part;  // [B,U,UNIT_MAX_SLICES] slice minima (used when gridDim.z > 1)
+  int32_t* ticket;    // [B,U] blocks of the pair that have finished this step; zero between steps
 };
 
-// grid = (U, B), block = UNIT_THREADS.  Dynamic shared memory: 2 floats per head of the unit.
+// grid = (U, B, slices), block = UNIT_THREADS.  Dynamic shared memory: one float per head of the unit.
 template <typename T, int D>
 __global__ void __launch_bounds__(UNIT_THREADS) tova_unit_policy_kernel(const StepParams p, const UnitParams up) {
   extern __shared__ __align__(16) float usm[];
@@ -52,6 +65,11 @@ __global__ void __launch_bounds__(UNIT_THREADS) tova_unit_policy_kernel(const St
   __shared__ int red_p[NW];
   __shared__ float s_wnew;
   __shared__ int s_victim;
+  __shared__ int s_last;
+  const int nz = gridDim.z, z = blockIdx.z;
+  const int slice = (p.n + 1 + nz - 1) / nz;             // candidates 0..n (n = the new token) in nz slices
+  const int j_lo = z * slice, j_hi = min(p.n + 1, j_lo + slice);
+  const bool owns_new = (p.n >= j_lo && p.n < j_hi);     // exactly one slice holds the new token
 
   const int pos_t = *p.cur_pos;
   int32_t* table = up.table + ((size_t)b * up.units + u) * p.cap;
@@ -82,7 +100,7 @@ __global__ void __launch_bounds__(UNIT_THREADS) tova_unit_policy_kernel(const St
   const float* lg = p.logits + ((size_t)b * p.H + h0) * p.ld;
   float val = INFINITY;
   int idx = 0x7fffffff, cpos = pos_t;
-  for (int j = tid; j <= p.n; j += UNIT_THREADS) {
+  for (int j = j_lo + tid; j < j_hi; j += UNIT_THREADS) {
     float w = 0.f;
 #pragma unroll 8
     for (int h = 0; h < nh; ++h) w += exp2f(lg[(size_t)h * p.ld + j] + hc[h]);
@@ -98,6 +116,7 @@ __global__ void __launch_bounds__(UNIT_THREADS) tova_unit_policy_kernel(const St
   }
 
   if (!p.do_evict) {                     // g(t) = min(t, k) not reached: the new token takes the next free row
+    if (!owns_new) return;               // (the other slices only had scores to add)
     __syncthreads();
     for (int i = tid; i < kv_n * (D * (int)sizeof(T) / 16); i += UNIT_THREADS) {
       constexpr int RB16 = D * (int)sizeof(T) / 16;
@@ -129,6 +148,33 @@ __global__ void __launch_bounds__(UNIT_THREADS) tova_unit_policy_kernel(const St
   if (tid == 0) {
     for (int w = 1; w < NW; ++w)
       if (red_v[w] < val || (red_v[w] == val && red_i[w] < idx)) { val = red_v[w]; idx = red_i[w]; cpos = red_p[w]; }
+    s_last = 1;
+    if (nz > 1) {
+      // This slice's minimum goes to global memory; the block that draws the last ticket merges them all.
+      UnitPartial* part = up.part + ((size_t)b * up.units + u) * UNIT_MAX_SLICES;
+      int32_t* ticket = up.ticket + (size_t)b * up.units + u;
+      UnitPartial mine;
+      mine.val = val; mine.idx = idx; mine.pos = cpos; mine.wnew = owns_new ? s_wnew : 0.f;
+      part[z] = mine;
+      __threadfence();                   // the partial and (through the barrier above) the block's scores, before the ticket
+      s_last = (atomicAdd(ticket, 1) == nz - 1);
+      if (s_last) {
+        __threadfence();
+        val = INFINITY; idx = 0x7fffffff; cpos = pos_t;
+        for (int q = 0; q < nz; ++q) {   // slice order = slot order: strict < keeps the lowest slot
+          const volatile UnitPartial* o = part + q;
+          const float ov = o->val;
+          const int oi = o->idx;
+          if (ov < val || (ov == val && oi < idx)) { val = ov; idx = oi; cpos = o->pos; }
+          if (p.n >= q * slice && p.n < q * slice + slice) s_wnew = o->wnew;
+        }
+        *ticket = 0;                     // ready for the next step (stream order)
+      }
+    }
+  }
+  __syncthreads();
+  if (!s_last) return;
+  if (tid == 0) {
     if (idx < 0 || idx > p.cap) { atomicExch(p.status, DEV_ERR_BAD_VICTIM); idx = p.cap; cpos = pos_t; }
     s_victim = idx;
     if (idx < p.cap) {

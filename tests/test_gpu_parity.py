@@ -461,6 +461,17 @@ def test_unit_policies_against_the_checker(policy, recent, shape):
     assert rep.evictions == w.batch * U * 50
 
 
+@pytest.mark.parametrize("policy,recent", [("h2o_layer", 0), ("h2o_layer", 40), ("tova_head", 0), ("h2o_head", 0)])
+def test_unit_policies_with_sliced_candidates(policy, recent):
+    """A state long enough that the (unit, sequence) pairs' candidates are cut into slices of thread blocks (701
+    candidates: three slices, the last one ragged, the new token in it) whose minima the last block merges: same
+    dropped positions, slot tables, outputs and scores as the checker, through the filling phase and beyond."""
+    w = MISTRAL.scaled(batch=2, n_q_heads=8, n_kv_heads=2, capacity=700)
+    U = 1 if policy == "h2o_layer" else w.n_kv_heads
+    rep = run_lockstep_units(w, 700 + 120, policy, recent, block=60)
+    assert rep.evictions == w.batch * U * 120
+
+
 def test_unit_policy_hand_worked_traces_on_gpu():
     from test_oracle_unit_policies import parse_unit_golden
     toks, _ = parse_golden()
