@@ -387,9 +387,18 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, boo
                                     (int)POSCOMP_SMEM_LIMIT)) != cudaSuccess) return e;
       pc_configured[c->device] = true;
     }
-    tova::tova_poscomp_kernel<T, D><<<p.B, tova::POSCOMP_THREADS, tova::poscomp_smem_bytes(p.cap, D), st>>>(p, c->poscomp);
+    // (the table's sines and cosines in double are the bulk of that kernel: a sequence's entries are shared out
+    //  among as many blocks as one wave of the GPU holds, at least 8 table rows each)
+    int pc_blocks = std::max(1, c->sm_count / p.B);
+    pc_blocks = std::max(1, std::min(pc_blocks, (p.n + 1 + 7) / 8));
+    tova::tova_poscomp_kernel<T, D><<<dim3(p.B, pc_blocks), tova::POSCOMP_THREADS, tova::poscomp_smem_bytes(p.cap, D), st>>>(
+        p, c->poscomp);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    tova::tova_split_rope_kernel<T, D><<<grid, 32, 0, st>>>(p, c->poscomp);
+    switch (tova::rope_unit_heads(p.G)) {
+      case 1: tova::tova_split_rope_kernel<T, D, 1><<<grid, 32, 0, st>>>(p, c->poscomp); break;
+      case 2: tova::tova_split_rope_kernel<T, D, 2><<<grid, 32, 0, st>>>(p, c->poscomp); break;
+      default: tova::tova_split_rope_kernel<T, D, 4><<<grid, 32, 0, st>>>(p, c->poscomp); break;
+    }
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if ((e = launch_combine<T, D>(c->device, p, st)) != cudaSuccess) return e;
     c->launches += 3;
@@ -660,10 +669,10 @@ void step_params(tova_cache* c, const void* q, const void* k, const void* v, int
   p.fuse_out = (c->fuse_merge && fused_merge_fits(cfg, c->chunk_rows, c->sm_count)) ? 1 : 0;
   p.merge_ctas = p.fuse_out ? (p.n_chunks + tova::SPLIT_MERGE_MAX_WARPS - 1) / tova::SPLIT_MERGE_MAX_WARPS : 1;
   if (p.merge_ctas < 1) p.merge_ctas = 1;
-  if (c->poscomp_ws) {         // the rotating streaming kernel: partials through global memory, 4 heads per warp
+  if (c->poscomp_ws) {         // the rotating streaming kernel: partials through global memory, up to 4 heads per warp
     p.fuse_out = 0;
     p.merge_ctas = 1;
-    p.hgroups = (p.G + tova::ROPE_UNIT_HEADS - 1) / tova::ROPE_UNIT_HEADS;
+    p.hgroups = (p.G + tova::rope_unit_heads(p.G) - 1) / tova::rope_unit_heads(p.G);
   }
   if (p.fuse_out && defer) {   // the split kernel keeps copies of the new token's rows for the later insert
     p.k_stage = base + c->lay.df_k;
@@ -1118,6 +1127,10 @@ int tova_cache_set_position_compression(tova_cache* c, void* dev_mem, size_t dev
   c->poscomp.q_rot = reinterpret_cast<float*>(ws + L.q_rot);
   c->poscomp.cpos = reinterpret_cast<double*>(ws + L.cpos);
   c->poscomp.rope_base = (double)rope_base;
+  static_assert(sizeof(c->poscomp.inv_freq) / sizeof(double) >= 64, "table of inverse frequencies");
+  if (c->cfg.head_dim > 128) return TOVA_ERR_UNSUPPORTED;
+  for (int d = 0; d < c->cfg.head_dim / 2; ++d)
+    c->poscomp.inv_freq[d] = std::pow((double)rope_base, -2.0 * (double)d / (double)c->cfg.head_dim);
   c->poscomp_ws = ws;
   return TOVA_OK;
 }

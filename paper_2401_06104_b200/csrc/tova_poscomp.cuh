@@ -9,10 +9,11 @@
 // ordinary step.  Attention depends on differences of positions only, so the
 // earliest retained token is put at 0.
 //
-//   tova_poscomp_kernel     per sequence: rank of every candidate by position,
-//                           the chain of compressed positions (in double, summed
-//                           in position order), a (cos, sin) table per candidate
-//                           and frequency, and the rotated query in fp32;
+//   tova_poscomp_kernel     per sequence: the candidates sorted by position (bitonic
+//                           sort in shared memory), the chain of compressed positions
+//                           (in double, prefix sums in position order), a (cos, sin)
+//                           table per candidate and frequency (angles reduced in
+//                           double, fp32 from there), and the rotated query in fp32;
 //   tova_split_rope_kernel  the streaming kernel of this mode: one warp per
 //                           (sequence, KV head, group of up to 4 query heads,
 //                           chunk of rows); rows come by plain 16-byte loads,
@@ -31,21 +32,46 @@
 namespace tova {
 
 constexpr int POSCOMP_THREADS = 512;
-constexpr int ROPE_UNIT_HEADS = 4;     // query heads one warp of the rotating streaming kernel carries
+constexpr int ROPE_UNIT_HEADS = 4;     // query heads one warp of the rotating streaming kernel carries at most
+// ... and for a group of G heads: 1, 2 or 4 (a warp carrying fewer heads than its template holds would repeat work)
+__host__ __device__ inline int rope_unit_heads(int G) { return G >= 3 ? 4 : (G == 2 ? 2 : 1); }
 
 struct PosCompParams {
   float2* table;      // [B,cap+1,D/2] (cos, sin) of candidate j (slot order, the new token at index n) and frequency d
   float* q_rot;       // [B,H,D] the query after rotary embedding at the new token's compressed position
   double* cpos;       // [B,cap+1] compressed positions (kept for inspection)
   double rope_base;
+  double inv_freq[64];   // rope_base^(-2d/D) for d < D/2 (head_dim <= 128), computed once on the host
 };
 
 __device__ __forceinline__ double compress_gap(int g) { return (g <= 10) ? (double)g : log(log((double)g)); }
 
-// grid = (B), block = POSCOMP_THREADS.  Dynamic shared memory (poscomp_smem_bytes): per candidate a double (the
-// chain) and three ints (position, rank, position by rank), plus D/2 doubles (inverse frequencies).
+// (cos, sin) of a non-negative angle given in double, to fp32 accuracy: the angle is reduced to [-pi/4, pi/4] in
+// double (x - k * pi/2; with k < 2^20 the one-term reduction is exact to ~1e-10), the remainder goes through the
+// fp32 routine, and the quadrant k mod 4 picks the signs.  A sixth of the cost of the double-precision routine.
+__device__ __forceinline__ float2 cos_sin_f32(double x) {
+  const double k = rint(x * 0.63661977236758134308);           // 2 / pi
+  const float r = (float)fma(-k, 1.57079632679489661923, x);   // pi / 2
+  float sr, cr;
+  sincosf(r, &sr, &cr);
+  const int q = (int)((long long)k & 3);
+  const float c = (q & 1) ? sr : cr, s2 = (q & 1) ? cr : sr;
+  // q = 0: (c, s); 1: (-s, c); 2: (-c, -s); 3: (s, -c)
+  return make_float2((q == 1 || q == 2) ? -c : c, (q >= 2) ? -s2 : s2);
+}
+
+__host__ __device__ inline int poscomp_sort_size(int cap) {   // the smallest power of two >= 32 that holds cap + 1 keys
+  int n = 32;
+  while (n < cap + 1) n <<= 1;
+  return n;
+}
+
+// grid = (B, blocks per sequence), block = POSCOMP_THREADS.  Dynamic shared memory (poscomp_smem_bytes): the sort
+// keys (64 bits each, a power of two of them), per candidate a double (the chain) and an int (its rank), plus D/2
+// doubles (inverse frequencies).
 __host__ __device__ inline size_t poscomp_smem_bytes(int cap, int D) {
-  return sizeof(double) * ((size_t)cap + 1 + D / 2) + sizeof(int32_t) * 3 * ((size_t)cap + 1);
+  return sizeof(unsigned long long) * (size_t)poscomp_sort_size(cap) + sizeof(double) * ((size_t)cap + 1 + D / 2) +
+         sizeof(int32_t) * ((size_t)cap + 1);
 }
 template <typename T, int D>
 __global__ void __launch_bounds__(POSCOMP_THREADS) tova_poscomp_kernel(const StepParams p, const PosCompParams pc) {
@@ -53,53 +79,84 @@ __global__ void __launch_bounds__(POSCOMP_THREADS) tova_poscomp_kernel(const Ste
   extern __shared__ __align__(16) unsigned char pcs_raw[];
   const int b = blockIdx.x, tid = threadIdx.x;
   const int m = p.n + 1;                                   // candidates: the live rows, then the new token
-  double* chain = reinterpret_cast<double*>(pcs_raw);      // [m] compressed position by rank
+  const int N = poscomp_sort_size(p.cap);
+  unsigned long long* key = reinterpret_cast<unsigned long long*>(pcs_raw);   // [N] (position, candidate), sorted below
+  double* chain = reinterpret_cast<double*>(key + N);      // [m] compressed position by rank
   double* inv_freq = chain + m;                            // [HALF]
-  int32_t* spos = reinterpret_cast<int32_t*>(inv_freq + HALF);   // [m] position by candidate
-  int32_t* rank = spos + m;                                // [m] rank of the candidate in position order
-  int32_t* sorted = rank + m;                              // [m] position by rank
+  int32_t* rank = reinterpret_cast<int32_t*>(inv_freq + HALF);   // [m] rank of the candidate in position order
   const int pos_t = (p.pos_t < 0) ? *p.cur_pos + 1 : p.pos_t;    // the streaming kernel of this step updates cur_pos later
 
-  for (int j = tid; j < m; j += NT) spos[j] = (j < p.n) ? p.pos[(size_t)b * p.cap + j] : pos_t;
-  for (int d = tid; d < HALF; d += NT) inv_freq[d] = pow(pc.rope_base, -2.0 * (double)d / (double)D);
+  // Candidates in position order (equal positions, which a caller could pass, in candidate order): a bitonic sort
+  // of (position, candidate) keys in shared memory, padded with keys beyond every position.
+  for (int j = tid; j < N; j += NT) {
+    const int pj = (j < p.n) ? p.pos[(size_t)b * p.cap + j] : pos_t;
+    key[j] = (j < m) ? (((unsigned long long)(unsigned int)pj << 32) | (unsigned int)j) : ~0ull;
+  }
+  for (int d = tid; d < HALF; d += NT) inv_freq[d] = pc.inv_freq[d];
   __syncthreads();
-  for (int j = tid; j < m; j += NT) {                      // positions are distinct: the rank is a permutation
-    const int pj = spos[j];
-    int r = 0;
-    for (int i = 0; i < m; ++i) r += (spos[i] < pj || (spos[i] == pj && i < j)) ? 1 : 0;
-    rank[j] = r;
+  for (int k = 2; k <= N; k <<= 1) {
+    // partners 32 or more apart: through shared memory, one pair per thread and turn
+    for (int j = k >> 1; j >= 32; j >>= 1) {
+      for (int u = tid; u < N / 2; u += NT) {
+        const int t = ((u & ~(j - 1)) << 1) | (u & (j - 1));   // the pair's lower index: bit j clear
+        const unsigned long long a = key[t], c = key[t | j];
+        if (((t & k) == 0) ? (a > c) : (a < c)) { key[t] = c; key[t | j] = a; }
+      }
+      __syncthreads();
+    }
+    // partners inside a warp's 32 consecutive keys: in registers, by shuffle
+    for (int t = tid; t < N; t += NT) {                        // N is a multiple of 32: whole warps
+      unsigned long long v = key[t];
+      const bool up = (t & k) == 0;
+      for (int j = min(k >> 1, 16); j > 0; j >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xffffffffu, v, j);
+        const bool lower = (t & j) == 0;
+        v = (lower == up) ? (v < o ? v : o) : (v > o ? v : o);
+      }
+      key[t] = v;
+    }
+    __syncthreads();
+  }
+  // rank of every candidate, then the compressed gap to the predecessor in position order
+  for (int r = tid; r < m; r += NT) {
+    rank[(int)(key[r] & 0xffffffffu)] = r;
+    chain[r] = (r > 0) ? compress_gap((int)(key[r] >> 32) - (int)(key[r - 1] >> 32)) : 0.0;
   }
   __syncthreads();
-  // positions by rank, then the compressed gap to the predecessor in position order
-  for (int j = tid; j < m; j += NT) sorted[rank[j]] = spos[j];
-  __syncthreads();
-  for (int r = tid; r < m; r += NT) chain[r] = (r > 0) ? compress_gap(sorted[r] - sorted[r - 1]) : 0.0;
-  __syncthreads();
-  if (tid == 0) {                                          // the chain, summed in position order
-    double acc = 0.0;
-    for (int r = 0; r < m; ++r) {
+  if (tid < 32) {
+    // The chain: prefix sums in position order, in double.  Every lane sums a run of consecutive ranks, the
+    // runs' totals are scanned across the warp, then every lane writes its run's prefixes.
+    const int per = (m + 31) / 32, r_lo = min(tid * per, m), r_hi = min(r_lo + per, m);
+    double run = 0.0;
+    for (int r = r_lo; r < r_hi; ++r) run += chain[r];
+    double incl = run;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const double up = __shfl_up_sync(0xffffffffu, incl, o);
+      if (tid >= o) incl += up;
+    }
+    double acc = incl - run;                               // total of the runs before this lane's
+    for (int r = r_lo; r < r_hi; ++r) {
       acc += chain[r];
       chain[r] = acc;
     }
   }
   __syncthreads();
-  // table of (cos, sin) and the compressed positions, by candidate
-  for (int j = tid; j < m; j += NT) pc.cpos[(size_t)b * (p.cap + 1) + j] = chain[rank[j]];
+  // table of (cos, sin) by candidate: the blocks of a sequence (gridDim.y of them, each having rebuilt the chain
+  // for itself) take the table's entries in turn; block 0 also stores the compressed positions and the query
   float2* tab = pc.table + (size_t)b * (p.cap + 1) * HALF;
-  for (int i = tid; i < m * HALF; i += NT) {
+  for (int i = blockIdx.y * NT + tid; i < m * HALF; i += NT * gridDim.y) {
     const int j = i / HALF, d = i % HALF;
-    double s, c;
-    sincos(chain[rank[j]] * inv_freq[d], &s, &c);
-    tab[i] = make_float2((float)c, (float)s);
+    tab[i] = cos_sin_f32(chain[rank[j]] * inv_freq[d]);
   }
-  __syncthreads();                                         // the new token's table row is complete (same block wrote it)
+  if (blockIdx.y != 0) return;
+  for (int j = tid; j < m; j += NT) pc.cpos[(size_t)b * (p.cap + 1) + j] = chain[rank[j]];
   // the query, rotated at the new token's position (fp32)
   const double pq = chain[rank[p.n]];
   for (int i = tid; i < p.H * HALF; i += NT) {
     const int h = i / HALF, d = i % HALF;
-    double s, c;
-    sincos(pq * inv_freq[d], &s, &c);
-    const float cf = (float)c, sf = (float)s;
+    const float2 cs = cos_sin_f32(pq * inv_freq[d]);
+    const float cf = cs.x, sf = cs.y;
     const T* qh = static_cast<const T*>(p.q) + ((size_t)b * p.H + h) * D;
     const float a = (float)qh[d], bb = (float)qh[d + HALF];
     float* dst = pc.q_rot + ((size_t)b * p.H + h) * D;
@@ -108,10 +165,10 @@ __global__ void __launch_bounds__(POSCOMP_THREADS) tova_poscomp_kernel(const Ste
   }
 }
 
-// grid = (max(n_chunks,1), Hkv*hgroups, B), block = one warp.  hgroups = ceil(G / ROPE_UNIT_HEADS).
-template <typename T, int D>
+// grid = (max(n_chunks,1), Hkv*hgroups, B), block = one warp.  hgroups = ceil(G / GU), GU = rope_unit_heads(G).
+template <typename T, int D, int GU>
 __global__ void __launch_bounds__(32) tova_split_rope_kernel(const StepParams p, const PosCompParams pc) {
-  constexpr int GU = ROPE_UNIT_HEADS;
+  static_assert(GU == 1 || GU == 2 || GU == 4, "heads per warp");
   constexpr int EPL = Vec16<T>::N;          // elements per lane
   constexpr int RB = D * (int)sizeof(T);
   constexpr int LPR = RB / 16;              // lanes per row
@@ -149,12 +206,13 @@ __global__ void __launch_bounds__(32) tova_split_rope_kernel(const StepParams p,
     wo.z = __shfl_xor_sync(0xffffffffu, w.z, LPR / 2);
     wo.w = __shfl_xor_sync(0xffffffffu, w.w, LPR / 2);
     Vec16<T>::unpack(wo, oth);
-    const float2* tr = tab + (size_t)j * HALF + d0;
+    const float4* tr = reinterpret_cast<const float4*>(tab + (size_t)j * HALF + d0);   // EPL is even, rows are 16-byte aligned
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      const float2 cs = __ldg(tr + e);
+    for (int e = 0; e < EPL; e += 2) {
+      const float4 cs = __ldg(tr + e / 2);                  // (cos, sin) of two neighbouring frequencies
       // lower half: a*c - b*s with a = own, b = partner; upper half: b*c + a*s with b = own, a = partner
       kf[e] = upper ? fmaf(oth[e], cs.y, own[e] * cs.x) : fmaf(-oth[e], cs.y, own[e] * cs.x);
+      kf[e + 1] = upper ? fmaf(oth[e + 1], cs.w, own[e + 1] * cs.z) : fmaf(-oth[e + 1], cs.w, own[e + 1] * cs.z);
     }
   };
 
@@ -190,13 +248,31 @@ __global__ void __launch_bounds__(32) tova_split_rope_kernel(const StepParams p,
   }
   const unsigned char* k_src = static_cast<const unsigned char*>(p.K) + (((size_t)b * p.Hkv + kvh) * p.cap + row_begin) * RB;
   const unsigned char* v_src = static_cast<const unsigned char*>(p.V) + (((size_t)b * p.Hkv + kvh) * p.cap + row_begin) * RB;
-#pragma unroll 4
+  // One head per warp: a pass is a short chain of dependent steps (rotation, reduction over the row's lanes,
+  // soft-max update) that cannot hide a trip to DRAM, so the rows of the next two passes are requested before the
+  // current one is worked on.  With more heads per warp a pass is long enough, and the registers are better spent
+  // on keeping more warps resident (measured: the look-ahead costs 30 % there).
+  constexpr int AHEAD = (GU == 1) ? 2 : 0;
+  uint4 kq[AHEAD + 1], vq[AHEAD + 1];
+#pragma unroll
+  for (int a = 0; a < AHEAD; ++a) {
+    const int rr = min(a * RPW + sub, rows - 1);
+    kq[a] = __ldg(reinterpret_cast<const uint4*>(k_src + (size_t)rr * RB) + lig);
+    vq[a] = __ldg(reinterpret_cast<const uint4*>(v_src + (size_t)rr * RB) + lig);
+  }
+#pragma unroll(AHEAD > 0 ? 2 : 4)
   for (int r0 = 0; r0 < rows; r0 += RPW) {          // uniform trip count: the shuffles need the whole warp
     const int r = r0 + sub;
     const bool live = r < rows;
     const int rr = live ? r : rows - 1;
-    const uint4 kw = __ldg(reinterpret_cast<const uint4*>(k_src + (size_t)rr * RB) + lig);
-    const uint4 vw = __ldg(reinterpret_cast<const uint4*>(v_src + (size_t)rr * RB) + lig);
+    {
+      const int rn = min(r0 + AHEAD * RPW + sub, rows - 1);   // AHEAD = 0: this pass's own rows
+      kq[AHEAD] = __ldg(reinterpret_cast<const uint4*>(k_src + (size_t)rn * RB) + lig);
+      vq[AHEAD] = __ldg(reinterpret_cast<const uint4*>(v_src + (size_t)rn * RB) + lig);
+    }
+    const uint4 kw = kq[0], vw = vq[0];
+#pragma unroll
+    for (int a = 0; a < AHEAD; ++a) { kq[a] = kq[a + 1]; vq[a] = vq[a + 1]; }
     float kf[EPL], vf[EPL];
     rotate(kw, row_begin + rr, kf);
     Vec16<T>::unpack(vw, vf);
