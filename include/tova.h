@@ -233,8 +233,9 @@ int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows);
  * TOVA_ERR_BAD_SHAPE; an unknown policy gives TOVA_ERR_UNSUPPORTED.  Positions
  * passed to the step calls must be >= 0, distinct and increasing for Window, "+i"
  * and H2O to mean what the paper describes; ties go to the lowest slot as
- * everywhere.  Head-wise and H2O policies process prompts token by token and
- * ignore deferred eviction.  Not available through tova_decode_step_static. */
+ * everywhere.  Head-wise and H2O policies process prompts token by token; with
+ * deferred eviction their victim choice and insert run on the cache's stream like
+ * the layer policies'.  Not available through tova_decode_step_static. */
 #define TOVA_POLICY_TOVA 0
 #define TOVA_POLICY_WINDOW 1
 #define TOVA_POLICY_TOVA_HEAD 2
@@ -268,7 +269,7 @@ int32_t tova_cache_units(const tova_cache* c);
  *        B*(capacity+1)*D/2 pairs, the rotated query, the positions.
  *   tova_cache_set_position_compression  dev_mem: 256-byte aligned device
  *        memory of that size, owned by the caller, to outlive the handle (NULL:
- *        off); only while the state is empty; capacity up to about 8000 rows
+ *        off); only while the state is empty; capacity up to about 7000 rows
  *        (TOVA_ERR_UNSUPPORTED beyond, and together with head-wise policies or
  *        sharding).  The step then takes three launches and a slower streaming
  *        kernel (a table read and a rotation per cached row); prompts go token

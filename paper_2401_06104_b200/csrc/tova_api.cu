@@ -458,8 +458,23 @@ cudaError_t launch_step(tova_cache* c, const StepParams& p, cudaStream_t st, boo
     int slices = (2 * c->sm_count) / (c->units * p.B);
     slices = std::min(slices, (p.n + 1 + 255) / 256);
     slices = std::max(1, std::min(slices, tova::UNIT_MAX_SLICES));
-    tova::tova_unit_policy_kernel<T, D><<<dim3(c->units, p.B, slices), tova::UNIT_THREADS, sizeof(float) * nh, st>>>(p, up);
+    // Deferred: victim choice and insert run on the side stream, from the copies of the new token's rows that the
+    // streaming kernel (or the outputs launch) left in the cache block, and overlap whatever the caller enqueues next.
+    StepParams pu = p;
+    cudaStream_t ust = st;
+    if (defer) {
+      if ((e = cudaEventRecord(c->ev_fork, st)) != cudaSuccess) return e;
+      if ((e = cudaStreamWaitEvent(c->side, c->ev_fork, 0)) != cudaSuccess) return e;
+      pu.k_new = c->base + c->lay.df_k;
+      pu.v_new = c->base + c->lay.df_v;
+      ust = c->side;
+    }
+    tova::tova_unit_policy_kernel<T, D><<<dim3(c->units, p.B, slices), tova::UNIT_THREADS, sizeof(float) * nh, ust>>>(pu, up);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if (defer) {
+      if ((e = cudaEventRecord(c->ev_join, c->side)) != cudaSuccess) return e;
+      c->pending = true;
+    }
     c->launches += n_launch;
     return cudaSuccess;
   }
@@ -685,7 +700,7 @@ int step_impl(tova_cache* c, const void* q, const void* k, const void* v, int32_
   const tova_config& cfg = c->cfg;
   if (c->len >= cfg.capacity && !cfg.evict) return TOVA_ERR_FULL;
   if (c->shard_on) return TOVA_ERR_BAD_SHAPE;   // a sharded layer steps through its two-phase calls
-  const bool defer = c->deferred && allow_defer && c->units == 0 && !c->poscomp_ws;
+  const bool defer = c->deferred && allow_defer && !c->poscomp_ws;
   StepParams p{};
   step_params(c, q, k, v, pos, out, evicted_pos, defer, p);
   cudaError_t e;

@@ -472,6 +472,51 @@ def test_unit_policies_with_sliced_candidates(policy, recent):
     assert rep.evictions == w.batch * U * 120
 
 
+@pytest.mark.parametrize("policy", ["tova_head", "h2o_layer", "h2o_head"])
+@pytest.mark.parametrize("fused", [True, False])
+def test_unit_policies_deferred_eviction_gives_identical_results(policy, fused):
+    """Head-wise and H2O policies with victim choice and insert on the cache's side stream, two caches taking
+    turns like the layers of a model, the caller's k and v buffers overwritten right after every call: same
+    outputs, dropped positions, slot tables, rows and scores as the default mode."""
+    w = MISTRAL.scaled(batch=2, n_q_heads=8, n_kv_heads=4, capacity=90)
+    T = 200
+    code = {"tova_head": tova.TOVA_POLICY_TOVA_HEAD, "h2o_layer": tova.TOVA_POLICY_H2O_LAYER,
+            "h2o_head": tova.TOVA_POLICY_H2O_HEAD}[policy]
+    U = 1 if policy == "h2o_layer" else w.n_kv_heads
+    streams = [W.tokens(w, 0, T, layer=l) for l in range(2)]
+    ref = [make_cache(w, fused_merge=fused) for _ in range(2)]
+    dfr = [make_cache(w, fused_merge=fused) for _ in range(2)]
+    for c in ref + dfr:
+        c.tova_cache_set_policy(code, 0)
+    for c in dfr:
+        c.tova_cache_set_deferred_eviction(True)
+    dev = [[tova.to_device(a, w.dtype) for a in s] for s in streams]
+    shape = (T, w.batch, w.n_q_heads, w.head_dim)
+    o_ref = [torch.empty(shape, device="cuda:0") for _ in range(2)]
+    o_dfr = [torch.empty(shape, device="cuda:0") for _ in range(2)]
+    e_ref = [torch.full((T, w.batch, U), -7, dtype=torch.int32, device="cuda:0") for _ in range(2)]
+    e_dfr = [torch.full((T, w.batch, U), -7, dtype=torch.int32, device="cuda:0") for _ in range(2)]
+    kbuf, vbuf = torch.empty_like(dev[0][1][0]), torch.empty_like(dev[0][2][0])
+    for t in range(T):
+        for l in range(2):
+            q, k, v = dev[l]
+            ref[l].tova_decode_step(q[t], k[t], v[t], t, o_ref[l][t], e_ref[l][t])
+            kbuf.copy_(k[t]); vbuf.copy_(v[t])
+            dfr[l].tova_decode_step(q[t], kbuf, vbuf, t, o_dfr[l][t], e_dfr[l][t])
+            kbuf.zero_(); vbuf.zero_()          # the library keeps its own copies for the later insert
+    for c in dfr:
+        c.tova_cache_join()
+    torch.cuda.synchronize()
+    for l in range(2):
+        assert torch.equal(o_ref[l], o_dfr[l]) and torch.equal(e_ref[l], e_dfr[l])
+        a, b = ref[l].tova_cache_read(want_kv=True), dfr[l].tova_cache_read(want_kv=True)
+        assert a["status"] == 0 and b["status"] == 0
+        for key in ("len", "positions", "K", "V"):
+            assert torch.equal(a[key], b[key]), key
+        if policy.startswith("h2o"):
+            assert torch.equal(ref[l].tova_cache_read_scores(), dfr[l].tova_cache_read_scores())
+
+
 def test_unit_policy_hand_worked_traces_on_gpu():
     from test_oracle_unit_policies import parse_unit_golden
     toks, _ = parse_golden()
