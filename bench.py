@@ -67,6 +67,8 @@ def parse_args():
                          "(-1: as many tokens as the state holds); a step is one whole prompt")
     ap.add_argument("--no-bulk-prefill", action="store_true", help="with --prefill: every prompt token takes the decode kernels")
     ap.add_argument("--warp-mma-prefill", action="store_true", help="with --prefill: bulk fill through the warp-level MMA kernel")
+    ap.add_argument("--chunk-barriers", type=int, default=0, choices=[0, 2],
+                    help="with --prefill: 2 = the deletion kernel's cluster meets twice per token (0 = once where it fits)")
     ap.add_argument("--chunk-cluster", type=int, default=0,
                     help="with --prefill: thread blocks per sequence in the kernel that replays a chunk's deletions (0 = auto)")
     ap.add_argument("--no-chunked-prefill", action="store_true",
@@ -534,6 +536,8 @@ def run_prefill(args):
             ws = c.tova_cache_set_prefill_workspace(ws)          # one workspace serves all: calls share a stream
             if args.chunk_cluster:
                 c.tova_cache_set_chunk_cluster(args.chunk_cluster)
+            if args.chunk_barriers:
+                c.tova_cache_set_chunk_barriers(args.chunk_barriers)
         caches.append(c)
     torch.cuda.synchronize()
     for c in caches[:warm]:

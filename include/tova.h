@@ -160,6 +160,14 @@ int tova_cache_set_prefill_workspace(tova_cache* c, void* dev_mem, size_t dev_by
  * beyond floating-point summation order.  Other values: TOVA_ERR_BAD_SHAPE. */
 int tova_cache_set_chunk_cluster(tova_cache* c, int32_t ctas);
 
+/* ... and how the blocks of such a cluster meet.  0 (default): once per token
+ * where the logits of two tokens fit the shared memory (a token's normaliser is
+ * then the row sum minus the terms of the rows dropped so far, and candidates
+ * are scored in one pass), else twice per token; 2: always twice (normaliser
+ * summed over the live rows, then the scores).  Same results up to
+ * floating-point summation order.  Other values: TOVA_ERR_BAD_SHAPE. */
+int tova_cache_set_chunk_barriers(tova_cache* c, int32_t per_token);
+
 /* tova_decode_step with HOST buffers; returns after `cuda_stream` has been
  * synchronised, when out (and evicted_pos if not NULL) hold the results.
  * Page-locked buffers (pinned or registered, 16-byte aligned; all of them):

@@ -86,6 +86,8 @@ def lib() -> ctypes.CDLL:
         L.tova_decode_step_commit.argtypes = [vp, vp, vp, vp, vp]
         L.tova_cache_set_chunk_cluster.restype = ctypes.c_int
         L.tova_cache_set_chunk_cluster.argtypes = [vp, i32]
+        L.tova_cache_set_chunk_barriers.restype = ctypes.c_int
+        L.tova_cache_set_chunk_barriers.argtypes = [vp, i32]
         L.tova_cache_read_scores.restype = ctypes.c_int
         L.tova_cache_read_scores.argtypes = [vp, vp, vp]
         L.tova_cache_units.restype = i32
@@ -261,6 +263,9 @@ class TovaCache:
 
     def tova_cache_set_chunk_cluster(self, ctas: int) -> None:
         _check(lib().tova_cache_set_chunk_cluster(self._h, int(ctas)), "tova_cache_set_chunk_cluster")
+
+    def tova_cache_set_chunk_barriers(self, per_token: int) -> None:
+        _check(lib().tova_cache_set_chunk_barriers(self._h, int(per_token)), "tova_cache_set_chunk_barriers")
 
     def tova_cache_set_chunk_rows(self, rows: int) -> None:
         _check(lib().tova_cache_set_chunk_rows(self._h, int(rows)), "tova_cache_set_chunk_rows")

@@ -146,6 +146,7 @@ struct tova_cache {
   tova::ShardParams shard;
   unsigned char* chunk_ws;
   int chunk_cluster;       // 0: automatic; 1, 2, 4, 8: CTAs per sequence of the deletion kernel; -1: the one-CTA kernel
+  int chunk_two_barriers;  // 1: the cluster kernel with two barriers per token even where the one-barrier kernel fits
   ChunkLayout chunk_lay;
   CUtensorMap chunk_map_k, chunk_map_v;
   int32_t len;          // rows per sequence (host mirror; sequences move in lock step)
@@ -831,12 +832,19 @@ cudaError_t launch_chunk_d(tova_cache* c, const tova::ChunkParams& p, cudaStream
     while (nc > 1 && (long long)p.B * nc > c->sm_count) nc >>= 1;
     if (c->chunk_cluster > 0) nc = c->chunk_cluster;
     const int S = ((p.cap + nc - 1) / nc + 3) / 4 * 4;
+    // Two or more tokens' logits staged: the kernel with one cluster barrier per token; one: the kernel with two.
+    int nstage1 = tova::CHUNK_STAGES_MAX;
+    while (nstage1 > 0 && tova::chunk_cluster1_smem(p.H, S, nstage1) > CHUNK_CLUSTER_SMEM_LIMIT) --nstage1;
+    const bool one_barrier = nstage1 >= 2 && c->chunk_two_barriers == 0;
     int nstage = tova::CHUNK_STAGES_MAX;
     while (nstage > 0 && tova::chunk_cluster_smem(p.H, S, nstage) > CHUNK_CLUSTER_SMEM_LIMIT) --nstage;
+    if (one_barrier) nstage = nstage1;
     if (nstage > 0 && c->chunk_cluster >= 0) {
       static std::atomic<bool> cl_configured[64];
       if (c->device >= 0 && c->device < 64 && !cl_configured[c->device]) {
         if ((e = cudaFuncSetAttribute(tova::tova_chunk_resolve_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)CHUNK_CLUSTER_SMEM_LIMIT)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(tova::tova_chunk_resolve_cluster1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)CHUNK_CLUSTER_SMEM_LIMIT)) != cudaSuccess) return e;
         cl_configured[c->device] = true;
       }
@@ -845,7 +853,7 @@ cudaError_t launch_chunk_d(tova_cache* c, const tova::ChunkParams& p, cudaStream
       int nt = 256;                            // about one thread per candidate of a CTA
       while (nt < tova::CHUNK_CLUSTER_THREADS_MAX && nt < S + 1) nt *= 2;
       cfg.blockDim = dim3(nt);
-      cfg.dynamicSmemBytes = tova::chunk_cluster_smem(p.H, S, nstage);
+      cfg.dynamicSmemBytes = one_barrier ? tova::chunk_cluster1_smem(p.H, S, nstage) : tova::chunk_cluster_smem(p.H, S, nstage);
       cfg.stream = st;
       cudaLaunchAttribute at[1];
       at[0].id = cudaLaunchAttributeClusterDimension;
@@ -854,7 +862,8 @@ cudaError_t launch_chunk_d(tova_cache* c, const tova::ChunkParams& p, cudaStream
       at[0].val.clusterDim.z = 1;
       cfg.attrs = at;
       cfg.numAttrs = 1;
-      e = cudaLaunchKernelEx(&cfg, tova::tova_chunk_resolve_cluster_kernel, p, S, nstage);
+      e = one_barrier ? cudaLaunchKernelEx(&cfg, tova::tova_chunk_resolve_cluster1_kernel, p, S, nstage)
+                      : cudaLaunchKernelEx(&cfg, tova::tova_chunk_resolve_cluster_kernel, p, S, nstage);
     } else {
       tova::tova_chunk_resolve_kernel<<<p.B, tova::CHUNK_RESOLVE_THREADS, chunk_resolve_smem(c->cfg), st>>>(p);
       e = cudaGetLastError();
@@ -1002,6 +1011,7 @@ int tova_cache_init(tova_cache** out, const tova_config* cfg, void* dev_mem, siz
   c->shard_on = false;
   c->shard_scored = false;
   c->chunk_cluster = 0;
+  c->chunk_two_barriers = 0;
   c->deferred = false;
   c->pending = false;
   c->side = nullptr;
@@ -1236,6 +1246,13 @@ int tova_cache_set_chunk_cluster(tova_cache* c, int32_t ctas) {
   if (!c) return TOVA_ERR_NULL;
   if (ctas != -1 && ctas != 0 && ctas != 1 && ctas != 2 && ctas != 4 && ctas != 8) return TOVA_ERR_BAD_SHAPE;
   c->chunk_cluster = ctas;
+  return TOVA_OK;
+}
+
+int tova_cache_set_chunk_barriers(tova_cache* c, int32_t per_token) {
+  if (!c) return TOVA_ERR_NULL;
+  if (per_token != 0 && per_token != 2) return TOVA_ERR_BAD_SHAPE;
+  c->chunk_two_barriers = per_token == 2 ? 1 : 0;
   return TOVA_OK;
 }
 

@@ -16,8 +16,11 @@
 //             earlier tokens - plus each query's row maximum R and the sum T of
 //             exp2(logit - R) over all those columns (tova_chunk_attn_kernel,
 //             MODE 0; warp-level bf16 MMAs, as in the bulk fill);
-//   resolve   one thread block per sequence replays the chunk's deletions in
-//             order from those logits alone (tova_chunk_resolve_kernel): for
+//   resolve   one thread block per sequence - or a cluster of blocks that share
+//             out the slots, with the logits staged in shared memory
+//             (tova_chunk_resolve_cluster1_kernel, one cluster barrier per token;
+//             tova_chunk_resolve_cluster_kernel, two) - replays the chunk's
+//             deletions in order from those logits alone (tova_chunk_resolve_kernel): for
 //             token i it removes the rows dropped by tokens < i from the
 //             normaliser (L = T - their terms), scores the k+1 live candidates
 //             by the head-averaged soft-max weight (Eq. 4, Algorithm 1), takes
@@ -77,6 +80,13 @@ struct ChunkParams {
 };
 
 constexpr int32_t CHUNK_ALIVE = 0x7fffffff;
+
+// 2^x by the special-function unit alone; results below the smallest normal number become zero.
+__device__ __forceinline__ float exp2_fast(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
 // The chunk's keys/values into the staging tiles (rows past the chunk are zeroed: they are read with weight zero),
 // every column's death step reset, the first position fixed for the later kernels.
@@ -609,6 +619,233 @@ __global__ void __launch_bounds__(CHUNK_CLUSTER_THREADS_MAX) tova_chunk_resolve_
     }
     __syncthreads();                                     // the buffer has been read by everybody; occl is up to date
     if (warp == 0 && i + nstage < p.C) {
+      fence_proxy_async_smem();
+      request(i + nstage);
+    }
+  }
+  if (!ok && tid == 0) atomicExch(p.status, DEV_ERR_COPY_TIMEOUT);
+  for (int t = tid; t < n_loc; t += NT) {
+    p.pos[(size_t)b * p.cap + s_begin + t] = posv[t];
+    p.slot_token[(size_t)b * p.cap + s_begin + t] = (occl[t] >= S) ? occl[t] - S : -1;
+  }
+}
+
+// The same replay with ONE cluster barrier per token (used where at least two tokens' logits fit in shared memory).
+// The normaliser of a token needs no pass of its own: L = T - (terms of the columns dropped so far), T being the
+// row sum over all columns that the logits pass left behind.  Every CTA keeps the list of the columns that died in
+// ITS slots (CTA 0 also of the tokens that dropped themselves) and, while token i is being decided, adds up their
+// terms for token i+1; the column that dies AT token i is not known before the barrier, so every CTA sends, with its
+// candidate for the arg-min, that candidate's terms for token i+1.  After the barrier every CTA holds the same
+// arg-min, the winner's terms and all partial corrections: L of token i+1 follows without another exchange, and the
+// candidates are scored in a single pass (exp2 of logit - R - log2(L H), summed over the heads).
+__host__ __device__ inline size_t chunk_cluster1_smem(int H, int S, int nstage) {
+  return sizeof(float) * ((size_t)nstage * H * (S + CHUNK_TOKENS) + 2 * (size_t)CHUNK_TOKENS * H +
+                          4 * (size_t)CHUNK_CLUSTER_MAX * H + 2 * (size_t)H) +
+         sizeof(int32_t) * 2 * (size_t)S + 64;
+}
+
+__global__ void __launch_bounds__(CHUNK_CLUSTER_THREADS_MAX) tova_chunk_resolve_cluster1_kernel(const ChunkParams p,
+                                                                                            const int S, const int nstage) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cl = cg::this_cluster();
+  constexpr int NWM = CHUNK_CLUSTER_THREADS_MAX / 32, NCM = CHUNK_CLUSTER_MAX;
+  const int NT = (int)blockDim.x, NW = NT / 32;
+  const int NC = (int)cl.num_blocks(), r = (int)cl.block_rank();
+  const int b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int H = p.H, SW = S + CHUNK_TOKENS;
+
+  extern __shared__ __align__(16) float csm3[];
+  float* stage = csm3;                                        // [nstage][H][SW]
+  float* Rs = stage + (size_t)nstage * H * SW;               // [64][H] row maxima of the chunk's queries
+  float* Ts = Rs + (size_t)CHUNK_TOKENS * H;                 // [64][H] row sums over all columns
+  float* xen = Ts + (size_t)CHUNK_TOKENS * H;                // [2][NCM][H] every CTA's candidate: its terms for the next token
+  float* xco = xen + 2 * (size_t)NCM * H;                    // [2][NCM][H] every CTA's correction for the next token
+  float* hc = xco + 2 * (size_t)NCM * H;                     // [H] -R - log2(L * H) of the current token
+  float* s_co = hc + H;                                      // [H] this CTA's correction for the next token
+  int32_t* occl = reinterpret_cast<int32_t*>(s_co + H);   // [S] staged column holding the slot's occupant
+  int32_t* posv = occl + S;                                  // [S] position it holds
+  __shared__ __align__(8) uint64_t full[CHUNK_STAGES_MAX];
+  __shared__ float2 best[2][NCM];                            // (value, slot) of every CTA, double-buffered
+  __shared__ float red_v[NWM];
+  __shared__ int red_i[NWM], red_c[NWM];
+  __shared__ int32_t dead[CHUNK_TOKENS];                     // staged columns that died in this CTA's care
+  __shared__ int s_ndead;
+
+  const int s_begin = r * S;
+  const int n_loc = max(0, min(S, p.cap - s_begin));          // slots this CTA really owns
+  const int n_cand = n_loc + (r == 0 ? 1 : 0);                // plus the new token
+  const int first = *p.first;
+  const float* lgb = p.lg + (size_t)b * CHUNK_TOKENS * H * p.ldc;
+
+  if (tid == 0) {
+    for (int s = 0; s < nstage; ++s) mbar_init(&full[s], 1);
+    mbar_fence_init();
+    s_ndead = 0;
+  }
+  for (int t = tid; t < S; t += NT) {
+    occl[t] = t;
+    posv[t] = (t < n_loc) ? p.pos[(size_t)b * p.cap + s_begin + t] : 0;
+  }
+  for (int t = tid; t < CHUNK_TOKENS * H; t += NT) {
+    const int i = t / H, h = t % H;
+    const float2 e = (i < p.C) ? p.rt[((size_t)b * H + h) * CHUNK_TOKENS + i] : make_float2(0.f, 1.f);
+    Rs[t] = e.x;
+    Ts[t] = e.y;
+  }
+  __syncthreads();
+  for (int h = tid; h < H; h += NT) {                        // token 0: nothing has been dropped yet
+    hc[h] = -Rs[h] - __log2f(Ts[h] * (float)H);
+    if (r == 0) p.ml[((size_t)b * H + h) * CHUNK_TOKENS] = make_float2(Rs[h], Ts[h]);
+  }
+  // logits of token i into buffer i % nstage: per head the CTA's state columns and the chunk's columns, 2 H bulk
+  // copies shared out among the warps (a lane issues its copies one after the other: one warp alone would spend
+  // more time issuing them than the token's arithmetic takes).  `arm` comes first, from one thread.
+  auto arm = [&](int i) { mbar_expect_tx(&full[i % nstage], (uint32_t)H * (uint32_t)SW * 4u); };
+  auto request = [&](int i) {
+    uint64_t* bar = &full[i % nstage];
+    float* dst = stage + (size_t)(i % nstage) * H * SW;
+    const float* src = lgb + (size_t)i * H * p.ldc;
+    if (lane < 4) {
+      for (int j = warp * 4 + lane; j < 2 * H; j += NW * 4) {
+        const int h = j >> 1;
+        if (j & 1) bulk_g2s(dst + (size_t)h * SW + S, src + (size_t)h * p.ldc + p.capA, (uint32_t)CHUNK_TOKENS * 4u, bar);
+        else bulk_g2s(dst + (size_t)h * SW, src + (size_t)h * p.ldc + s_begin, (uint32_t)S * 4u, bar);
+      }
+    }
+  };
+  if (tid == 0)
+    for (int i = 0; i < min(nstage, p.C); ++i) arm(i);
+  __syncthreads();
+  for (int i = 0; i < min(nstage, p.C); ++i) request(i);
+  cl.sync();                                                  // every CTA of the cluster runs: its shared memory may be written
+
+  bool ok = true;
+  for (int i = 0; i < p.C; ++i) {
+    const int pos_i = first + i;
+    const int par = i & 1;
+    const bool more = i + 1 < p.C;
+    const float* st = stage + (size_t)(i % nstage) * H * SW;
+    const float* st1 = stage + (size_t)((i + 1) % nstage) * H * SW;   // the next token's logits (more)
+    ok = warp_wait(&full[i % nstage], (uint32_t)((i / nstage) & 1)) && ok;
+    // ---- head-averaged weight of this CTA's candidates, lowest (value, slot) -----------------------------
+    float val = INFINITY;
+    int idx = 0x7fffffff, ccol = -1;
+    for (int t = tid; t < n_cand; t += NT) {
+      const int c = (t < n_loc) ? occl[t] : S + i;
+      const int pj = (t < n_loc) ? posv[t] : pos_i;
+      const float* col = st + c;
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;       // fixed order: heads h = 0,4,8,.. / 1,5,.. / 2,6,.. / 3,7,..
+      int h = 0;
+      for (; h + 7 < H; h += 8) {                         // eight heads' logits requested before the first is used
+        float x[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) x[u] = col[(h + u) * SW] + hc[h + u];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) x[u] = exp2_fast(x[u]);
+        a0 += x[0] + x[4];
+        a1 += x[1] + x[5];
+        a2 += x[2] + x[6];
+        a3 += x[3] + x[7];
+      }
+      for (; h < H; ++h) a0 += exp2_fast(col[h * SW] + hc[h]);
+      float a = (a0 + a1) + (a2 + a3);
+      if (pj < p.keep_first) a = INFINITY;
+      const int g = (t < n_loc) ? s_begin + t : p.cap;
+      if (a < val) { val = a; idx = g; ccol = c; }      // t ascends and with it the slot: strict < keeps the lowest
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, val, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+      const int oc = __shfl_xor_sync(0xffffffffu, ccol, o);
+      if (ov < val || (ov == val && oi < idx)) { val = ov; idx = oi; ccol = oc; }
+    }
+    if (lane == 0) { red_v[warp] = val; red_i[warp] = idx; red_c[warp] = ccol; }
+    // ---- this CTA's correction for token i+1: the terms of the columns that died in its care so far --------
+    if (more) {
+      ok = warp_wait(&full[(i + 1) % nstage], (uint32_t)(((i + 1) / nstage) & 1)) && ok;
+      const int nd = s_ndead;
+      for (int h = warp; h < H; h += NW) {                  // a warp per head, a lane per dead column
+        const float R1 = Rs[(i + 1) * H + h];
+        float g = 0.f;
+        for (int d = lane; d < nd; d += 32) g += exp2_fast(st1[h * SW + dead[d]] - R1);
+        g = warp_sum(g);
+        if (lane == 0) s_co[h] = g;
+      }
+    }
+    __syncthreads();
+    if (warp == 0) {
+      val = (lane < NW) ? red_v[lane] : INFINITY;
+      idx = (lane < NW) ? red_i[lane] : 0x7fffffff;
+      ccol = (lane < NW) ? red_c[lane] : -1;
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, val, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+        const int oc = __shfl_xor_sync(0xffffffffu, ccol, o);
+        if (ov < val || (ov == val && oi < idx)) { val = ov; idx = oi; ccol = oc; }
+      }
+      // the candidate to every CTA, and with it what the next token's normaliser loses if this candidate is the
+      // one to go (its terms for token i+1) and this CTA's correction
+      if (lane < NC) *cl.map_shared_rank(&best[par][r], lane) = make_float2(val, __int_as_float(idx));
+      if (more) {
+        for (int h = lane; h < H; h += 32) {
+          const float en = (ccol >= 0) ? exp2_fast(st1[h * SW + ccol] - Rs[(i + 1) * H + h]) : 0.f;
+          const float co = s_co[h];
+          for (int q = 0; q < NC; ++q) {
+            *cl.map_shared_rank(&xen[((size_t)par * NCM + r) * H + h], q) = en;
+            *cl.map_shared_rank(&xco[((size_t)par * NCM + r) * H + h], q) = co;
+          }
+        }
+      }
+    }
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    // ---- the same arg-min in every CTA; the slot's owner lets the token in; the next token's normaliser ----------
+    float bv = INFINITY;
+    int bi = 0x7fffffff, rw = 0;
+    for (int rr = 0; rr < NC; ++rr) {
+      const float2 e = best[par][rr];
+      const int ei = __float_as_int(e.y);
+      if (e.x < bv || (e.x == bv && ei < bi)) { bv = e.x; bi = ei; rw = rr; }
+    }
+    if (bi < 0 || bi > p.cap) {                          // cannot happen with finite logits: report, drop the token
+      if (tid == 0 && r == 0) atomicExch(p.status, DEV_ERR_BAD_VICTIM);
+      bi = p.cap;
+      rw = 0;
+    }
+    if (more) {
+      for (int h = tid; h < H; h += NT) {
+        float gone = xen[((size_t)par * NCM + rw) * H + h];
+        for (int rr = 0; rr < NC; ++rr) gone += xco[((size_t)par * NCM + rr) * H + h];
+        const float R1 = Rs[(i + 1) * H + h];
+        const float L = Ts[(i + 1) * H + h] - gone;
+        hc[h] = -R1 - __log2f(L * (float)H);
+        if (r == 0) p.ml[((size_t)b * H + h) * CHUNK_TOKENS + i + 1] = make_float2(R1, L);
+      }
+    }
+    if (tid == 0) {
+      if (i + nstage < p.C) arm(i + nstage);             // (this buffer's phase of token i was consumed above)
+      if (bi < p.cap) {
+        const int l = bi - s_begin;
+        if (l >= 0 && l < n_loc) {                      // Eq. 9 in place: the token takes the dropped row's slot
+          const int old = occl[l];
+          p.death[(size_t)b * p.ldc + (old < S ? s_begin + old : p.capA + (old - S))] = i;
+          if (p.evicted) p.evicted[(size_t)i * p.B + b] = posv[l];
+          occl[l] = S + i;
+          posv[l] = pos_i;
+          dead[s_ndead] = old;
+          s_ndead = s_ndead + 1;
+        }
+      } else if (r == 0) {                               // the token itself had the lowest weight
+        p.death[(size_t)b * p.ldc + p.capA + i] = i;
+        if (p.evicted) p.evicted[(size_t)i * p.B + b] = pos_i;
+        dead[s_ndead] = S + i;
+        s_ndead = s_ndead + 1;
+      }
+    }
+    __syncthreads();                                     // the buffer has been read by everybody; occl, hc, dead are up to date
+    if (i + nstage < p.C) {
       fence_proxy_async_smem();
       request(i + nstage);
     }

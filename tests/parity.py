@@ -61,7 +61,7 @@ POLICIES = {"tova": tova.TOVA_POLICY_TOVA, "window": tova.TOVA_POLICY_WINDOW,
 
 def make_cache(w: W.Workload, sm_scale: float = 0.0, evict: bool = True, chunk_rows: int = 0,
                fused_merge: bool = True, policy: str = "tova", keep_first: int = 0, prefill_ws: bool = False,
-               chunk_cluster: int = 0, rope_base: float = 0.0):
+               chunk_cluster: int = 0, rope_base: float = 0.0, chunk_barriers: int = 0):
     c = tova.TovaCache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, dtype=w.dtype,
                        sm_scale=sm_scale, evict=evict)
     if chunk_rows:
@@ -76,6 +76,8 @@ def make_cache(w: W.Workload, sm_scale: float = 0.0, evict: bool = True, chunk_r
         c.tova_cache_set_prefill_workspace()
         if chunk_cluster:
             c.tova_cache_set_chunk_cluster(chunk_cluster)
+        if chunk_barriers:
+            c.tova_cache_set_chunk_barriers(chunk_barriers)
     return c
 
 
@@ -100,7 +102,7 @@ def run_lockstep(w: W.Workload, n_tokens: int, *, seqs: Optional[Sequence[int]] 
                  first_pos: int = 0, check_state_every: int = 4, direct_fill: bool = False,
                  fused_merge: bool = True, policy: str = "tova", keep_first: int = 0,
                  period: int = 0, prefill_ws: bool = False, chunk_cluster: int = 0,
-                 rope_base: float = 0.0) -> ParityReport:
+                 rope_base: float = 0.0, chunk_barriers: int = 0) -> ParityReport:
     """Feed n_tokens tokens to both sides and compare at every token.
 
     direct_fill: while the state is filling nothing is dropped (Section 3.3), so
@@ -117,7 +119,7 @@ def run_lockstep(w: W.Workload, n_tokens: int, *, seqs: Optional[Sequence[int]] 
     own = cache is None
     cache = cache or make_cache(w, sm_scale=sm_scale, chunk_rows=chunk_rows, fused_merge=fused_merge,
                                 policy=policy, keep_first=keep_first, prefill_ws=prefill_ws,
-                                chunk_cluster=chunk_cluster, rope_base=rope_base)
+                                chunk_cluster=chunk_cluster, rope_base=rope_base, chunk_barriers=chunk_barriers)
     orc = oracle or OracleCache(len(seqs), w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity,
                                 sm_scale=sm_scale, precision="f32", policy=policy, keep_first=keep_first,
                                 rope_base=rope_base)

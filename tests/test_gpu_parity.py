@@ -189,16 +189,27 @@ def test_chunked_prompt_against_the_checker(H, Hkv, D, cap, B, block, keep):
             assert np.array_equal(st["V"][b, :, s].numpy(), v[pos[b, s], b])
 
 
+@pytest.mark.parametrize("barriers", [0, 2])
 @pytest.mark.parametrize("ctas", [-1, 1, 2, 4, 8])
-def test_chunked_prompt_every_cluster_size(ctas):
+def test_chunked_prompt_every_cluster_size(ctas, barriers):
     """The deletion kernel as one thread block reading global memory (-1) and as clusters of 1 to 8 blocks
-    with staged logits; capacity 333 leaves the last block of a cluster a ragged share (8 x 44 > 333)."""
+    with staged logits, meeting once per token (the normaliser from the row sum minus the dropped rows' terms)
+    or twice; capacity 333 leaves the last block of a cluster a ragged share (8 x 44 > 333)."""
+    if ctas == -1 and barriers:
+        pytest.skip("one block per sequence: no cluster")
     w = MISTRAL.scaled(batch=2, n_q_heads=8, n_kv_heads=2, capacity=333)
-    rep = run_lockstep(w, 333 + 64 + 40, block=64, prefill_ws=True, chunk_cluster=ctas, check_state_every=1)
+    rep = run_lockstep(w, 333 + 64 + 40, block=64, prefill_ws=True, chunk_cluster=ctas, check_state_every=1,
+                       chunk_barriers=barriers)
     assert rep.evictions == 2 * 104
     w = LLAMA.scaled(batch=1, n_q_heads=4, n_kv_heads=4, capacity=20)      # fewer slots than blocks can share out
-    rep = run_lockstep(w, 20 + 64 * 2, block=64, prefill_ws=True, chunk_cluster=ctas, check_state_every=1)
+    rep = run_lockstep(w, 20 + 64 * 2, block=64, prefill_ws=True, chunk_cluster=ctas, check_state_every=1,
+                       chunk_barriers=barriers)
     assert rep.evictions == 128
+    # protected positions and a token that drops itself now and then (keep_first leaves few candidates)
+    w = MISTRAL.scaled(batch=2, n_q_heads=8, n_kv_heads=2, capacity=70)
+    rep = run_lockstep(w, 70 + 64 * 3 + 9, block=64, prefill_ws=True, chunk_cluster=ctas, check_state_every=1,
+                       chunk_barriers=barriers, keep_first=4)
+    assert rep.evictions == 2 * (64 * 3 + 9)
 
 
 def test_chunked_prompt_equals_token_by_token_processing():
