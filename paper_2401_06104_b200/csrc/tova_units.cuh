@@ -102,8 +102,17 @@ __global__ void __launch_bounds__(UNIT_THREADS) tova_unit_policy_kernel(const St
   int idx = 0x7fffffff, cpos = pos_t;
   for (int j = j_lo + tid; j < j_hi; j += UNIT_THREADS) {
     float w = 0.f;
-#pragma unroll 8
-    for (int h = 0; h < nh; ++h) w += exp2f(lg[(size_t)h * p.ld + j] + hc[h]);
+    {
+      int h = 0;
+      for (; h + 7 < nh; h += 8) {          // eight heads' logits requested before the first is used
+        float x[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) x[e] = lg[(size_t)(h + e) * p.ld + j] + hc[h + e];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) w += exp2f(x[e]);
+      }
+      for (; h < nh; ++h) w += exp2f(lg[(size_t)h * p.ld + j] + hc[h]);
+    }
     float key = w;
     const int pj = (j < p.n) ? table[j] : pos_t;
     if (up.h2o && j < p.n) {             // the row's weight at this step joins its sum before the choice
