@@ -189,14 +189,11 @@ def test_chunked_prompt_against_the_checker(H, Hkv, D, cap, B, block, keep):
             assert np.array_equal(st["V"][b, :, s].numpy(), v[pos[b, s], b])
 
 
-@pytest.mark.parametrize("barriers", [0, 2])
-@pytest.mark.parametrize("ctas", [-1, 1, 2, 4, 8])
+@pytest.mark.parametrize("ctas,barriers", [(-1, 0)] + [(c, nb) for c in (1, 2, 4, 8) for nb in (0, 2)])
 def test_chunked_prompt_every_cluster_size(ctas, barriers):
     """The deletion kernel as one thread block reading global memory (-1) and as clusters of 1 to 8 blocks
     with staged logits, meeting once per token (the normaliser from the row sum minus the dropped rows' terms)
     or twice; capacity 333 leaves the last block of a cluster a ragged share (8 x 44 > 333)."""
-    if ctas == -1 and barriers:
-        pytest.skip("one block per sequence: no cluster")
     w = MISTRAL.scaled(batch=2, n_q_heads=8, n_kv_heads=2, capacity=333)
     rep = run_lockstep(w, 333 + 64 + 40, block=64, prefill_ws=True, chunk_cluster=ctas, check_state_every=1,
                        chunk_barriers=barriers)
