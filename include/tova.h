@@ -241,9 +241,11 @@ int tova_cache_set_chunk_rows(tova_cache* c, int32_t rows);
  * TOVA_ERR_BAD_SHAPE; an unknown policy gives TOVA_ERR_UNSUPPORTED.  Positions
  * passed to the step calls must be >= 0, distinct and increasing for Window, "+i"
  * and H2O to mean what the paper describes; ties go to the lowest slot as
- * everywhere.  Head-wise and H2O policies process prompts token by token; with
- * deferred eviction their victim choice and insert run on the cache's stream like
- * the layer policies'.  Not available through tova_decode_step_static. */
+ * everywhere.  H2O processes prompts token by token (its scores accumulate from
+ * the first token on); head-wise TOVA takes the bulk route for prompt tokens that
+ * find free rows and goes token by token from there.  With deferred eviction
+ * their victim choice and insert run on the cache's stream like the layer
+ * policies'.  Not available through tova_decode_step_static. */
 #define TOVA_POLICY_TOVA 0
 #define TOVA_POLICY_WINDOW 1
 #define TOVA_POLICY_TOVA_HEAD 2

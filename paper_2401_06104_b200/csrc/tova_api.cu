@@ -780,6 +780,8 @@ int launch_fill(tova_cache* c, const void* q, const void* k, const void* v, int 
   p.cur_pos = reinterpret_cast<int32_t*>(base + c->lay.cur_pos);
   p.status = reinterpret_cast<int32_t*>(base + c->lay.status);
   p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.evicted = evicted_pos;
+  p.units = c->units > 1 ? c->units : 1;
+  p.upos = c->units > 1 ? reinterpret_cast<int32_t*>(base + c->lay.upos) : nullptr;
   p.B = c->cfg.batch; p.H = c->cfg.n_q_heads; p.Hkv = c->cfg.n_kv_heads; p.G = p.H / p.Hkv;
   p.cap = c->cfg.capacity;
   p.n0 = c->len;
@@ -1286,8 +1288,9 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
   {
     const int room = c->cfg.capacity - c->len;
     const int F = n_tokens < room ? n_tokens : room;
-    // (the per-unit policies keep their own slot tables and scores: token by token)
-    if (c->bulk_fill && c->fill_maps && F >= BULK_FILL_MIN_TOKENS && c->units == 0 && !c->poscomp_ws) {
+    // (H2O accumulates scores from the first token on: token by token; head-wise TOVA only needs its slot tables)
+    const bool unit_ok = c->units == 0 || c->policy == tova::POLICY_TOVA_HEAD;
+    if (c->bulk_fill && c->fill_maps && F >= BULK_FILL_MIN_TOKENS && unit_ok && !c->poscomp_ws) {
       rc = launch_fill(c, q, k, v, F, first_pos, out, evicted_pos, static_cast<cudaStream_t>(cuda_stream));
       if (rc != TOVA_OK) return rc;
       done = F;

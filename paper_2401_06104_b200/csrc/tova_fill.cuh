@@ -41,7 +41,9 @@ struct FillParams {
   const void* k_new;       // [F,B,Hkv,D]
   const void* v_new;
   float* out;              // [F,B,H,D]
-  int32_t* evicted;        // [F,B] or null
+  int32_t* evicted;        // [F,B] ([F,B,units] with per-unit tables) or null
+  int32_t* upos;           // [B,units,cap] per-unit slot tables (head-wise TOVA), or null
+  int units;               // units that own rows: 1 (the layer) or Hkv
   int B, H, Hkv, G, cap;
   int n0;                  // rows held before the run
   int F;                   // tokens in the run (n0 + F <= cap)
@@ -71,7 +73,14 @@ __global__ void tova_fill_rows_kernel(const FillParams p) {
     const int b = (int)(i % p.B);
     const int t = (int)(i / p.B);
     p.pos[(size_t)b * p.cap + p.n0 + t] = first + t;
-    if (p.evicted) p.evicted[i] = -1;
+    if (p.upos) {                      // every unit holds the same tokens while nothing is dropped
+      for (int u = 0; u < p.units; ++u) {
+        p.upos[((size_t)b * p.units + u) * p.cap + p.n0 + t] = first + t;
+        if (p.evicted) p.evicted[i * p.units + u] = -1;
+      }
+    } else if (p.evicted) {
+      p.evicted[i] = -1;
+    }
   }
 }
 

@@ -158,6 +158,40 @@ def test_bulk_prefill_against_decode_steps(H, Hkv, D, cap, T0, T1, mode):
     assert a.tova_cache_launches() < b.tova_cache_launches()
 
 
+def test_bulk_prefill_head_wise_tova_against_decode_steps():
+    """Head-wise TOVA: the prompt tokens that find free rows take the bulk route too (every KV head's slot table
+    gets the same positions, nothing is dropped); per-unit dropped positions, slot tables, rows and all later outputs
+    bit-identical to decode steps, outputs of the bulk tokens within the output tolerance."""
+    w = MISTRAL.scaled(batch=2, n_q_heads=8, n_kv_heads=4, capacity=150)
+    T0, T1 = 90, 140
+    T, U = T0 + T1, w.n_kv_heads
+    q, k, v = W.tokens(w, 0, T)
+    dq, dk, dv = (tova.to_device(x, w.dtype) for x in (q, k, v))
+    caches, outs, evs = [], [], []
+    for bulk in (True, False):
+        c = make_cache(w)
+        c.tova_cache_set_policy(tova.TOVA_POLICY_TOVA_HEAD, 0)
+        out = torch.empty(T, w.batch, w.n_q_heads, w.head_dim, dtype=torch.float32, device="cuda:0")
+        ev = torch.full((T, w.batch, U), -12345, dtype=torch.int32, device="cuda:0")
+        if bulk:
+            c.tova_prefill(dq[:T0], dk[:T0], dv[:T0], T0, 0, out[:T0], ev[:T0])
+            c.tova_prefill(dq[T0:], dk[T0:], dv[T0:], T1, T0, out[T0:], ev[T0:])
+        else:
+            for t in range(T):
+                c.tova_decode_step(dq[t], dk[t], dv[t], t, out[t], ev[t])
+        torch.cuda.synchronize()
+        caches.append(c); outs.append(out.cpu().numpy()); evs.append(ev.cpu().numpy())
+    assert np.array_equal(evs[0], evs[1])
+    assert np.all(evs[0][:w.capacity] == -1) and np.any(evs[0][w.capacity:] >= 0)
+    assert np.abs(outs[0][:w.capacity] - outs[1][:w.capacity]).max() <= out_tol(w)
+    assert np.array_equal(outs[0][w.capacity:], outs[1][w.capacity:])
+    sa, sb = (c.tova_cache_read(want_kv=True) for c in caches)
+    assert sa["status"] == 0 and sb["status"] == 0
+    for key in ("len", "positions", "K", "V"):
+        assert torch.equal(sa[key], sb[key]), key
+    assert caches[0].tova_cache_launches() < caches[1].tova_cache_launches()
+
+
 # ---------------------------------------------------------------------------
 # prompt tokens that meet a full state, in chunks (appendix "Experimental Details": whole chunks at once,
 # the attention masked according to the layer's attention weights)
