@@ -16,13 +16,14 @@
 //             earlier tokens - plus each query's row maximum R and the sum T of
 //             exp2(logit - R) over all those columns (tova_chunk_attn_kernel,
 //             MODE 0; warp-level bf16 MMAs, as in the bulk fill);
-//   resolve   one thread block per sequence - or a cluster of blocks that share
-//             out the slots, with the logits staged in shared memory
+//   resolve   a cluster of thread blocks per sequence that share out the slots,
+//             with the logits staged in shared memory
 //             (tova_chunk_resolve_cluster1_kernel, one cluster barrier per token;
-//             tova_chunk_resolve_cluster_kernel, two) - replays the chunk's
-//             deletions in order from those logits alone (tova_chunk_resolve_kernel): for
-//             token i it removes the rows dropped by tokens < i from the
-//             normaliser (L = T - their terms), scores the k+1 live candidates
+//             tova_chunk_resolve_cluster_kernel, two) - or one block per sequence
+//             reading global memory (tova_chunk_resolve_kernel) - replays the
+//             chunk's deletions in order from those logits alone: for token i it
+//             removes the rows dropped by tokens < i from the normaliser
+//             (L = T - their terms), scores the k+1 live candidates
 //             by the head-averaged soft-max weight (Eq. 4, Algorithm 1), takes
 //             the arg-min - lowest slot on ties, the token itself being slot k -
 //             records the dropped position and lets the token take the slot.
