@@ -524,7 +524,6 @@ def run_prefill(args):
     steps, warm = min(args.steps, 8), min(max(args.warmup, 3), 3)
     q, k, v = (tova.to_device(a, w.dtype, dev) for a in W.tokens(w, 0, T))
     out = torch.empty(T, B, H, D, dtype=torch.float32, device=dev)
-    ev = torch.empty(T, B, dtype=torch.int32, device=dev)
     caches = []
     chunked = not (args.no_chunked_prefill or args.no_bulk_prefill) and w.dtype == W.DTYPE_BF16 and T > cap
     ws = None
@@ -532,6 +531,10 @@ def run_prefill(args):
         c = tova.TovaCache(B, H, Hkv, D, cap, dtype=w.dtype, device=dev)
         if args.no_bulk_prefill or args.warp_mma_prefill:
             c.tova_cache_set_bulk_prefill(0 if args.no_bulk_prefill else 2)
+        if args.policy != "tova" or args.keep_first:
+            c.tova_cache_set_policy({"tova": tova.TOVA_POLICY_TOVA, "window": tova.TOVA_POLICY_WINDOW,
+                                     "tova_head": tova.TOVA_POLICY_TOVA_HEAD, "h2o_layer": tova.TOVA_POLICY_H2O_LAYER,
+                                     "h2o_head": tova.TOVA_POLICY_H2O_HEAD}[args.policy], args.keep_first)
         if chunked:
             ws = c.tova_cache_set_prefill_workspace(ws)          # one workspace serves all: calls share a stream
             if args.chunk_cluster:
@@ -539,6 +542,7 @@ def run_prefill(args):
             if args.chunk_barriers:
                 c.tova_cache_set_chunk_barriers(args.chunk_barriers)
         caches.append(c)
+    ev = torch.empty(T, B, caches[0].tova_cache_units(), dtype=torch.int32, device=dev)   # per unit for head-wise policies
     torch.cuda.synchronize()
     for c in caches[:warm]:
         c.tova_prefill(q, k, v, T, 0, out, ev)

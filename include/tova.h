@@ -145,7 +145,7 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
  *        shared by caches of one shape whose calls are ordered on one stream.
  *        TOVA_ERR_UNSUPPORTED for fp32 states and for capacities beyond what the
  *        deletion kernel's shared memory holds (about 25,000 rows).
- * Used for the TOVA policy (with or without protected first positions) on bf16
+ * Used for the TOVA and Window policies (with or without protected first positions) on bf16
  * states, for runs of at least 8 tokens; everything else takes the per-token
  * route as before. */
 size_t tova_prefill_workspace_bytes(const tova_config* cfg);

@@ -918,6 +918,7 @@ int launch_chunk(tova_cache* c, const void* q, const void* k, const void* v, int
   p.C = C;
   p.first_pos = first_pos;
   p.keep_first = c->keep_first;
+  p.window = c->policy == tova::POLICY_WINDOW ? 1 : 0;
   p.scale2 = c->scale2;
   const cudaError_t e = c->cfg.head_dim == 128 ? launch_chunk_d<128>(c, p, st) : launch_chunk_d<64>(c, p, st);
   return e == cudaSuccess ? TOVA_OK : TOVA_ERR_CUDA;
@@ -1297,9 +1298,9 @@ int tova_prefill(tova_cache* c, const void* q, const void* k, const void* v, int
     }
   }
   // Tokens that meet a full state: chunks of up to 64 through the caller's workspace, where one was given
-  // (TOVA policy, with or without protected first positions; bf16 states).
-  const bool chunked = c->chunk_ws && c->bulk_fill && c->cfg.evict && c->units == 0 && c->policy == tova::POLICY_TOVA &&
-                       !c->poscomp_ws;
+  // (TOVA or Window, with or without protected first positions; bf16 states).
+  const bool chunked = c->chunk_ws && c->bulk_fill && c->cfg.evict && c->units == 0 &&
+                       (c->policy == tova::POLICY_TOVA || c->policy == tova::POLICY_WINDOW) && !c->poscomp_ws;
   for (int32_t t = done; t < n_tokens;) {
     if (chunked && c->len == c->cfg.capacity && n_tokens - t >= CHUNK_MIN_TOKENS) {
       const int C = n_tokens - t < tova::CHUNK_TOKENS ? n_tokens - t : tova::CHUNK_TOKENS;

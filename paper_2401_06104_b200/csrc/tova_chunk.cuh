@@ -77,6 +77,7 @@ struct ChunkParams {
   int C;                   // tokens in this chunk (1..64)
   int first_pos;           // position of the chunk's first token, or < 0: current position + 1
   int keep_first;          // rows holding positions 0..keep_first-1 are never dropped
+  int window;              // 1: the Window policy - the row holding the earliest droppable position goes
   float scale2;
 };
 
@@ -391,6 +392,7 @@ __global__ void __launch_bounds__(CHUNK_RESOLVE_THREADS) tova_chunk_resolve_kern
       float a = 0.f;
 #pragma unroll 8
       for (int h = 0; h < p.H; ++h) a += exp2f(col[h * hstride] + hc[h]);
+      if (p.window) a = (float)(pj - pos_i);             // Window: the earliest position goes (ages are below 2^24: exact)
       if (pj < p.keep_first) a = INFINITY;               // one of the first i token states: never dropped
       if (a < val) { val = a; idx = s; }                 // s ascends: strict < keeps the lowest slot
     }
@@ -566,6 +568,7 @@ __global__ void __launch_bounds__(CHUNK_CLUSTER_THREADS_MAX) tova_chunk_resolve_
       }
       for (; h < H; ++h) a0 = fmaf(col[(size_t)h * SW], invLH[h], a0);
       float a = (a0 + a1) + (a2 + a3);
+      if (p.window) a = (float)(pj - pos_i);             // Window: the earliest position goes
       if (pj < p.keep_first) a = INFINITY;
       const int g = (t < n_loc) ? s_begin + t : p.cap;
       if (a < val) { val = a; idx = g; }               // t ascends and with it the slot: strict < keeps the lowest
@@ -750,6 +753,7 @@ __global__ void __launch_bounds__(CHUNK_CLUSTER_THREADS_MAX) tova_chunk_resolve_
       }
       for (; h < H; ++h) a0 += exp2_fast(col[h * SW] + hc[h]);
       float a = (a0 + a1) + (a2 + a3);
+      if (p.window) a = (float)(pj - pos_i);             // Window: the earliest position goes
       if (pj < p.keep_first) a = INFINITY;
       const int g = (t < n_loc) ? s_begin + t : p.cap;
       if (a < val) { val = a; idx = g; ccol = c; }      // t ascends and with it the slot: strict < keeps the lowest

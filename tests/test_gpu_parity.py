@@ -243,6 +243,22 @@ def test_chunked_prompt_every_cluster_size(ctas, barriers):
     assert rep.evictions == 2 * (64 * 3 + 9)
 
 
+@pytest.mark.parametrize("keep,ctas,barriers", [(0, 0, 0), (4, 2, 0), (4, 4, 2), (0, -1, 0)])
+def test_chunked_prompt_window_policy(keep, ctas, barriers):
+    """Window and Window+4 on the chunked route (the row holding the earliest droppable position goes, the
+    normalisers and outputs come from the same passes): every token against the checker, and the state ends up
+    holding exactly the protected positions and the latest ones."""
+    w = MISTRAL.scaled(batch=2, n_q_heads=8, n_kv_heads=2, capacity=150)
+    n = 150 + 64 * 3 + 20
+    rep = run_lockstep(w, n, block=64, prefill_ws=True, policy="window", keep_first=keep, chunk_cluster=ctas,
+                       chunk_barriers=barriers, check_state_every=1)
+    assert rep.evictions == 2 * (n - 150)
+    held = rep.cache.tova_cache_read()["positions"].numpy()
+    want = sorted(list(range(keep)) + list(range(n - (150 - keep), n)))
+    for b in range(w.batch):
+        assert sorted(held[b].tolist()) == want
+
+
 def test_chunked_prompt_equals_token_by_token_processing():
     """Same prompt through the chunked route and through decode steps: the same dropped positions, the same
     state, outputs within the output tolerance; later decode steps bit-identical.  Also: no outputs wanted,
