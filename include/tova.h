@@ -279,7 +279,7 @@ int32_t tova_cache_units(const tova_cache* c);
  *        B*(capacity+1)*D/2 pairs, the rotated query, the positions.
  *   tova_cache_set_position_compression  dev_mem: 256-byte aligned device
  *        memory of that size, owned by the caller, to outlive the handle (NULL:
- *        off); only while the state is empty; capacity up to about 7000 rows
+ *        off); only while the state is empty; capacity up to 8191 rows
  *        (TOVA_ERR_UNSUPPORTED beyond, and together with head-wise policies or
  *        sharding).  The step then takes three launches and a slower streaming
  *        kernel (a table read and a rotation per cached row); prompts go token
