@@ -87,6 +87,7 @@ def test_null_handles_are_rejected():
     assert L.tova_cache_units(None) == -1
     assert L.tova_cache_set_prefill_workspace(None, None, 0) == -1
     assert L.tova_cache_set_chunk_cluster(None, 0) == -1
+    assert L.tova_cache_set_chunk_barriers(None, 0) == -1
     assert L.tova_cache_set_position_compression(None, None, 0, 10000.0) == -1
     assert L.tova_cache_read_compressed_positions(None, None, None) == -1
     assert L.tova_position_workspace_bytes(ctypes.byref(cfg())) > 2 * 101 * 64 * 8

@@ -302,6 +302,11 @@ def test_prefill_workspace_argument_errors():
     for bad in (3, 16, -2):
         with pytest.raises(tova.TovaError):
             c.tova_cache_set_chunk_cluster(bad)
+    for bad in (1, 3, -1):
+        with pytest.raises(tova.TovaError):
+            c.tova_cache_set_chunk_barriers(bad)
+    c.tova_cache_set_chunk_barriers(2)
+    c.tova_cache_set_chunk_barriers(0)
 
 
 def test_bulk_prefill_mode_argument():
